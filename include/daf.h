@@ -1,0 +1,184 @@
+/*
+ * daf.h -- C ABI of the B200 (sm_100a) activation compress / decompress library.
+ *
+ * The library implements the data-parallel hot path of the Dynamic Activation
+ * Framework: saved activations are quantized group by group after the forward
+ * pass and dequantized before the backward pass (Sec. 2.3 of the paper).
+ *
+ * Conventions for every entry point
+ *   - Pointers named d_* are DEVICE pointers owned by the caller; h_* are HOST
+ *     pointers.  The library never allocates or frees device memory: inputs,
+ *     outputs and scratch ("workspace") all belong to the caller.
+ *   - `stream` is a cudaStream_t passed as void*.  GPU work is enqueued on it
+ *     and the call returns without waiting; outputs are valid once the stream
+ *     has reached that point.
+ *   - The return value is a daf_status.  Argument errors are detected on the
+ *     host before anything is launched.  Errors that only the device can see
+ *     (packed buffer too small, a bounded wait that ran out) are recorded in a
+ *     status word inside the workspace and read back with daf_poll_status; the
+ *     kernels never store out of bounds, trap or spin without limit.
+ *   - Device pointers must be 16-byte aligned unless stated otherwise.
+ *   - No entry point throws; none keeps global state between calls.
+ *
+ * Data layout (all tensors are flat, contiguous, row-major)
+ *   group   : G consecutive elements (G a power of two, 32 <= G <= window_elems)
+ *   window  : window_elems consecutive elements = the unit over which the
+ *             average bit budget is enforced and the unit of parallel work
+ *   packed  : for group g, G*b_g/8 bytes at byte offset sum_{h<g} G*b_h/8; code i
+ *             of the group occupies bits [i*b_g, (i+1)*b_g) of that byte string,
+ *             least significant bit first (little-endian 32-bit words with
+ *             code i at shift (i*b_g) mod 32); no padding anywhere
+ *   bits    : one byte per group, the width b_g itself
+ *   min, scale : one float per group (binary32 for every input dtype)
+ *   window_offsets : n_windows+1 uint64 byte offsets of each window's first
+ *             group in `packed`; the last entry is the total packed size
+ */
+#ifndef DAF_H
+#define DAF_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum daf_status {
+    DAF_OK = 0,
+    DAF_ERR_INVALID_ARG = 1,  /* null / misaligned pointer, bad group or window size, bad mask */
+    DAF_ERR_SHAPE = 2,        /* numel is zero or not a multiple of the group size            */
+    DAF_ERR_BUDGET = 3,       /* bit budget below the smallest allowed width                   */
+    DAF_ERR_CAPACITY = 4,     /* packed buffer or workspace too small                          */
+    DAF_ERR_CUDA = 5,         /* a CUDA runtime call failed                                    */
+    DAF_ERR_TIMEOUT = 6,      /* a bounded device-side wait ran out                            */
+    DAF_ERR_UNSUPPORTED = 7   /* valid request this build does not implement                   */
+} daf_status;
+
+typedef enum daf_dtype { DAF_F32 = 0, DAF_F16 = 1, DAF_BF16 = 2 } daf_dtype;
+typedef enum daf_round { DAF_ROUND_STOCHASTIC = 0, DAF_ROUND_NEAREST = 1 } daf_round;
+
+typedef void *daf_stream;     /* a cudaStream_t */
+
+/* Description of one tensor and of how it is (was) compressed. */
+typedef struct daf_params {
+    uint32_t struct_size;     /* sizeof(daf_params), for ABI checking                               */
+    uint32_t dtype;           /* daf_dtype of the input of compress / the output of decompress      */
+    uint64_t numel;           /* elements; a positive multiple of group_size                        */
+    uint32_t group_size;      /* G: power of two, 32 <= G <= window_elems                           */
+    uint32_t window_elems;    /* 0 means 16384; supported: 4096, 8192, 16384                        */
+    uint32_t width_mask;      /* bit b set <=> width b allowed; non-empty subset of {1,2,4,8}       */
+    float    bit_budget;      /* average bits per element per window; floor(budget*256)/256 is used */
+    uint32_t rounding;        /* daf_round                                                          */
+    uint32_t reserved;        /* must be 0                                                          */
+    uint64_t seed;            /* Philox key                                                         */
+    uint64_t elem_index_base; /* global index of element 0 (a multiple of 8); 0 unless the tensor
+                                 is a shard of a larger one compressed with the same seed          */
+} daf_params;
+
+/*
+ * Sizes that follow from the parameters (host only, launches nothing).
+ *   n_groups = numel / G, n_windows = ceil(n_groups / (window_elems / G)),
+ *   packed_capacity_bytes = sum over windows of floor(beta_q8 * n / 256) * G / 8 with n the
+ *   window's group count and beta_q8 = floor(bit_budget * 256): an upper bound on the packed
+ *   size that the budget guarantees,
+ *   workspace_bytes = scratch needed by daf_compress / daf_decompress for this tensor.
+ * Any output pointer may be NULL.  Errors: INVALID_ARG, SHAPE, BUDGET, UNSUPPORTED.
+ */
+daf_status daf_sizes(const daf_params *params, uint64_t *n_groups, uint64_t *n_windows,
+                     uint64_t *packed_capacity_bytes, uint64_t *workspace_bytes);
+
+/*
+ * Compress one tensor (Eq. 1 applied per group; widths chosen greedily per window by
+ * importance per bit under the budget, Sec. 3.4.1; codes packed compactly, Sec. 3.3).
+ *   d_in             in : numel elements of params->dtype
+ *   d_packed         out: packed codes, at most packed_capacity bytes are written
+ *   d_bits           out: n_groups bytes        d_min, d_scale  out: n_groups floats each
+ *   d_window_offsets out: n_windows + 1 uint64
+ *   d_workspace          : workspace_bytes of scratch, contents irrelevant on entry; also
+ *                          holds the device status word afterwards (see daf_poll_status)
+ * One fused kernel reads the input once.  If the packed output of a window would pass
+ * packed_capacity, nothing of that window is stored and the status word becomes
+ * DAF_ERR_CAPACITY.  Inputs must be finite; behaviour on NaN / Inf is unspecified but
+ * memory safe.  Calls sharing a workspace must not overlap on the GPU.
+ */
+daf_status daf_compress(const daf_params *params, const void *d_in, void *d_packed,
+                        uint64_t packed_capacity, uint8_t *d_bits, float *d_min, float *d_scale,
+                        uint64_t *d_window_offsets, void *d_workspace, uint64_t workspace_bytes,
+                        daf_stream stream);
+
+/*
+ * Decompress (Sec. 2.3: stored activations are dequantized to their original precision
+ * for the gradient computation): x_hat = fma(code, scale, min), rounded to nearest even
+ * into params->dtype.  Inputs are the outputs of daf_compress for the same params;
+ * d_out receives numel elements.  The workspace is not used by this version and may be NULL.
+ */
+daf_status daf_decompress(const daf_params *params, const void *d_packed, const uint8_t *d_bits,
+                          const float *d_min, const float *d_scale,
+                          const uint64_t *d_window_offsets, void *d_out, void *d_workspace,
+                          uint64_t workspace_bytes, daf_stream stream);
+
+/*
+ * Device-wide exclusive prefix sum of the group byte lengths G*b_g/8 ("layout
+ * concatenation", Sec. 3.3): d_offsets[g] = sum_{h<g} G*bits[h]/8 for g = 0..n_groups.
+ * Single pass with a bounded decoupled look-back.  d_ws: daf_group_offsets_workspace(n_groups)
+ * bytes of scratch.  d_bits needs no alignment; d_offsets must be 8-byte aligned.
+ */
+daf_status daf_group_offsets(const uint8_t *d_bits, uint64_t n_groups, uint32_t group_size,
+                             uint64_t *d_offsets, void *d_ws, uint64_t ws_bytes, daf_stream stream);
+uint64_t   daf_group_offsets_workspace(uint64_t n_groups);
+
+/*
+ * Wait for `stream` and return the device status word of a workspace that was last used by
+ * daf_compress, daf_compress_batch or daf_group_offsets: DAF_OK, DAF_ERR_CAPACITY or
+ * DAF_ERR_TIMEOUT (DAF_ERR_CUDA if the copy itself fails).
+ */
+daf_status daf_poll_status(const void *d_workspace, daf_stream stream);
+
+/*
+ * Batched forms for sets of activations (one launch per up to DAF_BATCH_MAX tensors): the
+ * result for tensor i is exactly that of the single-tensor call with params[i] and the i-th
+ * pointers.  All arrays are HOST arrays of n entries holding device pointers / capacities;
+ * every tensor of a batch must share dtype, group_size, window_elems, width_mask, bit_budget
+ * and rounding (seed and elem_index_base may differ).  One workspace serves the whole batch:
+ * daf_batch_workspace(n, params) bytes.
+ */
+#define DAF_BATCH_MAX 64   /* tensors per batched call */
+uint64_t   daf_batch_workspace(uint32_t n, const daf_params *params);
+daf_status daf_compress_batch(uint32_t n, const daf_params *params, const void *const *d_in,
+                              void *const *d_packed, const uint64_t *packed_capacity,
+                              uint8_t *const *d_bits, float *const *d_min, float *const *d_scale,
+                              uint64_t *const *d_window_offsets, void *d_workspace,
+                              uint64_t workspace_bytes, daf_stream stream);
+daf_status daf_decompress_batch(uint32_t n, const daf_params *params, const void *const *d_packed,
+                                const uint8_t *const *d_bits, const float *const *d_min,
+                                const float *const *d_scale,
+                                const uint64_t *const *d_window_offsets, void *const *d_out,
+                                daf_stream stream);
+
+/*
+ * Host-side page pool for packed buffers (Sec. 3.4.2: one preallocated contiguous arena,
+ * page-granular first-fit allocation; Sec. 3.4.3: every allocation carries an importance,
+ * and the least important one is evicted first).  The pool does bookkeeping only: it never
+ * touches the arena's memory, which the caller allocates (device or host) and describes by
+ * its size.  Not thread safe.  Handles are positive; 0 means "no allocation".
+ */
+typedef struct daf_pool daf_pool;
+typedef struct daf_pool_stats {
+    uint64_t arena_bytes, page_bytes, pages_total, pages_used, live_allocations,
+             bytes_requested, largest_free_run_pages, evictions;
+} daf_pool_stats;
+daf_pool  *daf_pool_create(uint64_t arena_bytes, uint64_t page_bytes /* 0 => 65536 */);
+void       daf_pool_destroy(daf_pool *pool);
+/* Returns a handle and the byte offset of the run inside the arena, or 0 if no run fits. */
+uint64_t   daf_pool_alloc(daf_pool *pool, uint64_t bytes, double importance, uint64_t *offset);
+daf_status daf_pool_free(daf_pool *pool, uint64_t handle);
+/* Frees the live allocation with the lowest importance per byte; returns its handle (0 if none). */
+uint64_t   daf_pool_evict_lowest(daf_pool *pool);
+daf_status daf_pool_get_stats(const daf_pool *pool, daf_pool_stats *stats);
+
+const char *daf_status_string(daf_status status);
+uint32_t    daf_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DAF_H */

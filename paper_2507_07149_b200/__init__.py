@@ -1,0 +1,294 @@
+"""B200-native activation compress / decompress (the DAF hot path): thin Python binding.
+
+Every function here only marshals arguments for the C ABI declared in ``include/daf.h``
+(``libdaf.so``, hand-written sm_100a kernels).  PyTorch supplies device memory and streams;
+all arithmetic of the path runs in the CUDA library.  There is no CPU fallback: if the
+library is missing or fails to load, the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdaf.so")
+
+OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_BUDGET, ERR_CAPACITY, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED = range(8)
+F32, F16, BF16 = 0, 1, 2
+ROUND_STOCHASTIC, ROUND_NEAREST = 0, 1
+BATCH_MAX = 64
+DEFAULT_WINDOW = 16384
+
+
+class daf_params(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("dtype", ctypes.c_uint32), ("numel", ctypes.c_uint64),
+                ("group_size", ctypes.c_uint32), ("window_elems", ctypes.c_uint32), ("width_mask", ctypes.c_uint32),
+                ("bit_budget", ctypes.c_float), ("rounding", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
+                ("seed", ctypes.c_uint64), ("elem_index_base", ctypes.c_uint64)]
+
+
+class daf_pool_stats(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_uint64) for n in ("arena_bytes", "page_bytes", "pages_total", "pages_used",
+                                               "live_allocations", "bytes_requested", "largest_free_run_pages",
+                                               "evictions")]
+
+
+class DafError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().daf_status_string(status).decode() if _lib is not None else str(status)
+        super().__init__(f"{where}: {msg} (status {status})")
+
+
+_lib = None
+_u64p = ctypes.POINTER(ctypes.c_uint64)
+_vp = ctypes.c_void_p
+
+# name -> (restype, argtypes): every symbol include/daf.h declares
+SIGNATURES = {
+    "daf_sizes": (ctypes.c_int, [ctypes.POINTER(daf_params), _u64p, _u64p, _u64p, _u64p]),
+    "daf_compress": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, ctypes.c_uint64, _vp, _vp, _vp, _vp, _vp,
+                                    ctypes.c_uint64, _vp]),
+    "daf_decompress": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_uint64, _vp]),
+    "daf_group_offsets": (ctypes.c_int, [_vp, ctypes.c_uint64, ctypes.c_uint32, _vp, _vp, ctypes.c_uint64, _vp]),
+    "daf_group_offsets_workspace": (ctypes.c_uint64, [ctypes.c_uint64]),
+    "daf_poll_status": (ctypes.c_int, [_vp, _vp]),
+    "daf_batch_workspace": (ctypes.c_uint64, [ctypes.c_uint32, ctypes.POINTER(daf_params)]),
+    "daf_compress_batch": (ctypes.c_int, [ctypes.c_uint32, ctypes.POINTER(daf_params), _vp, _vp, _u64p, _vp, _vp, _vp, _vp,
+                                          _vp, ctypes.c_uint64, _vp]),
+    "daf_decompress_batch": (ctypes.c_int, [ctypes.c_uint32, ctypes.POINTER(daf_params), _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "daf_pool_create": (_vp, [ctypes.c_uint64, ctypes.c_uint64]),
+    "daf_pool_destroy": (None, [_vp]),
+    "daf_pool_alloc": (ctypes.c_uint64, [_vp, ctypes.c_uint64, ctypes.c_double, _u64p]),
+    "daf_pool_free": (ctypes.c_int, [_vp, ctypes.c_uint64]),
+    "daf_pool_evict_lowest": (ctypes.c_uint64, [_vp]),
+    "daf_pool_get_stats": (ctypes.c_int, [_vp, ctypes.POINTER(daf_pool_stats)]),
+    "daf_status_string": (ctypes.c_char_p, [ctypes.c_int]),
+    "daf_version": (ctypes.c_uint32, []),
+}
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C-ABI library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2507_07149_b200.build` "
+                               "(nvcc, sm_100a); there is no CPU fallback")
+        handle = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = handle
+    return _lib
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise DafError(status, where)
+
+
+# ------------------------------------------------------------------------------------ params / sizes
+def width_mask(widths) -> int:
+    m = 0
+    for b in widths:
+        m |= 1 << int(b)
+    return m
+
+
+def make_params(dtype: int, numel: int, group_size: int, widths, bit_budget: float, *, window_elems: int = 0,
+                rounding: int = ROUND_STOCHASTIC, seed: int = 0, elem_index_base: int = 0) -> daf_params:
+    return daf_params(ctypes.sizeof(daf_params), dtype, numel, group_size, window_elems, width_mask(widths),
+                      bit_budget, rounding, 0, seed, elem_index_base)
+
+
+@dataclass
+class Sizes:
+    n_groups: int
+    n_windows: int
+    packed_capacity: int
+    workspace: int
+
+
+def daf_sizes(params: daf_params) -> Sizes:
+    v = [ctypes.c_uint64() for _ in range(4)]
+    _check(lib().daf_sizes(ctypes.byref(params), *[ctypes.byref(x) for x in v]), "daf_sizes")
+    return Sizes(*[int(x.value) for x in v])
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def dtype_code(t) -> int:
+    torch = _torch()
+    return {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}[t.dtype]
+
+
+def _stream(stream=None) -> int:
+    torch = _torch()
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(s.cuda_stream)
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else int(t.data_ptr())
+
+
+# ------------------------------------------------------------------------------------ raw entry points
+def daf_compress(params, d_in, d_packed, packed_capacity, d_bits, d_min, d_scale, d_window_offsets, d_workspace,
+                 workspace_bytes, stream=None):
+    """Tensors (or None) in, status checked; everything else is the C call."""
+    _check(lib().daf_compress(ctypes.byref(params), _ptr(d_in), _ptr(d_packed), packed_capacity, _ptr(d_bits), _ptr(d_min),
+                              _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_workspace), workspace_bytes, _stream(stream)),
+           "daf_compress")
+
+
+def daf_decompress(params, d_packed, d_bits, d_min, d_scale, d_window_offsets, d_out, d_workspace=None,
+                   workspace_bytes=0, stream=None):
+    _check(lib().daf_decompress(ctypes.byref(params), _ptr(d_packed), _ptr(d_bits), _ptr(d_min), _ptr(d_scale),
+                                _ptr(d_window_offsets), _ptr(d_out), _ptr(d_workspace), workspace_bytes, _stream(stream)),
+           "daf_decompress")
+
+
+def daf_group_offsets_workspace(n_groups: int) -> int:
+    return int(lib().daf_group_offsets_workspace(n_groups))
+
+
+def daf_group_offsets(d_bits, n_groups, group_size, d_offsets, d_ws, ws_bytes, stream=None):
+    _check(lib().daf_group_offsets(_ptr(d_bits), n_groups, group_size, _ptr(d_offsets), _ptr(d_ws), ws_bytes,
+                                   _stream(stream)), "daf_group_offsets")
+
+
+def daf_poll_status(d_workspace, stream=None) -> int:
+    return int(lib().daf_poll_status(_ptr(d_workspace), _stream(stream)))
+
+
+def _ptr_array(tensors):
+    return (ctypes.c_void_p * len(tensors))(*[_ptr(t) for t in tensors])
+
+
+def daf_batch_workspace(params_list) -> int:
+    arr = (daf_params * len(params_list))(*params_list)
+    return int(lib().daf_batch_workspace(len(params_list), arr))
+
+
+def daf_compress_batch(params_list, d_in, d_packed, capacities, d_bits, d_min, d_scale, d_window_offsets, d_workspace,
+                       workspace_bytes, stream=None):
+    n = len(params_list)
+    arr = (daf_params * n)(*params_list)
+    caps = (ctypes.c_uint64 * n)(*capacities)
+    _check(lib().daf_compress_batch(n, arr, _ptr_array(d_in), _ptr_array(d_packed), caps, _ptr_array(d_bits),
+                                    _ptr_array(d_min), _ptr_array(d_scale), _ptr_array(d_window_offsets), _ptr(d_workspace),
+                                    workspace_bytes, _stream(stream)), "daf_compress_batch")
+
+
+def daf_decompress_batch(params_list, d_packed, d_bits, d_min, d_scale, d_window_offsets, d_out, stream=None):
+    n = len(params_list)
+    arr = (daf_params * n)(*params_list)
+    _check(lib().daf_decompress_batch(n, arr, _ptr_array(d_packed), _ptr_array(d_bits), _ptr_array(d_min),
+                                      _ptr_array(d_scale), _ptr_array(d_window_offsets), _ptr_array(d_out), _stream(stream)),
+           "daf_decompress_batch")
+
+
+def daf_version() -> int:
+    return int(lib().daf_version())
+
+
+def daf_status_string(status: int) -> str:
+    return lib().daf_status_string(status).decode()
+
+
+# ------------------------------------------------------------------------------------ conveniences (allocation only)
+@dataclass
+class CompressedTensor:
+    """Device buffers written by daf_compress for one tensor (owned by torch)."""
+    params: daf_params
+    shape: tuple
+    packed: object
+    bits: object
+    min: object
+    scale: object
+    window_offsets: object
+    workspace: object
+    sizes: Sizes
+
+    def packed_bytes(self) -> int:
+        return int(self.window_offsets[-1].item())
+
+
+def alloc_outputs(params: daf_params, device, shape=None) -> CompressedTensor:
+    torch = _torch()
+    sz = daf_sizes(params)
+    return CompressedTensor(
+        params, tuple(shape) if shape is not None else (int(params.numel),),
+        torch.empty(max(sz.packed_capacity, 16), dtype=torch.uint8, device=device),
+        torch.empty(sz.n_groups, dtype=torch.uint8, device=device),
+        torch.empty(sz.n_groups, dtype=torch.float32, device=device),
+        torch.empty(sz.n_groups, dtype=torch.float32, device=device),
+        torch.empty(sz.n_windows + 1, dtype=torch.int64, device=device),
+        torch.empty(sz.workspace, dtype=torch.uint8, device=device), sz)
+
+
+def compress(x, group_size: int, widths, bit_budget: float, *, window_elems: int = 0, rounding: int = ROUND_STOCHASTIC,
+             seed: int = 0, elem_index_base: int = 0, out: CompressedTensor | None = None, check: bool = False,
+             stream=None) -> CompressedTensor:
+    """Allocate outputs with torch (unless given) and call daf_compress on the current stream."""
+    if not x.is_cuda or not x.is_contiguous():
+        raise ValueError("compress expects a contiguous CUDA tensor")
+    params = make_params(dtype_code(x), x.numel(), group_size, widths, bit_budget, window_elems=window_elems,
+                         rounding=rounding, seed=seed, elem_index_base=elem_index_base)
+    c = out if out is not None else alloc_outputs(params, x.device, x.shape)
+    c.params = params
+    daf_compress(params, x, c.packed, c.sizes.packed_capacity, c.bits, c.min, c.scale, c.window_offsets, c.workspace,
+                 c.sizes.workspace, stream)
+    if check:
+        _check(daf_poll_status(c.workspace, stream), "daf_compress (device status)")
+    return c
+
+
+def decompress(c: CompressedTensor, out=None, stream=None):
+    torch = _torch()
+    dt = {F32: torch.float32, F16: torch.float16, BF16: torch.bfloat16}[int(c.params.dtype)]
+    if out is None:
+        out = torch.empty(c.shape, dtype=dt, device=c.packed.device)
+    daf_decompress(c.params, c.packed, c.bits, c.min, c.scale, c.window_offsets, out, None, 0, stream)
+    return out
+
+
+class Pool:
+    """Host-side page pool (bookkeeping only) over a caller-owned arena."""
+
+    def __init__(self, arena_bytes: int, page_bytes: int = 0):
+        self._h = lib().daf_pool_create(arena_bytes, page_bytes)
+        if not self._h:
+            raise DafError(ERR_INVALID_ARG, "daf_pool_create")
+
+    def alloc(self, nbytes: int, importance: float):
+        off = ctypes.c_uint64()
+        h = int(lib().daf_pool_alloc(self._h, nbytes, importance, ctypes.byref(off)))
+        return (h, int(off.value)) if h else (0, None)
+
+    def free(self, handle: int):
+        _check(lib().daf_pool_free(self._h, handle), "daf_pool_free")
+
+    def evict_lowest(self) -> int:
+        return int(lib().daf_pool_evict_lowest(self._h))
+
+    def stats(self) -> dict:
+        s = daf_pool_stats()
+        _check(lib().daf_pool_get_stats(self._h, ctypes.byref(s)), "daf_pool_get_stats")
+        return {n: int(getattr(s, n)) for n, _ in daf_pool_stats._fields_}
+
+    def close(self):
+        if self._h:
+            lib().daf_pool_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,236 @@
+// Decompress kernel: unpack + dequantize (Sec. 2.3 of the paper: stored activations return to
+// their original precision before the gradient computation).  One CTA per window; no CTA
+// depends on another because compress stored every window's byte offset.
+//
+//   bits of the window's groups -> intra-window exclusive scan of the group byte lengths
+//   -> each lane reads the b bytes holding its 8 consecutive codes, widens them with the
+//      power-of-two offset of Eq. 5 (bits | 0x4B000000 is the float 2^23 + code),
+//      x_hat = fma(code, scale, min), rounds to the output type and stores 32 (or 16) bytes.
+#include "common.cuh"
+
+namespace daf {
+
+struct DecTensor {
+    const uint8_t *packed;
+    const uint8_t *bits;
+    const float *mn;
+    const float *scale;
+    const uint64_t *woff;
+    void *out;
+    uint64_t numel;
+    uint32_t first_window;
+    uint32_t n_windows;
+};
+
+template <int NT> struct DecompressArgs {
+    uint32_t total_windows, n_tensors, G, log2G;
+    DecTensor t[NT];
+};
+
+struct DecRec {
+    float mn, scale;
+    uint32_t b, off;
+};
+
+template <int B> __device__ __forceinline__ void decode8(uint32_t w0, uint32_t w1, float mn, float scale, float (&y)[8])
+{
+    constexpr uint32_t L = (1u << B) - 1u;
+#pragma unroll
+    for (int i = 0; i < 8; i++) {
+        uint32_t f;
+        if (B == 8) {
+            // byte i of the pair of words into the low byte of 0x4B0000xx in one permute
+            f = __byte_perm(i < 4 ? w0 : w1, 0x4B000000u, 0x7540u | (uint32_t)(i & 3));
+        } else {
+            f = ((w0 >> (B * i)) & L) | 0x4B000000u;
+        }
+        const float q = __fsub_rn(__uint_as_float(f), 8388608.0f);   // exact: f is the float 2^23 + code
+        y[i] = __fmaf_rn(q, scale, mn);
+    }
+}
+
+template <typename T, int CHUNKS, bool BATCH>
+__global__ void __launch_bounds__(kThreads)
+decompress_kernel(const __grid_constant__ DecompressArgs<BATCH ? DAF_BATCH_MAX : 1> a)
+{
+    constexpr uint32_t WE = kThreads * kLaneElems * CHUNKS;
+    __shared__ __align__(16) DecRec s_grp[kMaxGroups];
+    __shared__ uint32_t s_wtot[kWarps];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t G = a.G, log2G = a.log2G;
+    const uint32_t gw = blockIdx.x;
+
+    uint32_t ti = 0;
+    if (BATCH) {
+        uint32_t lo = 0, hi = a.n_tensors - 1;
+        while (lo < hi) {
+            uint32_t mid = (lo + hi + 1) >> 1;
+            if (a.t[mid].first_window <= gw) lo = mid; else hi = mid - 1;
+        }
+        ti = lo;
+    }
+    const DecTensor &td = a.t[ti];
+    const uint32_t w = gw - td.first_window;
+    const uint64_t wbase = (uint64_t)w * WE;
+    const uint64_t left = td.numel - wbase;
+    const uint32_t n_elems = left < WE ? (uint32_t)left : WE;
+    const uint32_t n = n_elems >> log2G;
+    const uint64_t g0 = wbase >> log2G;
+
+    // group records: width, min, scale and the group's byte offset inside the window
+    uint32_t b = 0, size = 0;
+    float mn = 0.0f, scale = 0.0f;
+    if ((uint32_t)tid < n) {
+        b = td.bits[g0 + tid];
+        mn = td.mn[g0 + tid];
+        scale = td.scale[g0 + tid];
+        size = (G >> 3) * b;
+    }
+    uint32_t incl = size;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        uint32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+        if (lane >= off) incl += y;
+    }
+    if (lane == 31) s_wtot[warp] = incl;
+    __syncthreads();
+    uint32_t before = 0;
+#pragma unroll
+    for (int i = 0; i < kWarps; i++)
+        if (i < warp) before += s_wtot[i];
+    if ((uint32_t)tid < n) {
+        DecRec rec;
+        rec.mn = mn;
+        rec.scale = scale;
+        rec.b = b;
+        rec.off = before + incl - size;
+        s_grp[tid] = rec;
+    }
+    __syncthreads();
+
+    const uint8_t *src = td.packed + td.woff[w];
+    char *out = reinterpret_cast<char *>(td.out) + wbase * Elem<T>::kBytes;
+#pragma unroll
+    for (int c = 0; c < CHUNKS; c++) {
+        const uint32_t e = (uint32_t)((warp * CHUNKS + c) * 256 + lane * 8);
+        if (e >= n_elems) continue;
+        const DecRec rec = s_grp[e >> log2G];
+        const uint8_t *p = src + rec.off + ((e & (G - 1u)) >> 3) * rec.b;
+        float y[8];
+        switch (rec.b) {
+        case 1: decode8<1>(*p, 0u, rec.mn, rec.scale, y); break;
+        case 2: decode8<2>(*reinterpret_cast<const uint16_t *>(p), 0u, rec.mn, rec.scale, y); break;
+        case 4: decode8<4>(*reinterpret_cast<const uint32_t *>(p), 0u, rec.mn, rec.scale, y); break;
+        default: {
+            uint32_t w0, w1;
+            if (G >= 64u) {
+                const uint2 v = *reinterpret_cast<const uint2 *>(p);
+                w0 = v.x;
+                w1 = v.y;
+            } else {                                              // G = 32: groups are only 4-byte aligned
+                w0 = reinterpret_cast<const uint32_t *>(p)[0];
+                w1 = reinterpret_cast<const uint32_t *>(p)[1];
+            }
+            decode8<8>(w0, w1, rec.mn, rec.scale, y);
+            break;
+        }
+        }
+        Elem<T>::store8(out + (size_t)e * Elem<T>::kBytes, y);
+    }
+}
+
+template <typename T, int CHUNKS, bool BATCH>
+static cudaError_t launch(const DecompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
+{
+    decompress_kernel<T, CHUNKS, BATCH><<<args.total_windows, kThreads, 0, stream>>>(args);
+    return cudaGetLastError();
+}
+
+template <bool BATCH>
+static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, const DecompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
+                            cudaStream_t stream)
+{
+#define DAF_CASE(T)                                                     \
+    switch (chunks) {                                                   \
+    case 1: return launch<T, 1, BATCH>(args, stream);                   \
+    case 2: return launch<T, 2, BATCH>(args, stream);                   \
+    default: return launch<T, 4, BATCH>(args, stream);                  \
+    }
+    if (dtype == DAF_F32) { DAF_CASE(float) }
+    if (dtype == DAF_F16) { DAF_CASE(__half) }
+    DAF_CASE(__nv_bfloat16)
+#undef DAF_CASE
+}
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static daf_status check_ptrs(const void *packed, const uint8_t *bits, const float *mn, const float *scale,
+                             const uint64_t *woff, const void *out)
+{
+    if (!packed || !bits || !mn || !scale || !woff || !out) return DAF_ERR_INVALID_ARG;
+    if (!aligned16(packed) || !aligned16(out) || (reinterpret_cast<uintptr_t>(mn) & 3u) ||
+        (reinterpret_cast<uintptr_t>(scale) & 3u) || (reinterpret_cast<uintptr_t>(woff) & 7u))
+        return DAF_ERR_INVALID_ARG;
+    return DAF_OK;
+}
+
+}  // namespace daf
+
+using namespace daf;
+
+extern "C" daf_status daf_decompress(const daf_params *params, const void *d_packed, const uint8_t *d_bits,
+                                     const float *d_min, const float *d_scale, const uint64_t *d_window_offsets,
+                                     void *d_out, void *d_workspace, uint64_t workspace_bytes, daf_stream stream)
+{
+    (void)d_workspace;
+    (void)workspace_bytes;
+    Plan pl;
+    daf_status st = make_plan(params, &pl);
+    if (st != DAF_OK) return st;
+    st = check_ptrs(d_packed, d_bits, d_min, d_scale, d_window_offsets, d_out);
+    if (st != DAF_OK) return st;
+    if (pl.n_windows > 0x7FFFFFFFull) return DAF_ERR_UNSUPPORTED;
+    DecompressArgs<1> a;
+    a.total_windows = (uint32_t)pl.n_windows;
+    a.n_tensors = 1;
+    a.G = pl.G;
+    a.log2G = pl.log2G;
+    a.t[0] = DecTensor{reinterpret_cast<const uint8_t *>(d_packed), d_bits, d_min, d_scale, d_window_offsets, d_out,
+                       params->numel, 0u, (uint32_t)pl.n_windows};
+    return dispatch<false>(params->dtype, pl.chunks, a, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? DAF_OK
+                                                                                                                 : DAF_ERR_CUDA;
+}
+
+extern "C" daf_status daf_decompress_batch(uint32_t n, const daf_params *params, const void *const *d_packed,
+                                           const uint8_t *const *d_bits, const float *const *d_min,
+                                           const float *const *d_scale, const uint64_t *const *d_window_offsets,
+                                           void *const *d_out, daf_stream stream)
+{
+    if (n == 0 || n > DAF_BATCH_MAX || !params || !d_packed || !d_bits || !d_min || !d_scale || !d_window_offsets || !d_out)
+        return DAF_ERR_INVALID_ARG;
+    Plan pl0;
+    daf_status st = make_plan(&params[0], &pl0);
+    if (st != DAF_OK) return st;
+    DecompressArgs<DAF_BATCH_MAX> a;
+    a.n_tensors = n;
+    a.G = pl0.G;
+    a.log2G = pl0.log2G;
+    uint64_t windows = 0;
+    for (uint32_t i = 0; i < n; i++) {
+        Plan pl;
+        st = make_plan(&params[i], &pl);
+        if (st != DAF_OK) return st;
+        if (params[i].dtype != params[0].dtype || pl.G != pl0.G || pl.We != pl0.We) return DAF_ERR_INVALID_ARG;
+        st = check_ptrs(d_packed[i], d_bits[i], d_min[i], d_scale[i], d_window_offsets[i], d_out[i]);
+        if (st != DAF_OK) return st;
+        if (windows + pl.n_windows > 0x7FFFFFFFull) return DAF_ERR_UNSUPPORTED;
+        a.t[i] = DecTensor{reinterpret_cast<const uint8_t *>(d_packed[i]), d_bits[i], d_min[i], d_scale[i],
+                           d_window_offsets[i], d_out[i], params[i].numel, (uint32_t)windows, (uint32_t)pl.n_windows};
+        windows += pl.n_windows;
+    }
+    a.total_windows = (uint32_t)windows;
+    return dispatch<true>(params[0].dtype, pl0.chunks, a, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? DAF_OK
+               : DAF_ERR_CUDA;
+}

@@ -1,0 +1,283 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs -- group min / scale, widths, offsets, codes and packed bytes bit-exact;
+dequantized values 0 ulp (fp16 / bf16) and within 1 ulp (fp32)."""
+import numpy as np
+import pytest
+
+import oracle
+import paper_2507_07149_b200 as daf
+from paper_2507_07149_b200 import workloads as wl
+
+from gpu_util import (assert_compress_parity, assert_decompress_parity, gpu_compress, to_device, to_host)
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+
+def _gen(cfg, ti, spec):
+    return wl.generate(cfg, ti, spec)
+
+
+# ------------------------------------------------------------------ the five workloads (small enough for the oracle)
+def test_cfg1_full():
+    w = wl.workload(1)
+    a = _gen(1, 0, w.tensors[0])
+    x, c, ref = assert_compress_parity(a, "f32", w.group_size, w.widths, w.bit_budget, seed=0, label="cfg1")
+    assert set(np.unique(ref.bits)) == {4}                    # ranges differ by far less than the 4 -> 8 threshold
+    assert_decompress_parity(c, ref, "f32", "cfg1")
+
+
+@pytest.mark.parametrize("ti", [3, 20, 56])                   # relu 64x56x56 block, a 28x28 conv, the last 7x7 relu
+def test_cfg2_tensors_at_batch_4(ti):
+    w = wl.workload(2, batch=4)
+    spec = w.tensors[ti]
+    a = _gen(2, ti, spec)
+    x, c, ref = assert_compress_parity(a, "f32", w.group_size, w.widths, w.bit_budget, seed=spec.philox_seed,
+                                       label=f"cfg2/{spec.name}")
+    assert sorted(np.unique(ref.bits)) == [2, 4]              # half the groups at 2 bits, half at 4
+    assert_decompress_parity(c, ref, "f32", f"cfg2/{spec.name}")
+
+
+@pytest.mark.parametrize("ti", [1, 12, 31])                   # includes 960x7x7 (ragged last window)
+def test_cfg3_tensors_at_batch_4(ti):
+    w = wl.workload(3, batch=4)
+    spec = w.tensors[ti]
+    a = _gen(3, ti, spec)
+    x, c, ref = assert_compress_parity(a, "f16", w.group_size, w.widths, w.bit_budget, seed=spec.philox_seed,
+                                       label=f"cfg3/{spec.name}")
+    assert_decompress_parity(c, ref, "f16", f"cfg3/{spec.name}")
+
+
+@pytest.mark.parametrize("ti", [0, 1])
+def test_cfg4_tensors_at_batch_2(ti):
+    w = wl.workload(4, batch=2, layers=1)
+    spec = w.tensors[ti]
+    a = _gen(4, ti, spec)
+    x, c, ref = assert_compress_parity(a, "bf16", w.group_size, w.widths, w.bit_budget, seed=spec.philox_seed,
+                                       label=f"cfg4/{spec.name}")
+    assert len(np.unique(ref.bits)) == 3                      # outlier groups force all three widths
+    assert_decompress_parity(c, ref, "bf16", f"cfg4/{spec.name}")
+
+
+@pytest.mark.parametrize("G", wl.SWEEP_GROUPS)
+@pytest.mark.parametrize("beta", wl.SWEEP_BUDGETS)
+def test_cfg5_sweep_point_on_a_slice(G, beta):
+    w = wl.workload(5, numel=1 << 21, group_size=G, bit_budget=beta)
+    a = _gen(5, 0, w.tensors[0])
+    x, c, ref = assert_compress_parity(a, "f32", G, w.widths, beta, label=f"cfg5/G{G}/b{beta}")
+    assert_decompress_parity(c, ref, "f32", f"cfg5/G{G}/b{beta}")
+
+
+# ------------------------------------------------------------------ stress inputs
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+@pytest.mark.parametrize("G", [32, 64, 128, 256, 512, 1024, 4096, 16384])
+def test_mixed_widths_in_one_window(dtype, G):
+    """Per-group scales spread over four decades: every width appears inside single windows."""
+    rng = np.random.default_rng(G)
+    n = 16384 * 3 + G * (3 if G < 16384 else 0)               # ragged last window unless G is the window
+    scale = 10.0 ** rng.uniform(-2, 2, n // G)
+    a32 = (rng.standard_normal(n) * np.repeat(scale, G)).astype(np.float32)
+    a = a32 if dtype == "f32" else (a32.astype(np.float16) if dtype == "f16" else wl.f32_to_bf16_bits(a32))
+    for widths, beta in (((1, 2, 4, 8), 3.0), ((1, 2, 4, 8), 2.5), ((2, 4, 8), 4.0)):
+        x, c, ref = assert_compress_parity(a, dtype, G, widths, beta, seed=G + 1, label=f"mixed/{dtype}/G{G}/{widths}/{beta}")
+        if G <= 4096:
+            assert len(np.unique(ref.bits)) >= 2
+        assert_decompress_parity(c, ref, dtype, f"mixed/{dtype}/G{G}")
+
+
+@pytest.mark.parametrize("widths", [(1,), (2,), (4,), (8,), (1, 2), (1, 4), (1, 8), (2, 4), (2, 8), (4, 8), (1, 2, 4), (1, 2, 8),
+                                    (1, 4, 8), (2, 4, 8), (1, 2, 4, 8)])
+def test_every_width_subset(widths):
+    rng = np.random.default_rng(len(widths) * 100 + sum(widths))
+    G, n = 64, 16384 * 2 + 64 * 5
+    a = (rng.standard_normal(n) * np.repeat(10.0 ** rng.uniform(-1, 1, n // G), G)).astype(np.float32)
+    for beta in (float(min(widths)), min(widths) + 0.8, 3.3, 8.0):
+        if beta < min(widths):
+            continue
+        x, c, ref = assert_compress_parity(a, "f32", G, widths, beta, seed=3, label=f"subset/{widths}/{beta}")
+        assert_decompress_parity(c, ref, "f32", f"subset/{widths}/{beta}")
+
+
+def test_degenerate_groups_zero_constant_and_signed_zero():
+    G = 128
+    vals = np.float32([0.0, -0.0, 1.0, -3.5, 6.0, 1e-30, 3e38, -3e38])
+    a = np.repeat(vals, G).astype(np.float32)
+    a = np.concatenate([a, np.tile(np.float32([0.0, -0.0]), G // 2), np.tile(np.float32([-0.0, 1.0]), G // 2),
+                        np.random.default_rng(0).standard_normal(16384).astype(np.float32)])
+    # subnormal-range group: range below 2^-118 is treated as constant
+    tiny = np.zeros(G, np.float32)
+    tiny[5] = np.float32(2.0 ** -120)
+    a = np.concatenate([a, tiny]).astype(np.float32)
+    x, c, ref = assert_compress_parity(a, "f32", G, (1, 2, 4, 8), 3.0, label="degenerate")
+    assert np.all(ref.scale[:8] == 0)
+    assert ref.mn.view(np.uint32)[8] == 0x80000000            # -0.0 orders below +0.0
+    assert_decompress_parity(c, ref, "f32", "degenerate")
+
+
+def test_heavy_ties_relu6_saturation():
+    """Most groups share the same range (clip at 0 and 6): the tie order by group index decides."""
+    rng = np.random.default_rng(4)
+    G, n = 128, 16384 * 4
+    a = np.clip(rng.standard_normal(n) * 2, 0, 6).astype(np.float16)
+    for beta in (1.5, 2.0, 2.75, 3.0):
+        x, c, ref = assert_compress_parity(a, "f16", G, (1, 2, 4, 8), beta, seed=9, label=f"ties/{beta}")
+        assert_decompress_parity(c, ref, "f16", f"ties/{beta}")
+
+
+@pytest.mark.parametrize("We", [4096, 8192, 16384])
+@pytest.mark.parametrize("rounding", [daf.ROUND_STOCHASTIC, daf.ROUND_NEAREST])
+def test_window_sizes_rounding_modes_and_shards(We, rounding):
+    rng = np.random.default_rng(We + rounding)
+    G, n = 256, We * 7 + 256 * 9
+    a = (rng.laplace(size=n) * np.repeat(10.0 ** rng.uniform(-1, 1, n // G), G)).astype(np.float32)
+    seed = 0xDEADBEEF12345678
+    x, c, ref = assert_compress_parity(a, "f32", G, (1, 2, 4, 8), 3.0, window_elems=We, rounding=rounding, seed=seed,
+                                       label=f"We{We}/r{rounding}")
+    assert_decompress_parity(c, ref, "f32", f"We{We}/r{rounding}")
+    # a window-aligned shard compressed with its element base reproduces the same bytes
+    lo, hi = 2 * We, 5 * We
+    xs, cs, refs = assert_compress_parity(a[lo:hi], "f32", G, (1, 2, 4, 8), 3.0, window_elems=We, rounding=rounding,
+                                          seed=seed, base=lo, label="shard")
+    full = c.packed[: c.packed_bytes()].cpu().numpy()
+    woff = c.window_offsets.cpu().numpy()
+    assert np.array_equal(cs.packed[: cs.packed_bytes()].cpu().numpy(), full[int(woff[2]):int(woff[5])])
+
+
+def test_large_element_index_base_uses_the_high_counter_word():
+    rng = np.random.default_rng(8)
+    a = rng.standard_normal(16384 * 2).astype(np.float32)
+    base = (1 << 35) + 16384 * 3
+    x, c, ref = assert_compress_parity(a, "f32", 256, (2, 4), 3.0, seed=77, base=base, label="bigbase")
+
+
+def test_single_group_and_single_window():
+    rng = np.random.default_rng(2)
+    for n, G in ((32, 32), (256, 256), (16384, 16384), (16384, 64), (4096, 128)):
+        a = rng.standard_normal(n).astype(np.float32)
+        x, c, ref = assert_compress_parity(a, "f32", G, (1, 2, 4, 8), 4.0, label=f"tiny/{n}/{G}")
+        assert_decompress_parity(c, ref, "f32", f"tiny/{n}/{G}")
+
+
+# ------------------------------------------------------------------ decompress fed with oracle buffers
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+def test_decompress_of_oracle_buffers(dtype):
+    rng = np.random.default_rng(12)
+    G, n = 64, 16384 * 2 + 64 * 7
+    a32 = (rng.standard_normal(n) * np.repeat(10.0 ** rng.uniform(-2, 2, n // G), G)).astype(np.float32)
+    a = a32 if dtype == "f32" else (a32.astype(np.float16) if dtype == "f16" else wl.f32_to_bf16_bits(a32))
+    ref = oracle.compress(a, G, (1, 2, 4, 8), 3.0, dtype="bf16" if dtype == "bf16" else None, seed=5)
+    p = daf.make_params({"f32": daf.F32, "f16": daf.F16, "bf16": daf.BF16}[dtype], n, G, (1, 2, 4, 8), 3.0, seed=5)
+    packed = torch.zeros(ref.packed.size + 16, dtype=torch.uint8, device="cuda")
+    packed[: ref.packed.size] = torch.from_numpy(ref.packed).cuda()
+    out = torch.empty(n, dtype={"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}[dtype], device="cuda")
+    daf.daf_decompress(p, packed, torch.from_numpy(ref.bits).cuda(), torch.from_numpy(ref.mn).cuda(),
+                       torch.from_numpy(ref.scale).cuda(), torch.from_numpy(ref.window_offsets.view(np.int64)).cuda(), out)
+    torch.cuda.synchronize()
+    got, want = to_host(out, dtype), oracle.decompress(ref)
+    assert np.array_equal(got.view(np.uint32 if dtype == "f32" else np.uint16),
+                          want.view(np.uint32 if dtype == "f32" else np.uint16))
+
+
+# ------------------------------------------------------------------ standalone scan
+@pytest.mark.parametrize("n_groups", [1, 31, 8192, 8193, 100_003, 3_000_000])
+def test_group_offsets_against_oracle(n_groups):
+    rng = np.random.default_rng(n_groups)
+    bits = rng.choice(np.uint8([1, 2, 4, 8]), n_groups)
+    for G, misalign in ((64, 0), (4096, 0), (256, 3)):
+        buf = torch.zeros(n_groups + 16, dtype=torch.uint8, device="cuda")
+        d_bits = buf[misalign: misalign + n_groups]
+        d_bits.copy_(torch.from_numpy(bits))
+        off = torch.empty(n_groups + 1, dtype=torch.int64, device="cuda")
+        ws_bytes = daf.daf_group_offsets_workspace(n_groups)
+        ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+        daf.daf_group_offsets(d_bits, n_groups, G, off, ws, ws_bytes)
+        assert daf.daf_poll_status(ws) == daf.OK
+        assert np.array_equal(off.cpu().numpy().view(np.uint64), oracle.offsets(bits, G))
+
+
+# ------------------------------------------------------------------ device-detected errors, guard bands
+def test_capacity_error_is_reported_and_nothing_is_written_out_of_bounds():
+    rng = np.random.default_rng(3)
+    n, G = 16384 * 6, 256
+    a = rng.standard_normal(n).astype(np.float32)
+    x = to_device(a, "f32")
+    p = daf.make_params(daf.F32, n, G, (4,), 4.0)
+    c = daf.alloc_outputs(p, x.device)
+    cap = 16384 * 4 // 8 * 3                                   # room for three of the six windows
+    c.packed.fill_(0xA5)
+    daf.daf_compress(p, x, c.packed, cap, c.bits, c.min, c.scale, c.window_offsets, c.workspace, c.sizes.workspace)
+    assert daf.daf_poll_status(c.workspace) == daf.ERR_CAPACITY
+    assert bool((c.packed[cap:] == 0xA5).all())
+    ref = oracle.compress(a, G, (4,), 4.0)
+    assert np.array_equal(c.packed[:cap].cpu().numpy(), ref.packed[:cap])
+    # the same buffers with enough room work again (the workspace is reset by every call)
+    daf.daf_compress(p, x, c.packed, c.sizes.packed_capacity, c.bits, c.min, c.scale, c.window_offsets, c.workspace,
+                     c.sizes.workspace)
+    assert daf.daf_poll_status(c.workspace) == daf.OK
+    assert np.array_equal(c.packed[: ref.packed.size].cpu().numpy(), ref.packed)
+
+
+def test_outputs_have_intact_guard_bands():
+    rng = np.random.default_rng(6)
+    n, G = 16384 * 3 + 128 * 5, 128
+    a = rng.standard_normal(n).astype(np.float16)
+    x = to_device(a, "f16")
+    p = daf.make_params(daf.F16, n, G, (1, 2, 4, 8), 2.5, seed=1)
+    sz = daf.daf_sizes(p)
+    pad = 256
+
+    def guarded(nbytes):
+        t = torch.full((nbytes + 2 * pad,), 0xA5, dtype=torch.uint8, device="cuda")
+        return t, t[pad: pad + nbytes]
+
+    bufs = {k: guarded(nb) for k, nb in (("packed", sz.packed_capacity), ("bits", sz.n_groups), ("mn", 4 * sz.n_groups),
+                                         ("scale", 4 * sz.n_groups), ("woff", 8 * (sz.n_windows + 1)), ("out", 2 * n))}
+    ws = torch.empty(sz.workspace, dtype=torch.uint8, device="cuda")
+    daf.daf_compress(p, x, bufs["packed"][1], sz.packed_capacity, bufs["bits"][1], bufs["mn"][1], bufs["scale"][1],
+                     bufs["woff"][1], ws, sz.workspace)
+    assert daf.daf_poll_status(ws) == daf.OK
+    daf.daf_decompress(p, bufs["packed"][1], bufs["bits"][1], bufs["mn"][1], bufs["scale"][1], bufs["woff"][1],
+                       bufs["out"][1])
+    torch.cuda.synchronize()
+    for name, (full, inner) in bufs.items():
+        assert bool((full[:pad] == 0xA5).all()) and bool((full[pad + inner.numel():] == 0xA5).all()), name
+    ref = oracle.compress(a, G, (1, 2, 4, 8), 2.5, seed=1)
+    assert np.array_equal(bufs["out"][1].cpu().numpy().view(np.uint16), oracle.decompress(ref).view(np.uint16))
+
+
+# ------------------------------------------------------------------ batched calls
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_batched_calls_equal_single_calls(dtype):
+    rng = np.random.default_rng(30)
+    G, widths, beta = 128, (1, 2, 4, 8), 3.0
+    sizes = [16384 * 2 + 128, 128, 16384, 16384 * 5 + 128 * 77, 4096]
+    arrays = []
+    for n in sizes:
+        a32 = (rng.standard_normal(n) * np.repeat(10.0 ** rng.uniform(-1, 1, n // G), G)).astype(np.float32)
+        arrays.append(a32 if dtype == "f32" else wl.f32_to_bf16_bits(a32))
+    xs = [to_device(a, dtype) for a in arrays]
+    code = {"f32": daf.F32, "bf16": daf.BF16}[dtype]
+    params = [daf.make_params(code, a.size, G, widths, beta, seed=100 + i) for i, a in enumerate(arrays)]
+    outs = [daf.alloc_outputs(p, "cuda") for p in params]
+    ws_bytes = daf.daf_batch_workspace(params)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    daf.daf_compress_batch(params, xs, [o.packed for o in outs], [o.sizes.packed_capacity for o in outs],
+                           [o.bits for o in outs], [o.min for o in outs], [o.scale for o in outs],
+                           [o.window_offsets for o in outs], ws, ws_bytes)
+    assert daf.daf_poll_status(ws) == daf.OK
+    ys = [torch.empty_like(x) for x in xs]
+    daf.daf_decompress_batch(params, [o.packed for o in outs], [o.bits for o in outs], [o.min for o in outs],
+                             [o.scale for o in outs], [o.window_offsets for o in outs], ys)
+    torch.cuda.synchronize()
+    for i, a in enumerate(arrays):
+        ref = oracle.compress(a, G, widths, beta, dtype="bf16" if dtype == "bf16" else None, seed=100 + i)
+        o = outs[i]
+        assert np.array_equal(o.bits.cpu().numpy(), ref.bits), i
+        assert np.array_equal(o.window_offsets.cpu().numpy().view(np.uint64), ref.window_offsets), i
+        assert np.array_equal(o.packed[: ref.packed.size].cpu().numpy(), ref.packed), i
+        assert np.array_equal(o.min.cpu().numpy().view(np.uint32), ref.mn.view(np.uint32)), i
+        assert np.array_equal(o.scale.cpu().numpy().view(np.uint32), ref.scale.view(np.uint32)), i
+        want = oracle.decompress(ref)
+        got = to_host(ys[i], dtype)
+        assert np.array_equal(got.view(np.uint32 if dtype == "f32" else np.uint16),
+                              want.view(np.uint32 if dtype == "f32" else np.uint16)), i
