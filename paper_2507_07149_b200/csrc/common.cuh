@@ -79,12 +79,11 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, const Ke
     uint32_t c2 = 0u, c3 = 0u;
 #pragma unroll
     for (int r = 0; r < 10; r++) {
-        uint32_t hi0 = __umulhi(kPhiloxM0, c0), lo0 = kPhiloxM0 * c0;
-        uint32_t hi1 = __umulhi(kPhiloxM1, c2), lo1 = kPhiloxM1 * c2;
-        c0 = hi1 ^ c1 ^ keys.k0[r];
-        c1 = lo1;
-        c2 = hi0 ^ c3 ^ keys.k1[r];
-        c3 = lo0;
+        const uint64_t p0 = (uint64_t)kPhiloxM0 * c0, p1 = (uint64_t)kPhiloxM1 * c2;   // one wide multiply each
+        c0 = (uint32_t)(p1 >> 32) ^ c1 ^ keys.k0[r];
+        c1 = (uint32_t)p1;
+        c2 = (uint32_t)(p0 >> 32) ^ c3 ^ keys.k1[r];
+        c3 = (uint32_t)p0;
     }
     o[0] = c0; o[1] = c1; o[2] = c2; o[3] = c3;
 }
@@ -101,12 +100,11 @@ __device__ __forceinline__ void philox4x32_10<PhiloxSeedKeys>(uint32_t c0, uint3
     uint32_t c2 = 0u, c3 = 0u;
 #pragma unroll
     for (int r = 0; r < 10; r++) {
-        uint32_t hi0 = __umulhi(kPhiloxM0, c0), lo0 = kPhiloxM0 * c0;
-        uint32_t hi1 = __umulhi(kPhiloxM1, c2), lo1 = kPhiloxM1 * c2;
-        c0 = hi1 ^ c1 ^ (s.lo + (uint32_t)r * kPhiloxW0);
-        c1 = lo1;
-        c2 = hi0 ^ c3 ^ (s.hi + (uint32_t)r * kPhiloxW1);
-        c3 = lo0;
+        const uint64_t p0 = (uint64_t)kPhiloxM0 * c0, p1 = (uint64_t)kPhiloxM1 * c2;
+        c0 = (uint32_t)(p1 >> 32) ^ c1 ^ (s.lo + (uint32_t)r * kPhiloxW0);
+        c1 = (uint32_t)p1;
+        c2 = (uint32_t)(p0 >> 32) ^ c3 ^ (s.hi + (uint32_t)r * kPhiloxW1);
+        c3 = (uint32_t)p0;
     }
     o[0] = c0; o[1] = c1; o[2] = c2; o[3] = c3;
 }

@@ -1,18 +1,24 @@
 // Fused compress kernel: one persistent CTA processes one window (window_elems elements) at a
 // time and reads the input from HBM exactly once.
 //
-//   load window into registers (8 consecutive elements per lane and chunk, 256-bit loads)
-//   -> per-group min / max (lane-local 3-input min/max, warp redux or segmented shuffles)
-//   -> per-window greedy bit-width choice (Sec. 3.4.1 of the paper: importance per bit)
-//   -> intra-window exclusive scan of the group byte lengths, device-wide window offset by a
-//      bounded decoupled look-back over 64-bit descriptors
-//   -> Eq. 1 quantization with stochastic rounding (Philox4x32-10, 16 bits per element, float
-//      -> uint through the power-of-two offset of Eq. 5) and lane-local LSB-first packing
-//   -> stores of the packed bytes and of bits / min / scale.
+//   - the next window is staged into shared memory by one bulk asynchronous copy (TMA,
+//     completion on an mbarrier) while the current one is processed;
+//   - staged window -> registers (8 consecutive elements per lane and chunk), per-group
+//     min / max (3-input min/max, warp redux or segmented shuffles);
+//   - per-window greedy bit-width choice (Sec. 3.4.1 of the paper: importance per bit);
+//   - intra-window exclusive scan of the group byte lengths; the window's byte count is
+//     published at once in a 64-bit descriptor;
+//   - Eq. 1 quantization with stochastic rounding (Philox4x32-10, 16 bits per element, the
+//     float -> uint step done with the power-of-two offset of Eq. 5) and lane-local LSB-first
+//     packing into a shared-memory buffer;
+//   - the window's device-wide byte offset comes from a bounded decoupled look-back over the
+//     descriptors, resolved opportunistically after the quantize pass and otherwise one
+//     window later, so that no CTA waits for its neighbours; the packed window then leaves
+//     shared memory as one bulk asynchronous store.
 //
 // Windows are handed out by an atomic ticket, so every window with a smaller index than the
-// one a CTA holds is already owned by a running (or finished) CTA and the look-back always
-// makes progress; it is bounded all the same.
+// one a CTA holds is owned by a running (or finished) CTA and the look-back always makes
+// progress; every wait is bounded all the same.
 #include "common.cuh"
 
 namespace daf {
@@ -32,13 +38,18 @@ struct TensorDesc {
     uint32_t n_windows;
 };
 
+struct SmemLayout {          // byte offsets into dynamic shared memory
+    uint32_t out0, out_stride, umn, umx, key, cum, grp, total;
+};
+
 template <int NT> struct CompressArgs {
     WorkspaceHeader *hdr;
     uint64_t *flags;
     uint32_t total_windows, n_tensors;
-    uint32_t G, log2G, beta_q8, m, nearest;
+    uint32_t G, log2G, beta_q8, m, nearest, bulk_store, n_max;
     uint32_t S[kMaxLevels], cost[kMaxLevels];
     float v[kMaxLevels];
+    SmemLayout lay;
     PhiloxKeys keys;          // round keys of tensor 0 (single-tensor launches)
     TensorDesc t[NT];
 };
@@ -51,8 +62,10 @@ struct GroupRec {             // what the quantize pass needs per group (one 16-
 // ------------------------------------------------------------------------------------------
 // Eight codes of width B from eight values; o[] holds eight 16-bit random lanes (two per word).
 // s = fma(x - mn, inv, 256) lies in [256, 512) where one ulp is 2^-15, so its mantissa field
-// is the fixed-point quotient; adding a 15-bit random offset and dropping 15 bits rounds
-// stochastically (offset 2^14 = round half up).
+// is the fixed-point quotient; adding a 15-bit random offset r15 and dropping 15 bits rounds
+// stochastically (r15 = 2^14: round half up).  With h = 2*r15 + (one more random bit),
+// (fixed + r15) >> 15 == (2*bits(s) + h - 2*bits(256)) >> 16, which needs one add, one shift
+// and one fused subtract-and-clamp per element.
 // ------------------------------------------------------------------------------------------
 template <int B>
 __device__ __forceinline__ void quantize8(const float (&x)[8], float mn, float inv, const uint32_t (&o)[4],
@@ -63,11 +76,11 @@ __device__ __forceinline__ void quantize8(const float (&x)[8], float mn, float i
     w1 = 0u;
 #pragma unroll
     for (int i = 0; i < 8; i++) {
-        float d = __fsub_rn(x[i], mn);
-        float s = __fmaf_rn(d, inv, 256.0f);
-        uint32_t r15 = (i & 1) ? (o[i >> 1] >> 17) : ((o[i >> 1] >> 1) & 0x7FFFu);
-        uint32_t t = __float_as_uint(s) - 0x43800000u + r15;
-        uint32_t q = min(t >> 15, L);
+        const float d = __fsub_rn(x[i], mn);
+        const float s = __fmaf_rn(d, inv, 256.0f);
+        const uint32_t h = (i & 1) ? (o[i >> 1] >> 16) : (o[i >> 1] & 0xFFFFu);
+        const uint32_t u = (__float_as_uint(s) << 1) + h;         // mod 2^32; 2*bits(256) = 0x87000000
+        const uint32_t q = min((u >> 16) - 0x8700u, L);
         if (B == 8) {
             if (i < 4) w0 |= q << (8 * i);
             else w1 |= q << (8 * (i - 4));
@@ -78,54 +91,198 @@ __device__ __forceinline__ void quantize8(const float (&x)[8], float mn, float i
 }
 
 // ------------------------------------------------------------------------------------------
-// Decoupled look-back over the window descriptors, executed by one full warp.  Returns the
-// exclusive prefix (bytes before this window); *failed is set when a predecessor is poisoned
-// or the bounded wait runs out.
+// Decoupled look-back over the window descriptors, executed by one full warp.  Each round
+// inspects DEPTH * 32 predecessors with all loads in flight at once.  Returns 1 when the
+// exclusive prefix was found (*excl), 0 when a needed descriptor is still empty and `block`
+// is false, -1 on a poisoned predecessor, -2 when the bounded wait ran out.
 // ------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint64_t lookback(uint64_t *flags, uint32_t gw, uint32_t first, uint64_t total,
-                                             int lane, int *failed, int *timed_out)
+constexpr int kLookDepth = 10;
+
+template <int DEPTH>
+__device__ __forceinline__ int lookback(const uint64_t *flags, uint32_t gw, uint32_t first, int lane, bool block,
+                                        uint64_t *excl_out)
 {
     uint64_t excl = 0;
-    int bad = 0, tmo = 0;
-    if (gw == first) {
-        if (lane == 0) st_relaxed_u64(flags + gw, (kFlagPrefix << kFlagShift) | total);
-        *failed = 0;
-        *timed_out = 0;
-        return 0;
-    }
-    if (lane == 0) st_relaxed_u64(flags + gw, (kFlagAggregate << kFlagShift) | total);
-    int64_t idx = (int64_t)gw - 1 - lane;
+    int64_t idx = (int64_t)gw - 1 - lane;                         // lane's nearest predecessor of this round
+    unsigned polls = 0;
     for (;;) {
-        uint64_t f = 0;
-        unsigned polls = 0;
-        unsigned ready_mask, stop_mask;
+        uint64_t f[DEPTH];
+        bool done = false;                                        // a prefix (or poison) ends the walk in this round
         for (;;) {
-            f = (idx >= (int64_t)first) ? ld_relaxed_u64(flags + idx) : (kFlagPrefix << kFlagShift);
-            uint32_t st = (uint32_t)(f >> kFlagShift);
-            stop_mask = __ballot_sync(0xFFFFFFFFu, st == kFlagPrefix || st == kFlagPoison);
-            unsigned empty_mask = __ballot_sync(0xFFFFFFFFu, st == kFlagEmpty);
-            // only descriptors up to and including the first prefix / poison matter
-            unsigned upto = stop_mask ? ((2u << (__ffs(stop_mask) - 1)) - 1u) : 0xFFFFFFFFu;
-            ready_mask = upto;
-            if ((empty_mask & upto) == 0u) break;
-            if (++polls > kMaxPolls) { tmo = 1; break; }
+#pragma unroll
+            for (int j = 0; j < DEPTH; j++) {
+                const int64_t i = idx - 32 * j;
+                f[j] = (i >= (int64_t)first) ? ld_relaxed_u64(flags + i) : (kFlagPrefix << kFlagShift);
+            }
+            bool ready = true;                                    // walk the chunks from the nearest predecessor outward
+            done = false;
+#pragma unroll
+            for (int j = 0; j < DEPTH; j++) {
+                if (!done && ready) {
+                    const uint32_t st = (uint32_t)(f[j] >> kFlagShift);
+                    const unsigned stop_mask = __ballot_sync(0xFFFFFFFFu, st == kFlagPrefix || st == kFlagPoison);
+                    const unsigned empty_mask = __ballot_sync(0xFFFFFFFFu, st == kFlagEmpty);
+                    const unsigned upto = stop_mask ? ((2u << (__ffs(stop_mask) - 1)) - 1u) : 0xFFFFFFFFu;
+                    if (empty_mask & upto) ready = false;
+                    else if (stop_mask) done = true;
+                }
+            }
+            if (ready) break;
+            if (!block) return 0;
+            if (++polls > kMaxPolls) return -2;
             __nanosleep(64);
         }
-        if (tmo) { bad = 1; break; }
-        uint32_t st = (uint32_t)(f >> kFlagShift);
-        if (__ballot_sync(0xFFFFFFFFu, st == kFlagPoison) & ready_mask) { bad = 1; break; }
-        uint64_t v = ((ready_mask >> lane) & 1u) ? (f & kFlagValueMask) : 0ull;
+        // accumulate up to and including the first prefix; a poisoned predecessor fails the window
+        uint64_t v = 0;
+        bool stop = false, bad = false;
+#pragma unroll
+        for (int j = 0; j < DEPTH; j++) {
+            if (!stop) {
+                const uint32_t st = (uint32_t)(f[j] >> kFlagShift);
+                const unsigned stop_mask = __ballot_sync(0xFFFFFFFFu, st == kFlagPrefix || st == kFlagPoison);
+                const unsigned upto = stop_mask ? ((2u << (__ffs(stop_mask) - 1)) - 1u) : 0xFFFFFFFFu;
+                if (__ballot_sync(0xFFFFFFFFu, st == kFlagPoison) & upto) bad = true;
+                if ((upto >> lane) & 1u) v += f[j] & kFlagValueMask;
+                if (stop_mask) stop = true;
+            }
+        }
+        if (bad) return -1;
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
         excl += v;
-        if (stop_mask) break;
-        idx -= 32;
+        if (done) break;
+        idx -= 32 * DEPTH;
     }
-    if (lane == 0)
-        st_relaxed_u64(flags + gw, bad ? (kFlagPoison << kFlagShift) : ((kFlagPrefix << kFlagShift) | (excl + total)));
-    *failed = bad;
-    *timed_out = tmo;
-    return excl;
+    *excl_out = excl;
+    return 1;
+}
+
+// ------------------------------------------------------------------------------------------
+// Bulk asynchronous copies (TMA, non-tensor form) and the mbarrier that signals a landed
+// window.  All waits are bounded.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_load(void *dst_smem, const void *src, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_addr(dst_smem)),
+                 "l"(src), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_store(void *dst, const void *src_smem, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_addr(src_smem)), "r"(bytes)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// Orders this thread's earlier writes to shared memory before later reads by the async proxy.
+__device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok)
+                 : "r"(smem_addr(bar)), "r"(parity)
+                 : "memory");
+    return ok != 0;
+}
+// Returns false if the copy did not land within the poll budget (try_wait itself blocks for a
+// hardware-defined interval, so the loop turns slowly).
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity)
+{
+    for (unsigned polls = 0; polls < kMaxPolls; polls++)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+
+// Eight consecutive elements of a lane from the staged window.  For 4-byte elements a lane
+// owns 32 bytes; the two 16-byte halves are read in an order that depends on the lane so
+// that each quarter-warp touches all 32 banks, then swapped back into element order.
+template <typename T> __device__ __forceinline__ void load8_staged(const unsigned char *chunk, int lane, float (&x)[8]);
+
+template <> __device__ __forceinline__ void load8_staged<float>(const unsigned char *chunk, int lane, float (&x)[8])
+{
+    const bool odd = (lane >> 2) & 1;
+    const unsigned char *p = chunk + lane * 32;
+    const float4 a = *reinterpret_cast<const float4 *>(p + (odd ? 16 : 0));
+    const float4 b = *reinterpret_cast<const float4 *>(p + (odd ? 0 : 16));
+    x[0] = odd ? b.x : a.x; x[1] = odd ? b.y : a.y; x[2] = odd ? b.z : a.z; x[3] = odd ? b.w : a.w;
+    x[4] = odd ? a.x : b.x; x[5] = odd ? a.y : b.y; x[6] = odd ? a.z : b.z; x[7] = odd ? a.w : b.w;
+}
+template <> __device__ __forceinline__ void load8_staged<__half>(const unsigned char *chunk, int lane, float (&x)[8])
+{
+    const uint4 v = *reinterpret_cast<const uint4 *>(chunk + lane * 16);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
+        x[2 * i] = f.x;
+        x[2 * i + 1] = f.y;
+    }
+}
+template <> __device__ __forceinline__ void load8_staged<__nv_bfloat16>(const unsigned char *chunk, int lane, float (&x)[8])
+{
+    const uint4 v = *reinterpret_cast<const uint4 *>(chunk + lane * 16);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+        x[2 * i] = __uint_as_float(w[i] << 16);
+        x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+}
+
+// Staged window -> registers, then min / max per unit of LPU lanes (a full warp uses the
+// redux instruction) written to shared memory.  Chunks past a ragged window's end read
+// stale bytes; their results are never used.
+template <typename T, int CHUNKS, int LPU>
+__device__ __forceinline__ void load_and_reduce(const unsigned char *stage, int warp, int lane, float (&x)[CHUNKS][8],
+                                                float *s_umn, float *s_umx)
+{
+    constexpr int kChunkBytes = 256 * Elem<T>::kBytes;
+#pragma unroll
+    for (int c = 0; c < CHUNKS; c++) load8_staged<T>(stage + (warp * CHUNKS + c) * kChunkBytes, lane, x[c]);
+#pragma unroll
+    for (int c = 0; c < CHUNKS; c++) {
+        float lo = fmin3(fmin3(x[c][0], x[c][1], x[c][2]), fmin3(x[c][3], x[c][4], x[c][5]), fmin2(x[c][6], x[c][7]));
+        float hi = fmax3(fmax3(x[c][0], x[c][1], x[c][2]), fmax3(x[c][3], x[c][4], x[c][5]), fmax2(x[c][6], x[c][7]));
+        if (LPU == 32) {
+            asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(lo) : "f"(lo));
+            asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(hi) : "f"(hi));
+        } else {
+#pragma unroll
+            for (int off = 1; off < LPU; off <<= 1) {
+                lo = fmin2(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, off));
+                hi = fmax2(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, off));
+            }
+        }
+        if ((lane & (LPU - 1)) == 0) {
+            const int u = (warp * CHUNKS + c) * (32 / LPU) + lane / LPU;
+            s_umn[u] = lo;
+            s_umx[u] = hi;
+        }
+    }
+}
+
+template <int NT> __device__ __forceinline__ uint32_t find_tensor(const CompressArgs<NT> &a, uint32_t gw)
+{
+    uint32_t lo = 0, hi = a.n_tensors - 1;                        // last tensor whose first window is <= gw
+    while (lo < hi) {
+        const uint32_t mid = (lo + hi + 1) >> 1;
+        if (a.t[mid].first_window <= gw) lo = mid; else hi = mid - 1;
+    }
+    return lo;
 }
 
 template <typename T, int CHUNKS, bool BATCH>
@@ -134,228 +291,279 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
 {
     constexpr uint32_t WE = kThreads * kLaneElems * CHUNKS;
 
-    __shared__ float s_umn[kMaxGroups], s_umx[kMaxGroups];      // per unit (min(G,256) elements)
-    __shared__ float s_R[kMaxGroups], s_mn[kMaxGroups];
-    __shared__ uint32_t s_key[kMaxLevels - 1][kMaxGroups];
-    __shared__ uint32_t s_cum[kMaxLevels - 1][kMaxGroups];
-    __shared__ __align__(16) GroupRec s_grp[kMaxGroups];
+    extern __shared__ __align__(128) unsigned char smem[];       // [stage | out0 | out1 | group arrays]
     __shared__ uint32_t s_wmin[kWarps], s_wmax[kWarps], s_wtot[kWarps];
-    __shared__ uint32_t s_ticket;
-    __shared__ uint64_t s_woff;
-    __shared__ int s_skip;
+    __shared__ __align__(8) uint64_t s_full;                     // mbarrier: staged window has landed
+    __shared__ uint32_t s_next;                                  // ticket of the staged window
+    __shared__ uint64_t s_woff;                                  // offset of the window being copied out (plain-store path)
+    __shared__ uint32_t s_wbytes;
+
+    unsigned char *const s_stage = smem;
+    float *const s_umn = reinterpret_cast<float *>(smem + a.lay.umn);
+    float *const s_umx = reinterpret_cast<float *>(smem + a.lay.umx);
+    uint32_t *const s_key = reinterpret_cast<uint32_t *>(smem + a.lay.key);   // [level][n_max]
+    uint32_t *const s_cum = reinterpret_cast<uint32_t *>(smem + a.lay.cum);
+    GroupRec *const s_grp = reinterpret_cast<GroupRec *>(smem + a.lay.grp);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t G = a.G, log2G = a.log2G, m = a.m;
-    const uint32_t U = G < 256u ? G : 256u;                      // unit: elements reduced inside one warp pass
-    const uint32_t log2U = G < 256u ? log2G : 8u;
-    const uint32_t lpu = U >> 3;                                  // lanes per unit
+    const uint32_t G = a.G, log2G = a.log2G, m = a.m, n_max = a.n_max;
+    const uint32_t e0 = (uint32_t)(warp * CHUNKS * 256 + lane * 8);    // this lane's first element of chunk 0
 
-    for (;;) {
-        if (tid == 0) s_ticket = atomicAdd(&a.hdr->ticket, 1u);
-        __syncthreads();
-        const uint32_t gw = s_ticket;
-        if (gw >= a.total_windows) return;
-
-        uint32_t ti = 0;
-        if (BATCH) {                                              // last tensor whose first window is <= gw
-            uint32_t lo = 0, hi = a.n_tensors - 1;
-            while (lo < hi) {
-                uint32_t mid = (lo + hi + 1) >> 1;
-                if (a.t[mid].first_window <= gw) lo = mid; else hi = mid - 1;
-            }
-            ti = lo;
+    // Thread 0 takes a ticket and starts the bulk copy of that window into the stage.
+    auto stage_next = [&]() {
+        const uint32_t t = atomicAdd(&a.hdr->ticket, 1u);
+        if (t < a.total_windows) {
+            const TensorDesc &nd = a.t[BATCH ? find_tensor(a, t) : 0u];
+            const uint64_t base = (uint64_t)(t - nd.first_window) * WE;
+            const uint64_t left = nd.numel - base;
+            const uint32_t bytes = (uint32_t)(left < WE ? left : WE) * Elem<T>::kBytes;
+            mbar_expect_tx(&s_full, bytes);
+            bulk_load(s_stage, reinterpret_cast<const char *>(nd.in) + base * Elem<T>::kBytes, bytes, &s_full);
         }
-        const TensorDesc &td = a.t[ti];
+        s_next = t;
+    };
+    auto record_error = [&](unsigned code, uint32_t window) {
+        if (atomicCAS(&a.hdr->status, 0u, code) == 0u) a.hdr->fail_window = window;
+    };
+
+    if (tid == 0) {
+        mbar_init(&s_full, 1);
+        stage_next();
+    }
+    __syncthreads();
+
+    // State of the previous window, whose packed bytes still sit in shared memory (warp 0).
+    bool have_prev = false;                                       // uniform over the CTA
+    uint32_t p_gw = 0, p_total = 0;
+    uint64_t p_excl = 0;
+    int p_state = 0;                                              // 0 unresolved, 1 resolved, < 0 failed
+    uint32_t gw = s_next;
+    uint32_t landed_phase = 0;
+
+    for (uint32_t iter = 0;; iter++) {
+        const bool valid = gw < a.total_windows;
+        if (!valid && !have_prev) break;
+        unsigned char *const s_out = smem + a.lay.out0 + (iter & 1u) * a.lay.out_stride;
+        unsigned char *const s_out_prev = smem + a.lay.out0 + ((iter & 1u) ^ 1u) * a.lay.out_stride;
+
+        const TensorDesc &td = a.t[BATCH ? find_tensor(a, valid ? gw : 0u) : 0u];
         const uint32_t w = gw - td.first_window;
         const uint64_t wbase = (uint64_t)w * WE;
         const uint64_t left = td.numel - wbase;
         const uint32_t n_elems = left < WE ? (uint32_t)left : WE;
-        const uint32_t n = n_elems >> log2G;                      // groups in this window
+        const uint32_t n = valid ? (n_elems >> log2G) : 0u;       // groups in this window
+        const uint32_t owners = (n + 31u) >> 5;                   // warps that own group records
         const uint64_t g0 = wbase >> log2G;                       // first group of the window in the tensor
 
-        // ---------------------------------------------------------------- load + unit min/max
+        // ---------------------------------------------------------------- staged window -> registers, unit min/max
         float x[CHUNKS][8];
-        uint32_t e[CHUNKS];
-#pragma unroll
-        for (int c = 0; c < CHUNKS; c++) {
-            e[c] = (uint32_t)((warp * CHUNKS + c) * 256 + lane * 8);
-            if (e[c] < n_elems) {
-                Elem<T>::load8(reinterpret_cast<const char *>(td.in) + (wbase + e[c]) * Elem<T>::kBytes, x[c]);
-            } else {
-#pragma unroll
-                for (int i = 0; i < 8; i++) x[c][i] = 0.0f;
+        bool landed = true;
+        if (valid) {
+            landed = mbar_wait_bounded(&s_full, landed_phase);
+            if (G >= 256u) load_and_reduce<T, CHUNKS, 32>(s_stage, warp, lane, x, s_umn, s_umx);
+            else if (G == 128u) load_and_reduce<T, CHUNKS, 16>(s_stage, warp, lane, x, s_umn, s_umx);
+            else if (G == 64u) load_and_reduce<T, CHUNKS, 8>(s_stage, warp, lane, x, s_umn, s_umx);
+            else load_and_reduce<T, CHUNKS, 4>(s_stage, warp, lane, x, s_umn, s_umx);
+        }
+        // unit stats visible; every thread has left the stage; did the copy land for all of them?
+        const bool landed_all = __syncthreads_and(landed) != 0;
+        const bool live = valid && landed_all;                    // this window is processed
+        if (tid == 0) {
+            if (live) stage_next();                               // the copy of the next window overlaps everything below
+            else s_next = 0xFFFFFFFFu;
+            if (valid && !landed_all) {                           // lost copy: poison the descriptor, report, stop after flushing
+                st_relaxed_u64(a.flags + gw, kFlagPoison << kFlagShift);
+                record_error(DAF_ERR_TIMEOUT, gw);
             }
         }
-#pragma unroll
-        for (int c = 0; c < CHUNKS; c++) {
-            float lo = fmin3(fmin3(x[c][0], x[c][1], x[c][2]), fmin3(x[c][3], x[c][4], x[c][5]), fmin2(x[c][6], x[c][7]));
-            float hi = fmax3(fmax3(x[c][0], x[c][1], x[c][2]), fmax3(x[c][3], x[c][4], x[c][5]), fmax2(x[c][6], x[c][7]));
-            for (uint32_t off = 1; off < lpu; off <<= 1) {
-                lo = fmin2(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, off));
-                hi = fmax2(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, off));
-            }
-            if ((lane & (lpu - 1u)) == 0u && e[c] < n_elems) {
-                s_umn[e[c] >> log2U] = lo;
-                s_umx[e[c] >> log2U] = hi;
-            }
-        }
-        __syncthreads();
+        landed_phase ^= 1u;
 
-        // ---------------------------------------------------------------- group range and keys
-        const uint64_t T = ((uint64_t)a.beta_q8 * n) >> 8;        // bit units of the window
-        const uint32_t rem = (uint32_t)(T - (uint64_t)a.S[0] * n);
-        // largest level every group can be raised to within the budget
-        uint32_t ell = 0;
-        while (ell + 1 < m && (a.S[ell + 1] - a.S[0]) * n <= rem) ell++;
-        const uint32_t rem_after = rem - (a.S[ell] - a.S[0]) * n;
+        uint32_t total = 0;
+        if (live) {
+            // ------------------------------------------------------------ group range and keys (owner warps)
+            const uint64_t Tbits = ((uint64_t)a.beta_q8 * n) >> 8; // bit units of the window
+            const uint32_t rem = (uint32_t)(Tbits - (uint64_t)a.S[0] * n);
+            uint32_t ell = 0;                                     // largest level every group can be raised to
+            while (ell + 1 < m && (a.S[ell + 1] - a.S[0]) * n <= rem) ell++;
+            const uint32_t rem_after = rem - (a.S[ell] - a.S[0]) * n;
+            const bool all_max = (ell + 1 == m);
+            // the best raise of level ell does not fit: the outcome is uniform iff the levels separate
+            const bool need_sep = !all_max && rem_after < a.cost[ell];
 
-        float mn = 0.0f, R = 0.0f;
-        uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
-        if ((uint32_t)tid < n) {
-            float mx;
-            if (G > 256u) {
-                const uint32_t r = G >> 8;
-                mn = s_umn[tid * r];
-                mx = s_umx[tid * r];
-                for (uint32_t j = 1; j < r; j++) {
-                    mn = fmin2(mn, s_umn[tid * r + j]);
-                    mx = fmax2(mx, s_umx[tid * r + j]);
-                }
-            } else {
-                mn = s_umn[tid];
-                mx = s_umx[tid];
-            }
-            R = __fsub_rn(mx, mn);
-            if (R < 0x1p-118f) R = 0.0f;                          // degenerate group: constant
-            s_mn[tid] = mn;
-            s_R[tid] = R;
-            for (uint32_t k = 0; k + 1 < m; k++) {
-                uint32_t key = __float_as_uint(__fmul_rn(R, a.v[k]));
-                s_key[k][tid] = key;
-                s_cum[k][tid] = 0u;
-                if (k + 1 == ell) kmin = key;
-                if (k == ell) kmax = key;
-            }
-        }
-        kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
-        kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
-        if (lane == 0) {
-            s_wmin[warp] = kmin;
-            s_wmax[warp] = kmax;
-        }
-        __syncthreads();
-        kmin = 0xFFFFFFFFu;
-        kmax = 0u;
-#pragma unroll
-        for (int i = 0; i < kWarps; i++) {
-            kmin = min(kmin, s_wmin[i]);
-            kmax = max(kmax, s_wmax[i]);
-        }
-
-        // ---------------------------------------------------------------- bit choice
-        // Uniform outcome: every raise below level ell sorts ahead of every raise from level
-        // ell upward, they all fit, and the best raise of level ell does not.
-        uint32_t level = ell;
-        const bool uniform = (ell + 1 == m) || (rem_after < a.cost[ell] && (ell == 0 || kmin >= kmax));
-        if (!uniform) {
-            // General case.  For each candidate (group g, raise k) add up the cost of all
-            // candidates that sort at or ahead of it (key descending, level ascending, group
-            // ascending); the candidate is accepted iff that total fits in the budget.
-            const uint32_t nl = m - 1;
-            const uint32_t items = n * nl * nl;
-            for (uint32_t it = tid; it < items; it += kThreads) {
-                const uint32_t g = it % n, kk = it / n;
-                const uint32_t k = kk / nl, k2 = kk % nl;
-                const uint32_t key = s_key[k][g];
-                uint32_t cnt = 0;
-                if (k2 < k) {
-                    for (uint32_t h = 0; h < n; h++) cnt += (s_key[k2][h] >= key);
-                } else if (k2 > k) {
-                    for (uint32_t h = 0; h < n; h++) cnt += (s_key[k2][h] > key);
-                } else {
-                    for (uint32_t h = 0; h < n; h++) {
-                        const uint32_t kh = s_key[k][h];
-                        cnt += (kh > key) || (kh == key && h <= g);
+            float mn = 0.0f, R = 0.0f;
+            if ((uint32_t)warp < owners) {
+                uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+                if ((uint32_t)tid < n) {
+                    float mx;
+                    if (G > 256u) {
+                        const uint32_t r = G >> 8;
+                        mn = s_umn[tid * r];
+                        mx = s_umx[tid * r];
+                        for (uint32_t j = 1; j < r; j++) {
+                            mn = fmin2(mn, s_umn[tid * r + j]);
+                            mx = fmax2(mx, s_umx[tid * r + j]);
+                        }
+                    } else {
+                        mn = s_umn[tid];
+                        mx = s_umx[tid];
+                    }
+                    R = __fsub_rn(mx, mn);
+                    if (R < 0x1p-118f) R = 0.0f;                  // degenerate group: constant
+                    if (!all_max) {
+                        for (uint32_t k = 0; k + 1 < m; k++) {
+                            const uint32_t key = __float_as_uint(__fmul_rn(R, a.v[k]));
+                            s_key[k * n_max + tid] = key;
+                            s_cum[k * n_max + tid] = 0u;
+                            if (k + 1 == ell) kmin = key;
+                            if (k == ell) kmax = key;
+                        }
                     }
                 }
-                atomicAdd(&s_cum[k][g], cnt * a.cost[k2]);
+                if (need_sep && ell > 0) {
+                    kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+                    kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+                    if (lane == 0) {
+                        s_wmin[warp] = kmin;
+                        s_wmax[warp] = kmax;
+                    }
+                }
             }
-            __syncthreads();
-            level = 0;
-            if ((uint32_t)tid < n)
-                for (uint32_t k = 0; k + 1 < m; k++) level += (s_cum[k][tid] <= rem);
-        }
 
-        // ---------------------------------------------------------------- group parameters, sizes, scan
-        uint32_t size = 0, b = 0;
-        float inv = 0.0f;
-        if ((uint32_t)tid < n) {
-            b = a.S[level];
-            const float Lf = (float)((1u << b) - 1u);
-            const float scale = R > 0.0f ? __fdiv_rn(R, Lf) : 0.0f;
-            inv = R > 0.0f ? __fdiv_rn(Lf, R) : 0.0f;
-            td.bits[g0 + tid] = (uint8_t)b;
-            td.mn[g0 + tid] = mn;
-            td.scale[g0 + tid] = scale;
-            size = (G >> 3) * b;
-        }
-        uint32_t incl = size;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            uint32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-            if (lane >= off) incl += y;
-        }
-        if (lane == 31) s_wtot[warp] = incl;
-        __syncthreads();
-        uint32_t wbase_bytes = 0, total = 0;
-#pragma unroll
-        for (int i = 0; i < kWarps; i++) {
-            const uint32_t t = s_wtot[i];
-            if (i < warp) wbase_bytes += t;
-            total += t;
-        }
-        if ((uint32_t)tid < n) {
-            GroupRec rec;
-            rec.mn = mn;
-            rec.inv = inv;
-            rec.b = b;
-            rec.off = wbase_bytes + incl - size;
-            s_grp[tid] = rec;
-        }
-        __syncthreads();
+            // ------------------------------------------------------------ bit choice
+            uint32_t level = ell;
+            if (!all_max) {
+                __syncthreads();                                  // keys and per-warp extremes visible
+                bool uniform = need_sep;
+                if (need_sep && ell > 0) {
+                    // Uniform outcome: every raise below level ell sorts ahead of every raise from
+                    // level ell upward (ties go to the lower level), they all fit, the next does not.
+                    uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+                    for (uint32_t i = 0; i < owners; i++) {
+                        kmin = min(kmin, s_wmin[i]);
+                        kmax = max(kmax, s_wmax[i]);
+                    }
+                    uniform = kmin >= kmax;
+                }
+                if (!uniform) {
+                    // General case.  For each candidate (group g, raise k) add up the cost of all
+                    // candidates that sort at or ahead of it (key descending, level ascending, group
+                    // ascending); the candidate is accepted iff that total fits in the budget.
+                    const uint32_t nl = m - 1;
+                    const uint32_t items = n * nl * nl;
+                    for (uint32_t it = tid; it < items; it += kThreads) {
+                        const uint32_t g = it % n, kk = it / n;
+                        const uint32_t k = kk / nl, k2 = kk % nl;
+                        const uint32_t key = s_key[k * n_max + g];
+                        const uint32_t *row = s_key + k2 * n_max;
+                        uint32_t cnt = 0;
+                        if (k2 < k) {
+                            for (uint32_t h = 0; h < n; h++) cnt += (row[h] >= key);
+                        } else if (k2 > k) {
+                            for (uint32_t h = 0; h < n; h++) cnt += (row[h] > key);
+                        } else {
+                            for (uint32_t h = 0; h < n; h++) cnt += (row[h] > key) || (row[h] == key && h <= g);
+                        }
+                        atomicAdd(&s_cum[k * n_max + g], cnt * a.cost[k2]);
+                    }
+                    __syncthreads();
+                    level = 0;
+                    if ((uint32_t)tid < n)
+                        for (uint32_t k = 0; k + 1 < m; k++) level += (s_cum[k * n_max + tid] <= rem);
+                }
+            }
 
-        // ---------------------------------------------------------------- window offset (warp 0)
-        if (warp == 0) {
-            int failed = 0, timed_out = 0;
-            const uint64_t excl = lookback(a.flags, gw, td.first_window, total, lane, &failed, &timed_out);
+            // ------------------------------------------------------------ group parameters, sizes, scan (owner warps)
+            uint32_t size = 0, b = 0, incl = 0;
+            float inv = 0.0f;
+            if ((uint32_t)warp < owners) {
+                if ((uint32_t)tid < n) {
+                    b = a.S[level];
+                    const float Lf = (float)((1u << b) - 1u);
+                    const float scale = R > 0.0f ? __fdiv_rn(R, Lf) : 0.0f;
+                    inv = R > 0.0f ? __fdiv_rn(Lf, R) : 0.0f;
+                    td.bits[g0 + tid] = (uint8_t)b;
+                    td.mn[g0 + tid] = mn;
+                    td.scale[g0 + tid] = scale;
+                    size = (G >> 3) * b;
+                }
+                incl = size;
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                    const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                    if (lane >= off) incl += y;
+                }
+                if (lane == 31) s_wtot[warp] = incl;
+                total = __shfl_sync(0xFFFFFFFFu, incl, 31);       // complete when a single warp owns all groups
+            }
+            uint32_t before = 0;
+            if (owners > 1) {
+                __syncthreads();
+                if ((uint32_t)warp < owners) {
+                    total = 0;
+                    for (uint32_t i = 0; i < owners; i++) {
+                        const uint32_t t = s_wtot[i];
+                        if (i < (uint32_t)warp) before += t;
+                        total += t;
+                    }
+                }
+            }
+            if ((uint32_t)tid < n) {
+                GroupRec rec;
+                rec.mn = mn;
+                rec.inv = inv;
+                rec.b = b;
+                rec.off = before + incl - size;
+                s_grp[tid] = rec;
+            }
+            // the window's byte count is known: publish it at once (warp 0 always owns groups)
+            if (tid == 0) {
+                const bool first = (gw == td.first_window);
+                st_relaxed_u64(a.flags + gw, ((first ? kFlagPrefix : kFlagAggregate) << kFlagShift) | total);
+            }
+        }
+        if (tid == 0) bulk_store_wait_read();                     // the store issued one window ago has left its buffer
+        __syncthreads();                                          // group records and s_next visible
+        const uint32_t gw_next = s_next;
+
+        // ---------------------------------------------------------------- previous window: offset, then out of shared memory
+        if (have_prev && warp == 0) {
+            const TensorDesc &pd = a.t[BATCH ? find_tensor(a, p_gw) : 0u];
+            if (p_state == 0) {                                   // not resolved opportunistically: wait (bounded) now
+                p_state = lookback<4>(a.flags, p_gw, pd.first_window, lane, true, &p_excl);
+                if (lane == 0)
+                    st_relaxed_u64(a.flags + p_gw, p_state == 1 ? ((kFlagPrefix << kFlagShift) | (p_excl + p_total))
+                                                                  : (kFlagPoison << kFlagShift));
+            }
             if (lane == 0) {
-                int skip = failed;
-                if (!failed) {
-                    td.woff[w] = excl;
-                    if (w + 1 == td.n_windows) td.woff[w + 1] = excl + total;
-                    if (excl + total > td.capacity) skip = 1;
+                const uint32_t pw = p_gw - pd.first_window;
+                bool skip = p_state != 1;
+                if (!skip) {
+                    pd.woff[pw] = p_excl;
+                    if (pw + 1 == pd.n_windows) pd.woff[pw + 1] = p_excl + p_total;
+                    skip = p_excl + p_total > pd.capacity;
                 }
-                if (skip) {
-                    const unsigned code = timed_out ? DAF_ERR_TIMEOUT : DAF_ERR_CAPACITY;
-                    if (atomicCAS(&a.hdr->status, 0u, code) == 0u) a.hdr->fail_window = gw;
+                if (skip) record_error(p_state == -2 ? DAF_ERR_TIMEOUT : DAF_ERR_CAPACITY, p_gw);
+                if (a.bulk_store) {
+                    if (!skip && p_total) bulk_store(pd.packed + p_excl, s_out_prev, p_total);
+                } else {
+                    s_woff = p_excl;
+                    s_wbytes = skip ? 0u : p_total;
                 }
-                s_woff = excl;
-                s_skip = skip;
             }
         }
 
-        // ---------------------------------------------------------------- quantize + pack (registers)
-        uint32_t pk0[CHUNKS], pk1[CHUNKS], pb[CHUNKS], poff[CHUNKS];
+        // ---------------------------------------------------------------- quantize + pack into shared memory
+        if (live) {
+            const uint64_t blk0 = ((td.elem_base + wbase) >> 3) + (e0 >> 3);
 #pragma unroll
-        for (int c = 0; c < CHUNKS; c++) {
-            pk0[c] = pk1[c] = pb[c] = poff[c] = 0u;
-            if (e[c] < n_elems) {
-                const GroupRec rec = s_grp[e[c] >> log2G];
+            for (int c = 0; c < CHUNKS; c++) {
+                const uint32_t e = e0 + 256u * c;
+                const GroupRec rec = s_grp[e >> log2G];
                 uint32_t o[4];
                 if (a.nearest) {
-                    o[0] = o[1] = o[2] = o[3] = 0x80008000u;       // every 15-bit lane = 2^14
+                    o[0] = o[1] = o[2] = o[3] = 0x80008000u;       // every 16-bit lane = 2 * 2^14
                 } else {
-                    const uint64_t blk = (td.elem_base + wbase + e[c]) >> 3;
+                    const uint64_t blk = blk0 + 32u * c;
                     if (BATCH) {
                         PhiloxSeedKeys sk{(uint32_t)td.seed, (uint32_t)(td.seed >> 32)};
                         philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), sk, o);
@@ -363,63 +571,112 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                         philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), a.keys, o);
                     }
                 }
-                switch (rec.b) {
-                case 1: quantize8<1>(x[c], rec.mn, rec.inv, o, pk0[c], pk1[c]); break;
-                case 2: quantize8<2>(x[c], rec.mn, rec.inv, o, pk0[c], pk1[c]); break;
-                case 4: quantize8<4>(x[c], rec.mn, rec.inv, o, pk0[c], pk1[c]); break;
-                default: quantize8<8>(x[c], rec.mn, rec.inv, o, pk0[c], pk1[c]); break;
-                }
-                pb[c] = rec.b;
-                poff[c] = rec.off + ((e[c] & (G - 1u)) >> 3) * rec.b;
-            }
-        }
-        __syncthreads();
-
-        // ---------------------------------------------------------------- store
-        if (!s_skip) {
-            uint8_t *dst = td.packed + s_woff;
-#pragma unroll
-            for (int c = 0; c < CHUNKS; c++) {
-                if (e[c] < n_elems) {
-                    uint8_t *p = dst + poff[c];
-                    switch (pb[c]) {
-                    case 1: *p = (uint8_t)pk0[c]; break;
-                    case 2: *reinterpret_cast<uint16_t *>(p) = (uint16_t)pk0[c]; break;
-                    case 4: *reinterpret_cast<uint32_t *>(p) = pk0[c]; break;
+                uint32_t w0, w1;
+                unsigned char *p = s_out + rec.off + ((e & (G - 1u)) >> 3) * rec.b;
+                if (e < n_elems) {
+                    switch (rec.b) {
+                    case 1: quantize8<1>(x[c], rec.mn, rec.inv, o, w0, w1); *p = (unsigned char)w0; break;
+                    case 2: quantize8<2>(x[c], rec.mn, rec.inv, o, w0, w1); *reinterpret_cast<uint16_t *>(p) = (uint16_t)w0; break;
+                    case 4: quantize8<4>(x[c], rec.mn, rec.inv, o, w0, w1); *reinterpret_cast<uint32_t *>(p) = w0; break;
                     default:
+                        quantize8<8>(x[c], rec.mn, rec.inv, o, w0, w1);
                         if (G >= 64u) {
-                            *reinterpret_cast<uint2 *>(p) = make_uint2(pk0[c], pk1[c]);
+                            *reinterpret_cast<uint2 *>(p) = make_uint2(w0, w1);
                         } else {                                   // G = 32: groups are only 4-byte aligned
-                            reinterpret_cast<uint32_t *>(p)[0] = pk0[c];
-                            reinterpret_cast<uint32_t *>(p)[1] = pk1[c];
+                            reinterpret_cast<uint32_t *>(p)[0] = w0;
+                            reinterpret_cast<uint32_t *>(p)[1] = w1;
                         }
                         break;
                     }
                 }
             }
+            if (a.bulk_store) fence_async_shared();               // packed bytes visible to the bulk store issued later
         }
-        // the next iteration's first barrier orders these reads of shared memory before any rewrite
+
+        // ---------------------------------------------------------------- plain-store path for the previous window
+        if (!a.bulk_store && have_prev) {
+            __syncthreads();                                      // s_woff / s_wbytes visible
+            const TensorDesc &pd = a.t[BATCH ? find_tensor(a, p_gw) : 0u];
+            uint32_t *dst = reinterpret_cast<uint32_t *>(pd.packed + s_woff);
+            const uint32_t *src = reinterpret_cast<const uint32_t *>(s_out_prev);
+            const uint32_t words = s_wbytes >> 2;
+            for (uint32_t i = tid; i < words; i += kThreads) dst[i] = src[i];
+        }
+
+        // ---------------------------------------------------------------- this window becomes the previous one
+        if (warp == 0) {
+            p_gw = gw;
+            p_total = __shfl_sync(0xFFFFFFFFu, total, 0);
+            p_excl = 0;
+            p_state = 0;
+            if (live) {
+                if (gw == td.first_window) {
+                    p_state = 1;                                  // already published as a prefix
+                } else {                                          // opportunistic, non-blocking look-back
+                    p_state = lookback<kLookDepth>(a.flags, gw, td.first_window, lane, false, &p_excl);
+                    if (lane == 0 && p_state != 0)
+                        st_relaxed_u64(a.flags + gw, p_state == 1 ? ((kFlagPrefix << kFlagShift) | (p_excl + p_total))
+                                                                    : (kFlagPoison << kFlagShift));
+                }
+            }
+        }
+        have_prev = live;
+        gw = live ? gw_next : 0xFFFFFFFFu;
+        if (valid && !landed_all) {                               // give the lost copy one more bounded chance before leaving
+            mbar_wait_bounded(&s_full, landed_phase ^ 1u);
+        }
     }
+    if (tid == 0) bulk_store_wait_all();
 }
 
 // ------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------
+// Shared-memory carve-up for one launch configuration.
+static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint32_t window_cap_bytes)
+{
+    auto up = [](uint32_t v) { return (v + 127u) & ~127u; };
+    const uint32_t n_max = we / G, units = we / (G < 256u ? G : 256u);
+    SmemLayout l;
+    uint32_t at = up(we * elem_bytes);
+    l.out0 = at;
+    l.out_stride = up(window_cap_bytes < 16u ? 16u : window_cap_bytes);
+    at += 2u * l.out_stride;
+    l.umn = at; at += up(4u * units);
+    l.umx = at; at += up(4u * units);
+    l.key = at; at += up(4u * (kMaxLevels - 1) * n_max);
+    l.cum = at; at += up(4u * (kMaxLevels - 1) * n_max);
+    l.grp = at; at += up(16u * n_max);
+    l.total = at;
+    return l;
+}
+
 template <typename T, int CHUNKS, bool BATCH>
 static cudaError_t launch(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
-    static int max_ctas = 0;                                      // resident CTAs on the current device
-    if (max_ctas == 0) {
-        int dev = 0, sms = 0, per_sm = 0;
-        cudaError_t e = cudaGetDevice(&dev);
+    static int sms = 0, smem_set = 0, cached_smem = -1, cached_ctas = 0;   // per instantiation, current device
+    const int smem = (int)args.lay.total;
+    cudaError_t e = cudaSuccess;
+    if (sms == 0) {
+        int dev = 0;
+        e = cudaGetDevice(&dev);
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e == cudaSuccess)
-            e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel<T, CHUNKS, BATCH>, kThreads, 0);
         if (e != cudaSuccess) return e;
-        max_ctas = sms * (per_sm > 0 ? per_sm : 1);
     }
-    const uint32_t grid = args.total_windows < (uint32_t)max_ctas ? args.total_windows : (uint32_t)max_ctas;
-    compress_kernel<T, CHUNKS, BATCH><<<grid, kThreads, 0, stream>>>(args);
+    if (smem > smem_set) {
+        e = cudaFuncSetAttribute(compress_kernel<T, CHUNKS, BATCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        smem_set = smem;
+    }
+    if (smem != cached_smem) {
+        int per_sm = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel<T, CHUNKS, BATCH>, kThreads, smem);
+        if (e != cudaSuccess) return e;
+        cached_smem = smem;
+        cached_ctas = sms * (per_sm > 0 ? per_sm : 1);
+    }
+    const uint32_t grid = args.total_windows < (uint32_t)cached_ctas ? args.total_windows : (uint32_t)cached_ctas;
+    compress_kernel<T, CHUNKS, BATCH><<<grid, kThreads, smem, stream>>>(args);
     return cudaGetLastError();
 }
 
@@ -448,6 +705,10 @@ template <int NT> static void fill_common(CompressArgs<NT> &a, const Plan &pl, c
     a.beta_q8 = pl.beta_q8;
     a.m = pl.m;
     a.nearest = p->rounding == DAF_ROUND_NEAREST;
+    a.bulk_store = pl.G >= 128u;                                  // every group is then a multiple of 16 bytes
+    a.n_max = pl.We / pl.G;
+    const uint32_t elem_bytes = p->dtype == DAF_F32 ? 4u : 2u;
+    a.lay = make_layout(pl.We, elem_bytes, pl.G, (uint32_t)((((uint64_t)pl.beta_q8 * pl.W) >> 8) * pl.G / 8));
     for (int k = 0; k < kMaxLevels; k++) {
         a.S[k] = pl.S[k];
         a.cost[k] = pl.cost[k];

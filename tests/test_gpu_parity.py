@@ -114,6 +114,20 @@ def test_degenerate_groups_zero_constant_and_signed_zero():
     assert_decompress_parity(c, ref, "f32", "degenerate")
 
 
+@pytest.mark.parametrize("G", [256, 1024, 16384])
+def test_signed_zero_minimum_in_full_warp_groups(G):
+    """Groups of 256 and more are reduced by the warp-wide redux path: -0.0 must still order below +0.0."""
+    rng = np.random.default_rng(G)
+    n = 16384 * 2
+    a = np.abs(rng.standard_normal(n)).astype(np.float32)
+    a[rng.integers(0, n, n // 8)] = 0.0
+    a[rng.integers(0, n, n // 8)] = -0.0                      # smallest values are a mix of +0.0 and -0.0
+    a[:G] = np.where(np.arange(G) % 2 == 0, np.float32(0.0), np.float32(-0.0))   # max must be +0.0, min -0.0
+    x, c, ref = assert_compress_parity(a, "f32", G, (1, 2, 4, 8), 3.0, label=f"signed-zero/G{G}")
+    assert ref.mn.view(np.uint32)[0] == 0x80000000
+    assert_decompress_parity(c, ref, "f32", f"signed-zero/G{G}")
+
+
 def test_heavy_ties_relu6_saturation():
     """Most groups share the same range (clip at 0 and 6): the tie order by group index decides."""
     rng = np.random.default_rng(4)
