@@ -47,6 +47,7 @@ template <int NT> struct CompressArgs {
     uint64_t *flags;
     uint32_t total_windows, n_tensors;
     uint32_t G, log2G, beta_q8, m, nearest, bulk_store, n_max;
+    uint32_t full_ell, full_rem, full_rem_after;   // budget arithmetic of a full window (n_max groups)
     uint32_t S[kMaxLevels], cost[kMaxLevels];
     float v[kMaxLevels];
     SmemLayout lay;
@@ -67,7 +68,7 @@ struct GroupRec {             // what the quantize pass needs per group (one 16-
 // (fixed + r15) >> 15 == (2*bits(s) + h - 2*bits(256)) >> 16, which needs one add, one shift
 // and one fused subtract-and-clamp per element.
 // ------------------------------------------------------------------------------------------
-template <int B>
+template <int B, bool CLAMP>
 __device__ __forceinline__ void quantize8(const float (&x)[8], float mn, float inv, const uint32_t (&o)[4],
                                           uint32_t &w0, uint32_t &w1)
 {
@@ -79,14 +80,19 @@ __device__ __forceinline__ void quantize8(const float (&x)[8], float mn, float i
         const float d = __fsub_rn(x[i], mn);
         const float s = __fmaf_rn(d, inv, 256.0f);
         const uint32_t h = (i & 1) ? (o[i >> 1] >> 16) : (o[i >> 1] & 0xFFFFu);
-        const uint32_t u = (__float_as_uint(s) << 1) + h;         // mod 2^32; 2*bits(256) = 0x87000000
-        const uint32_t q = min((u >> 16) - 0x8700u, L);
-        if (B == 8) {
-            if (i < 4) w0 |= q << (8 * i);
-            else w1 |= q << (8 * (i - 4));
+        const uint32_t t = (__float_as_uint(s) << 1) + h;         // mod 2^32; 2*bits(256) = 0x87000000
+        const int pos = (B * i) & 31;                             // bit position of code i in its word (unrolled: constant)
+        uint32_t field;
+        if (CLAMP) {
+            field = min((t >> 16) - 0x8700u, L) << pos;
         } else {
-            w0 |= q << (B * i);
+            // the code is the B-bit field of t at bit 16 (never above L when 1/scale is a normal
+            // number): move it to its place and mask, without materialising it
+            const uint32_t moved = pos < 16 ? (t >> (16 - pos)) : (pos == 16 ? t : (t << (pos - 16)));
+            field = moved & (L << pos);
         }
+        if (B == 8 && i >= 4) w1 |= field;
+        else w0 |= field;
     }
 }
 
@@ -96,7 +102,7 @@ __device__ __forceinline__ void quantize8(const float (&x)[8], float mn, float i
 // exclusive prefix was found (*excl), 0 when a needed descriptor is still empty and `block`
 // is false, -1 on a poisoned predecessor, -2 when the bounded wait ran out.
 // ------------------------------------------------------------------------------------------
-constexpr int kLookDepth = 10;
+constexpr int kLookDepth = 16;
 
 template <int DEPTH>
 __device__ __forceinline__ int lookback(const uint64_t *flags, uint32_t gw, uint32_t first, int lane, bool block,
@@ -207,19 +213,16 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity
     return false;
 }
 
-// Eight consecutive elements of a lane from the staged window.  For 4-byte elements a lane
-// owns 32 bytes; the two 16-byte halves are read in an order that depends on the lane so
-// that each quarter-warp touches all 32 banks, then swapped back into element order.
+// Eight consecutive elements of a lane from the staged window (two 16-byte shared loads for
+// 4-byte elements, one for 2-byte elements).
 template <typename T> __device__ __forceinline__ void load8_staged(const unsigned char *chunk, int lane, float (&x)[8]);
 
 template <> __device__ __forceinline__ void load8_staged<float>(const unsigned char *chunk, int lane, float (&x)[8])
 {
-    const bool odd = (lane >> 2) & 1;
-    const unsigned char *p = chunk + lane * 32;
-    const float4 a = *reinterpret_cast<const float4 *>(p + (odd ? 16 : 0));
-    const float4 b = *reinterpret_cast<const float4 *>(p + (odd ? 0 : 16));
-    x[0] = odd ? b.x : a.x; x[1] = odd ? b.y : a.y; x[2] = odd ? b.z : a.z; x[3] = odd ? b.w : a.w;
-    x[4] = odd ? a.x : b.x; x[5] = odd ? a.y : b.y; x[6] = odd ? a.z : b.z; x[7] = odd ? a.w : b.w;
+    const float4 a = *reinterpret_cast<const float4 *>(chunk + lane * 32);
+    const float4 b = *reinterpret_cast<const float4 *>(chunk + lane * 32 + 16);
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
+    x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
 }
 template <> __device__ __forceinline__ void load8_staged<__half>(const unsigned char *chunk, int lane, float (&x)[8])
 {
@@ -285,18 +288,66 @@ template <int NT> __device__ __forceinline__ uint32_t find_tensor(const Compress
     return lo;
 }
 
+// What the rest of the CTA needs to know about a window once its widths are chosen.
+struct WindowInfo {
+    uint32_t total;        // packed bytes of the window
+    uint32_t fast_b;       // common width when every group got the same one and no clamp is needed, else 0
+};
+
+// The CTA is 16 compute warps plus one control warp.  Hardware barrier 1 ("stage"): the
+// compute warps have consumed the staged window and finished the previous window's packed
+// bytes; barrier 2 ("widths"): the window's group records are ready; barrier 3 is private to
+// the warps that own group records.
+constexpr int kComputeWarps = kWarps;
+constexpr int kCompressThreads = kThreads + 32;
+constexpr uint32_t kBarStage = 1, kBarWidths = 2, kBarOwners = 3;
+
+__device__ __forceinline__ void bar_sync(uint32_t id, uint32_t threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+__device__ __forceinline__ void bar_arrive(uint32_t id, uint32_t threads)
+{
+    __threadfence_block();                                        // this thread's shared-memory writes first
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// Quantize + pack one window whose groups all have width B (no clamp needed): no per-chunk
+// decisions, packed position computed from the element index alone.
+template <typename KEYS, int CHUNKS, int B>
+__device__ __forceinline__ void quantize_uniform(const float (&x)[CHUNKS][8], const GroupRec *s_grp, uint32_t log2G,
+                                                 uint32_t e0, uint64_t blk0, const KEYS &keys, unsigned char *s_out)
+{
+    unsigned char *const out = s_out + (e0 >> 3) * B;
+#pragma unroll
+    for (int c = 0; c < CHUNKS; c++) {
+        const float2 mi = *reinterpret_cast<const float2 *>(&s_grp[(e0 + 256u * c) >> log2G]);   // mn, inv
+        uint32_t o[4];
+        const uint64_t blk = blk0 + 32u * c;
+        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), keys, o);
+        uint32_t w0, w1;
+        quantize8<B, false>(x[c], mi.x, mi.y, o, w0, w1);
+        unsigned char *p = out + 32 * B * c;
+        if (B == 1) *p = (unsigned char)w0;
+        else if (B == 2) *reinterpret_cast<uint16_t *>(p) = (uint16_t)w0;
+        else if (B == 4) *reinterpret_cast<uint32_t *>(p) = w0;
+        else *reinterpret_cast<uint2 *>(p) = make_uint2(w0, w1);
+    }
+}
+
 template <typename T, int CHUNKS, bool BATCH>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kCompressThreads, 2)
 compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> a)
 {
     constexpr uint32_t WE = kThreads * kLaneElems * CHUNKS;
 
     extern __shared__ __align__(128) unsigned char smem[];       // [stage | out0 | out1 | group arrays]
-    __shared__ uint32_t s_wmin[kWarps], s_wmax[kWarps], s_wtot[kWarps];
+    __shared__ uint32_t s_wtot[kComputeWarps];
     __shared__ __align__(8) uint64_t s_full;                     // mbarrier: staged window has landed
     __shared__ uint32_t s_next;                                  // ticket of the staged window
-    __shared__ uint64_t s_woff;                                  // offset of the window being copied out (plain-store path)
-    __shared__ uint32_t s_wbytes;
+    __shared__ uint32_t s_lost;                                  // a staged copy did not land in time
+    __shared__ WindowInfo s_win[2];
+    __shared__ uint32_t s_slow[2];                               // a group of the window needs the clamped quantizer
 
     unsigned char *const s_stage = smem;
     float *const s_umn = reinterpret_cast<float *>(smem + a.lay.umn);
@@ -306,11 +357,10 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     GroupRec *const s_grp = reinterpret_cast<GroupRec *>(smem + a.lay.grp);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t G = a.G, log2G = a.log2G, m = a.m, n_max = a.n_max;
-    const uint32_t e0 = (uint32_t)(warp * CHUNKS * 256 + lane * 8);    // this lane's first element of chunk 0
+    const uint32_t G = a.G, log2G = a.log2G;
 
-    // Thread 0 takes a ticket and starts the bulk copy of that window into the stage.
-    auto stage_next = [&]() {
+    // Control lane: takes a ticket and starts the bulk copy of that window into the stage.
+    auto stage_next = [&]() -> uint32_t {
         const uint32_t t = atomicAdd(&a.hdr->ticket, 1u);
         if (t < a.total_windows) {
             const TensorDesc &nd = a.t[BATCH ? find_tensor(a, t) : 0u];
@@ -321,184 +371,234 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             bulk_load(s_stage, reinterpret_cast<const char *>(nd.in) + base * Elem<T>::kBytes, bytes, &s_full);
         }
         s_next = t;
+        return t;
     };
     auto record_error = [&](unsigned code, uint32_t window) {
         if (atomicCAS(&a.hdr->status, 0u, code) == 0u) a.hdr->fail_window = window;
     };
 
-    if (tid == 0) {
+    if (tid == kThreads) {
         mbar_init(&s_full, 1);
+        s_lost = 0u;
+        s_slow[0] = s_slow[1] = 0u;
         stage_next();
     }
     __syncthreads();
-
-    // State of the previous window, whose packed bytes still sit in shared memory (warp 0).
-    bool have_prev = false;                                       // uniform over the CTA
-    uint32_t p_gw = 0, p_total = 0;
-    uint64_t p_excl = 0;
-    int p_state = 0;                                              // 0 unresolved, 1 resolved, < 0 failed
     uint32_t gw = s_next;
-    uint32_t landed_phase = 0;
 
-    for (uint32_t iter = 0;; iter++) {
-        const bool valid = gw < a.total_windows;
-        if (!valid && !have_prev) break;
+    if (warp == kComputeWarps) {
+        // ============================================================ control warp
+        // Per window i: wait until the compute warps have consumed stage(i) and finished the
+        // packed bytes of window i-1; start the copy of window i+1; then, off the compute
+        // warps' critical path, find window i-1's byte offset by look-back, publish its
+        // inclusive prefix, and send its packed bytes to global memory.
+        bool have_prev = false;
+        uint32_t p_gw = 0;
+        for (uint32_t iter = 0;; iter++) {
+            const bool valid = gw < a.total_windows;
+            bar_sync(kBarStage, kCompressThreads);
+            const bool lost = s_lost != 0u;
+            uint32_t next = 0xFFFFFFFFu;
+            if (valid) {
+                if (lane == 0) {
+                    if (!lost) stage_next();
+                    else s_next = 0xFFFFFFFFu;
+                    bulk_store_wait_read();                       // the buffer window i+1 will be packed into is free again
+                }
+                __syncwarp();
+                next = lost ? 0xFFFFFFFFu : s_next;
+                bar_arrive(kBarWidths, kCompressThreads);
+            }
+            if (have_prev) {
+                const TensorDesc &pd = a.t[BATCH ? find_tensor(a, p_gw) : 0u];
+                const uint32_t p_total = s_win[(iter & 1u) ^ 1u].total;
+                const unsigned char *src = smem + a.lay.out0 + ((iter & 1u) ^ 1u) * a.lay.out_stride;
+                uint64_t excl = 0;
+                int state = 1;
+                if (p_gw != pd.first_window) {
+                    state = lookback<kLookDepth>(a.flags, p_gw, pd.first_window, lane, true, &excl);
+                    if (lane == 0)
+                        st_relaxed_u64(a.flags + p_gw, state == 1 ? ((kFlagPrefix << kFlagShift) | (excl + p_total))
+                                                                    : (kFlagPoison << kFlagShift));
+                }
+                const uint32_t pw = p_gw - pd.first_window;
+                bool skip = state != 1;
+                if (!skip) {
+                    if (lane == 0) {
+                        pd.woff[pw] = excl;
+                        if (pw + 1 == pd.n_windows) pd.woff[pw + 1] = excl + p_total;
+                    }
+                    skip = excl + p_total > pd.capacity;
+                }
+                if (skip) {
+                    if (lane == 0) record_error(state == -2 ? DAF_ERR_TIMEOUT : DAF_ERR_CAPACITY, p_gw);
+                } else if (a.bulk_store) {
+                    if (lane == 0 && p_total) bulk_store(pd.packed + excl, src, p_total);
+                } else {                                          // groups of 32 / 64: windows are only 4-byte aligned
+                    uint32_t *dst = reinterpret_cast<uint32_t *>(pd.packed + excl);
+                    const uint32_t *s32 = reinterpret_cast<const uint32_t *>(src);
+                    for (uint32_t i = lane; i < (p_total >> 2); i += 32) dst[i] = s32[i];
+                }
+            }
+            if (!valid) break;
+            if (lost) {
+                if (lane == 0) {
+                    record_error(DAF_ERR_TIMEOUT, gw);
+                    st_relaxed_u64(a.flags + gw, kFlagPoison << kFlagShift);
+                    mbar_wait_bounded(&s_full, iter & 1u);        // one more bounded chance for the lost copy
+                }
+                have_prev = false;
+            } else {
+                have_prev = true;
+                p_gw = gw;
+            }
+            gw = next;
+        }
+        if (lane == 0) bulk_store_wait_all();
+        return;
+    }
+
+    // ================================================================ compute warps
+    const uint32_t e0 = (uint32_t)(warp * CHUNKS * 256 + lane * 8);    // this lane's first element of chunk 0
+    for (uint32_t iter = 0; gw < a.total_windows; iter++) {
         unsigned char *const s_out = smem + a.lay.out0 + (iter & 1u) * a.lay.out_stride;
-        unsigned char *const s_out_prev = smem + a.lay.out0 + ((iter & 1u) ^ 1u) * a.lay.out_stride;
-
-        const TensorDesc &td = a.t[BATCH ? find_tensor(a, valid ? gw : 0u) : 0u];
+        const TensorDesc &td = a.t[BATCH ? find_tensor(a, gw) : 0u];
         const uint32_t w = gw - td.first_window;
         const uint64_t wbase = (uint64_t)w * WE;
         const uint64_t left = td.numel - wbase;
         const uint32_t n_elems = left < WE ? (uint32_t)left : WE;
-        const uint32_t n = valid ? (n_elems >> log2G) : 0u;       // groups in this window
+        const uint32_t n = n_elems >> log2G;                      // groups in this window
         const uint32_t owners = (n + 31u) >> 5;                   // warps that own group records
-        const uint64_t g0 = wbase >> log2G;                       // first group of the window in the tensor
 
         // ---------------------------------------------------------------- staged window -> registers, unit min/max
         float x[CHUNKS][8];
-        bool landed = true;
-        if (valid) {
-            landed = mbar_wait_bounded(&s_full, landed_phase);
-            if (G >= 256u) load_and_reduce<T, CHUNKS, 32>(s_stage, warp, lane, x, s_umn, s_umx);
-            else if (G == 128u) load_and_reduce<T, CHUNKS, 16>(s_stage, warp, lane, x, s_umn, s_umx);
-            else if (G == 64u) load_and_reduce<T, CHUNKS, 8>(s_stage, warp, lane, x, s_umn, s_umx);
-            else load_and_reduce<T, CHUNKS, 4>(s_stage, warp, lane, x, s_umn, s_umx);
-        }
-        // unit stats visible; every thread has left the stage; did the copy land for all of them?
-        const bool landed_all = __syncthreads_and(landed) != 0;
-        const bool live = valid && landed_all;                    // this window is processed
-        if (tid == 0) {
-            if (live) stage_next();                               // the copy of the next window overlaps everything below
-            else s_next = 0xFFFFFFFFu;
-            if (valid && !landed_all) {                           // lost copy: poison the descriptor, report, stop after flushing
-                st_relaxed_u64(a.flags + gw, kFlagPoison << kFlagShift);
-                record_error(DAF_ERR_TIMEOUT, gw);
-            }
-        }
-        landed_phase ^= 1u;
+        if (!mbar_wait_bounded(&s_full, iter & 1u)) s_lost = 1u;
+        if (G >= 256u) load_and_reduce<T, CHUNKS, 32>(s_stage, warp, lane, x, s_umn, s_umx);
+        else if (G == 128u) load_and_reduce<T, CHUNKS, 16>(s_stage, warp, lane, x, s_umn, s_umx);
+        else if (G == 64u) load_and_reduce<T, CHUNKS, 8>(s_stage, warp, lane, x, s_umn, s_umx);
+        else load_and_reduce<T, CHUNKS, 4>(s_stage, warp, lane, x, s_umn, s_umx);
 
-        uint32_t total = 0;
-        if (live) {
-            // ------------------------------------------------------------ group range and keys (owner warps)
-            const uint64_t Tbits = ((uint64_t)a.beta_q8 * n) >> 8; // bit units of the window
-            const uint32_t rem = (uint32_t)(Tbits - (uint64_t)a.S[0] * n);
-            uint32_t ell = 0;                                     // largest level every group can be raised to
-            while (ell + 1 < m && (a.S[ell + 1] - a.S[0]) * n <= rem) ell++;
-            const uint32_t rem_after = rem - (a.S[ell] - a.S[0]) * n;
+        // ---------------------------------------------------------------- widths of the window (owner warps only)
+        if ((uint32_t)warp < owners) {
+            bar_sync(kBarStage, kCompressThreads);                // every warp's unit min / max is visible
+            const uint32_t m = a.m, n_max = a.n_max;
+            const uint64_t g0 = wbase >> log2G;                   // first group of the window in the tensor
+            // Budget arithmetic of the window: precomputed on the host for full windows.
+            uint32_t ell = a.full_ell, rem = a.full_rem, rem_after = a.full_rem_after;
+            if (n != n_max) {
+                const uint64_t Tbits = ((uint64_t)a.beta_q8 * n) >> 8;    // bit units of the window
+                rem = (uint32_t)(Tbits - (uint64_t)a.S[0] * n);
+                ell = 0;                                          // largest level every group can be raised to
+                while (ell + 1 < m && (a.S[ell + 1] - a.S[0]) * n <= rem) ell++;
+                rem_after = rem - (a.S[ell] - a.S[0]) * n;
+            }
             const bool all_max = (ell + 1 == m);
             // the best raise of level ell does not fit: the outcome is uniform iff the levels separate
             const bool need_sep = !all_max && rem_after < a.cost[ell];
+            const bool mine = (uint32_t)tid < n;
+            if (tid == 0) s_slow[(iter & 1u) ^ 1u] = 0u;          // reset the flag of the next window
 
+            // range of this thread's group
             float mn = 0.0f, R = 0.0f;
-            if ((uint32_t)warp < owners) {
-                uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
-                if ((uint32_t)tid < n) {
-                    float mx;
-                    if (G > 256u) {
-                        const uint32_t r = G >> 8;
-                        mn = s_umn[tid * r];
-                        mx = s_umx[tid * r];
-                        for (uint32_t j = 1; j < r; j++) {
-                            mn = fmin2(mn, s_umn[tid * r + j]);
-                            mx = fmax2(mx, s_umx[tid * r + j]);
-                        }
-                    } else {
-                        mn = s_umn[tid];
-                        mx = s_umx[tid];
+            if (mine) {
+                float mx;
+                if (G > 256u) {
+                    const uint32_t r = G >> 8;
+                    mn = s_umn[tid * r];
+                    mx = s_umx[tid * r];
+                    for (uint32_t j = 1; j < r; j++) {
+                        mn = fmin2(mn, s_umn[tid * r + j]);
+                        mx = fmax2(mx, s_umx[tid * r + j]);
                     }
-                    R = __fsub_rn(mx, mn);
-                    if (R < 0x1p-118f) R = 0.0f;                  // degenerate group: constant
-                    if (!all_max) {
-                        for (uint32_t k = 0; k + 1 < m; k++) {
-                            const uint32_t key = __float_as_uint(__fmul_rn(R, a.v[k]));
-                            s_key[k * n_max + tid] = key;
-                            s_cum[k * n_max + tid] = 0u;
-                            if (k + 1 == ell) kmin = key;
-                            if (k == ell) kmax = key;
-                        }
-                    }
+                } else {
+                    mn = s_umn[tid];
+                    mx = s_umx[tid];
                 }
-                if (need_sep && ell > 0) {
-                    kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
-                    kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
-                    if (lane == 0) {
-                        s_wmin[warp] = kmin;
-                        s_wmax[warp] = kmax;
-                    }
-                }
+                R = __fsub_rn(mx, mn);
+                if (R < 0x1p-118f) R = 0.0f;                      // degenerate group: constant
             }
 
-            // ------------------------------------------------------------ bit choice
+            // bit choice
             uint32_t level = ell;
-            if (!all_max) {
-                __syncthreads();                                  // keys and per-warp extremes visible
-                bool uniform = need_sep;
-                if (need_sep && ell > 0) {
-                    // Uniform outcome: every raise below level ell sorts ahead of every raise from
-                    // level ell upward (ties go to the lower level), they all fit, the next does not.
-                    uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
-                    for (uint32_t i = 0; i < owners; i++) {
-                        kmin = min(kmin, s_wmin[i]);
-                        kmax = max(kmax, s_wmax[i]);
+            bool uniform = all_max || need_sep;
+            if (need_sep && ell > 0) {
+                // Uniform outcome: every raise below level ell sorts ahead of every raise from
+                // level ell upward (ties go to the lower level), they all fit, the next does not.
+                // Each owner warp evaluates the test over all groups itself (no exchange needed).
+                const float v_lo = a.v[ell - 1], v_hi = a.v[ell];
+                uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+                if (owners == 1) {
+                    if (mine) {
+                        kmin = __float_as_uint(__fmul_rn(R, v_lo));
+                        kmax = __float_as_uint(__fmul_rn(R, v_hi));
                     }
-                    uniform = kmin >= kmax;
-                }
-                if (!uniform) {
-                    // General case.  For each candidate (group g, raise k) add up the cost of all
-                    // candidates that sort at or ahead of it (key descending, level ascending, group
-                    // ascending); the candidate is accepted iff that total fits in the budget.
-                    const uint32_t nl = m - 1;
-                    const uint32_t items = n * nl * nl;
-                    for (uint32_t it = tid; it < items; it += kThreads) {
-                        const uint32_t g = it % n, kk = it / n;
-                        const uint32_t k = kk / nl, k2 = kk % nl;
-                        const uint32_t key = s_key[k * n_max + g];
-                        const uint32_t *row = s_key + k2 * n_max;
-                        uint32_t cnt = 0;
-                        if (k2 < k) {
-                            for (uint32_t h = 0; h < n; h++) cnt += (row[h] >= key);
-                        } else if (k2 > k) {
-                            for (uint32_t h = 0; h < n; h++) cnt += (row[h] > key);
-                        } else {
-                            for (uint32_t h = 0; h < n; h++) cnt += (row[h] > key) || (row[h] == key && h <= g);
-                        }
-                        atomicAdd(&s_cum[k * n_max + g], cnt * a.cost[k2]);
+                } else {                                          // groups of at most 256: one unit per group
+                    for (uint32_t g = lane; g < n; g += 32) {
+                        float Rg = __fsub_rn(s_umx[g], s_umn[g]);
+                        if (Rg < 0x1p-118f) Rg = 0.0f;
+                        kmin = min(kmin, __float_as_uint(__fmul_rn(Rg, v_lo)));
+                        kmax = max(kmax, __float_as_uint(__fmul_rn(Rg, v_hi)));
                     }
-                    __syncthreads();
-                    level = 0;
-                    if ((uint32_t)tid < n)
-                        for (uint32_t k = 0; k + 1 < m; k++) level += (s_cum[k * n_max + tid] <= rem);
                 }
+                kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+                kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+                uniform = kmin >= kmax;
             }
-
-            // ------------------------------------------------------------ group parameters, sizes, scan (owner warps)
-            uint32_t size = 0, b = 0, incl = 0;
-            float inv = 0.0f;
-            if ((uint32_t)warp < owners) {
-                if ((uint32_t)tid < n) {
+            uint32_t size = 0, b = 0, incl = 0, total = 0, before = 0;
+            if (uniform) {
+                b = a.S[ell];
+                size = (G >> 3) * b;
+                incl = (uint32_t)(tid + 1) * size;                // group g starts at g * size
+                total = n * size;
+            } else {
+                // General case.  For each candidate (group g, raise k) add up the cost of all
+                // candidates that sort at or ahead of it (key descending, level ascending, group
+                // ascending); the candidate is accepted iff that total fits in the budget.
+                if (mine) {
+#pragma unroll
+                    for (int k = 0; k < kMaxLevels - 1; k++) {
+                        s_key[k * n_max + tid] = __float_as_uint(__fmul_rn(R, a.v[k]));
+                        s_cum[k * n_max + tid] = 0u;
+                    }
+                }
+                if (owners > 1) bar_sync(kBarOwners, owners * 32u);
+                else __syncwarp();
+                const uint32_t nl = m - 1;
+                const uint32_t items = n * nl * nl;
+                for (uint32_t it = tid; it < items; it += owners * 32u) {
+                    const uint32_t g = it % n, kk = it / n;
+                    const uint32_t k = kk / nl, k2 = kk % nl;
+                    const uint32_t kg = s_key[k * n_max + g];
+                    const uint32_t *row = s_key + k2 * n_max;
+                    uint32_t cnt = 0;
+                    if (k2 < k) {
+                        for (uint32_t h = 0; h < n; h++) cnt += (row[h] >= kg);
+                    } else if (k2 > k) {
+                        for (uint32_t h = 0; h < n; h++) cnt += (row[h] > kg);
+                    } else {
+                        for (uint32_t h = 0; h < n; h++) cnt += (row[h] > kg) || (row[h] == kg && h <= g);
+                    }
+                    atomicAdd(&s_cum[k * n_max + g], cnt * a.cost[k2]);
+                }
+                if (owners > 1) bar_sync(kBarOwners, owners * 32u);
+                else __syncwarp();
+                level = 0;
+                if (mine) {
+                    for (uint32_t k = 0; k + 1 < m; k++) level += (s_cum[k * n_max + tid] <= rem);
                     b = a.S[level];
-                    const float Lf = (float)((1u << b) - 1u);
-                    const float scale = R > 0.0f ? __fdiv_rn(R, Lf) : 0.0f;
-                    inv = R > 0.0f ? __fdiv_rn(Lf, R) : 0.0f;
-                    td.bits[g0 + tid] = (uint8_t)b;
-                    td.mn[g0 + tid] = mn;
-                    td.scale[g0 + tid] = scale;
                     size = (G >> 3) * b;
                 }
+                // byte offset of each group inside the window: exclusive scan of the sizes
                 incl = size;
 #pragma unroll
                 for (int off = 1; off < 32; off <<= 1) {
                     const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, off);
                     if (lane >= off) incl += y;
                 }
-                if (lane == 31) s_wtot[warp] = incl;
-                total = __shfl_sync(0xFFFFFFFFu, incl, 31);       // complete when a single warp owns all groups
-            }
-            uint32_t before = 0;
-            if (owners > 1) {
-                __syncthreads();
-                if ((uint32_t)warp < owners) {
+                total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                if (owners > 1) {
+                    if (lane == 0) s_wtot[warp] = total;
+                    bar_sync(kBarOwners, owners * 32u);
                     total = 0;
                     for (uint32_t i = 0; i < owners; i++) {
                         const uint32_t t = s_wtot[i];
@@ -507,7 +607,17 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                     }
                 }
             }
-            if ((uint32_t)tid < n) {
+
+            // group parameters and metadata
+            if (mine) {
+                const float Lf = (float)((1u << b) - 1u);
+                const float scale = R > 0.0f ? __fdiv_rn(R, Lf) : 0.0f;
+                const float inv = R > 0.0f ? __fdiv_rn(Lf, R) : 0.0f;
+                // 1/scale not a normal number: codes may need the clamp, take the careful path
+                if (R > 0.0f && inv < 0x1p-126f) s_slow[iter & 1u] = 1u;
+                td.bits[g0 + tid] = (uint8_t)b;
+                td.mn[g0 + tid] = mn;
+                td.scale[g0 + tid] = scale;
                 GroupRec rec;
                 rec.mn = mn;
                 rec.inv = inv;
@@ -515,46 +625,43 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 rec.off = before + incl - size;
                 s_grp[tid] = rec;
             }
-            // the window's byte count is known: publish it at once (warp 0 always owns groups)
             if (tid == 0) {
+                // the window's byte count is known: publish it at once (a lost copy poisons it instead)
                 const bool first = (gw == td.first_window);
-                st_relaxed_u64(a.flags + gw, ((first ? kFlagPrefix : kFlagAggregate) << kFlagShift) | total);
+                if (s_lost == 0u)
+                    st_relaxed_u64(a.flags + gw, ((first ? kFlagPrefix : kFlagAggregate) << kFlagShift) | total);
+                s_win[iter & 1u].total = total;
+                s_win[iter & 1u].fast_b = (uniform && n_elems == WE && !a.nearest) ? b : 0u;
             }
+        } else {
+            bar_arrive(kBarStage, kCompressThreads);
         }
-        if (tid == 0) bulk_store_wait_read();                     // the store issued one window ago has left its buffer
-        __syncthreads();                                          // group records and s_next visible
+        bar_sync(kBarWidths, kCompressThreads);                   // group records, window info and s_next visible
         const uint32_t gw_next = s_next;
-
-        // ---------------------------------------------------------------- previous window: offset, then out of shared memory
-        if (have_prev && warp == 0) {
-            const TensorDesc &pd = a.t[BATCH ? find_tensor(a, p_gw) : 0u];
-            if (p_state == 0) {                                   // not resolved opportunistically: wait (bounded) now
-                p_state = lookback<4>(a.flags, p_gw, pd.first_window, lane, true, &p_excl);
-                if (lane == 0)
-                    st_relaxed_u64(a.flags + p_gw, p_state == 1 ? ((kFlagPrefix << kFlagShift) | (p_excl + p_total))
-                                                                  : (kFlagPoison << kFlagShift));
-            }
-            if (lane == 0) {
-                const uint32_t pw = p_gw - pd.first_window;
-                bool skip = p_state != 1;
-                if (!skip) {
-                    pd.woff[pw] = p_excl;
-                    if (pw + 1 == pd.n_windows) pd.woff[pw + 1] = p_excl + p_total;
-                    skip = p_excl + p_total > pd.capacity;
-                }
-                if (skip) record_error(p_state == -2 ? DAF_ERR_TIMEOUT : DAF_ERR_CAPACITY, p_gw);
-                if (a.bulk_store) {
-                    if (!skip && p_total) bulk_store(pd.packed + p_excl, s_out_prev, p_total);
-                } else {
-                    s_woff = p_excl;
-                    s_wbytes = skip ? 0u : p_total;
-                }
-            }
-        }
+        const uint32_t fast_b = s_slow[iter & 1u] ? 0u : s_win[iter & 1u].fast_b;
+        if (s_lost != 0u) break;
 
         // ---------------------------------------------------------------- quantize + pack into shared memory
-        if (live) {
-            const uint64_t blk0 = ((td.elem_base + wbase) >> 3) + (e0 >> 3);
+        const uint64_t blk0 = ((td.elem_base + wbase) >> 3) + (e0 >> 3);
+        if (fast_b != 0u) {
+            // one width for the whole (full) window, stochastic rounding, no clamp needed
+            if (BATCH) {
+                const PhiloxSeedKeys sk{(uint32_t)td.seed, (uint32_t)(td.seed >> 32)};
+                switch (fast_b) {
+                case 1: quantize_uniform<PhiloxSeedKeys, CHUNKS, 1>(x, s_grp, log2G, e0, blk0, sk, s_out); break;
+                case 2: quantize_uniform<PhiloxSeedKeys, CHUNKS, 2>(x, s_grp, log2G, e0, blk0, sk, s_out); break;
+                case 4: quantize_uniform<PhiloxSeedKeys, CHUNKS, 4>(x, s_grp, log2G, e0, blk0, sk, s_out); break;
+                default: quantize_uniform<PhiloxSeedKeys, CHUNKS, 8>(x, s_grp, log2G, e0, blk0, sk, s_out); break;
+                }
+            } else {
+                switch (fast_b) {
+                case 1: quantize_uniform<PhiloxKeys, CHUNKS, 1>(x, s_grp, log2G, e0, blk0, a.keys, s_out); break;
+                case 2: quantize_uniform<PhiloxKeys, CHUNKS, 2>(x, s_grp, log2G, e0, blk0, a.keys, s_out); break;
+                case 4: quantize_uniform<PhiloxKeys, CHUNKS, 4>(x, s_grp, log2G, e0, blk0, a.keys, s_out); break;
+                default: quantize_uniform<PhiloxKeys, CHUNKS, 8>(x, s_grp, log2G, e0, blk0, a.keys, s_out); break;
+                }
+            }
+        } else {
 #pragma unroll
             for (int c = 0; c < CHUNKS; c++) {
                 const uint32_t e = e0 + 256u * c;
@@ -565,7 +672,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 } else {
                     const uint64_t blk = blk0 + 32u * c;
                     if (BATCH) {
-                        PhiloxSeedKeys sk{(uint32_t)td.seed, (uint32_t)(td.seed >> 32)};
+                        const PhiloxSeedKeys sk{(uint32_t)td.seed, (uint32_t)(td.seed >> 32)};
                         philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), sk, o);
                     } else {
                         philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), a.keys, o);
@@ -575,11 +682,11 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 unsigned char *p = s_out + rec.off + ((e & (G - 1u)) >> 3) * rec.b;
                 if (e < n_elems) {
                     switch (rec.b) {
-                    case 1: quantize8<1>(x[c], rec.mn, rec.inv, o, w0, w1); *p = (unsigned char)w0; break;
-                    case 2: quantize8<2>(x[c], rec.mn, rec.inv, o, w0, w1); *reinterpret_cast<uint16_t *>(p) = (uint16_t)w0; break;
-                    case 4: quantize8<4>(x[c], rec.mn, rec.inv, o, w0, w1); *reinterpret_cast<uint32_t *>(p) = w0; break;
+                    case 1: quantize8<1, true>(x[c], rec.mn, rec.inv, o, w0, w1); *p = (unsigned char)w0; break;
+                    case 2: quantize8<2, true>(x[c], rec.mn, rec.inv, o, w0, w1); *reinterpret_cast<uint16_t *>(p) = (uint16_t)w0; break;
+                    case 4: quantize8<4, true>(x[c], rec.mn, rec.inv, o, w0, w1); *reinterpret_cast<uint32_t *>(p) = w0; break;
                     default:
-                        quantize8<8>(x[c], rec.mn, rec.inv, o, w0, w1);
+                        quantize8<8, true>(x[c], rec.mn, rec.inv, o, w0, w1);
                         if (G >= 64u) {
                             *reinterpret_cast<uint2 *>(p) = make_uint2(w0, w1);
                         } else {                                   // G = 32: groups are only 4-byte aligned
@@ -590,43 +697,11 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                     }
                 }
             }
-            if (a.bulk_store) fence_async_shared();               // packed bytes visible to the bulk store issued later
         }
-
-        // ---------------------------------------------------------------- plain-store path for the previous window
-        if (!a.bulk_store && have_prev) {
-            __syncthreads();                                      // s_woff / s_wbytes visible
-            const TensorDesc &pd = a.t[BATCH ? find_tensor(a, p_gw) : 0u];
-            uint32_t *dst = reinterpret_cast<uint32_t *>(pd.packed + s_woff);
-            const uint32_t *src = reinterpret_cast<const uint32_t *>(s_out_prev);
-            const uint32_t words = s_wbytes >> 2;
-            for (uint32_t i = tid; i < words; i += kThreads) dst[i] = src[i];
-        }
-
-        // ---------------------------------------------------------------- this window becomes the previous one
-        if (warp == 0) {
-            p_gw = gw;
-            p_total = __shfl_sync(0xFFFFFFFFu, total, 0);
-            p_excl = 0;
-            p_state = 0;
-            if (live) {
-                if (gw == td.first_window) {
-                    p_state = 1;                                  // already published as a prefix
-                } else {                                          // opportunistic, non-blocking look-back
-                    p_state = lookback<kLookDepth>(a.flags, gw, td.first_window, lane, false, &p_excl);
-                    if (lane == 0 && p_state != 0)
-                        st_relaxed_u64(a.flags + gw, p_state == 1 ? ((kFlagPrefix << kFlagShift) | (p_excl + p_total))
-                                                                    : (kFlagPoison << kFlagShift));
-                }
-            }
-        }
-        have_prev = live;
-        gw = live ? gw_next : 0xFFFFFFFFu;
-        if (valid && !landed_all) {                               // give the lost copy one more bounded chance before leaving
-            mbar_wait_bounded(&s_full, landed_phase ^ 1u);
-        }
+        if (a.bulk_store) fence_async_shared();                   // packed bytes visible to the bulk store issued later
+        gw = gw_next;
     }
-    if (tid == 0) bulk_store_wait_all();
+    bar_arrive(kBarStage, kCompressThreads);                      // the last window's packed bytes are complete
 }
 
 // ------------------------------------------------------------------------------------------
@@ -670,13 +745,13 @@ static cudaError_t launch(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, c
     }
     if (smem != cached_smem) {
         int per_sm = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel<T, CHUNKS, BATCH>, kThreads, smem);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel<T, CHUNKS, BATCH>, kCompressThreads, smem);
         if (e != cudaSuccess) return e;
         cached_smem = smem;
         cached_ctas = sms * (per_sm > 0 ? per_sm : 1);
     }
     const uint32_t grid = args.total_windows < (uint32_t)cached_ctas ? args.total_windows : (uint32_t)cached_ctas;
-    compress_kernel<T, CHUNKS, BATCH><<<grid, kThreads, smem, stream>>>(args);
+    compress_kernel<T, CHUNKS, BATCH><<<grid, kCompressThreads, smem, stream>>>(args);
     return cudaGetLastError();
 }
 
@@ -708,6 +783,13 @@ template <int NT> static void fill_common(CompressArgs<NT> &a, const Plan &pl, c
     a.bulk_store = pl.G >= 128u;                                  // every group is then a multiple of 16 bytes
     a.n_max = pl.We / pl.G;
     const uint32_t elem_bytes = p->dtype == DAF_F32 ? 4u : 2u;
+    {
+        const uint32_t n = a.n_max;
+        a.full_rem = (uint32_t)((((uint64_t)pl.beta_q8 * n) >> 8) - (uint64_t)pl.S[0] * n);
+        a.full_ell = 0;
+        while (a.full_ell + 1 < pl.m && (pl.S[a.full_ell + 1] - pl.S[0]) * n <= a.full_rem) a.full_ell++;
+        a.full_rem_after = a.full_rem - (pl.S[a.full_ell] - pl.S[0]) * n;
+    }
     a.lay = make_layout(pl.We, elem_bytes, pl.G, (uint32_t)((((uint64_t)pl.beta_q8 * pl.W) >> 8) * pl.G / 8));
     for (int k = 0; k < kMaxLevels; k++) {
         a.S[k] = pl.S[k];
