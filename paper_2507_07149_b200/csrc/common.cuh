@@ -23,7 +23,8 @@ struct WorkspaceHeader {
     unsigned int status;        // daf_status recorded by the device (0 = OK)
     unsigned int ticket;        // next window to hand out
     unsigned int fail_window;   // first window that recorded an error (diagnostic)
-    unsigned int pad[61];
+    unsigned int fail_site;     // which wait or check recorded it (diagnostic)
+    unsigned int pad[60];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
 

@@ -46,7 +46,7 @@ template <int NT> struct CompressArgs {
     WorkspaceHeader *hdr;
     uint64_t *flags;
     uint32_t total_windows, n_tensors;
-    uint32_t G, log2G, beta_q8, m, nearest, bulk_store, n_max;
+    uint32_t G, log2G, beta_q8, m, nearest, bulk_store, n_max, nbuf;
     uint32_t full_ell, full_rem, full_rem_after;   // budget arithmetic of a full window (n_max groups)
     uint32_t S[kMaxLevels], cost[kMaxLevels];
     float v[kMaxLevels];
@@ -247,34 +247,37 @@ template <> __device__ __forceinline__ void load8_staged<__nv_bfloat16>(const un
 }
 
 // Staged window -> registers, then min / max per unit of LPU lanes (a full warp uses the
-// redux instruction) written to shared memory.  Chunks past a ragged window's end read
-// stale bytes; their results are never used.
+// redux instruction).  Every lane of a unit ends up with the unit's min / max (lo[c], hi[c]);
+// the unit's first lane also writes them to shared memory for the general bit choice.
+// Chunks past a ragged window's end read stale bytes; their results are never used.
 template <typename T, int CHUNKS, int LPU>
 __device__ __forceinline__ void load_and_reduce(const unsigned char *stage, int warp, int lane, float (&x)[CHUNKS][8],
-                                                float *s_umn, float *s_umx)
+                                                float (&lo)[CHUNKS], float (&hi)[CHUNKS], float *s_umn, float *s_umx)
 {
     constexpr int kChunkBytes = 256 * Elem<T>::kBytes;
 #pragma unroll
     for (int c = 0; c < CHUNKS; c++) load8_staged<T>(stage + (warp * CHUNKS + c) * kChunkBytes, lane, x[c]);
 #pragma unroll
     for (int c = 0; c < CHUNKS; c++) {
-        float lo = fmin3(fmin3(x[c][0], x[c][1], x[c][2]), fmin3(x[c][3], x[c][4], x[c][5]), fmin2(x[c][6], x[c][7]));
-        float hi = fmax3(fmax3(x[c][0], x[c][1], x[c][2]), fmax3(x[c][3], x[c][4], x[c][5]), fmax2(x[c][6], x[c][7]));
+        float l = fmin3(fmin3(x[c][0], x[c][1], x[c][2]), fmin3(x[c][3], x[c][4], x[c][5]), fmin2(x[c][6], x[c][7]));
+        float h = fmax3(fmax3(x[c][0], x[c][1], x[c][2]), fmax3(x[c][3], x[c][4], x[c][5]), fmax2(x[c][6], x[c][7]));
         if (LPU == 32) {
-            asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(lo) : "f"(lo));
-            asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(hi) : "f"(hi));
+            asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(l) : "f"(l));
+            asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(h) : "f"(h));
         } else {
 #pragma unroll
             for (int off = 1; off < LPU; off <<= 1) {
-                lo = fmin2(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, off));
-                hi = fmax2(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, off));
+                l = fmin2(l, __shfl_xor_sync(0xFFFFFFFFu, l, off));
+                h = fmax2(h, __shfl_xor_sync(0xFFFFFFFFu, h, off));
             }
         }
         if ((lane & (LPU - 1)) == 0) {
             const int u = (warp * CHUNKS + c) * (32 / LPU) + lane / LPU;
-            s_umn[u] = lo;
-            s_umx[u] = hi;
+            s_umn[u] = l;
+            s_umx[u] = h;
         }
+        lo[c] = l;
+        hi[c] = h;
     }
 }
 
@@ -288,19 +291,25 @@ template <int NT> __device__ __forceinline__ uint32_t find_tensor(const Compress
     return lo;
 }
 
-// What the rest of the CTA needs to know about a window once its widths are chosen.
-struct WindowInfo {
-    uint32_t total;        // packed bytes of the window
-    uint32_t fast_b;       // common width when every group got the same one and no clamp is needed, else 0
-};
-
-// The CTA is 16 compute warps plus one control warp.  Hardware barrier 1 ("stage"): the
-// compute warps have consumed the staged window and finished the previous window's packed
-// bytes; barrier 2 ("widths"): the window's group records are ready; barrier 3 is private to
-// the warps that own group records.
+// The CTA is 16 compute warps plus one control warp.
+//   barrier kBarWindow : the 16 compute warps meet once per window, after every warp has turned
+//                        its part of the staged window into registers and min / max; the control
+//                        warp only arrives there (it never makes the compute warps' wait longer
+//                        than its own work of the previous round), which also hands over the next
+//                        ticket and the guarantee that the packed-bytes buffer about to be
+//                        rewritten has left shared memory;
+//   barrier kBarWidths : compute warps only, used when a window needs the general bit choice;
+//   barrier kBarOwners : the warps that own group records in the general bit choice;
+//   mbarrier s_full    : the staged window has landed (bulk copy complete);
+//   mbarrier s_cons    : every compute warp has consumed the staged window and has finished
+//                        packing the previous window (16 arrivals);
+//   mbarrier s_done    : every compute warp has left its loop (16 arrivals, used once).
 constexpr int kComputeWarps = kWarps;
 constexpr int kCompressThreads = kThreads + 32;
-constexpr uint32_t kBarStage = 1, kBarWidths = 2, kBarOwners = 3;
+constexpr uint32_t kBarWindow = 1, kBarWidths = 2, kBarOwners = 3, kBarWindowOdd = 4;
+// Window barriers alternate between two hardware barriers: the control warp may arrive for
+// window i+1 while the compute warps are still gathering at the barrier of window i.
+__device__ __forceinline__ uint32_t window_barrier(uint32_t i) { return (i & 1u) ? kBarWindowOdd : kBarWindow; }
 
 __device__ __forceinline__ void bar_sync(uint32_t id, uint32_t threads)
 {
@@ -311,27 +320,44 @@ __device__ __forceinline__ void bar_arrive(uint32_t id, uint32_t threads)
     __threadfence_block();                                        // this thread's shared-memory writes first
     asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
 
-// Quantize + pack one window whose groups all have width B (no clamp needed): no per-chunk
-// decisions, packed position computed from the element index alone.
-template <typename KEYS, int CHUNKS, int B>
-__device__ __forceinline__ void quantize_uniform(const float (&x)[CHUNKS][8], const GroupRec *s_grp, uint32_t log2G,
-                                                 uint32_t e0, uint64_t blk0, const KEYS &keys, unsigned char *s_out)
+// Quantize + pack CHUNKS chunks that all have width B, with per-chunk (min, 1/scale) in
+// registers: no per-chunk decisions, packed position computed from the element index alone.
+template <typename KEYS, int CHUNKS, int B, bool CLAMP>
+__device__ __forceinline__ void quantize_uniform(const float (&x)[CHUNKS][8], const float (&mn)[CHUNKS],
+                                                 const float (&inv)[CHUNKS], uint32_t e0, uint64_t blk0, const KEYS &keys,
+                                                 unsigned char *s_out)
 {
     unsigned char *const out = s_out + (e0 >> 3) * B;
 #pragma unroll
     for (int c = 0; c < CHUNKS; c++) {
-        const float2 mi = *reinterpret_cast<const float2 *>(&s_grp[(e0 + 256u * c) >> log2G]);   // mn, inv
         uint32_t o[4];
         const uint64_t blk = blk0 + 32u * c;
         philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), keys, o);
         uint32_t w0, w1;
-        quantize8<B, false>(x[c], mi.x, mi.y, o, w0, w1);
+        quantize8<B, CLAMP>(x[c], mn[c], inv[c], o, w0, w1);
         unsigned char *p = out + 32 * B * c;
         if (B == 1) *p = (unsigned char)w0;
         else if (B == 2) *reinterpret_cast<uint16_t *>(p) = (uint16_t)w0;
         else if (B == 4) *reinterpret_cast<uint32_t *>(p) = w0;
         else *reinterpret_cast<uint2 *>(p) = make_uint2(w0, w1);
+    }
+}
+
+template <typename KEYS, int CHUNKS, bool CLAMP>
+__device__ __forceinline__ void quantize_uniform_b(uint32_t b, const float (&x)[CHUNKS][8], const float (&mn)[CHUNKS],
+                                                   const float (&inv)[CHUNKS], uint32_t e0, uint64_t blk0, const KEYS &keys,
+                                                   unsigned char *s_out)
+{
+    switch (b) {
+    case 1: quantize_uniform<KEYS, CHUNKS, 1, CLAMP>(x, mn, inv, e0, blk0, keys, s_out); break;
+    case 2: quantize_uniform<KEYS, CHUNKS, 2, CLAMP>(x, mn, inv, e0, blk0, keys, s_out); break;
+    case 4: quantize_uniform<KEYS, CHUNKS, 4, CLAMP>(x, mn, inv, e0, blk0, keys, s_out); break;
+    default: quantize_uniform<KEYS, CHUNKS, 8, CLAMP>(x, mn, inv, e0, blk0, keys, s_out); break;
     }
 }
 
@@ -341,13 +367,13 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
 {
     constexpr uint32_t WE = kThreads * kLaneElems * CHUNKS;
 
-    extern __shared__ __align__(128) unsigned char smem[];       // [stage | out0 | out1 | group arrays]
+    extern __shared__ __align__(128) unsigned char smem[];       // [stage | packed-bytes buffers | group arrays]
     __shared__ uint32_t s_wtot[kComputeWarps];
-    __shared__ __align__(8) uint64_t s_full;                     // mbarrier: staged window has landed
-    __shared__ uint32_t s_next;                                  // ticket of the staged window
-    __shared__ uint32_t s_lost;                                  // a staged copy did not land in time
-    __shared__ WindowInfo s_win[2];
-    __shared__ uint32_t s_slow[2];                               // a group of the window needs the clamped quantizer
+    __shared__ __align__(8) uint64_t s_full, s_cons, s_done;     // mbarriers
+    __shared__ uint32_t s_next[2];                               // ticket of window i at slot i & 1
+    __shared__ uint32_t s_lost;                                  // a bounded wait ran out
+    __shared__ uint32_t s_kmin[3], s_kmax[3];                    // extremes of the separation test, slot i % 3
+    __shared__ uint32_t s_tot[4];                                // packed bytes of window i at slot i & 3
 
     unsigned char *const s_stage = smem;
     float *const s_umn = reinterpret_cast<float *>(smem + a.lay.umn);
@@ -357,62 +383,78 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     GroupRec *const s_grp = reinterpret_cast<GroupRec *>(smem + a.lay.grp);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t G = a.G, log2G = a.log2G;
+    const uint32_t G = a.G, log2G = a.log2G, nbuf = a.nbuf;
 
-    // Control lane: takes a ticket and starts the bulk copy of that window into the stage.
-    auto stage_next = [&]() -> uint32_t {
-        const uint32_t t = atomicAdd(&a.hdr->ticket, 1u);
-        if (t < a.total_windows) {
-            const TensorDesc &nd = a.t[BATCH ? find_tensor(a, t) : 0u];
-            const uint64_t base = (uint64_t)(t - nd.first_window) * WE;
-            const uint64_t left = nd.numel - base;
-            const uint32_t bytes = (uint32_t)(left < WE ? left : WE) * Elem<T>::kBytes;
-            mbar_expect_tx(&s_full, bytes);
-            bulk_load(s_stage, reinterpret_cast<const char *>(nd.in) + base * Elem<T>::kBytes, bytes, &s_full);
+    auto record_error = [&](unsigned code, uint32_t window, unsigned site) {
+        if (atomicCAS(&a.hdr->status, 0u, code) == 0u) {
+            a.hdr->fail_window = window;
+            a.hdr->fail_site = site;
         }
-        s_next = t;
-        return t;
     };
-    auto record_error = [&](unsigned code, uint32_t window) {
-        if (atomicCAS(&a.hdr->status, 0u, code) == 0u) a.hdr->fail_window = window;
+    // Control lane: start the bulk copy of window `t` into the stage.
+    auto stage_window = [&](uint32_t t) {
+        const TensorDesc &nd = a.t[BATCH ? find_tensor(a, t) : 0u];
+        const uint64_t base = (uint64_t)(t - nd.first_window) * WE;
+        const uint64_t left = nd.numel - base;
+        const uint32_t bytes = (uint32_t)(left < WE ? left : WE) * Elem<T>::kBytes;
+        mbar_expect_tx(&s_full, bytes);
+        bulk_load(s_stage, reinterpret_cast<const char *>(nd.in) + base * Elem<T>::kBytes, bytes, &s_full);
     };
 
     if (tid == kThreads) {
         mbar_init(&s_full, 1);
+        mbar_init(&s_cons, kComputeWarps);
+        mbar_init(&s_done, kComputeWarps);
         s_lost = 0u;
-        s_slow[0] = s_slow[1] = 0u;
-        stage_next();
+        s_kmin[0] = s_kmin[1] = s_kmin[2] = 0xFFFFFFFFu;
+        s_kmax[0] = s_kmax[1] = s_kmax[2] = 0u;
+        const uint32_t t0 = atomicAdd(&a.hdr->ticket, 1u);
+        if (t0 < a.total_windows) stage_window(t0);
+        const uint32_t t1 = t0 < a.total_windows ? atomicAdd(&a.hdr->ticket, 1u) : 0xFFFFFFFFu;
+        s_next[0] = t0;
+        s_next[1] = t1;
     }
     __syncthreads();
-    uint32_t gw = s_next;
 
     if (warp == kComputeWarps) {
         // ============================================================ control warp
-        // Per window i: wait until the compute warps have consumed stage(i) and finished the
-        // packed bytes of window i-1; start the copy of window i+1; then, off the compute
-        // warps' critical path, find window i-1's byte offset by look-back, publish its
-        // inclusive prefix, and send its packed bytes to global memory.
-        bool have_prev = false;
+        // Round i: once the compute warps have consumed stage(i) (and finished packing window
+        // i-1), start the copy of window i+1, reserve the ticket of window i+2 and arrive at the
+        // window barrier of i+1; then, off the compute warps' critical path, find window i-1's
+        // byte offset by look-back, publish its inclusive prefix and send its packed bytes to
+        // global memory with one bulk store.
+        uint32_t t_cur = s_next[0], t_nxt = s_next[1];            // tickets of windows i and i+1
+        if (t_cur < a.total_windows) bar_arrive(window_barrier(0), kCompressThreads);
+        bool have_prev = false, lost = false;
         uint32_t p_gw = 0;
-        for (uint32_t iter = 0;; iter++) {
-            const bool valid = gw < a.total_windows;
-            bar_sync(kBarStage, kCompressThreads);
-            const bool lost = s_lost != 0u;
-            uint32_t next = 0xFFFFFFFFu;
+        for (uint32_t i = 0;; i++) {
+            const bool valid = t_cur < a.total_windows;
+            // compute warps: stage(i) consumed and window i-1 packed; after the last window they
+            // signal on a barrier of its own (they may get there before this round starts, and a
+            // parity wait must never be two phases behind)
+            if (!(valid ? mbar_wait_bounded(&s_cons, i & 1u) : mbar_wait_bounded(&s_done, 0u))) {
+                s_lost = 1u;
+                if (lane == 0) record_error(DAF_ERR_TIMEOUT, t_cur, 2u + 16u * i);
+            }
+            lost = lost || (s_lost != 0u);
+            uint32_t t_nn = 0xFFFFFFFFu;                          // ticket of window i+2
             if (valid) {
+                const bool nxt_valid = !lost && t_nxt < a.total_windows;
                 if (lane == 0) {
-                    if (!lost) stage_next();
-                    else s_next = 0xFFFFFFFFu;
-                    bulk_store_wait_read();                       // the buffer window i+1 will be packed into is free again
+                    if (nxt_valid) {
+                        stage_window(t_nxt);
+                        t_nn = atomicAdd(&a.hdr->ticket, 1u);
+                    }
+                    s_next[i & 1u] = t_nn;                        // slot of window i+2
                 }
-                __syncwarp();
-                next = lost ? 0xFFFFFFFFu : s_next;
-                bar_arrive(kBarWidths, kCompressThreads);
+                t_nn = __shfl_sync(0xFFFFFFFFu, t_nn, 0);
+                if (!nxt_valid) t_nxt = 0xFFFFFFFFu;
+                if (nbuf >= 3 && nxt_valid) bar_arrive(window_barrier(i + 1u), kCompressThreads);
             }
             if (have_prev) {
                 const TensorDesc &pd = a.t[BATCH ? find_tensor(a, p_gw) : 0u];
-                const uint32_t p_total = s_win[(iter & 1u) ^ 1u].total;
-                const unsigned char *src = smem + a.lay.out0 + ((iter & 1u) ^ 1u) * a.lay.out_stride;
+                const uint32_t p_total = s_tot[(i - 1u) & 3u];
+                const unsigned char *src = smem + a.lay.out0 + ((i - 1u) % nbuf) * a.lay.out_stride;
                 uint64_t excl = 0;
                 int state = 1;
                 if (p_gw != pd.first_window) {
@@ -431,28 +473,30 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                     skip = excl + p_total > pd.capacity;
                 }
                 if (skip) {
-                    if (lane == 0) record_error(state == -2 ? DAF_ERR_TIMEOUT : DAF_ERR_CAPACITY, p_gw);
+                    if (lane == 0) record_error(state == -2 ? DAF_ERR_TIMEOUT : DAF_ERR_CAPACITY, p_gw, state == 1 ? 5u : (state == -2 ? 3u : 4u));
                 } else if (a.bulk_store) {
-                    if (lane == 0 && p_total) bulk_store(pd.packed + excl, src, p_total);
+                    if (lane == 0 && p_total) {
+                        bulk_store(pd.packed + excl, src, p_total);
+                        bulk_store_wait_read();                   // the buffer may be rewritten from now on
+                    }
                 } else {                                          // groups of 32 / 64: windows are only 4-byte aligned
                     uint32_t *dst = reinterpret_cast<uint32_t *>(pd.packed + excl);
                     const uint32_t *s32 = reinterpret_cast<const uint32_t *>(src);
-                    for (uint32_t i = lane; i < (p_total >> 2); i += 32) dst[i] = s32[i];
+                    for (uint32_t k = lane; k < (p_total >> 2); k += 32) dst[k] = s32[k];
                 }
+                __syncwarp();
             }
+            if (valid && nbuf < 3 && t_nxt < a.total_windows) bar_arrive(window_barrier(i + 1u), kCompressThreads);
             if (!valid) break;
             if (lost) {
-                if (lane == 0) {
-                    record_error(DAF_ERR_TIMEOUT, gw);
-                    st_relaxed_u64(a.flags + gw, kFlagPoison << kFlagShift);
-                    mbar_wait_bounded(&s_full, iter & 1u);        // one more bounded chance for the lost copy
-                }
+                if (lane == 0) st_relaxed_u64(a.flags + t_cur, kFlagPoison << kFlagShift);
                 have_prev = false;
             } else {
                 have_prev = true;
-                p_gw = gw;
+                p_gw = t_cur;
             }
-            gw = next;
+            t_cur = t_nxt;
+            t_nxt = t_nn;
         }
         if (lane == 0) bulk_store_wait_all();
         return;
@@ -460,208 +504,271 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
 
     // ================================================================ compute warps
     const uint32_t e0 = (uint32_t)(warp * CHUNKS * 256 + lane * 8);    // this lane's first element of chunk 0
-    for (uint32_t iter = 0; gw < a.total_windows; iter++) {
-        unsigned char *const s_out = smem + a.lay.out0 + (iter & 1u) * a.lay.out_stride;
+    const uint32_t lpu = (G < 256u ? G : 256u) >> 3;              // lanes per unit
+    const bool local = G <= 256u * CHUNKS;                        // every group lives inside one warp's chunks
+    uint32_t gw = s_next[0];
+    uint32_t i = 0;
+    for (; gw < a.total_windows; i++) {
+        unsigned char *const s_out = smem + a.lay.out0 + (i % nbuf) * a.lay.out_stride;
         const TensorDesc &td = a.t[BATCH ? find_tensor(a, gw) : 0u];
         const uint32_t w = gw - td.first_window;
         const uint64_t wbase = (uint64_t)w * WE;
         const uint64_t left = td.numel - wbase;
         const uint32_t n_elems = left < WE ? (uint32_t)left : WE;
         const uint32_t n = n_elems >> log2G;                      // groups in this window
-        const uint32_t owners = (n + 31u) >> 5;                   // warps that own group records
+        const uint64_t g0 = wbase >> log2G;                       // first group of the window in the tensor
+
+        // Budget arithmetic of the window: precomputed on the host for full windows.
+        uint32_t ell = a.full_ell, rem = a.full_rem, rem_after = a.full_rem_after;
+        if (n != a.n_max) {
+            const uint64_t Tbits = ((uint64_t)a.beta_q8 * n) >> 8;        // bit units of the window
+            rem = (uint32_t)(Tbits - (uint64_t)a.S[0] * n);
+            ell = 0;                                              // largest level every group can be raised to
+            while (ell + 1 < a.m && (a.S[ell + 1] - a.S[0]) * n <= rem) ell++;
+            rem_after = rem - (a.S[ell] - a.S[0]) * n;
+        }
+        const bool all_max = (ell + 1 == a.m);
+        // the best raise of level ell does not fit: the outcome is uniform iff the levels separate
+        const bool need_sep = !all_max && rem_after < a.cost[ell];
+        // Fast path candidates: full window, stochastic rounding, groups local to a warp.
+        const bool fast_ok = local && n_elems == WE && !a.nearest && (all_max || need_sep);
+        const bool test_sep = fast_ok && need_sep && ell > 0;
 
         // ---------------------------------------------------------------- staged window -> registers, unit min/max
-        float x[CHUNKS][8];
-        if (!mbar_wait_bounded(&s_full, iter & 1u)) s_lost = 1u;
-        if (G >= 256u) load_and_reduce<T, CHUNKS, 32>(s_stage, warp, lane, x, s_umn, s_umx);
-        else if (G == 128u) load_and_reduce<T, CHUNKS, 16>(s_stage, warp, lane, x, s_umn, s_umx);
-        else if (G == 64u) load_and_reduce<T, CHUNKS, 8>(s_stage, warp, lane, x, s_umn, s_umx);
-        else load_and_reduce<T, CHUNKS, 4>(s_stage, warp, lane, x, s_umn, s_umx);
+        float x[CHUNKS][8], lo[CHUNKS], hi[CHUNKS];
+        if (!mbar_wait_bounded(&s_full, i & 1u)) {
+            s_lost = 1u;
+            if (lane == 0) record_error(DAF_ERR_TIMEOUT, gw, 1u + 16u * i);
+        }
+        if (lpu == 32u) load_and_reduce<T, CHUNKS, 32>(s_stage, warp, lane, x, lo, hi, s_umn, s_umx);
+        else if (lpu == 16u) load_and_reduce<T, CHUNKS, 16>(s_stage, warp, lane, x, lo, hi, s_umn, s_umx);
+        else if (lpu == 8u) load_and_reduce<T, CHUNKS, 8>(s_stage, warp, lane, x, lo, hi, s_umn, s_umx);
+        else load_and_reduce<T, CHUNKS, 4>(s_stage, warp, lane, x, lo, hi, s_umn, s_umx);
 
-        // ---------------------------------------------------------------- widths of the window (owner warps only)
-        if ((uint32_t)warp < owners) {
-            bar_sync(kBarStage, kCompressThreads);                // every warp's unit min / max is visible
-            const uint32_t m = a.m, n_max = a.n_max;
-            const uint64_t g0 = wbase >> log2G;                   // first group of the window in the tensor
-            // Budget arithmetic of the window: precomputed on the host for full windows.
-            uint32_t ell = a.full_ell, rem = a.full_rem, rem_after = a.full_rem_after;
-            if (n != n_max) {
-                const uint64_t Tbits = ((uint64_t)a.beta_q8 * n) >> 8;    // bit units of the window
-                rem = (uint32_t)(Tbits - (uint64_t)a.S[0] * n);
-                ell = 0;                                          // largest level every group can be raised to
-                while (ell + 1 < m && (a.S[ell + 1] - a.S[0]) * n <= rem) ell++;
-                rem_after = rem - (a.S[ell] - a.S[0]) * n;
-            }
-            const bool all_max = (ell + 1 == m);
-            // the best raise of level ell does not fit: the outcome is uniform iff the levels separate
-            const bool need_sep = !all_max && rem_after < a.cost[ell];
-            const bool mine = (uint32_t)tid < n;
-            if (tid == 0) s_slow[(iter & 1u) ^ 1u] = 0u;          // reset the flag of the next window
-
-            // range of this thread's group
-            float mn = 0.0f, R = 0.0f;
-            if (mine) {
-                float mx;
-                if (G > 256u) {
-                    const uint32_t r = G >> 8;
-                    mn = s_umn[tid * r];
-                    mx = s_umx[tid * r];
-                    for (uint32_t j = 1; j < r; j++) {
-                        mn = fmin2(mn, s_umn[tid * r + j]);
-                        mx = fmax2(mx, s_umx[tid * r + j]);
-                    }
-                } else {
-                    mn = s_umn[tid];
-                    mx = s_umx[tid];
+        float R[CHUNKS];
+        if (fast_ok) {
+            // groups of 512 / 1024 span 2 / 4 chunks of this warp
+            if (G == 512u) {
+#pragma unroll
+                for (int c = 0; c + 1 < CHUNKS; c += 2) {
+                    lo[c] = lo[c + 1] = fmin2(lo[c], lo[c + 1]);
+                    hi[c] = hi[c + 1] = fmax2(hi[c], hi[c + 1]);
                 }
-                R = __fsub_rn(mx, mn);
-                if (R < 0x1p-118f) R = 0.0f;                      // degenerate group: constant
+            } else if (G == 1024u && CHUNKS == 4) {
+                const float l = fmin2(fmin2(lo[0], lo[1]), fmin2(lo[2], lo[3]));
+                const float h = fmax2(fmax2(hi[0], hi[1]), fmax2(hi[2], hi[3]));
+#pragma unroll
+                for (int c = 0; c < CHUNKS; c++) {
+                    lo[c] = l;
+                    hi[c] = h;
+                }
             }
-
-            // bit choice
-            uint32_t level = ell;
-            bool uniform = all_max || need_sep;
-            if (need_sep && ell > 0) {
-                // Uniform outcome: every raise below level ell sorts ahead of every raise from
-                // level ell upward (ties go to the lower level), they all fit, the next does not.
-                // Each owner warp evaluates the test over all groups itself (no exchange needed).
+#pragma unroll
+            for (int c = 0; c < CHUNKS; c++) {
+                R[c] = __fsub_rn(hi[c], lo[c]);
+                if (R[c] < 0x1p-118f) R[c] = 0.0f;                // degenerate group: constant
+            }
+            if (test_sep) {
+                // separation test of the uniform outcome: min over groups of the key of the last
+                // raise taken, max over groups of the key of the first raise not taken
                 const float v_lo = a.v[ell - 1], v_hi = a.v[ell];
                 uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
-                if (owners == 1) {
-                    if (mine) {
-                        kmin = __float_as_uint(__fmul_rn(R, v_lo));
-                        kmax = __float_as_uint(__fmul_rn(R, v_hi));
-                    }
-                } else {                                          // groups of at most 256: one unit per group
-                    for (uint32_t g = lane; g < n; g += 32) {
-                        float Rg = __fsub_rn(s_umx[g], s_umn[g]);
-                        if (Rg < 0x1p-118f) Rg = 0.0f;
-                        kmin = min(kmin, __float_as_uint(__fmul_rn(Rg, v_lo)));
-                        kmax = max(kmax, __float_as_uint(__fmul_rn(Rg, v_hi)));
-                    }
-                }
-                kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
-                kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
-                uniform = kmin >= kmax;
-            }
-            uint32_t size = 0, b = 0, incl = 0, total = 0, before = 0;
-            if (uniform) {
-                b = a.S[ell];
-                size = (G >> 3) * b;
-                incl = (uint32_t)(tid + 1) * size;                // group g starts at g * size
-                total = n * size;
-            } else {
-                // General case.  For each candidate (group g, raise k) add up the cost of all
-                // candidates that sort at or ahead of it (key descending, level ascending, group
-                // ascending); the candidate is accepted iff that total fits in the budget.
-                if (mine) {
 #pragma unroll
-                    for (int k = 0; k < kMaxLevels - 1; k++) {
-                        s_key[k * n_max + tid] = __float_as_uint(__fmul_rn(R, a.v[k]));
-                        s_cum[k * n_max + tid] = 0u;
-                    }
+                for (int c = 0; c < CHUNKS; c++) {
+                    kmin = min(kmin, __float_as_uint(__fmul_rn(R[c], v_lo)));
+                    kmax = max(kmax, __float_as_uint(__fmul_rn(R[c], v_hi)));
                 }
-                if (owners > 1) bar_sync(kBarOwners, owners * 32u);
-                else __syncwarp();
-                const uint32_t nl = m - 1;
-                const uint32_t items = n * nl * nl;
-                for (uint32_t it = tid; it < items; it += owners * 32u) {
-                    const uint32_t g = it % n, kk = it / n;
-                    const uint32_t k = kk / nl, k2 = kk % nl;
-                    const uint32_t kg = s_key[k * n_max + g];
-                    const uint32_t *row = s_key + k2 * n_max;
-                    uint32_t cnt = 0;
-                    if (k2 < k) {
-                        for (uint32_t h = 0; h < n; h++) cnt += (row[h] >= kg);
-                    } else if (k2 > k) {
-                        for (uint32_t h = 0; h < n; h++) cnt += (row[h] > kg);
-                    } else {
-                        for (uint32_t h = 0; h < n; h++) cnt += (row[h] > kg) || (row[h] == kg && h <= g);
-                    }
-                    atomicAdd(&s_cum[k * n_max + g], cnt * a.cost[k2]);
+                if (lpu != 32u) {
+                    kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+                    kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
                 }
-                if (owners > 1) bar_sync(kBarOwners, owners * 32u);
-                else __syncwarp();
-                level = 0;
+                if (lane == 0) {
+                    atomicMin(&s_kmin[i % 3u], kmin);
+                    atomicMax(&s_kmax[i % 3u], kmax);
+                }
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_cons);                      // stage consumed, previous window packed
+
+        // ---------------------------------------------------------------- the one meeting point per window
+        bar_sync(window_barrier(i), kCompressThreads);
+        const uint32_t gw_next = s_next[(i + 1u) & 1u];
+        if (tid == 0) {
+            s_kmin[(i + 2u) % 3u] = 0xFFFFFFFFu;
+            s_kmax[(i + 2u) % 3u] = 0u;
+        }
+        if (s_lost != 0u) break;
+        const bool uniform = fast_ok && (!test_sep || s_kmin[i % 3u] >= s_kmax[i % 3u]);
+        const uint64_t blk0 = ((td.elem_base + wbase) >> 3) + (e0 >> 3);
+
+        if (uniform) {
+            // -------------------------------------------------------------- every group gets width S[ell]
+            const uint32_t b = a.S[ell];
+            const float Lf = (float)((1u << b) - 1u);
+            // lane j of a unit works out (scale, 1/scale) of chunk j's group, then the unit shares them
+            const int j = lane & (int)(lpu - 1u), sb = lane - j;
+            float Rj = 0.0f, mnj = 0.0f;
+#pragma unroll
+            for (int c = 0; c < CHUNKS; c++)
+                if (j == c) {
+                    Rj = R[c];
+                    mnj = lo[c];
+                }
+            const float scale_j = Rj > 0.0f ? __fdiv_rn(Rj, Lf) : 0.0f;
+            const float inv_j = Rj > 0.0f ? __fdiv_rn(Lf, Rj) : 0.0f;
+            if (j < CHUNKS) {
+                const uint32_t eu = (uint32_t)((warp * CHUNKS + j) * 256 + sb * 8);   // first element of the unit
+                if ((eu & (G - 1u)) == 0u) {                      // the unit opens a group: write its metadata
+                    const uint64_t g = g0 + (eu >> log2G);
+                    td.bits[g] = (uint8_t)b;
+                    td.mn[g] = mnj;
+                    td.scale[g] = scale_j;
+                }
+            }
+            float inv[CHUNKS];
+#pragma unroll
+            for (int c = 0; c < CHUNKS; c++) inv[c] = __shfl_sync(0xFFFFFFFFu, inv_j, sb + c);
+            // 1/scale not a normal number (range beyond 2^126 * L): the careful quantizer clamps
+            const bool careful = __any_sync(0xFFFFFFFFu, Rj > 0.0f && inv_j < 0x1p-126f) != 0;
+            if (tid == 0) {
+                const uint32_t total = n * (G >> 3) * b;
+                const bool first = (gw == td.first_window);
+                st_relaxed_u64(a.flags + gw, ((first ? kFlagPrefix : kFlagAggregate) << kFlagShift) | total);
+                s_tot[i & 3u] = total;
+            }
+            if (BATCH) {
+                const PhiloxSeedKeys sk{(uint32_t)td.seed, (uint32_t)(td.seed >> 32)};
+                if (careful) quantize_uniform_b<PhiloxSeedKeys, CHUNKS, true>(b, x, lo, inv, e0, blk0, sk, s_out);
+                else quantize_uniform_b<PhiloxSeedKeys, CHUNKS, false>(b, x, lo, inv, e0, blk0, sk, s_out);
+            } else {
+                if (careful) quantize_uniform_b<PhiloxKeys, CHUNKS, true>(b, x, lo, inv, e0, blk0, a.keys, s_out);
+                else quantize_uniform_b<PhiloxKeys, CHUNKS, false>(b, x, lo, inv, e0, blk0, a.keys, s_out);
+            }
+        } else {
+            // -------------------------------------------------------------- general bit choice (owner warps), then a generic pass
+            const uint32_t owners = (n + 31u) >> 5;               // warps that own group records
+            if ((uint32_t)warp < owners) {
+                const uint32_t m = a.m, n_max = a.n_max;
+                const bool mine = (uint32_t)tid < n;
+                float mn = 0.0f, Rg = 0.0f;
                 if (mine) {
-                    for (uint32_t k = 0; k + 1 < m; k++) level += (s_cum[k * n_max + tid] <= rem);
+                    float mx;
+                    if (G > 256u) {
+                        const uint32_t r = G >> 8;
+                        mn = s_umn[tid * r];
+                        mx = s_umx[tid * r];
+                        for (uint32_t k = 1; k < r; k++) {
+                            mn = fmin2(mn, s_umn[tid * r + k]);
+                            mx = fmax2(mx, s_umx[tid * r + k]);
+                        }
+                    } else {
+                        mn = s_umn[tid];
+                        mx = s_umx[tid];
+                    }
+                    Rg = __fsub_rn(mx, mn);
+                    if (Rg < 0x1p-118f) Rg = 0.0f;                // degenerate group: constant
+                }
+                uint32_t level = ell;
+                bool same = all_max;                              // every group ends at level ell
+                if (!all_max) {
+                    if (mine) {
+#pragma unroll
+                        for (int k = 0; k < kMaxLevels - 1; k++) {
+                            s_key[k * n_max + tid] = __float_as_uint(__fmul_rn(Rg, a.v[k]));
+                            s_cum[k * n_max + tid] = 0u;
+                        }
+                    }
+                    if (owners > 1) bar_sync(kBarOwners, owners * 32u);
+                    else __syncwarp();
+                    if (need_sep) {
+                        // Uniform outcome: every raise below level ell sorts ahead of every raise from
+                        // level ell upward (ties go to the lower level), they all fit, the next does not.
+                        same = true;
+                        if (ell > 0) {
+                            uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+                            for (uint32_t g = lane; g < n; g += 32) {
+                                kmin = min(kmin, s_key[(ell - 1) * n_max + g]);
+                                kmax = max(kmax, s_key[ell * n_max + g]);
+                            }
+                            kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+                            kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+                            same = kmin >= kmax;
+                        }
+                    }
+                    if (!same) {
+                        // For each candidate (group g, raise k) add up the cost of all candidates that
+                        // sort at or ahead of it (key descending, level ascending, group ascending);
+                        // the candidate is accepted iff that total fits in the budget.
+                        const uint32_t nl = m - 1;
+                        const uint32_t items = n * nl * nl;
+                        for (uint32_t it = tid; it < items; it += owners * 32u) {
+                            const uint32_t g = it % n, kk = it / n;
+                            const uint32_t k = kk / nl, k2 = kk % nl;
+                            const uint32_t kg = s_key[k * n_max + g];
+                            const uint32_t *row = s_key + k2 * n_max;
+                            uint32_t cnt = 0;
+                            if (k2 < k) {
+                                for (uint32_t h = 0; h < n; h++) cnt += (row[h] >= kg);
+                            } else if (k2 > k) {
+                                for (uint32_t h = 0; h < n; h++) cnt += (row[h] > kg);
+                            } else {
+                                for (uint32_t h = 0; h < n; h++) cnt += (row[h] > kg) || (row[h] == kg && h <= g);
+                            }
+                            atomicAdd(&s_cum[k * n_max + g], cnt * a.cost[k2]);
+                        }
+                        if (owners > 1) bar_sync(kBarOwners, owners * 32u);
+                        else __syncwarp();
+                        level = 0;
+                        if (mine)
+                            for (uint32_t k = 0; k + 1 < m; k++) level += (s_cum[k * n_max + tid] <= rem);
+                    }
+                }
+                uint32_t size = 0, b = 0;
+                float inv = 0.0f;
+                if (mine) {
                     b = a.S[level];
+                    const float Lf = (float)((1u << b) - 1u);
+                    const float scale = Rg > 0.0f ? __fdiv_rn(Rg, Lf) : 0.0f;
+                    inv = Rg > 0.0f ? __fdiv_rn(Lf, Rg) : 0.0f;
+                    td.bits[g0 + tid] = (uint8_t)b;
+                    td.mn[g0 + tid] = mn;
+                    td.scale[g0 + tid] = scale;
                     size = (G >> 3) * b;
                 }
                 // byte offset of each group inside the window: exclusive scan of the sizes
-                incl = size;
+                uint32_t incl = size;
 #pragma unroll
                 for (int off = 1; off < 32; off <<= 1) {
                     const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, off);
                     if (lane >= off) incl += y;
                 }
-                total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31), before = 0;
                 if (owners > 1) {
                     if (lane == 0) s_wtot[warp] = total;
                     bar_sync(kBarOwners, owners * 32u);
                     total = 0;
-                    for (uint32_t i = 0; i < owners; i++) {
-                        const uint32_t t = s_wtot[i];
-                        if (i < (uint32_t)warp) before += t;
+                    for (uint32_t k = 0; k < owners; k++) {
+                        const uint32_t t = s_wtot[k];
+                        if (k < (uint32_t)warp) before += t;
                         total += t;
                     }
                 }
-            }
-
-            // group parameters and metadata
-            if (mine) {
-                const float Lf = (float)((1u << b) - 1u);
-                const float scale = R > 0.0f ? __fdiv_rn(R, Lf) : 0.0f;
-                const float inv = R > 0.0f ? __fdiv_rn(Lf, R) : 0.0f;
-                // 1/scale not a normal number: codes may need the clamp, take the careful path
-                if (R > 0.0f && inv < 0x1p-126f) s_slow[iter & 1u] = 1u;
-                td.bits[g0 + tid] = (uint8_t)b;
-                td.mn[g0 + tid] = mn;
-                td.scale[g0 + tid] = scale;
-                GroupRec rec;
-                rec.mn = mn;
-                rec.inv = inv;
-                rec.b = b;
-                rec.off = before + incl - size;
-                s_grp[tid] = rec;
-            }
-            if (tid == 0) {
-                // the window's byte count is known: publish it at once (a lost copy poisons it instead)
-                const bool first = (gw == td.first_window);
-                if (s_lost == 0u)
+                if (mine) {
+                    GroupRec rec;
+                    rec.mn = mn;
+                    rec.inv = inv;
+                    rec.b = b;
+                    rec.off = before + incl - size;
+                    s_grp[tid] = rec;
+                }
+                if (tid == 0) {
+                    const bool first = (gw == td.first_window);
                     st_relaxed_u64(a.flags + gw, ((first ? kFlagPrefix : kFlagAggregate) << kFlagShift) | total);
-                s_win[iter & 1u].total = total;
-                s_win[iter & 1u].fast_b = (uniform && n_elems == WE && !a.nearest) ? b : 0u;
-            }
-        } else {
-            bar_arrive(kBarStage, kCompressThreads);
-        }
-        bar_sync(kBarWidths, kCompressThreads);                   // group records, window info and s_next visible
-        const uint32_t gw_next = s_next;
-        const uint32_t fast_b = s_slow[iter & 1u] ? 0u : s_win[iter & 1u].fast_b;
-        if (s_lost != 0u) break;
-
-        // ---------------------------------------------------------------- quantize + pack into shared memory
-        const uint64_t blk0 = ((td.elem_base + wbase) >> 3) + (e0 >> 3);
-        if (fast_b != 0u) {
-            // one width for the whole (full) window, stochastic rounding, no clamp needed
-            if (BATCH) {
-                const PhiloxSeedKeys sk{(uint32_t)td.seed, (uint32_t)(td.seed >> 32)};
-                switch (fast_b) {
-                case 1: quantize_uniform<PhiloxSeedKeys, CHUNKS, 1>(x, s_grp, log2G, e0, blk0, sk, s_out); break;
-                case 2: quantize_uniform<PhiloxSeedKeys, CHUNKS, 2>(x, s_grp, log2G, e0, blk0, sk, s_out); break;
-                case 4: quantize_uniform<PhiloxSeedKeys, CHUNKS, 4>(x, s_grp, log2G, e0, blk0, sk, s_out); break;
-                default: quantize_uniform<PhiloxSeedKeys, CHUNKS, 8>(x, s_grp, log2G, e0, blk0, sk, s_out); break;
-                }
-            } else {
-                switch (fast_b) {
-                case 1: quantize_uniform<PhiloxKeys, CHUNKS, 1>(x, s_grp, log2G, e0, blk0, a.keys, s_out); break;
-                case 2: quantize_uniform<PhiloxKeys, CHUNKS, 2>(x, s_grp, log2G, e0, blk0, a.keys, s_out); break;
-                case 4: quantize_uniform<PhiloxKeys, CHUNKS, 4>(x, s_grp, log2G, e0, blk0, a.keys, s_out); break;
-                default: quantize_uniform<PhiloxKeys, CHUNKS, 8>(x, s_grp, log2G, e0, blk0, a.keys, s_out); break;
+                    s_tot[i & 3u] = total;
                 }
             }
-        } else {
+            bar_sync(kBarWidths, kThreads);                       // group records visible to all compute warps
 #pragma unroll
             for (int c = 0; c < CHUNKS; c++) {
                 const uint32_t e = e0 + 256u * c;
@@ -701,14 +808,15 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         if (a.bulk_store) fence_async_shared();                   // packed bytes visible to the bulk store issued later
         gw = gw_next;
     }
-    bar_arrive(kBarStage, kCompressThreads);                      // the last window's packed bytes are complete
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&s_done);                          // the last window is packed (or the loop was left)
 }
 
 // ------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------
 // Shared-memory carve-up for one launch configuration.
-static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint32_t window_cap_bytes)
+static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint32_t window_cap_bytes, uint32_t nbuf)
 {
     auto up = [](uint32_t v) { return (v + 127u) & ~127u; };
     const uint32_t n_max = we / G, units = we / (G < 256u ? G : 256u);
@@ -716,7 +824,7 @@ static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint
     uint32_t at = up(we * elem_bytes);
     l.out0 = at;
     l.out_stride = up(window_cap_bytes < 16u ? 16u : window_cap_bytes);
-    at += 2u * l.out_stride;
+    at += nbuf * l.out_stride;
     l.umn = at; at += up(4u * units);
     l.umx = at; at += up(4u * units);
     l.key = at; at += up(4u * (kMaxLevels - 1) * n_max);
@@ -790,7 +898,15 @@ template <int NT> static void fill_common(CompressArgs<NT> &a, const Plan &pl, c
         while (a.full_ell + 1 < pl.m && (pl.S[a.full_ell + 1] - pl.S[0]) * n <= a.full_rem) a.full_ell++;
         a.full_rem_after = a.full_rem - (pl.S[a.full_ell] - pl.S[0]) * n;
     }
-    a.lay = make_layout(pl.We, elem_bytes, pl.G, (uint32_t)((((uint64_t)pl.beta_q8 * pl.W) >> 8) * pl.G / 8));
+    // Three packed-bytes buffers keep the control warp entirely off the compute warps' path;
+    // fall back to two when three would not leave room for two CTAs per SM (227 KiB).
+    const uint32_t cap = (uint32_t)((((uint64_t)pl.beta_q8 * pl.W) >> 8) * pl.G / 8);
+    a.nbuf = 3;
+    a.lay = make_layout(pl.We, elem_bytes, pl.G, cap, 3);
+    if (2u * (a.lay.total + 2048u) > 227u * 1024u) {
+        a.nbuf = 2;
+        a.lay = make_layout(pl.We, elem_bytes, pl.G, cap, 2);
+    }
     for (int k = 0; k < kMaxLevels; k++) {
         a.S[k] = pl.S[k];
         a.cost[k] = pl.cost[k];
