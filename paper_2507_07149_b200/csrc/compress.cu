@@ -291,34 +291,26 @@ template <int NT> __device__ __forceinline__ uint32_t find_tensor(const Compress
     return lo;
 }
 
-// The CTA is 16 compute warps plus one control warp.
-//   barrier kBarWindow : the 16 compute warps meet once per window, after every warp has turned
-//                        its part of the staged window into registers and min / max; the control
-//                        warp only arrives there (it never makes the compute warps' wait longer
-//                        than its own work of the previous round), which also hands over the next
-//                        ticket and the guarantee that the packed-bytes buffer about to be
-//                        rewritten has left shared memory;
-//   barrier kBarWidths : compute warps only, used when a window needs the general bit choice;
-//   barrier kBarOwners : the warps that own group records in the general bit choice;
-//   mbarrier s_full    : the staged window has landed (bulk copy complete);
-//   mbarrier s_cons    : every compute warp has consumed the staged window and has finished
-//                        packing the previous window (16 arrivals);
-//   mbarrier s_done    : every compute warp has left its loop (16 arrivals, used once).
+// One persistent CTA per SM: 16 compute warps plus one control warp, synchronised only through
+// shared-memory mbarriers (every wait on them is bounded) except inside the general bit choice.
+//   s_full[s]  : the bulk copy into stage s has landed (or the control warp has marked the
+//                window behind it as "no more work");
+//   s_cons[s]  : all compute warps have moved stage s into registers and have finished packing
+//                the previous window (16 arrivals);
+//   s_exch     : all compute warps have contributed their part of a window's min / max test
+//                (16 arrivals) -- arrival and wait are split so that the exchange of window
+//                j+1 completes while window j is being quantized;
+//   s_wid      : the group records of a window that needed the general bit choice are ready;
+//   s_done     : all compute warps have left their loop.
+// Window j uses stage j & 1, packed-bytes buffer j % 3 and slot j & 3 of the small per-window
+// arrays.  The control warp owns tickets, bulk copies in, look-back and bulk stores out.
 constexpr int kComputeWarps = kWarps;
 constexpr int kCompressThreads = kThreads + 32;
-constexpr uint32_t kBarWindow = 1, kBarWidths = 2, kBarOwners = 3, kBarWindowOdd = 4;
-// Window barriers alternate between two hardware barriers: the control warp may arrive for
-// window i+1 while the compute warps are still gathering at the barrier of window i.
-__device__ __forceinline__ uint32_t window_barrier(uint32_t i) { return (i & 1u) ? kBarWindowOdd : kBarWindow; }
+constexpr uint32_t kBarOwners = 3;
 
 __device__ __forceinline__ void bar_sync(uint32_t id, uint32_t threads)
 {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
-}
-__device__ __forceinline__ void bar_arrive(uint32_t id, uint32_t threads)
-{
-    __threadfence_block();                                        // this thread's shared-memory writes first
-    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
 {
@@ -361,29 +353,37 @@ __device__ __forceinline__ void quantize_uniform_b(uint32_t b, const float (&x)[
     }
 }
 
+// Budget arithmetic of a window of n groups.
+struct Budget {
+    uint32_t ell;          // largest level every group can be raised to
+    uint32_t rem;          // bit units left after the smallest width
+    bool all_max;          // every group reaches the largest width
+    bool need_sep;         // the best raise of level ell does not fit: uniform iff the levels separate
+};
+
 template <typename T, int CHUNKS, bool BATCH>
-__global__ void __launch_bounds__(kCompressThreads, 2)
+__global__ void __launch_bounds__(kCompressThreads, 1)
 compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> a)
 {
     constexpr uint32_t WE = kThreads * kLaneElems * CHUNKS;
+    constexpr uint32_t kStageBytes = WE * Elem<T>::kBytes;
 
-    extern __shared__ __align__(128) unsigned char smem[];       // [stage | packed-bytes buffers | group arrays]
+    extern __shared__ __align__(128) unsigned char smem[];       // [stage 0 | stage 1 | packed x3 | group arrays]
+    __shared__ __align__(8) uint64_t s_full[2], s_cons[2], s_exch, s_wid, s_done;   // mbarriers
+    __shared__ uint32_t s_next[4];                               // ticket of window j
+    __shared__ uint32_t s_kmin[4], s_kmax[4], s_flag[4];         // per-window exchange: key extremes, "a wait ran out"
+    __shared__ uint32_t s_tot[4];                                // packed bytes of window j
     __shared__ uint32_t s_wtot[kComputeWarps];
-    __shared__ __align__(8) uint64_t s_full, s_cons, s_done;     // mbarriers
-    __shared__ uint32_t s_next[2];                               // ticket of window i at slot i & 1
-    __shared__ uint32_t s_lost;                                  // a bounded wait ran out
-    __shared__ uint32_t s_kmin[3], s_kmax[3];                    // extremes of the separation test, slot i % 3
-    __shared__ uint32_t s_tot[4];                                // packed bytes of window i at slot i & 3
+    __shared__ uint32_t s_lost;
 
-    unsigned char *const s_stage = smem;
-    float *const s_umn = reinterpret_cast<float *>(smem + a.lay.umn);
+    float *const s_umn = reinterpret_cast<float *>(smem + a.lay.umn);    // [2][units]
     float *const s_umx = reinterpret_cast<float *>(smem + a.lay.umx);
     uint32_t *const s_key = reinterpret_cast<uint32_t *>(smem + a.lay.key);   // [level][n_max]
     uint32_t *const s_cum = reinterpret_cast<uint32_t *>(smem + a.lay.cum);
-    GroupRec *const s_grp = reinterpret_cast<GroupRec *>(smem + a.lay.grp);
+    GroupRec *const s_grp = reinterpret_cast<GroupRec *>(smem + a.lay.grp);   // [2][n_max]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t G = a.G, log2G = a.log2G, nbuf = a.nbuf;
+    const uint32_t G = a.G, log2G = a.log2G;
 
     auto record_error = [&](unsigned code, uint32_t window, unsigned site) {
         if (atomicCAS(&a.hdr->status, 0u, code) == 0u) {
@@ -391,70 +391,92 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             a.hdr->fail_site = site;
         }
     };
-    // Control lane: start the bulk copy of window `t` into the stage.
-    auto stage_window = [&](uint32_t t) {
-        const TensorDesc &nd = a.t[BATCH ? find_tensor(a, t) : 0u];
-        const uint64_t base = (uint64_t)(t - nd.first_window) * WE;
-        const uint64_t left = nd.numel - base;
-        const uint32_t bytes = (uint32_t)(left < WE ? left : WE) * Elem<T>::kBytes;
-        mbar_expect_tx(&s_full, bytes);
-        bulk_load(s_stage, reinterpret_cast<const char *>(nd.in) + base * Elem<T>::kBytes, bytes, &s_full);
+    auto tensor_of = [&](uint32_t gw) -> const TensorDesc & { return a.t[BATCH ? find_tensor(a, gw) : 0u]; };
+    auto budget_of = [&](uint32_t n) {
+        Budget b;
+        uint32_t rem_after = a.full_rem_after;
+        b.ell = a.full_ell;
+        b.rem = a.full_rem;
+        if (n != a.n_max) {                                       // ragged last window: work it out here
+            const uint64_t Tbits = ((uint64_t)a.beta_q8 * n) >> 8;
+            b.rem = (uint32_t)(Tbits - (uint64_t)a.S[0] * n);
+            b.ell = 0;
+            while (b.ell + 1 < a.m && (a.S[b.ell + 1] - a.S[0]) * n <= b.rem) b.ell++;
+            rem_after = b.rem - (a.S[b.ell] - a.S[0]) * n;
+        }
+        b.all_max = (b.ell + 1 == a.m);
+        b.need_sep = !b.all_max && rem_after < a.cost[b.ell];
+        return b;
     };
-
-    if (tid == kThreads) {
-        mbar_init(&s_full, 1);
-        mbar_init(&s_cons, kComputeWarps);
-        mbar_init(&s_done, kComputeWarps);
-        s_lost = 0u;
-        s_kmin[0] = s_kmin[1] = s_kmin[2] = 0xFFFFFFFFu;
-        s_kmax[0] = s_kmax[1] = s_kmax[2] = 0u;
-        const uint32_t t0 = atomicAdd(&a.hdr->ticket, 1u);
-        if (t0 < a.total_windows) stage_window(t0);
-        const uint32_t t1 = t0 < a.total_windows ? atomicAdd(&a.hdr->ticket, 1u) : 0xFFFFFFFFu;
-        s_next[0] = t0;
-        s_next[1] = t1;
-    }
-    __syncthreads();
 
     if (warp == kComputeWarps) {
         // ============================================================ control warp
-        // Round i: once the compute warps have consumed stage(i) (and finished packing window
-        // i-1), start the copy of window i+1, reserve the ticket of window i+2 and arrive at the
-        // window barrier of i+1; then, off the compute warps' critical path, find window i-1's
-        // byte offset by look-back, publish its inclusive prefix and send its packed bytes to
-        // global memory with one bulk store.
-        uint32_t t_cur = s_next[0], t_nxt = s_next[1];            // tickets of windows i and i+1
-        if (t_cur < a.total_windows) bar_arrive(window_barrier(0), kCompressThreads);
-        bool have_prev = false, lost = false;
-        uint32_t p_gw = 0;
-        for (uint32_t i = 0;; i++) {
-            const bool valid = t_cur < a.total_windows;
-            // compute warps: stage(i) consumed and window i-1 packed; after the last window they
-            // signal on a barrier of its own (they may get there before this round starts, and a
-            // parity wait must never be two phases behind)
-            if (!(valid ? mbar_wait_bounded(&s_cons, i & 1u) : mbar_wait_bounded(&s_done, 0u))) {
-                s_lost = 1u;
-                if (lane == 0) record_error(DAF_ERR_TIMEOUT, t_cur, 2u + 16u * i);
+        // Control lane: publish the ticket of window j and start its bulk copy into stage j & 1,
+        // or complete the stage's barrier empty-handed when there is no such window.
+        auto issue = [&](uint32_t j, uint32_t t) {
+            s_next[j & 3u] = t;
+            uint64_t *bar = &s_full[j & 1u];
+            if (t < a.total_windows) {
+                const TensorDesc &nd = tensor_of(t);
+                const uint64_t base = (uint64_t)(t - nd.first_window) * WE;
+                const uint64_t left = nd.numel - base;
+                const uint32_t bytes = (uint32_t)(left < WE ? left : WE) * Elem<T>::kBytes;
+                mbar_expect_tx(bar, bytes);
+                bulk_load(smem + (j & 1u) * kStageBytes, reinterpret_cast<const char *>(nd.in) + base * Elem<T>::kBytes, bytes, bar);
+            } else {
+                mbar_arrive(bar);
             }
-            lost = lost || (s_lost != 0u);
-            uint32_t t_nn = 0xFFFFFFFFu;                          // ticket of window i+2
-            if (valid) {
-                const bool nxt_valid = !lost && t_nxt < a.total_windows;
-                if (lane == 0) {
-                    if (nxt_valid) {
-                        stage_window(t_nxt);
-                        t_nn = atomicAdd(&a.hdr->ticket, 1u);
-                    }
-                    s_next[i & 1u] = t_nn;                        // slot of window i+2
+        };
+        uint32_t t0 = 0xFFFFFFFFu, t1 = 0xFFFFFFFFu;              // tickets of windows r and r+1
+        if (lane == 0) {
+            mbar_init(&s_full[0], 1);
+            mbar_init(&s_full[1], 1);
+            mbar_init(&s_cons[0], kComputeWarps);
+            mbar_init(&s_cons[1], kComputeWarps);
+            mbar_init(&s_exch, kComputeWarps);
+            mbar_init(&s_wid, kComputeWarps);
+            mbar_init(&s_done, kComputeWarps);
+            s_lost = 0u;
+            for (int k = 0; k < 4; k++) {
+                s_kmin[k] = 0xFFFFFFFFu;
+                s_kmax[k] = 0u;
+                s_flag[k] = 0u;
+            }
+            t0 = atomicAdd(&a.hdr->ticket, 1u);
+            issue(0, t0);
+            if (t0 < a.total_windows) {
+                t1 = atomicAdd(&a.hdr->ticket, 1u);
+                issue(1, t1);
+            }
+        }
+        t0 = __shfl_sync(0xFFFFFFFFu, t0, 0);
+        t1 = __shfl_sync(0xFFFFFFFFu, t1, 0);
+        __syncthreads();
+
+        bool have_prev = false;
+        uint32_t p_gw = 0;
+        for (uint32_t r = 0;; r++) {
+            const bool valid = t0 < a.total_windows && s_lost == 0u;
+            // round r: window r is in registers once s_cons fires; after the last window (or a
+            // lost wait) the compute warps sign off on s_done instead
+            bool ok = valid ? mbar_wait_bounded(&s_cons[r & 1u], (r >> 1) & 1u) : mbar_wait_bounded(&s_done, 0u);
+            if (!ok) {
+                s_lost = 1u;
+                if (lane == 0) record_error(DAF_ERR_TIMEOUT, t0, 2u + 16u * r);
+            }
+            uint32_t t2 = 0xFFFFFFFFu;                            // ticket of window r+2
+            if (valid && ok) {
+                if (lane == 0 && t1 < a.total_windows) {
+                    if (s_lost == 0u) t2 = atomicAdd(&a.hdr->ticket, 1u);
+                    issue(r + 2u, t2);                            // stage r & 1 is free again
                 }
-                t_nn = __shfl_sync(0xFFFFFFFFu, t_nn, 0);
-                if (!nxt_valid) t_nxt = 0xFFFFFFFFu;
-                if (nbuf >= 3 && nxt_valid) bar_arrive(window_barrier(i + 1u), kCompressThreads);
+                t2 = __shfl_sync(0xFFFFFFFFu, t2, 0);
             }
             if (have_prev) {
-                const TensorDesc &pd = a.t[BATCH ? find_tensor(a, p_gw) : 0u];
-                const uint32_t p_total = s_tot[(i - 1u) & 3u];
-                const unsigned char *src = smem + a.lay.out0 + ((i - 1u) % nbuf) * a.lay.out_stride;
+                // window r-1 is packed: find its byte offset, publish its inclusive prefix, store it
+                const TensorDesc &pd = tensor_of(p_gw);
+                const uint32_t p_total = s_tot[(r - 1u) & 3u];
+                const unsigned char *src = smem + a.lay.out0 + ((r - 1u) % 3u) * a.lay.out_stride;
                 uint64_t excl = 0;
                 int state = 1;
                 if (p_gw != pd.first_window) {
@@ -473,7 +495,8 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                     skip = excl + p_total > pd.capacity;
                 }
                 if (skip) {
-                    if (lane == 0) record_error(state == -2 ? DAF_ERR_TIMEOUT : DAF_ERR_CAPACITY, p_gw, state == 1 ? 5u : (state == -2 ? 3u : 4u));
+                    if (lane == 0)
+                        record_error(state == -2 ? DAF_ERR_TIMEOUT : DAF_ERR_CAPACITY, p_gw, state == 1 ? 5u : (state == -2 ? 3u : 4u));
                 } else if (a.bulk_store) {
                     if (lane == 0 && p_total) {
                         bulk_store(pd.packed + excl, src, p_total);
@@ -485,193 +508,254 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                     for (uint32_t k = lane; k < (p_total >> 2); k += 32) dst[k] = s32[k];
                 }
                 __syncwarp();
-            }
-            if (valid && nbuf < 3 && t_nxt < a.total_windows) bar_arrive(window_barrier(i + 1u), kCompressThreads);
-            if (!valid) break;
-            if (lost) {
-                if (lane == 0) st_relaxed_u64(a.flags + t_cur, kFlagPoison << kFlagShift);
                 have_prev = false;
-            } else {
-                have_prev = true;
-                p_gw = t_cur;
             }
-            t_cur = t_nxt;
-            t_nxt = t_nn;
+            if (!valid || !ok) {
+                // leaving: windows this CTA still holds tickets for will never be published
+                if (lane == 0) {
+                    if (t0 < a.total_windows) st_relaxed_u64(a.flags + t0, kFlagPoison << kFlagShift);
+                    if (t1 < a.total_windows) st_relaxed_u64(a.flags + t1, kFlagPoison << kFlagShift);
+                    // bulk copies still in flight must land before the CTA goes away
+                    if (t0 < a.total_windows) mbar_wait_bounded(&s_full[r & 1u], (r >> 1) & 1u);
+                    if (t1 < a.total_windows) mbar_wait_bounded(&s_full[(r + 1u) & 1u], ((r + 1u) >> 1) & 1u);
+                }
+                break;
+            }
+            have_prev = true;
+            p_gw = t0;
+            t0 = t1;
+            t1 = t2;
         }
         if (lane == 0) bulk_store_wait_all();
         return;
     }
 
     // ================================================================ compute warps
+    __syncthreads();                                              // barriers initialised by the control warp
     const uint32_t e0 = (uint32_t)(warp * CHUNKS * 256 + lane * 8);    // this lane's first element of chunk 0
     const uint32_t lpu = (G < 256u ? G : 256u) >> 3;              // lanes per unit
+    const uint32_t units = WE >> (G < 256u ? log2G : 8u);         // units per window
     const bool local = G <= 256u * CHUNKS;                        // every group lives inside one warp's chunks
-    uint32_t gw = s_next[0];
-    uint32_t i = 0;
-    for (; gw < a.total_windows; i++) {
-        unsigned char *const s_out = smem + a.lay.out0 + (i % nbuf) * a.lay.out_stride;
-        const TensorDesc &td = a.t[BATCH ? find_tensor(a, gw) : 0u];
-        const uint32_t w = gw - td.first_window;
-        const uint64_t wbase = (uint64_t)w * WE;
+
+    // the window being quantized (registers) and how
+    float x[CHUNKS][8];
+    float q_mn[CHUNKS], q_inv[CHUNKS];                            // uniform windows: per-chunk min and 1/scale
+    uint32_t q_b = 0;                                             // uniform windows: the width; 0 = use the group records
+    bool q_careful = false;
+    uint32_t q_gw = 0, q_elems = 0;
+    uint32_t n_generic = 0;                                       // windows that took the general bit choice so far
+    bool my_lost = false;
+
+    for (uint32_t j = 0;; j++) {
+        // ---------------------------------------------------------------- window j has landed (or there is none)
+        if (!mbar_wait_bounded(&s_full[j & 1u], (j >> 1) & 1u)) {
+            my_lost = true;
+            s_lost = 1u;
+            if (lane == 0) record_error(DAF_ERR_TIMEOUT, 0u, 1u + 16u * j);
+        }
+        const uint32_t gw = my_lost ? 0xFFFFFFFFu : s_next[j & 3u];
+        const bool valid = gw < a.total_windows;
+        const unsigned char *stage = smem + (j & 1u) * kStageBytes;
+
+        // ---------------------------------------------------------------- min / max of window j, contribution to its exchange
+        const TensorDesc &td = tensor_of(valid ? gw : 0u);
+        const uint64_t wbase = (uint64_t)(gw - td.first_window) * WE;
         const uint64_t left = td.numel - wbase;
         const uint32_t n_elems = left < WE ? (uint32_t)left : WE;
-        const uint32_t n = n_elems >> log2G;                      // groups in this window
-        const uint64_t g0 = wbase >> log2G;                       // first group of the window in the tensor
-
-        // Budget arithmetic of the window: precomputed on the host for full windows.
-        uint32_t ell = a.full_ell, rem = a.full_rem, rem_after = a.full_rem_after;
-        if (n != a.n_max) {
-            const uint64_t Tbits = ((uint64_t)a.beta_q8 * n) >> 8;        // bit units of the window
-            rem = (uint32_t)(Tbits - (uint64_t)a.S[0] * n);
-            ell = 0;                                              // largest level every group can be raised to
-            while (ell + 1 < a.m && (a.S[ell + 1] - a.S[0]) * n <= rem) ell++;
-            rem_after = rem - (a.S[ell] - a.S[0]) * n;
-        }
-        const bool all_max = (ell + 1 == a.m);
-        // the best raise of level ell does not fit: the outcome is uniform iff the levels separate
-        const bool need_sep = !all_max && rem_after < a.cost[ell];
+        const uint32_t n = n_elems >> log2G;                      // groups in window j
+        Budget bud = budget_of(valid ? n : a.n_max);
         // Fast path candidates: full window, stochastic rounding, groups local to a warp.
-        const bool fast_ok = local && n_elems == WE && !a.nearest && (all_max || need_sep);
-        const bool test_sep = fast_ok && need_sep && ell > 0;
-
-        // ---------------------------------------------------------------- staged window -> registers, unit min/max
-        float x[CHUNKS][8], lo[CHUNKS], hi[CHUNKS];
-        if (!mbar_wait_bounded(&s_full, i & 1u)) {
-            s_lost = 1u;
-            if (lane == 0) record_error(DAF_ERR_TIMEOUT, gw, 1u + 16u * i);
-        }
-        if (lpu == 32u) load_and_reduce<T, CHUNKS, 32>(s_stage, warp, lane, x, lo, hi, s_umn, s_umx);
-        else if (lpu == 16u) load_and_reduce<T, CHUNKS, 16>(s_stage, warp, lane, x, lo, hi, s_umn, s_umx);
-        else if (lpu == 8u) load_and_reduce<T, CHUNKS, 8>(s_stage, warp, lane, x, lo, hi, s_umn, s_umx);
-        else load_and_reduce<T, CHUNKS, 4>(s_stage, warp, lane, x, lo, hi, s_umn, s_umx);
-
-        float R[CHUNKS];
-        if (fast_ok) {
-            // groups of 512 / 1024 span 2 / 4 chunks of this warp
-            if (G == 512u) {
+        const bool fast_ok = local && n_elems == WE && !a.nearest && (bud.all_max || bud.need_sep);
+        const bool test_sep = fast_ok && bud.need_sep && bud.ell > 0;
+        float lo[CHUNKS], hi[CHUNKS];
+        if (valid) {
+            float y[CHUNKS][8];                                   // transient: only the min / max are kept
+            float *umn = s_umn + (j & 1u) * units, *umx = s_umx + (j & 1u) * units;
+            if (lpu == 32u) load_and_reduce<T, CHUNKS, 32>(stage, warp, lane, y, lo, hi, umn, umx);
+            else if (lpu == 16u) load_and_reduce<T, CHUNKS, 16>(stage, warp, lane, y, lo, hi, umn, umx);
+            else if (lpu == 8u) load_and_reduce<T, CHUNKS, 8>(stage, warp, lane, y, lo, hi, umn, umx);
+            else load_and_reduce<T, CHUNKS, 4>(stage, warp, lane, y, lo, hi, umn, umx);
+            if (fast_ok) {
+                // groups of 512 / 1024 span 2 / 4 chunks of this warp
+                if (G == 512u) {
 #pragma unroll
-                for (int c = 0; c + 1 < CHUNKS; c += 2) {
-                    lo[c] = lo[c + 1] = fmin2(lo[c], lo[c + 1]);
-                    hi[c] = hi[c + 1] = fmax2(hi[c], hi[c + 1]);
+                    for (int c = 0; c + 1 < CHUNKS; c += 2) {
+                        lo[c] = lo[c + 1] = fmin2(lo[c], lo[c + 1]);
+                        hi[c] = hi[c + 1] = fmax2(hi[c], hi[c + 1]);
+                    }
+                } else if (G == 1024u && CHUNKS == 4) {
+                    const float l = fmin2(fmin2(lo[0], lo[1]), fmin2(lo[2], lo[3]));
+                    const float h = fmax2(fmax2(hi[0], hi[1]), fmax2(hi[2], hi[3]));
+#pragma unroll
+                    for (int c = 0; c < CHUNKS; c++) {
+                        lo[c] = l;
+                        hi[c] = h;
+                    }
                 }
-            } else if (G == 1024u && CHUNKS == 4) {
-                const float l = fmin2(fmin2(lo[0], lo[1]), fmin2(lo[2], lo[3]));
-                const float h = fmax2(fmax2(hi[0], hi[1]), fmax2(hi[2], hi[3]));
+                if (test_sep) {
+                    // separation test of the uniform outcome: min over groups of the key of the last
+                    // raise taken, max over groups of the key of the first raise not taken
+                    const float v_lo = a.v[bud.ell - 1], v_hi = a.v[bud.ell];
+                    uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+#pragma unroll
+                    for (int c = 0; c < CHUNKS; c++) {
+                        float R = __fsub_rn(hi[c], lo[c]);
+                        if (R < 0x1p-118f) R = 0.0f;              // degenerate group: constant
+                        kmin = min(kmin, __float_as_uint(__fmul_rn(R, v_lo)));
+                        kmax = max(kmax, __float_as_uint(__fmul_rn(R, v_hi)));
+                    }
+                    if (lpu != 32u) {
+                        kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+                        kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+                    }
+                    if (lane == 0) {
+                        atomicMin(&s_kmin[j & 3u], kmin);
+                        atomicMax(&s_kmax[j & 3u], kmax);
+                    }
+                }
+            }
+            if (lane == 0 && s_lost != 0u) atomicOr(&s_flag[j & 3u], 1u);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s_exch);
+        }
+
+        // ---------------------------------------------------------------- quantize + pack window j-1 (registers -> shared)
+        if (j > 0) {
+            unsigned char *const s_out = smem + a.lay.out0 + ((j - 1u) % 3u) * a.lay.out_stride;
+            const TensorDesc &qd = tensor_of(q_gw);
+            const uint64_t qbase = (uint64_t)(q_gw - qd.first_window) * WE;
+            const uint64_t blk0 = ((qd.elem_base + qbase) >> 3) + (e0 >> 3);
+            if (q_b != 0u) {
+                if (BATCH) {
+                    const PhiloxSeedKeys sk{(uint32_t)qd.seed, (uint32_t)(qd.seed >> 32)};
+                    if (q_careful) quantize_uniform_b<PhiloxSeedKeys, CHUNKS, true>(q_b, x, q_mn, q_inv, e0, blk0, sk, s_out);
+                    else quantize_uniform_b<PhiloxSeedKeys, CHUNKS, false>(q_b, x, q_mn, q_inv, e0, blk0, sk, s_out);
+                } else {
+                    if (q_careful) quantize_uniform_b<PhiloxKeys, CHUNKS, true>(q_b, x, q_mn, q_inv, e0, blk0, a.keys, s_out);
+                    else quantize_uniform_b<PhiloxKeys, CHUNKS, false>(q_b, x, q_mn, q_inv, e0, blk0, a.keys, s_out);
+                }
+            } else {
+                const GroupRec *grp = s_grp + ((j - 1u) & 1u) * a.n_max;
 #pragma unroll
                 for (int c = 0; c < CHUNKS; c++) {
-                    lo[c] = l;
-                    hi[c] = h;
+                    const uint32_t e = e0 + 256u * c;
+                    const GroupRec rec = grp[e >> log2G];
+                    uint32_t o[4];
+                    if (a.nearest) {
+                        o[0] = o[1] = o[2] = o[3] = 0x80008000u;   // every 16-bit lane = 2 * 2^14
+                    } else {
+                        const uint64_t blk = blk0 + 32u * c;
+                        if (BATCH) {
+                            const PhiloxSeedKeys sk{(uint32_t)qd.seed, (uint32_t)(qd.seed >> 32)};
+                            philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), sk, o);
+                        } else {
+                            philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), a.keys, o);
+                        }
+                    }
+                    uint32_t w0, w1;
+                    unsigned char *p = s_out + rec.off + ((e & (G - 1u)) >> 3) * rec.b;
+                    if (e < q_elems) {
+                        switch (rec.b) {
+                        case 1: quantize8<1, true>(x[c], rec.mn, rec.inv, o, w0, w1); *p = (unsigned char)w0; break;
+                        case 2: quantize8<2, true>(x[c], rec.mn, rec.inv, o, w0, w1); *reinterpret_cast<uint16_t *>(p) = (uint16_t)w0; break;
+                        case 4: quantize8<4, true>(x[c], rec.mn, rec.inv, o, w0, w1); *reinterpret_cast<uint32_t *>(p) = w0; break;
+                        default:
+                            quantize8<8, true>(x[c], rec.mn, rec.inv, o, w0, w1);
+                            if (G >= 64u) {
+                                *reinterpret_cast<uint2 *>(p) = make_uint2(w0, w1);
+                            } else {                               // G = 32: groups are only 4-byte aligned
+                                reinterpret_cast<uint32_t *>(p)[0] = w0;
+                                reinterpret_cast<uint32_t *>(p)[1] = w1;
+                            }
+                            break;
+                        }
+                    }
+                }
+            }
+            if (a.bulk_store) fence_async_shared();               // packed bytes visible to the bulk store issued later
+        }
+        if (!valid) break;
+
+        // ---------------------------------------------------------------- the exchange of window j is complete: widths
+        if (!mbar_wait_bounded(&s_exch, j & 1u)) {
+            s_lost = 1u;
+            if (lane == 0) record_error(DAF_ERR_TIMEOUT, gw, 6u + 16u * j);
+            break;
+        }
+        if (s_flag[j & 3u] != 0u) break;                          // some warp ran out of patience: all leave together
+        if (tid == 0) {                                           // recycle the slot two windows ahead
+            s_kmin[(j + 2u) & 3u] = 0xFFFFFFFFu;
+            s_kmax[(j + 2u) & 3u] = 0u;
+        }
+        const bool uniform = fast_ok && (!test_sep || s_kmin[j & 3u] >= s_kmax[j & 3u]);
+        const uint64_t g0 = wbase >> log2G;                       // first group of the window in the tensor
+        if (uniform) {
+            // -------------------------------------------------------------- every group gets width S[ell]
+            const uint32_t b = a.S[bud.ell];
+            const float Lf = (float)((1u << b) - 1u);
+            // lane k of a unit works out (scale, 1/scale) of chunk k's group, then the unit shares them
+            const int k = lane & (int)(lpu - 1u), sb = lane - k;
+            float Rk = 0.0f, mnk = 0.0f;
+#pragma unroll
+            for (int c = 0; c < CHUNKS; c++)
+                if (k == c) {
+                    Rk = __fsub_rn(hi[c], lo[c]);
+                    mnk = lo[c];
+                }
+            if (Rk < 0x1p-118f) Rk = 0.0f;                        // degenerate group: constant
+            const float scale_k = Rk > 0.0f ? __fdiv_rn(Rk, Lf) : 0.0f;
+            const float inv_k = Rk > 0.0f ? __fdiv_rn(Lf, Rk) : 0.0f;
+            if (k < CHUNKS) {
+                const uint32_t eu = (uint32_t)((warp * CHUNKS + k) * 256 + sb * 8);   // first element of the unit
+                if ((eu & (G - 1u)) == 0u) {                      // the unit opens a group: write its metadata
+                    const uint64_t g = g0 + (eu >> log2G);
+                    td.bits[g] = (uint8_t)b;
+                    td.mn[g] = mnk;
+                    td.scale[g] = scale_k;
                 }
             }
 #pragma unroll
             for (int c = 0; c < CHUNKS; c++) {
-                R[c] = __fsub_rn(hi[c], lo[c]);
-                if (R[c] < 0x1p-118f) R[c] = 0.0f;                // degenerate group: constant
+                q_inv[c] = __shfl_sync(0xFFFFFFFFu, inv_k, sb + c);
+                q_mn[c] = lo[c];
             }
-            if (test_sep) {
-                // separation test of the uniform outcome: min over groups of the key of the last
-                // raise taken, max over groups of the key of the first raise not taken
-                const float v_lo = a.v[ell - 1], v_hi = a.v[ell];
-                uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
-#pragma unroll
-                for (int c = 0; c < CHUNKS; c++) {
-                    kmin = min(kmin, __float_as_uint(__fmul_rn(R[c], v_lo)));
-                    kmax = max(kmax, __float_as_uint(__fmul_rn(R[c], v_hi)));
-                }
-                if (lpu != 32u) {
-                    kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
-                    kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
-                }
-                if (lane == 0) {
-                    atomicMin(&s_kmin[i % 3u], kmin);
-                    atomicMax(&s_kmax[i % 3u], kmax);
-                }
-            }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&s_cons);                      // stage consumed, previous window packed
-
-        // ---------------------------------------------------------------- the one meeting point per window
-        bar_sync(window_barrier(i), kCompressThreads);
-        const uint32_t gw_next = s_next[(i + 1u) & 1u];
-        if (tid == 0) {
-            s_kmin[(i + 2u) % 3u] = 0xFFFFFFFFu;
-            s_kmax[(i + 2u) % 3u] = 0u;
-        }
-        if (s_lost != 0u) break;
-        const bool uniform = fast_ok && (!test_sep || s_kmin[i % 3u] >= s_kmax[i % 3u]);
-        const uint64_t blk0 = ((td.elem_base + wbase) >> 3) + (e0 >> 3);
-
-        if (uniform) {
-            // -------------------------------------------------------------- every group gets width S[ell]
-            const uint32_t b = a.S[ell];
-            const float Lf = (float)((1u << b) - 1u);
-            // lane j of a unit works out (scale, 1/scale) of chunk j's group, then the unit shares them
-            const int j = lane & (int)(lpu - 1u), sb = lane - j;
-            float Rj = 0.0f, mnj = 0.0f;
-#pragma unroll
-            for (int c = 0; c < CHUNKS; c++)
-                if (j == c) {
-                    Rj = R[c];
-                    mnj = lo[c];
-                }
-            const float scale_j = Rj > 0.0f ? __fdiv_rn(Rj, Lf) : 0.0f;
-            const float inv_j = Rj > 0.0f ? __fdiv_rn(Lf, Rj) : 0.0f;
-            if (j < CHUNKS) {
-                const uint32_t eu = (uint32_t)((warp * CHUNKS + j) * 256 + sb * 8);   // first element of the unit
-                if ((eu & (G - 1u)) == 0u) {                      // the unit opens a group: write its metadata
-                    const uint64_t g = g0 + (eu >> log2G);
-                    td.bits[g] = (uint8_t)b;
-                    td.mn[g] = mnj;
-                    td.scale[g] = scale_j;
-                }
-            }
-            float inv[CHUNKS];
-#pragma unroll
-            for (int c = 0; c < CHUNKS; c++) inv[c] = __shfl_sync(0xFFFFFFFFu, inv_j, sb + c);
             // 1/scale not a normal number (range beyond 2^126 * L): the careful quantizer clamps
-            const bool careful = __any_sync(0xFFFFFFFFu, Rj > 0.0f && inv_j < 0x1p-126f) != 0;
+            q_careful = __any_sync(0xFFFFFFFFu, Rk > 0.0f && inv_k < 0x1p-126f) != 0;
+            q_b = b;
             if (tid == 0) {
                 const uint32_t total = n * (G >> 3) * b;
                 const bool first = (gw == td.first_window);
                 st_relaxed_u64(a.flags + gw, ((first ? kFlagPrefix : kFlagAggregate) << kFlagShift) | total);
-                s_tot[i & 3u] = total;
-            }
-            if (BATCH) {
-                const PhiloxSeedKeys sk{(uint32_t)td.seed, (uint32_t)(td.seed >> 32)};
-                if (careful) quantize_uniform_b<PhiloxSeedKeys, CHUNKS, true>(b, x, lo, inv, e0, blk0, sk, s_out);
-                else quantize_uniform_b<PhiloxSeedKeys, CHUNKS, false>(b, x, lo, inv, e0, blk0, sk, s_out);
-            } else {
-                if (careful) quantize_uniform_b<PhiloxKeys, CHUNKS, true>(b, x, lo, inv, e0, blk0, a.keys, s_out);
-                else quantize_uniform_b<PhiloxKeys, CHUNKS, false>(b, x, lo, inv, e0, blk0, a.keys, s_out);
+                s_tot[j & 3u] = total;
             }
         } else {
-            // -------------------------------------------------------------- general bit choice (owner warps), then a generic pass
+            // -------------------------------------------------------------- general bit choice (owner warps), group records
             const uint32_t owners = (n + 31u) >> 5;               // warps that own group records
             if ((uint32_t)warp < owners) {
                 const uint32_t m = a.m, n_max = a.n_max;
+                const float *umn = s_umn + (j & 1u) * units, *umx = s_umx + (j & 1u) * units;
                 const bool mine = (uint32_t)tid < n;
                 float mn = 0.0f, Rg = 0.0f;
                 if (mine) {
                     float mx;
                     if (G > 256u) {
-                        const uint32_t r = G >> 8;
-                        mn = s_umn[tid * r];
-                        mx = s_umx[tid * r];
-                        for (uint32_t k = 1; k < r; k++) {
-                            mn = fmin2(mn, s_umn[tid * r + k]);
-                            mx = fmax2(mx, s_umx[tid * r + k]);
+                        const uint32_t rr = G >> 8;
+                        mn = umn[tid * rr];
+                        mx = umx[tid * rr];
+                        for (uint32_t k = 1; k < rr; k++) {
+                            mn = fmin2(mn, umn[tid * rr + k]);
+                            mx = fmax2(mx, umx[tid * rr + k]);
                         }
                     } else {
-                        mn = s_umn[tid];
-                        mx = s_umx[tid];
+                        mn = umn[tid];
+                        mx = umx[tid];
                     }
                     Rg = __fsub_rn(mx, mn);
                     if (Rg < 0x1p-118f) Rg = 0.0f;                // degenerate group: constant
                 }
-                uint32_t level = ell;
-                bool same = all_max;                              // every group ends at level ell
-                if (!all_max) {
+                uint32_t level = bud.ell;
+                bool same = bud.all_max;                          // every group ends at level ell
+                if (!bud.all_max) {
                     if (mine) {
 #pragma unroll
                         for (int k = 0; k < kMaxLevels - 1; k++) {
@@ -681,15 +765,15 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                     }
                     if (owners > 1) bar_sync(kBarOwners, owners * 32u);
                     else __syncwarp();
-                    if (need_sep) {
+                    if (bud.need_sep) {
                         // Uniform outcome: every raise below level ell sorts ahead of every raise from
                         // level ell upward (ties go to the lower level), they all fit, the next does not.
                         same = true;
-                        if (ell > 0) {
+                        if (bud.ell > 0) {
                             uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
                             for (uint32_t g = lane; g < n; g += 32) {
-                                kmin = min(kmin, s_key[(ell - 1) * n_max + g]);
-                                kmax = max(kmax, s_key[ell * n_max + g]);
+                                kmin = min(kmin, s_key[(bud.ell - 1) * n_max + g]);
+                                kmax = max(kmax, s_key[bud.ell * n_max + g]);
                             }
                             kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
                             kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
@@ -721,7 +805,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                         else __syncwarp();
                         level = 0;
                         if (mine)
-                            for (uint32_t k = 0; k + 1 < m; k++) level += (s_cum[k * n_max + tid] <= rem);
+                            for (uint32_t k = 0; k + 1 < m; k++) level += (s_cum[k * n_max + tid] <= bud.rem);
                     }
                 }
                 uint32_t size = 0, b = 0;
@@ -753,6 +837,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                         if (k < (uint32_t)warp) before += t;
                         total += t;
                     }
+                    bar_sync(kBarOwners, owners * 32u);           // s_wtot may be rewritten by the next general window
                 }
                 if (mine) {
                     GroupRec rec;
@@ -760,76 +845,58 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                     rec.inv = inv;
                     rec.b = b;
                     rec.off = before + incl - size;
-                    s_grp[tid] = rec;
+                    s_grp[(j & 1u) * n_max + tid] = rec;
                 }
                 if (tid == 0) {
                     const bool first = (gw == td.first_window);
                     st_relaxed_u64(a.flags + gw, ((first ? kFlagPrefix : kFlagAggregate) << kFlagShift) | total);
-                    s_tot[i & 3u] = total;
+                    s_tot[j & 3u] = total;
                 }
             }
-            bar_sync(kBarWidths, kThreads);                       // group records visible to all compute warps
-#pragma unroll
-            for (int c = 0; c < CHUNKS; c++) {
-                const uint32_t e = e0 + 256u * c;
-                const GroupRec rec = s_grp[e >> log2G];
-                uint32_t o[4];
-                if (a.nearest) {
-                    o[0] = o[1] = o[2] = o[3] = 0x80008000u;       // every 16-bit lane = 2 * 2^14
-                } else {
-                    const uint64_t blk = blk0 + 32u * c;
-                    if (BATCH) {
-                        const PhiloxSeedKeys sk{(uint32_t)td.seed, (uint32_t)(td.seed >> 32)};
-                        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), sk, o);
-                    } else {
-                        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), a.keys, o);
-                    }
-                }
-                uint32_t w0, w1;
-                unsigned char *p = s_out + rec.off + ((e & (G - 1u)) >> 3) * rec.b;
-                if (e < n_elems) {
-                    switch (rec.b) {
-                    case 1: quantize8<1, true>(x[c], rec.mn, rec.inv, o, w0, w1); *p = (unsigned char)w0; break;
-                    case 2: quantize8<2, true>(x[c], rec.mn, rec.inv, o, w0, w1); *reinterpret_cast<uint16_t *>(p) = (uint16_t)w0; break;
-                    case 4: quantize8<4, true>(x[c], rec.mn, rec.inv, o, w0, w1); *reinterpret_cast<uint32_t *>(p) = w0; break;
-                    default:
-                        quantize8<8, true>(x[c], rec.mn, rec.inv, o, w0, w1);
-                        if (G >= 64u) {
-                            *reinterpret_cast<uint2 *>(p) = make_uint2(w0, w1);
-                        } else {                                   // G = 32: groups are only 4-byte aligned
-                            reinterpret_cast<uint32_t *>(p)[0] = w0;
-                            reinterpret_cast<uint32_t *>(p)[1] = w1;
-                        }
-                        break;
-                    }
-                }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s_wid);
+            if (!mbar_wait_bounded(&s_wid, n_generic & 1u)) {     // group records visible to all compute warps
+                s_lost = 1u;
+                if (lane == 0) record_error(DAF_ERR_TIMEOUT, gw, 7u + 16u * j);
+                break;
             }
+            n_generic++;
+            q_b = 0u;
         }
-        if (a.bulk_store) fence_async_shared();                   // packed bytes visible to the bulk store issued later
-        gw = gw_next;
+        q_gw = gw;
+        q_elems = n_elems;
+
+        // ---------------------------------------------------------------- window j: stage -> registers, stage released
+        {
+            constexpr int kChunkBytes = 256 * Elem<T>::kBytes;
+#pragma unroll
+            for (int c = 0; c < CHUNKS; c++) load8_staged<T>(stage + (warp * CHUNKS + c) * kChunkBytes, lane, x[c]);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_cons[j & 1u]);              // stage consumed, previous window packed
     }
     __syncwarp();
-    if (lane == 0) mbar_arrive(&s_done);                          // the last window is packed (or the loop was left)
+    if (lane == 0) mbar_arrive(&s_done);                          // this warp is out of the loop
 }
 
 // ------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------
 // Shared-memory carve-up for one launch configuration.
-static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint32_t window_cap_bytes, uint32_t nbuf)
+static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint32_t window_cap_bytes)
 {
     auto up = [](uint32_t v) { return (v + 127u) & ~127u; };
     const uint32_t n_max = we / G, units = we / (G < 256u ? G : 256u);
     SmemLayout l;
-    uint32_t at = up(we * elem_bytes);
+    uint32_t at = 2u * up(we * elem_bytes);                       // two stages
     l.out0 = at;
     l.out_stride = up(window_cap_bytes < 16u ? 16u : window_cap_bytes);
-    at += nbuf * l.out_stride;
-    l.umn = at; at += up(4u * units);
-    l.umx = at; at += up(4u * units);
+    at += 3u * l.out_stride;                                      // three packed-bytes buffers
+    l.umn = at; at += up(2u * 4u * units);
+    l.umx = at; at += up(2u * 4u * units);
     l.key = at; at += up(4u * (kMaxLevels - 1) * n_max);
     l.cum = at; at += up(4u * (kMaxLevels - 1) * n_max);
-    l.grp = at; at += up(16u * n_max);
+    l.grp = at; at += up(2u * 16u * n_max);
     l.total = at;
     return l;
 }
@@ -898,15 +965,8 @@ template <int NT> static void fill_common(CompressArgs<NT> &a, const Plan &pl, c
         while (a.full_ell + 1 < pl.m && (pl.S[a.full_ell + 1] - pl.S[0]) * n <= a.full_rem) a.full_ell++;
         a.full_rem_after = a.full_rem - (pl.S[a.full_ell] - pl.S[0]) * n;
     }
-    // Three packed-bytes buffers keep the control warp entirely off the compute warps' path;
-    // fall back to two when three would not leave room for two CTAs per SM (227 KiB).
-    const uint32_t cap = (uint32_t)((((uint64_t)pl.beta_q8 * pl.W) >> 8) * pl.G / 8);
     a.nbuf = 3;
-    a.lay = make_layout(pl.We, elem_bytes, pl.G, cap, 3);
-    if (2u * (a.lay.total + 2048u) > 227u * 1024u) {
-        a.nbuf = 2;
-        a.lay = make_layout(pl.We, elem_bytes, pl.G, cap, 2);
-    }
+    a.lay = make_layout(pl.We, elem_bytes, pl.G, (uint32_t)((((uint64_t)pl.beta_q8 * pl.W) >> 8) * pl.G / 8));
     for (int k = 0; k < kMaxLevels; k++) {
         a.S[k] = pl.S[k];
         a.cost[k] = pl.cost[k];
