@@ -94,6 +94,10 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, const Ke
 struct PhiloxSeedKeys {
     uint32_t lo, hi;
 };
+__device__ __forceinline__ uint32_t philox_key0(const PhiloxKeys &k, int r) { return k.k0[r]; }
+__device__ __forceinline__ uint32_t philox_key1(const PhiloxKeys &k, int r) { return k.k1[r]; }
+__device__ __forceinline__ uint32_t philox_key0(const PhiloxSeedKeys &k, int r) { return k.lo + (uint32_t)r * kPhiloxW0; }
+__device__ __forceinline__ uint32_t philox_key1(const PhiloxSeedKeys &k, int r) { return k.hi + (uint32_t)r * kPhiloxW1; }
 template <>
 __device__ __forceinline__ void philox4x32_10<PhiloxSeedKeys>(uint32_t c0, uint32_t c1, const PhiloxSeedKeys &s,
                                                                uint32_t (&o)[4])

@@ -80,7 +80,7 @@ __device__ __forceinline__ void quantize8(const float (&x)[8], float mn, float i
         const float d = __fsub_rn(x[i], mn);
         const float s = __fmaf_rn(d, inv, 256.0f);
         const uint32_t h = (i & 1) ? (o[i >> 1] >> 16) : (o[i >> 1] & 0xFFFFu);
-        const uint32_t t = (__float_as_uint(s) << 1) + h;         // mod 2^32; 2*bits(256) = 0x87000000
+        const uint32_t t = __float_as_uint(s) * 2u + h;           // mod 2^32; 2*bits(256) = 0x87000000
         const int pos = (B * i) & 31;                             // bit position of code i in its word (unrolled: constant)
         uint32_t field;
         if (CLAMP) {
@@ -214,17 +214,32 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity
 }
 
 // Eight consecutive elements of a lane from the staged window (two 16-byte shared loads for
-// 4-byte elements, one for 2-byte elements).
-template <typename T> __device__ __forceinline__ void load8_staged(const unsigned char *chunk, int lane, float (&x)[8]);
+// 4-byte elements, one for 2-byte elements).  For 4-byte elements a lane owns 32 bytes; the
+// two halves are read in an order that depends on the lane so that each quarter-warp touches
+// all 32 banks.  ORDERED = false leaves the halves as read (enough for min / max).
+template <typename T, bool ORDERED> __device__ __forceinline__ void load8_staged(const unsigned char *chunk, int lane, float (&x)[8]);
 
-template <> __device__ __forceinline__ void load8_staged<float>(const unsigned char *chunk, int lane, float (&x)[8])
+template <> __device__ __forceinline__ void load8_staged<float, false>(const unsigned char *chunk, int lane, float (&x)[8])
 {
-    const float4 a = *reinterpret_cast<const float4 *>(chunk + lane * 32);
-    const float4 b = *reinterpret_cast<const float4 *>(chunk + lane * 32 + 16);
+    const int odd = (lane >> 2) & 1;
+    const unsigned char *p = chunk + lane * 32;
+    const float4 a = *reinterpret_cast<const float4 *>(p + odd * 16);
+    const float4 b = *reinterpret_cast<const float4 *>(p + (odd ^ 1) * 16);
     x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
     x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
 }
-template <> __device__ __forceinline__ void load8_staged<__half>(const unsigned char *chunk, int lane, float (&x)[8])
+template <> __device__ __forceinline__ void load8_staged<float, true>(const unsigned char *chunk, int lane, float (&x)[8])
+{
+    const bool odd = (lane >> 2) & 1;
+    float y[8];
+    load8_staged<float, false>(chunk, lane, y);
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+        x[i] = odd ? y[i + 4] : y[i];
+        x[i + 4] = odd ? y[i] : y[i + 4];
+    }
+}
+template <bool ORDERED> __device__ __forceinline__ void load8_staged_half(const unsigned char *chunk, int lane, float (&x)[8])
 {
     const uint4 v = *reinterpret_cast<const uint4 *>(chunk + lane * 16);
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
@@ -235,7 +250,7 @@ template <> __device__ __forceinline__ void load8_staged<__half>(const unsigned 
         x[2 * i + 1] = f.y;
     }
 }
-template <> __device__ __forceinline__ void load8_staged<__nv_bfloat16>(const unsigned char *chunk, int lane, float (&x)[8])
+template <bool ORDERED> __device__ __forceinline__ void load8_staged_bf16(const unsigned char *chunk, int lane, float (&x)[8])
 {
     const uint4 v = *reinterpret_cast<const uint4 *>(chunk + lane * 16);
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
@@ -245,6 +260,10 @@ template <> __device__ __forceinline__ void load8_staged<__nv_bfloat16>(const un
         x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
     }
 }
+template <> __device__ __forceinline__ void load8_staged<__half, false>(const unsigned char *c, int l, float (&x)[8]) { load8_staged_half<false>(c, l, x); }
+template <> __device__ __forceinline__ void load8_staged<__half, true>(const unsigned char *c, int l, float (&x)[8]) { load8_staged_half<true>(c, l, x); }
+template <> __device__ __forceinline__ void load8_staged<__nv_bfloat16, false>(const unsigned char *c, int l, float (&x)[8]) { load8_staged_bf16<false>(c, l, x); }
+template <> __device__ __forceinline__ void load8_staged<__nv_bfloat16, true>(const unsigned char *c, int l, float (&x)[8]) { load8_staged_bf16<true>(c, l, x); }
 
 // Staged window -> registers, then min / max per unit of LPU lanes (a full warp uses the
 // redux instruction).  Every lane of a unit ends up with the unit's min / max (lo[c], hi[c]);
@@ -256,7 +275,7 @@ __device__ __forceinline__ void load_and_reduce(const unsigned char *stage, int 
 {
     constexpr int kChunkBytes = 256 * Elem<T>::kBytes;
 #pragma unroll
-    for (int c = 0; c < CHUNKS; c++) load8_staged<T>(stage + (warp * CHUNKS + c) * kChunkBytes, lane, x[c]);
+    for (int c = 0; c < CHUNKS; c++) load8_staged<T, false>(stage + (warp * CHUNKS + c) * kChunkBytes, lane, x[c]);
 #pragma unroll
     for (int c = 0; c < CHUNKS; c++) {
         float l = fmin3(fmin3(x[c][0], x[c][1], x[c][2]), fmin3(x[c][3], x[c][4], x[c][5]), fmin2(x[c][6], x[c][7]));
@@ -291,7 +310,7 @@ template <int NT> __device__ __forceinline__ uint32_t find_tensor(const Compress
     return lo;
 }
 
-// One persistent CTA per SM: 16 compute warps plus one control warp, synchronised only through
+// One persistent CTA per SM: 16 compute warps plus three service warps, synchronised only through
 // shared-memory mbarriers (every wait on them is bounded) except inside the general bit choice.
 //   s_full[s]  : the bulk copy into stage s has landed (or the control warp has marked the
 //                window behind it as "no more work");
@@ -301,11 +320,11 @@ template <int NT> __device__ __forceinline__ uint32_t find_tensor(const Compress
 //                (16 arrivals) -- arrival and wait are split so that the exchange of window
 //                j+1 completes while window j is being quantized;
 //   s_wid      : the group records of a window that needed the general bit choice are ready;
-//   s_done     : all compute warps have left their loop.
-// Window j uses stage j & 1, packed-bytes buffer j % 3 and slot j & 3 of the small per-window
-// arrays.  The control warp owns tickets, bulk copies in, look-back and bulk stores out.
-constexpr int kComputeWarps = kWarps;
-constexpr int kCompressThreads = kThreads + 32;
+//   s_ready[b] : the window using packed-bytes buffer b is completely packed (16 arrivals);
+//   s_free[b]  : the packed bytes of the window that used buffer b have left shared memory.
+// Window j uses stage j & 1, packed-bytes buffer j % 3 and slot j & 3 (tickets: j & 7) of the
+// small per-window arrays.  A loader warp owns tickets and bulk copies in; two storer warps
+// alternate over the windows for look-back and bulk stores out.
 constexpr uint32_t kBarOwners = 3;
 
 __device__ __forceinline__ void bar_sync(uint32_t id, uint32_t threads)
@@ -317,6 +336,41 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
 }
 
+// Philox4x32-10 for CHUNKS consecutive counter blocks at once (blk0 + 32 c): the rounds of the
+// independent blocks are interleaved in program order so that their long dependency chains
+// overlap.
+template <typename KEYS, int CHUNKS>
+__device__ __forceinline__ void philox_chunks(uint64_t blk0, const KEYS &keys, uint32_t (&o)[CHUNKS][4])
+{
+    uint32_t c0[CHUNKS], c1[CHUNKS], c2[CHUNKS], c3[CHUNKS];
+#pragma unroll
+    for (int c = 0; c < CHUNKS; c++) {
+        const uint64_t blk = blk0 + 32u * c;
+        c0[c] = (uint32_t)blk;
+        c1[c] = (uint32_t)(blk >> 32);
+        c2[c] = 0u;
+        c3[c] = 0u;
+    }
+#pragma unroll
+    for (int r = 0; r < 10; r++) {
+#pragma unroll
+        for (int c = 0; c < CHUNKS; c++) {
+            const uint64_t p0 = (uint64_t)kPhiloxM0 * c0[c], p1 = (uint64_t)kPhiloxM1 * c2[c];
+            c0[c] = (uint32_t)(p1 >> 32) ^ c1[c] ^ philox_key0(keys, r);
+            c1[c] = (uint32_t)p1;
+            c2[c] = (uint32_t)(p0 >> 32) ^ c3[c] ^ philox_key1(keys, r);
+            c3[c] = (uint32_t)p0;
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < CHUNKS; c++) {
+        o[c][0] = c0[c];
+        o[c][1] = c1[c];
+        o[c][2] = c2[c];
+        o[c][3] = c3[c];
+    }
+}
+
 // Quantize + pack CHUNKS chunks that all have width B, with per-chunk (min, 1/scale) in
 // registers: no per-chunk decisions, packed position computed from the element index alone.
 template <typename KEYS, int CHUNKS, int B, bool CLAMP>
@@ -325,13 +379,12 @@ __device__ __forceinline__ void quantize_uniform(const float (&x)[CHUNKS][8], co
                                                  unsigned char *s_out)
 {
     unsigned char *const out = s_out + (e0 >> 3) * B;
+    uint32_t o[CHUNKS][4];
+    philox_chunks<KEYS, CHUNKS>(blk0, keys, o);
 #pragma unroll
     for (int c = 0; c < CHUNKS; c++) {
-        uint32_t o[4];
-        const uint64_t blk = blk0 + 32u * c;
-        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), keys, o);
         uint32_t w0, w1;
-        quantize8<B, CLAMP>(x[c], mn[c], inv[c], o, w0, w1);
+        quantize8<B, CLAMP>(x[c], mn[c], inv[c], o[c], w0, w1);
         unsigned char *p = out + 32 * B * c;
         if (B == 1) *p = (unsigned char)w0;
         else if (B == 2) *reinterpret_cast<uint16_t *>(p) = (uint16_t)w0;
@@ -361,20 +414,22 @@ struct Budget {
     bool need_sep;         // the best raise of level ell does not fit: uniform iff the levels separate
 };
 
-template <typename T, int CHUNKS, bool BATCH>
-__global__ void __launch_bounds__(kCompressThreads, 1)
+// T: element type; CHUNKS: 256-element chunks per compute warp; NW: compute warps.
+template <typename T, int CHUNKS, int NW, bool BATCH>
+__global__ void __launch_bounds__(NW * 32 + 96, 1)
 compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> a)
 {
-    constexpr uint32_t WE = kThreads * kLaneElems * CHUNKS;
+    constexpr int kComputeWarps = NW;
+    constexpr uint32_t WE = NW * 256u * CHUNKS;
     constexpr uint32_t kStageBytes = WE * Elem<T>::kBytes;
 
     extern __shared__ __align__(128) unsigned char smem[];       // [stage 0 | stage 1 | packed x3 | group arrays]
-    __shared__ __align__(8) uint64_t s_full[2], s_cons[2], s_exch, s_wid, s_done;   // mbarriers
-    __shared__ uint32_t s_next[4];                               // ticket of window j
+    __shared__ __align__(8) uint64_t s_full[2], s_cons[2], s_ready[3], s_free[3], s_exch, s_wid;   // mbarriers
+    __shared__ uint32_t s_next[8];                               // ticket of window j
     __shared__ uint32_t s_kmin[4], s_kmax[4], s_flag[4];         // per-window exchange: key extremes, "a wait ran out"
     __shared__ uint32_t s_tot[4];                                // packed bytes of window j
-    __shared__ uint32_t s_wtot[kComputeWarps];
-    __shared__ uint32_t s_lost;
+    __shared__ uint32_t s_wtot[NW];
+    __shared__ uint32_t s_lost, s_end;                           // s_end: number of windows this CTA packed (set on leaving)
 
     float *const s_umn = reinterpret_cast<float *>(smem + a.lay.umn);    // [2][units]
     float *const s_umx = reinterpret_cast<float *>(smem + a.lay.umx);
@@ -410,11 +465,12 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     };
 
     if (warp == kComputeWarps) {
-        // ============================================================ control warp
-        // Control lane: publish the ticket of window j and start its bulk copy into stage j & 1,
-        // or complete the stage's barrier empty-handed when there is no such window.
+        // ============================================================ loader warp
+        // Publishes the ticket of window j and starts its bulk copy into stage j & 1, or completes
+        // the stage's barrier empty-handed when there is no such window.  Round r: once the
+        // compute warps have moved window r into registers, stage r & 1 takes window r+2.
         auto issue = [&](uint32_t j, uint32_t t) {
-            s_next[j & 3u] = t;
+            s_next[j & 7u] = t;
             uint64_t *bar = &s_full[j & 1u];
             if (t < a.total_windows) {
                 const TensorDesc &nd = tensor_of(t);
@@ -427,16 +483,20 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 mbar_arrive(bar);
             }
         };
-        uint32_t t0 = 0xFFFFFFFFu, t1 = 0xFFFFFFFFu;              // tickets of windows r and r+1
+        uint32_t t0 = 0xFFFFFFFFu, t1 = 0xFFFFFFFFu, t2 = 0xFFFFFFFFu;   // tickets of windows r, r+1, r+2
         if (lane == 0) {
             mbar_init(&s_full[0], 1);
             mbar_init(&s_full[1], 1);
             mbar_init(&s_cons[0], kComputeWarps);
             mbar_init(&s_cons[1], kComputeWarps);
+            mbar_init(&s_free[0], 1);
+            mbar_init(&s_free[1], 1);
+            mbar_init(&s_free[2], 1);
             mbar_init(&s_exch, kComputeWarps);
             mbar_init(&s_wid, kComputeWarps);
-            mbar_init(&s_done, kComputeWarps);
+            for (int k = 0; k < 3; k++) mbar_init(&s_ready[k], kComputeWarps);
             s_lost = 0u;
+            s_end = 0xFFFFFFFFu;
             for (int k = 0; k < 4; k++) {
                 s_kmin[k] = 0xFFFFFFFFu;
                 s_kmax[k] = 0u;
@@ -444,87 +504,91 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             }
             t0 = atomicAdd(&a.hdr->ticket, 1u);
             issue(0, t0);
-            if (t0 < a.total_windows) {
-                t1 = atomicAdd(&a.hdr->ticket, 1u);
-                issue(1, t1);
-            }
+            if (t0 < a.total_windows) t1 = atomicAdd(&a.hdr->ticket, 1u);
+            issue(1, t1);
+            if (t1 < a.total_windows) t2 = atomicAdd(&a.hdr->ticket, 1u);   // reserved ahead: its latency is off the path
         }
-        t0 = __shfl_sync(0xFFFFFFFFu, t0, 0);
-        t1 = __shfl_sync(0xFFFFFFFFu, t1, 0);
         __syncthreads();
-
-        bool have_prev = false;
-        uint32_t p_gw = 0;
-        for (uint32_t r = 0;; r++) {
-            const bool valid = t0 < a.total_windows && s_lost == 0u;
-            // round r: window r is in registers once s_cons fires; after the last window (or a
-            // lost wait) the compute warps sign off on s_done instead
-            bool ok = valid ? mbar_wait_bounded(&s_cons[r & 1u], (r >> 1) & 1u) : mbar_wait_bounded(&s_done, 0u);
-            if (!ok) {
+        if (lane != 0) return;
+        for (uint32_t r = 0; t0 < a.total_windows; r++) {
+            if (!mbar_wait_bounded(&s_cons[r & 1u], (r >> 1) & 1u)) {
                 s_lost = 1u;
-                if (lane == 0) record_error(DAF_ERR_TIMEOUT, t0, 2u + 16u * r);
+                record_error(DAF_ERR_TIMEOUT, t0, 2u + 16u * r);
             }
-            uint32_t t2 = 0xFFFFFFFFu;                            // ticket of window r+2
-            if (valid && ok) {
-                if (lane == 0 && t1 < a.total_windows) {
-                    if (s_lost == 0u) t2 = atomicAdd(&a.hdr->ticket, 1u);
-                    issue(r + 2u, t2);                            // stage r & 1 is free again
+            if (s_lost != 0u) {
+                // leaving: windows still held will never be published; copies in flight must land
+                if (t1 < a.total_windows) {
+                    st_relaxed_u64(a.flags + t1, kFlagPoison << kFlagShift);
+                    mbar_wait_bounded(&s_full[(r + 1u) & 1u], ((r + 1u) >> 1) & 1u);
                 }
-                t2 = __shfl_sync(0xFFFFFFFFu, t2, 0);
-            }
-            if (have_prev) {
-                // window r-1 is packed: find its byte offset, publish its inclusive prefix, store it
-                const TensorDesc &pd = tensor_of(p_gw);
-                const uint32_t p_total = s_tot[(r - 1u) & 3u];
-                const unsigned char *src = smem + a.lay.out0 + ((r - 1u) % 3u) * a.lay.out_stride;
-                uint64_t excl = 0;
-                int state = 1;
-                if (p_gw != pd.first_window) {
-                    state = lookback<kLookDepth>(a.flags, p_gw, pd.first_window, lane, true, &excl);
-                    if (lane == 0)
-                        st_relaxed_u64(a.flags + p_gw, state == 1 ? ((kFlagPrefix << kFlagShift) | (excl + p_total))
-                                                                    : (kFlagPoison << kFlagShift));
-                }
-                const uint32_t pw = p_gw - pd.first_window;
-                bool skip = state != 1;
-                if (!skip) {
-                    if (lane == 0) {
-                        pd.woff[pw] = excl;
-                        if (pw + 1 == pd.n_windows) pd.woff[pw + 1] = excl + p_total;
-                    }
-                    skip = excl + p_total > pd.capacity;
-                }
-                if (skip) {
-                    if (lane == 0)
-                        record_error(state == -2 ? DAF_ERR_TIMEOUT : DAF_ERR_CAPACITY, p_gw, state == 1 ? 5u : (state == -2 ? 3u : 4u));
-                } else if (a.bulk_store) {
-                    if (lane == 0 && p_total) {
-                        bulk_store(pd.packed + excl, src, p_total);
-                        bulk_store_wait_read();                   // the buffer may be rewritten from now on
-                    }
-                } else {                                          // groups of 32 / 64: windows are only 4-byte aligned
-                    uint32_t *dst = reinterpret_cast<uint32_t *>(pd.packed + excl);
-                    const uint32_t *s32 = reinterpret_cast<const uint32_t *>(src);
-                    for (uint32_t k = lane; k < (p_total >> 2); k += 32) dst[k] = s32[k];
-                }
-                __syncwarp();
-                have_prev = false;
-            }
-            if (!valid || !ok) {
-                // leaving: windows this CTA still holds tickets for will never be published
-                if (lane == 0) {
-                    if (t0 < a.total_windows) st_relaxed_u64(a.flags + t0, kFlagPoison << kFlagShift);
-                    if (t1 < a.total_windows) st_relaxed_u64(a.flags + t1, kFlagPoison << kFlagShift);
-                    // bulk copies still in flight must land before the CTA goes away
-                    if (t0 < a.total_windows) mbar_wait_bounded(&s_full[r & 1u], (r >> 1) & 1u);
-                    if (t1 < a.total_windows) mbar_wait_bounded(&s_full[(r + 1u) & 1u], ((r + 1u) >> 1) & 1u);
-                }
+                if (t2 < a.total_windows) st_relaxed_u64(a.flags + t2, kFlagPoison << kFlagShift);
+                s_next[(r + 2u) & 7u] = 0xFFFFFFFFu;
+                mbar_arrive(&s_full[r & 1u]);
                 break;
             }
-            have_prev = true;
-            p_gw = t0;
-            t0 = t1;
-            t1 = t2;
+            if (t1 < a.total_windows) {
+                issue(r + 2u, t2);                                // stage r & 1 is free again
+                t0 = t1;
+                t1 = t2;
+                t2 = t1 < a.total_windows ? atomicAdd(&a.hdr->ticket, 1u) : 0xFFFFFFFFu;
+            } else {
+                t0 = t1;
+            }
+        }
+        return;
+    }
+    if (warp > kComputeWarps) {
+        // ============================================================ storer warps (two, alternating windows)
+        // For window p: once it is packed, find its byte offset by look-back, publish its inclusive
+        // prefix, send its packed bytes to global memory with one bulk store, free the buffer.
+        __syncthreads();
+        for (uint32_t p = (uint32_t)(warp - kComputeWarps - 1);; p += 2u) {
+            // s_ready[p % 3] fires when window p is packed -- or when the compute warps have left
+            // their loop without ever reaching a window p (s_end tells which)
+            const bool ok = mbar_wait_bounded(&s_ready[p % 3u], (p / 3u) & 1u);
+            if (ok && p >= s_end) break;
+            const uint32_t p_gw = s_next[p & 7u];
+            if (!ok || s_lost != 0u) {
+                s_lost = 1u;
+                if (lane == 0 && !ok) record_error(DAF_ERR_TIMEOUT, 0u, 8u + 16u * p);
+                if (lane == 0 && ok) st_relaxed_u64(a.flags + p_gw, kFlagPoison << kFlagShift);
+                break;
+            }
+            const TensorDesc &pd = tensor_of(p_gw);
+            const uint32_t p_total = s_tot[p & 3u];
+            const unsigned char *src = smem + a.lay.out0 + (p % 3u) * a.lay.out_stride;
+            uint64_t excl = 0;
+            int state = 1;
+            if (p_gw != pd.first_window) {
+                state = lookback<kLookDepth>(a.flags, p_gw, pd.first_window, lane, true, &excl);
+                if (lane == 0)
+                    st_relaxed_u64(a.flags + p_gw, state == 1 ? ((kFlagPrefix << kFlagShift) | (excl + p_total))
+                                                                : (kFlagPoison << kFlagShift));
+            }
+            const uint32_t pw = p_gw - pd.first_window;
+            bool skip = state != 1;
+            if (!skip) {
+                if (lane == 0) {
+                    pd.woff[pw] = excl;
+                    if (pw + 1 == pd.n_windows) pd.woff[pw + 1] = excl + p_total;
+                }
+                skip = excl + p_total > pd.capacity;
+            }
+            if (skip) {
+                if (lane == 0)
+                    record_error(state == -2 ? DAF_ERR_TIMEOUT : DAF_ERR_CAPACITY, p_gw, state == 1 ? 5u : (state == -2 ? 3u : 4u));
+            } else if (a.bulk_store) {
+                if (lane == 0 && p_total) {
+                    bulk_store(pd.packed + excl, src, p_total);
+                    bulk_store_wait_read();
+                }
+            } else {                                              // groups of 32 / 64: windows are only 4-byte aligned
+                uint32_t *dst = reinterpret_cast<uint32_t *>(pd.packed + excl);
+                const uint32_t *s32 = reinterpret_cast<const uint32_t *>(src);
+                for (uint32_t k = lane; k < (p_total >> 2); k += 32) dst[k] = s32[k];
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s_free[p % 3u]);          // the buffer may be rewritten from now on
         }
         if (lane == 0) bulk_store_wait_all();
         return;
@@ -535,38 +599,45 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     const uint32_t e0 = (uint32_t)(warp * CHUNKS * 256 + lane * 8);    // this lane's first element of chunk 0
     const uint32_t lpu = (G < 256u ? G : 256u) >> 3;              // lanes per unit
     const uint32_t units = WE >> (G < 256u ? log2G : 8u);         // units per window
-    const bool local = G <= 256u * CHUNKS;                        // every group lives inside one warp's chunks
+    // Launch-wide facts about full windows (the ragged last window of a tensor always takes the
+    // general path): can the quick uniform-width decision apply, and with which numbers?
+    const Budget fb = budget_of(a.n_max);
+    const bool fast_launch = G <= 256u * CHUNKS && !a.nearest && (fb.all_max || fb.need_sep);
+    const bool test_sep = fast_launch && fb.need_sep && fb.ell > 0;
+    const uint32_t fast_b = a.S[fb.ell];
+    const float fast_L = (float)((1u << fast_b) - 1u);
+    const float v_lo = a.v[fb.ell > 0 ? fb.ell - 1 : 0], v_hi = a.v[fb.ell];
+    // lane k of a unit looks after chunk k's group in the uniform case
+    const int uk = lane & (int)(lpu - 1u), usb = lane - uk;
+    const uint32_t unit_elem = (uint32_t)((warp * CHUNKS + uk) * 256 + usb * 8);   // first element of that unit
+    const bool meta_lane = uk < CHUNKS && (unit_elem & (G - 1u)) == 0u;            // the unit opens a group
 
     // the window being quantized (registers) and how
     float x[CHUNKS][8];
     float q_mn[CHUNKS], q_inv[CHUNKS];                            // uniform windows: per-chunk min and 1/scale
     uint32_t q_b = 0;                                             // uniform windows: the width; 0 = use the group records
-    bool q_careful = false;
     uint32_t q_gw = 0, q_elems = 0;
     uint32_t n_generic = 0;                                       // windows that took the general bit choice so far
+    uint32_t n_packed = 0;                                        // windows 0 .. n_packed-1 are packed
     bool my_lost = false;
 
-    for (uint32_t j = 0;; j++) {
+    uint32_t j = 0;
+    for (;; j++) {
         // ---------------------------------------------------------------- window j has landed (or there is none)
         if (!mbar_wait_bounded(&s_full[j & 1u], (j >> 1) & 1u)) {
             my_lost = true;
             s_lost = 1u;
             if (lane == 0) record_error(DAF_ERR_TIMEOUT, 0u, 1u + 16u * j);
         }
-        const uint32_t gw = my_lost ? 0xFFFFFFFFu : s_next[j & 3u];
+        const uint32_t gw = my_lost ? 0xFFFFFFFFu : s_next[j & 7u];
         const bool valid = gw < a.total_windows;
         const unsigned char *stage = smem + (j & 1u) * kStageBytes;
 
         // ---------------------------------------------------------------- min / max of window j, contribution to its exchange
         const TensorDesc &td = tensor_of(valid ? gw : 0u);
-        const uint64_t wbase = (uint64_t)(gw - td.first_window) * WE;
-        const uint64_t left = td.numel - wbase;
-        const uint32_t n_elems = left < WE ? (uint32_t)left : WE;
-        const uint32_t n = n_elems >> log2G;                      // groups in window j
-        Budget bud = budget_of(valid ? n : a.n_max);
-        // Fast path candidates: full window, stochastic rounding, groups local to a warp.
-        const bool fast_ok = local && n_elems == WE && !a.nearest && (bud.all_max || bud.need_sep);
-        const bool test_sep = fast_ok && bud.need_sep && bud.ell > 0;
+        const uint32_t w = gw - td.first_window;
+        const bool full = (uint64_t)(w + 1u) * WE <= td.numel;
+        const bool fast_ok = fast_launch && full;
         float lo[CHUNKS], hi[CHUNKS];
         if (valid) {
             float y[CHUNKS][8];                                   // transient: only the min / max are kept
@@ -592,26 +663,35 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                         hi[c] = h;
                     }
                 }
-                if (test_sep) {
-                    // separation test of the uniform outcome: min over groups of the key of the last
-                    // raise taken, max over groups of the key of the first raise not taken
-                    const float v_lo = a.v[bud.ell - 1], v_hi = a.v[bud.ell];
-                    uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+                // Contribution to the window's exchange: the separation test of the uniform outcome
+                // (min over groups of the key of the last raise taken, max over groups of the key of
+                // the first raise not taken) and "some range is so large that 1/scale is not a normal
+                // number" (bit 1 of the flag word: such windows take the careful general path).
+                uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+                float rmax = 0.0f;
 #pragma unroll
-                    for (int c = 0; c < CHUNKS; c++) {
-                        float R = __fsub_rn(hi[c], lo[c]);
-                        if (R < 0x1p-118f) R = 0.0f;              // degenerate group: constant
+                for (int c = 0; c < CHUNKS; c++) {
+                    float R = __fsub_rn(hi[c], lo[c]);
+                    if (R < 0x1p-118f) R = 0.0f;                  // degenerate group: constant
+                    rmax = fmax2(rmax, R);
+                    if (test_sep) {
                         kmin = min(kmin, __float_as_uint(__fmul_rn(R, v_lo)));
                         kmax = max(kmax, __float_as_uint(__fmul_rn(R, v_hi)));
                     }
-                    if (lpu != 32u) {
+                }
+                if (lpu != 32u) {
+                    if (test_sep) {
                         kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
                         kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
                     }
-                    if (lane == 0) {
+                    rmax = __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(rmax)));   // rmax >= 0
+                }
+                if (lane == 0) {
+                    if (test_sep) {
                         atomicMin(&s_kmin[j & 3u], kmin);
                         atomicMax(&s_kmax[j & 3u], kmax);
                     }
+                    if (!(rmax < 0x1p126f)) atomicOr(&s_flag[j & 3u], 2u);
                 }
             }
             if (lane == 0 && s_lost != 0u) atomicOr(&s_flag[j & 3u], 1u);
@@ -622,17 +702,19 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         // ---------------------------------------------------------------- quantize + pack window j-1 (registers -> shared)
         if (j > 0) {
             unsigned char *const s_out = smem + a.lay.out0 + ((j - 1u) % 3u) * a.lay.out_stride;
+            if (j > 3u && !mbar_wait_bounded(&s_free[(j - 1u) % 3u], (((j - 1u) / 3u) - 1u) & 1u)) {
+                s_lost = 1u;                                      // the buffer's previous window never left: give up
+                if (lane == 0) record_error(DAF_ERR_TIMEOUT, q_gw, 9u + 16u * j);
+                break;
+            }
             const TensorDesc &qd = tensor_of(q_gw);
-            const uint64_t qbase = (uint64_t)(q_gw - qd.first_window) * WE;
-            const uint64_t blk0 = ((qd.elem_base + qbase) >> 3) + (e0 >> 3);
+            const uint64_t blk0 = ((qd.elem_base >> 3) + (uint64_t)(q_gw - qd.first_window) * (WE / 8u)) + (e0 >> 3);
             if (q_b != 0u) {
                 if (BATCH) {
                     const PhiloxSeedKeys sk{(uint32_t)qd.seed, (uint32_t)(qd.seed >> 32)};
-                    if (q_careful) quantize_uniform_b<PhiloxSeedKeys, CHUNKS, true>(q_b, x, q_mn, q_inv, e0, blk0, sk, s_out);
-                    else quantize_uniform_b<PhiloxSeedKeys, CHUNKS, false>(q_b, x, q_mn, q_inv, e0, blk0, sk, s_out);
+                    quantize_uniform_b<PhiloxSeedKeys, CHUNKS, false>(q_b, x, q_mn, q_inv, e0, blk0, sk, s_out);
                 } else {
-                    if (q_careful) quantize_uniform_b<PhiloxKeys, CHUNKS, true>(q_b, x, q_mn, q_inv, e0, blk0, a.keys, s_out);
-                    else quantize_uniform_b<PhiloxKeys, CHUNKS, false>(q_b, x, q_mn, q_inv, e0, blk0, a.keys, s_out);
+                    quantize_uniform_b<PhiloxKeys, CHUNKS, false>(q_b, x, q_mn, q_inv, e0, blk0, a.keys, s_out);
                 }
             } else {
                 const GroupRec *grp = s_grp + ((j - 1u) & 1u) * a.n_max;
@@ -673,6 +755,9 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 }
             }
             if (a.bulk_store) fence_async_shared();               // packed bytes visible to the bulk store issued later
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s_ready[(j - 1u) % 3u]);  // this warp's share of window j-1 is packed
+            n_packed = j;
         }
         if (!valid) break;
 
@@ -682,53 +767,52 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             if (lane == 0) record_error(DAF_ERR_TIMEOUT, gw, 6u + 16u * j);
             break;
         }
-        if (s_flag[j & 3u] != 0u) break;                          // some warp ran out of patience: all leave together
-        if (tid == 0) {                                           // recycle the slot two windows ahead
+        const uint32_t flag = s_flag[j & 3u];
+        if (flag & 1u) break;                                     // some warp ran out of patience: all leave together
+        if (tid == 0) {                                           // recycle the slots two windows ahead
             s_kmin[(j + 2u) & 3u] = 0xFFFFFFFFu;
             s_kmax[(j + 2u) & 3u] = 0u;
+            s_flag[(j + 2u) & 3u] = 0u;
         }
-        const bool uniform = fast_ok && (!test_sep || s_kmin[j & 3u] >= s_kmax[j & 3u]);
-        const uint64_t g0 = wbase >> log2G;                       // first group of the window in the tensor
+        const bool uniform = fast_ok && flag == 0u && (!test_sep || s_kmin[j & 3u] >= s_kmax[j & 3u]);
         if (uniform) {
             // -------------------------------------------------------------- every group gets width S[ell]
-            const uint32_t b = a.S[bud.ell];
-            const float Lf = (float)((1u << b) - 1u);
             // lane k of a unit works out (scale, 1/scale) of chunk k's group, then the unit shares them
-            const int k = lane & (int)(lpu - 1u), sb = lane - k;
             float Rk = 0.0f, mnk = 0.0f;
 #pragma unroll
             for (int c = 0; c < CHUNKS; c++)
-                if (k == c) {
+                if (uk == c) {
                     Rk = __fsub_rn(hi[c], lo[c]);
                     mnk = lo[c];
                 }
             if (Rk < 0x1p-118f) Rk = 0.0f;                        // degenerate group: constant
-            const float scale_k = Rk > 0.0f ? __fdiv_rn(Rk, Lf) : 0.0f;
-            const float inv_k = Rk > 0.0f ? __fdiv_rn(Lf, Rk) : 0.0f;
-            if (k < CHUNKS) {
-                const uint32_t eu = (uint32_t)((warp * CHUNKS + k) * 256 + sb * 8);   // first element of the unit
-                if ((eu & (G - 1u)) == 0u) {                      // the unit opens a group: write its metadata
-                    const uint64_t g = g0 + (eu >> log2G);
-                    td.bits[g] = (uint8_t)b;
-                    td.mn[g] = mnk;
-                    td.scale[g] = scale_k;
-                }
+            const float scale_k = Rk > 0.0f ? __fdiv_rn(Rk, fast_L) : 0.0f;
+            const float inv_k = Rk > 0.0f ? __fdiv_rn(fast_L, Rk) : 0.0f;
+            if (meta_lane) {
+                const uint64_t g = (((uint64_t)w * WE) >> log2G) + (unit_elem >> log2G);
+                td.bits[g] = (uint8_t)fast_b;
+                td.mn[g] = mnk;
+                td.scale[g] = scale_k;
             }
 #pragma unroll
             for (int c = 0; c < CHUNKS; c++) {
-                q_inv[c] = __shfl_sync(0xFFFFFFFFu, inv_k, sb + c);
+                q_inv[c] = __shfl_sync(0xFFFFFFFFu, inv_k, usb + c);
                 q_mn[c] = lo[c];
             }
-            // 1/scale not a normal number (range beyond 2^126 * L): the careful quantizer clamps
-            q_careful = __any_sync(0xFFFFFFFFu, Rk > 0.0f && inv_k < 0x1p-126f) != 0;
-            q_b = b;
+            q_b = fast_b;
             if (tid == 0) {
-                const uint32_t total = n * (G >> 3) * b;
-                const bool first = (gw == td.first_window);
+                const uint32_t total = a.n_max * (G >> 3) * fast_b;
+                const bool first = (w == 0u);
                 st_relaxed_u64(a.flags + gw, ((first ? kFlagPrefix : kFlagAggregate) << kFlagShift) | total);
                 s_tot[j & 3u] = total;
             }
         } else {
+            const uint64_t wbase = (uint64_t)w * WE;
+            const uint64_t left = td.numel - wbase;
+            const uint32_t n_elems = left < WE ? (uint32_t)left : WE;
+            const uint32_t n = n_elems >> log2G;                  // groups in window j
+            const Budget bud = budget_of(n);
+            const uint64_t g0 = wbase >> log2G;                   // first group of the window in the tensor
             // -------------------------------------------------------------- general bit choice (owner warps), group records
             const uint32_t owners = (n + 31u) >> 5;               // warps that own group records
             if ((uint32_t)warp < owners) {
@@ -862,21 +946,30 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             }
             n_generic++;
             q_b = 0u;
+            q_elems = n_elems;
         }
         q_gw = gw;
-        q_elems = n_elems;
 
         // ---------------------------------------------------------------- window j: stage -> registers, stage released
         {
             constexpr int kChunkBytes = 256 * Elem<T>::kBytes;
 #pragma unroll
-            for (int c = 0; c < CHUNKS; c++) load8_staged<T>(stage + (warp * CHUNKS + c) * kChunkBytes, lane, x[c]);
+            for (int c = 0; c < CHUNKS; c++) load8_staged<T, true>(stage + (warp * CHUNKS + c) * kChunkBytes, lane, x[c]);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&s_cons[j & 1u]);              // stage consumed, previous window packed
     }
+    // Out of the loop with windows 0 .. n_packed-1 packed: wake the two storer warps, which wait
+    // for windows n_packed and n_packed+1.  The wake-up goes through the same barriers as a packed
+    // window, so it honours the same rule: never before the buffer's previous window has left.
+    if (tid == 0) s_end = n_packed;
+    for (uint32_t q = n_packed; q < n_packed + 2u; q++)
+        if (q >= 3u) mbar_wait_bounded(&s_free[q % 3u], ((q / 3u) - 1u) & 1u);
     __syncwarp();
-    if (lane == 0) mbar_arrive(&s_done);                          // this warp is out of the loop
+    if (lane == 0) {
+        mbar_arrive(&s_ready[n_packed % 3u]);
+        mbar_arrive(&s_ready[(n_packed + 1u) % 3u]);
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -901,9 +994,10 @@ static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint
     return l;
 }
 
-template <typename T, int CHUNKS, bool BATCH>
+template <typename T, int CHUNKS, int NW, bool BATCH>
 static cudaError_t launch(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
+    constexpr int kBlock = NW * 32 + 96;
     static int sms = 0, smem_set = 0, cached_smem = -1, cached_ctas = 0;   // per instantiation, current device
     const int smem = (int)args.lay.total;
     cudaError_t e = cudaSuccess;
@@ -914,31 +1008,33 @@ static cudaError_t launch(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, c
         if (e != cudaSuccess) return e;
     }
     if (smem > smem_set) {
-        e = cudaFuncSetAttribute(compress_kernel<T, CHUNKS, BATCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        e = cudaFuncSetAttribute(compress_kernel<T, CHUNKS, NW, BATCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         smem_set = smem;
     }
     if (smem != cached_smem) {
         int per_sm = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel<T, CHUNKS, BATCH>, kCompressThreads, smem);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel<T, CHUNKS, NW, BATCH>, kBlock, smem);
         if (e != cudaSuccess) return e;
         cached_smem = smem;
         cached_ctas = sms * (per_sm > 0 ? per_sm : 1);
     }
     const uint32_t grid = args.total_windows < (uint32_t)cached_ctas ? args.total_windows : (uint32_t)cached_ctas;
-    compress_kernel<T, CHUNKS, BATCH><<<grid, kCompressThreads, smem, stream>>>(args);
+    compress_kernel<T, CHUNKS, NW, BATCH><<<grid, kBlock, smem, stream>>>(args);
     return cudaGetLastError();
 }
 
+// `chunks4k` = window_elems / 4096: the window is spread over 16 compute warps (a CTA holds at
+// most 1024 threads, and the control warp takes one of its 32 warp slots).
 template <bool BATCH>
-static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
+static cudaError_t dispatch(uint32_t dtype, uint32_t chunks4k, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
                             cudaStream_t stream)
 {
 #define DAF_CASE(T)                                                     \
-    switch (chunks) {                                                   \
-    case 1: return launch<T, 1, BATCH>(args, stream);                   \
-    case 2: return launch<T, 2, BATCH>(args, stream);                   \
-    default: return launch<T, 4, BATCH>(args, stream);                  \
+    switch (chunks4k) {                                                 \
+    case 1: return launch<T, 1, 16, BATCH>(args, stream);               \
+    case 2: return launch<T, 2, 16, BATCH>(args, stream);               \
+    default: return launch<T, 4, 16, BATCH>(args, stream);              \
     }
     if (dtype == DAF_F32) { DAF_CASE(float) }
     if (dtype == DAF_F16) { DAF_CASE(__half) }

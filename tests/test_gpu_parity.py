@@ -128,6 +128,22 @@ def test_signed_zero_minimum_in_full_warp_groups(G):
     assert_decompress_parity(c, ref, "f32", f"signed-zero/G{G}")
 
 
+@pytest.mark.parametrize("G", [64, 256, 2048])
+def test_huge_ranges_where_the_inverse_scale_is_subnormal(G):
+    """Ranges beyond 2^126: 1/scale is a subnormal number and the code clamp can become active."""
+    rng = np.random.default_rng(G + 7)
+    n = 16384 * 3
+    a = rng.random(n).astype(np.float32)
+    big = rng.integers(0, n // G, 8)
+    for g in big:
+        a[g * G:(g + 1) * G] = (rng.random(G) * 1.6e38).astype(np.float32)     # range up to about 2^127
+        a[g * G] = np.float32(1.6e38)
+        a[g * G + 1] = np.float32(0.0)
+    for widths, beta in (((1, 2, 4, 8), 8.0), ((1,), 1.0), ((1, 2, 4, 8), 3.0)):
+        x, c, ref = assert_compress_parity(a, "f32", G, widths, beta, seed=11, label=f"huge/G{G}/{widths}/{beta}")
+        assert_decompress_parity(c, ref, "f32", f"huge/G{G}")
+
+
 def test_heavy_ties_relu6_saturation():
     """Most groups share the same range (clip at 0 and 6): the tie order by group index decides."""
     rng = np.random.default_rng(4)
