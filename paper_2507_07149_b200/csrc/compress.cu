@@ -414,9 +414,11 @@ struct Budget {
     bool need_sep;         // the best raise of level ell does not fit: uniform iff the levels separate
 };
 
-// T: element type; CHUNKS: 256-element chunks per compute warp; NW: compute warps.
-template <typename T, int CHUNKS, int NW, bool BATCH>
-__global__ void __launch_bounds__(NW * 32 + 96, 1)
+// T: element type; CHUNKS: 256-element chunks per compute warp; NW: compute warps; NSTAGE: staged
+// windows per CTA (2: one CTA per SM with a window of look-ahead; 1: two CTAs per SM that cover
+// each other's copy latency); NSTO: storer warps.
+template <typename T, int CHUNKS, int NW, int NSTAGE, int NSTO, bool BATCH>
+__global__ void __launch_bounds__(NW * 32 + 32 + 32 * NSTO, NSTAGE == 1 ? 2 : 1)
 compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> a)
 {
     constexpr int kComputeWarps = NW;
@@ -424,7 +426,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     constexpr uint32_t kStageBytes = WE * Elem<T>::kBytes;
 
     extern __shared__ __align__(128) unsigned char smem[];       // [stage 0 | stage 1 | packed x3 | group arrays]
-    __shared__ __align__(8) uint64_t s_full[2], s_cons[2], s_ready[3], s_free[3], s_exch, s_wid;   // mbarriers
+    __shared__ __align__(8) uint64_t s_full[NSTAGE], s_cons[NSTAGE], s_ready[3], s_free[3], s_exch, s_wid;   // mbarriers
     __shared__ uint32_t s_next[8];                               // ticket of window j
     __shared__ uint32_t s_kmin[4], s_kmax[4], s_flag[4];         // per-window exchange: key extremes, "a wait ran out"
     __shared__ uint32_t s_tot[4];                                // packed bytes of window j
@@ -471,30 +473,38 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         // compute warps have moved window r into registers, stage r & 1 takes window r+2.
         auto issue = [&](uint32_t j, uint32_t t) {
             s_next[j & 7u] = t;
-            uint64_t *bar = &s_full[j & 1u];
+            uint64_t *bar = &s_full[j % NSTAGE];
             if (t < a.total_windows) {
                 const TensorDesc &nd = tensor_of(t);
                 const uint64_t base = (uint64_t)(t - nd.first_window) * WE;
                 const uint64_t left = nd.numel - base;
                 const uint32_t bytes = (uint32_t)(left < WE ? left : WE) * Elem<T>::kBytes;
                 mbar_expect_tx(bar, bytes);
-                bulk_load(smem + (j & 1u) * kStageBytes, reinterpret_cast<const char *>(nd.in) + base * Elem<T>::kBytes, bytes, bar);
+                bulk_load(smem + (j % NSTAGE) * kStageBytes, reinterpret_cast<const char *>(nd.in) + base * Elem<T>::kBytes, bytes, bar);
             } else {
                 mbar_arrive(bar);
             }
         };
-        uint32_t t0 = 0xFFFFFFFFu, t1 = 0xFFFFFFFFu, t2 = 0xFFFFFFFFu;   // tickets of windows r, r+1, r+2
+        uint32_t next_w = 0;                                      // next window index to issue
+        uint32_t tk = 0xFFFFFFFFu;                                // its ticket, reserved ahead of time
+        bool more = true;                                         // no "no more work" window issued yet
+        auto issue_next = [&]() {
+            issue(next_w, tk);
+            more = tk < a.total_windows;
+            next_w++;
+            if (more) tk = atomicAdd(&a.hdr->ticket, 1u);         // its latency is off the compute warps' path
+        };
         if (lane == 0) {
-            mbar_init(&s_full[0], 1);
-            mbar_init(&s_full[1], 1);
-            mbar_init(&s_cons[0], kComputeWarps);
-            mbar_init(&s_cons[1], kComputeWarps);
-            mbar_init(&s_free[0], 1);
-            mbar_init(&s_free[1], 1);
-            mbar_init(&s_free[2], 1);
+            for (int k = 0; k < NSTAGE; k++) {
+                mbar_init(&s_full[k], 1);
+                mbar_init(&s_cons[k], kComputeWarps);
+            }
+            for (int k = 0; k < 3; k++) {
+                mbar_init(&s_ready[k], kComputeWarps);
+                mbar_init(&s_free[k], 1);
+            }
             mbar_init(&s_exch, kComputeWarps);
             mbar_init(&s_wid, kComputeWarps);
-            for (int k = 0; k < 3; k++) mbar_init(&s_ready[k], kComputeWarps);
             s_lost = 0u;
             s_end = 0xFFFFFFFFu;
             for (int k = 0; k < 4; k++) {
@@ -502,47 +512,45 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 s_kmax[k] = 0u;
                 s_flag[k] = 0u;
             }
-            t0 = atomicAdd(&a.hdr->ticket, 1u);
-            issue(0, t0);
-            if (t0 < a.total_windows) t1 = atomicAdd(&a.hdr->ticket, 1u);
-            issue(1, t1);
-            if (t1 < a.total_windows) t2 = atomicAdd(&a.hdr->ticket, 1u);   // reserved ahead: its latency is off the path
+            tk = atomicAdd(&a.hdr->ticket, 1u);
+            for (int k = 0; k < NSTAGE && more; k++) issue_next();
         }
         __syncthreads();
         if (lane != 0) return;
-        for (uint32_t r = 0; t0 < a.total_windows; r++) {
-            if (!mbar_wait_bounded(&s_cons[r & 1u], (r >> 1) & 1u)) {
+        // Round r: once the compute warps have moved window r into registers, its stage takes
+        // window r + NSTAGE.  Windows 0 .. next_w-1 have been issued, the last of them possibly
+        // as "no more work".
+        for (uint32_t r = 0; more || r + 1u < next_w; r++) {
+            if (!mbar_wait_bounded(&s_cons[r % NSTAGE], (r / NSTAGE) & 1u)) {
                 s_lost = 1u;
-                record_error(DAF_ERR_TIMEOUT, t0, 2u + 16u * r);
+                record_error(DAF_ERR_TIMEOUT, s_next[r & 7u], 2u + 16u * r);
             }
             if (s_lost != 0u) {
                 // leaving: windows still held will never be published; copies in flight must land
-                if (t1 < a.total_windows) {
-                    st_relaxed_u64(a.flags + t1, kFlagPoison << kFlagShift);
-                    mbar_wait_bounded(&s_full[(r + 1u) & 1u], ((r + 1u) >> 1) & 1u);
+                for (uint32_t q = r + 1u; q < next_w; q++) {
+                    const uint32_t t = s_next[q & 7u];
+                    if (t < a.total_windows) {
+                        st_relaxed_u64(a.flags + t, kFlagPoison << kFlagShift);
+                        mbar_wait_bounded(&s_full[q % NSTAGE], (q / NSTAGE) & 1u);
+                    }
                 }
-                if (t2 < a.total_windows) st_relaxed_u64(a.flags + t2, kFlagPoison << kFlagShift);
-                s_next[(r + 2u) & 7u] = 0xFFFFFFFFu;
-                mbar_arrive(&s_full[r & 1u]);
+                if (more && tk < a.total_windows) st_relaxed_u64(a.flags + tk, kFlagPoison << kFlagShift);
+                if (more) {                                       // release anyone still waiting for the next window
+                    tk = 0xFFFFFFFFu;
+                    issue_next();
+                }
                 break;
             }
-            if (t1 < a.total_windows) {
-                issue(r + 2u, t2);                                // stage r & 1 is free again
-                t0 = t1;
-                t1 = t2;
-                t2 = t1 < a.total_windows ? atomicAdd(&a.hdr->ticket, 1u) : 0xFFFFFFFFu;
-            } else {
-                t0 = t1;
-            }
+            if (more) issue_next();
         }
         return;
     }
     if (warp > kComputeWarps) {
-        // ============================================================ storer warps (two, alternating windows)
+        // ============================================================ storer warps (taking windows in turn)
         // For window p: once it is packed, find its byte offset by look-back, publish its inclusive
         // prefix, send its packed bytes to global memory with one bulk store, free the buffer.
         __syncthreads();
-        for (uint32_t p = (uint32_t)(warp - kComputeWarps - 1);; p += 2u) {
+        for (uint32_t p = (uint32_t)(warp - kComputeWarps - 1);; p += NSTO) {
             // s_ready[p % 3] fires when window p is packed -- or when the compute warps have left
             // their loop without ever reaching a window p (s_end tells which)
             const bool ok = mbar_wait_bounded(&s_ready[p % 3u], (p / 3u) & 1u);
@@ -624,14 +632,14 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     uint32_t j = 0;
     for (;; j++) {
         // ---------------------------------------------------------------- window j has landed (or there is none)
-        if (!mbar_wait_bounded(&s_full[j & 1u], (j >> 1) & 1u)) {
+        if (!mbar_wait_bounded(&s_full[j % NSTAGE], (j / NSTAGE) & 1u)) {
             my_lost = true;
             s_lost = 1u;
             if (lane == 0) record_error(DAF_ERR_TIMEOUT, 0u, 1u + 16u * j);
         }
         const uint32_t gw = my_lost ? 0xFFFFFFFFu : s_next[j & 7u];
         const bool valid = gw < a.total_windows;
-        const unsigned char *stage = smem + (j & 1u) * kStageBytes;
+        const unsigned char *stage = smem + (j % NSTAGE) * kStageBytes;
 
         // ---------------------------------------------------------------- min / max of window j, contribution to its exchange
         const TensorDesc &td = tensor_of(valid ? gw : 0u);
@@ -957,31 +965,29 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             for (int c = 0; c < CHUNKS; c++) load8_staged<T, true>(stage + (warp * CHUNKS + c) * kChunkBytes, lane, x[c]);
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(&s_cons[j & 1u]);              // stage consumed, previous window packed
+        if (lane == 0) mbar_arrive(&s_cons[j % NSTAGE]);          // stage consumed
     }
-    // Out of the loop with windows 0 .. n_packed-1 packed: wake the two storer warps, which wait
-    // for windows n_packed and n_packed+1.  The wake-up goes through the same barriers as a packed
+    // Out of the loop with windows 0 .. n_packed-1 packed: wake the storer warps, which wait for the
+    // windows from n_packed on.  The wake-up goes through the same barriers as a packed
     // window, so it honours the same rule: never before the buffer's previous window has left.
     if (tid == 0) s_end = n_packed;
-    for (uint32_t q = n_packed; q < n_packed + 2u; q++)
+    for (uint32_t q = n_packed; q < n_packed + NSTO; q++)
         if (q >= 3u) mbar_wait_bounded(&s_free[q % 3u], ((q / 3u) - 1u) & 1u);
     __syncwarp();
-    if (lane == 0) {
-        mbar_arrive(&s_ready[n_packed % 3u]);
-        mbar_arrive(&s_ready[(n_packed + 1u) % 3u]);
-    }
+    if (lane == 0)
+        for (uint32_t q = n_packed; q < n_packed + NSTO; q++) mbar_arrive(&s_ready[q % 3u]);
 }
 
 // ------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------
 // Shared-memory carve-up for one launch configuration.
-static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint32_t window_cap_bytes)
+static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint32_t window_cap_bytes, uint32_t nstage)
 {
     auto up = [](uint32_t v) { return (v + 127u) & ~127u; };
     const uint32_t n_max = we / G, units = we / (G < 256u ? G : 256u);
     SmemLayout l;
-    uint32_t at = 2u * up(we * elem_bytes);                       // two stages
+    uint32_t at = nstage * up(we * elem_bytes);                   // the stages
     l.out0 = at;
     l.out_stride = up(window_cap_bytes < 16u ? 16u : window_cap_bytes);
     at += 3u * l.out_stride;                                      // three packed-bytes buffers
@@ -994,10 +1000,14 @@ static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint
     return l;
 }
 
-template <typename T, int CHUNKS, int NW, bool BATCH>
+// Staged windows per CTA.  Two stages and one CTA per SM measured faster on B200 than one stage
+// and two CTAs per SM (which leaves 56 registers per thread and spills).
+constexpr uint32_t kStages = 2, kStorers = 2;
+
+template <typename T, int CHUNKS, int NW, int NSTAGE, int NSTO, bool BATCH>
 static cudaError_t launch(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
-    constexpr int kBlock = NW * 32 + 96;
+    constexpr int kBlock = NW * 32 + 32 + 32 * NSTO;
     static int sms = 0, smem_set = 0, cached_smem = -1, cached_ctas = 0;   // per instantiation, current device
     const int smem = (int)args.lay.total;
     cudaError_t e = cudaSuccess;
@@ -1008,33 +1018,33 @@ static cudaError_t launch(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, c
         if (e != cudaSuccess) return e;
     }
     if (smem > smem_set) {
-        e = cudaFuncSetAttribute(compress_kernel<T, CHUNKS, NW, BATCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        e = cudaFuncSetAttribute(compress_kernel<T, CHUNKS, NW, NSTAGE, NSTO, BATCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         smem_set = smem;
     }
     if (smem != cached_smem) {
         int per_sm = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel<T, CHUNKS, NW, BATCH>, kBlock, smem);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel<T, CHUNKS, NW, NSTAGE, NSTO, BATCH>, kBlock, smem);
         if (e != cudaSuccess) return e;
         cached_smem = smem;
         cached_ctas = sms * (per_sm > 0 ? per_sm : 1);
     }
     const uint32_t grid = args.total_windows < (uint32_t)cached_ctas ? args.total_windows : (uint32_t)cached_ctas;
-    compress_kernel<T, CHUNKS, NW, BATCH><<<grid, kBlock, smem, stream>>>(args);
+    compress_kernel<T, CHUNKS, NW, NSTAGE, NSTO, BATCH><<<grid, kBlock, smem, stream>>>(args);
     return cudaGetLastError();
 }
 
 // `chunks4k` = window_elems / 4096: the window is spread over 16 compute warps (a CTA holds at
-// most 1024 threads, and the control warp takes one of its 32 warp slots).
+// most 1024 threads, and the service warps take some of its 32 warp slots).
 template <bool BATCH>
 static cudaError_t dispatch(uint32_t dtype, uint32_t chunks4k, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
                             cudaStream_t stream)
 {
-#define DAF_CASE(T)                                                     \
-    switch (chunks4k) {                                                 \
-    case 1: return launch<T, 1, 16, BATCH>(args, stream);               \
-    case 2: return launch<T, 2, 16, BATCH>(args, stream);               \
-    default: return launch<T, 4, 16, BATCH>(args, stream);              \
+#define DAF_CASE(T)                                                                     \
+    switch (chunks4k) {                                                                 \
+    case 1: return launch<T, 1, 16, kStages, kStorers, BATCH>(args, stream);            \
+    case 2: return launch<T, 2, 16, kStages, kStorers, BATCH>(args, stream);            \
+    default: return launch<T, 4, 16, kStages, kStorers, BATCH>(args, stream);           \
     }
     if (dtype == DAF_F32) { DAF_CASE(float) }
     if (dtype == DAF_F16) { DAF_CASE(__half) }
@@ -1062,7 +1072,7 @@ template <int NT> static void fill_common(CompressArgs<NT> &a, const Plan &pl, c
         a.full_rem_after = a.full_rem - (pl.S[a.full_ell] - pl.S[0]) * n;
     }
     a.nbuf = 3;
-    a.lay = make_layout(pl.We, elem_bytes, pl.G, (uint32_t)((((uint64_t)pl.beta_q8 * pl.W) >> 8) * pl.G / 8));
+    a.lay = make_layout(pl.We, elem_bytes, pl.G, (uint32_t)((((uint64_t)pl.beta_q8 * pl.W) >> 8) * pl.G / 8), kStages);
     for (int k = 0; k < kMaxLevels; k++) {
         a.S[k] = pl.S[k];
         a.cost[k] = pl.cost[k];
