@@ -204,3 +204,13 @@ def workload(cfg: int, **kw) -> Workload:
 
 SWEEP_GROUPS = (64, 256, 1024, 4096)
 SWEEP_BUDGETS = (1.0, 2.0, 4.0, 8.0)
+
+
+def shard_range(numel: int, window_elems: int, rank: int, world: int):
+    """Window-aligned slice [lo, hi) of a flat tensor for one rank: whole windows, as even as possible.
+    Compressing the slice with elem_index_base=lo reproduces the bytes of the unsharded run."""
+    n_windows = -(-numel // window_elems)
+    per, extra = divmod(n_windows, world)
+    w_lo = rank * per + min(rank, extra)
+    w_hi = w_lo + per + (1 if rank < extra else 0)
+    return min(w_lo * window_elems, numel), min(w_hi * window_elems, numel)
