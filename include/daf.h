@@ -155,6 +155,37 @@ daf_status daf_decompress_batch(uint32_t n, const daf_params *params, const void
                                 daf_stream stream);
 
 /*
+ * daf_compress without a caller-supplied workspace.  (The paper has no counterpart: this entry
+ * point exists for callers of this library, not for the method.)
+ *
+ * Some callers cannot hand the library scratch memory because they cannot allocate any at the
+ * point where activations are compressed: a training job that has given every free byte of the
+ * device to its own preallocated arena, so that a further cudaMalloc fails; code running inside
+ * a framework allocator's out-of-memory or free-memory callback, where asking that allocator
+ * for a workspace tensor would re-enter it; paths that cannot afford the device-wide
+ * synchronisation an allocation may imply.  For them the scratch of the compress kernel (the
+ * 256-byte header with ticket and status word, and one 64-bit look-back descriptor per window)
+ * lives in a fixed array inside the library's device image: DAF_STATIC_MAX_WINDOWS descriptors,
+ * 512.25 KiB, held by every GPU that loads the library until the process exits.
+ *
+ * Arguments as for daf_compress, minus the workspace.  d_status (device, 4-byte aligned, may be
+ * NULL) receives the device status word (a daf_status) once the stream reaches that point.
+ *   - Tensors with more than DAF_STATIC_MAX_WINDOWS windows (2^30 elements at the default window
+ *     of 16384) are rejected with DAF_ERR_CAPACITY before anything is enqueued.
+ *   - The call allocates and frees nothing, on host or device.  The first call on each device
+ *     looks up the array's device address (with that device current); make that first call
+ *     outside any stream capture.
+ *   - Every call uses the same array.  The part a call needs is cleared on the stream first, so
+ *     stale contents of an earlier call never matter, but two calls that overlap on the GPU (on
+ *     different streams, or from different threads) race on it: serialise them.
+ */
+#define DAF_STATIC_MAX_WINDOWS 65536
+daf_status daf_compress_static(const daf_params *params, const void *d_in, void *d_packed,
+                               uint64_t packed_capacity, uint8_t *d_bits, float *d_min,
+                               float *d_scale, uint64_t *d_window_offsets, uint32_t *d_status,
+                               daf_stream stream);
+
+/*
  * Host-side page pool for packed buffers (Sec. 3.4.2: one preallocated contiguous arena,
  * page-granular first-fit allocation; Sec. 3.4.3: every allocation carries an importance,
  * and the least important one is evicted first).  The pool does bookkeeping only: it never

@@ -50,6 +50,7 @@ SIGNATURES = {
     "daf_sizes": (ctypes.c_int, [ctypes.POINTER(daf_params), _u64p, _u64p, _u64p, _u64p]),
     "daf_compress": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, ctypes.c_uint64, _vp, _vp, _vp, _vp, _vp,
                                     ctypes.c_uint64, _vp]),
+    "daf_compress_static": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, ctypes.c_uint64, _vp, _vp, _vp, _vp, _vp, _vp]),
     "daf_decompress": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_uint64, _vp]),
     "daf_group_offsets": (ctypes.c_int, [_vp, ctypes.c_uint64, ctypes.c_uint32, _vp, _vp, ctypes.c_uint64, _vp]),
     "daf_group_offsets_workspace": (ctypes.c_uint64, [ctypes.c_uint64]),
@@ -144,6 +145,19 @@ def daf_compress(params, d_in, d_packed, packed_capacity, d_bits, d_min, d_scale
     _check(lib().daf_compress(ctypes.byref(params), _ptr(d_in), _ptr(d_packed), packed_capacity, _ptr(d_bits), _ptr(d_min),
                               _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_workspace), workspace_bytes, _stream(stream)),
            "daf_compress")
+
+
+STATIC_MAX_WINDOWS = 65536
+
+
+def daf_compress_static(params, d_in, d_packed, packed_capacity, d_bits, d_min, d_scale, d_window_offsets, d_status=None,
+                        stream=None):
+    """daf_compress for callers that cannot allocate a workspace: the kernel's scratch is a fixed
+    array inside the library (at most STATIC_MAX_WINDOWS windows; calls must not overlap on the GPU).
+    d_status: optional int32 tensor of one element that receives the device status word."""
+    _check(lib().daf_compress_static(ctypes.byref(params), _ptr(d_in), _ptr(d_packed), packed_capacity, _ptr(d_bits),
+                                     _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_status), _stream(stream)),
+           "daf_compress_static")
 
 
 def daf_decompress(params, d_packed, d_bits, d_min, d_scale, d_window_offsets, d_out, d_workspace=None,

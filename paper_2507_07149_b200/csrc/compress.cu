@@ -1114,6 +1114,57 @@ extern "C" daf_status daf_compress(const daf_params *params, const void *d_in, v
     return dispatch<false>(params->dtype, pl.chunks, a, s) == cudaSuccess ? DAF_OK : DAF_ERR_CUDA;
 }
 
+// ------------------------------------------------------------------------------------------
+// Compress with the kernel's scratch in a fixed device array instead of a caller's workspace,
+// for callers that cannot allocate one (see include/daf.h).  In host code the array's name is
+// only a handle: the address a kernel can use comes from cudaGetSymbolAddress, looked up once
+// per device with that device current.
+// ------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[sizeof(WorkspaceHeader) + 8ull * DAF_STATIC_MAX_WINDOWS];
+
+extern "C" daf_status daf_compress_static(const daf_params *params, const void *d_in, void *d_packed,
+                                          uint64_t packed_capacity, uint8_t *d_bits, float *d_min, float *d_scale,
+                                          uint64_t *d_window_offsets, uint32_t *d_status, daf_stream stream)
+{
+    Plan pl;
+    daf_status st = make_plan(params, &pl);
+    if (st != DAF_OK) return st;
+    if (!d_in || !d_packed || !d_bits || !d_min || !d_scale || !d_window_offsets) return DAF_ERR_INVALID_ARG;
+    if (!aligned16(d_in) || !aligned16(d_packed) || (reinterpret_cast<uintptr_t>(d_min) & 3u) ||
+        (reinterpret_cast<uintptr_t>(d_scale) & 3u) || (reinterpret_cast<uintptr_t>(d_window_offsets) & 7u) ||
+        (reinterpret_cast<uintptr_t>(d_status) & 3u))
+        return DAF_ERR_INVALID_ARG;
+    if (pl.n_windows > DAF_STATIC_MAX_WINDOWS) return DAF_ERR_CAPACITY;      // the fixed array has no room for more
+
+    // device address of the array, once per device
+    constexpr int kMaxDevices = 64;
+    static void *scratch_of[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return DAF_ERR_CUDA;
+    if (!scratch_of[dev]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return DAF_ERR_CUDA;
+        scratch_of[dev] = ptr;
+    }
+    void *scratch = scratch_of[dev];
+
+    CompressArgs<1> a;
+    fill_common(a, pl, params, scratch);
+    a.total_windows = (uint32_t)pl.n_windows;
+    a.n_tensors = 1;
+    a.keys = philox_keys(params->seed);
+    a.t[0] = TensorDesc{d_in, reinterpret_cast<uint8_t *>(d_packed), packed_capacity, d_bits, d_min, d_scale,
+                        d_window_offsets, params->numel, params->elem_index_base, params->seed, 0u,
+                        (uint32_t)pl.n_windows};
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    // header (ticket, status) and this call's descriptors must start at zero: the array keeps the last call's contents
+    if (cudaMemsetAsync(scratch, 0, pl.workspace, s) != cudaSuccess) return DAF_ERR_CUDA;
+    if (dispatch<false>(params->dtype, pl.chunks, a, s) != cudaSuccess) return DAF_ERR_CUDA;
+    if (d_status && cudaMemcpyAsync(d_status, scratch, sizeof(uint32_t), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+        return DAF_ERR_CUDA;
+    return DAF_OK;
+}
+
 extern "C" uint64_t daf_batch_workspace(uint32_t n, const daf_params *params)
 {
     uint64_t windows = 0;
