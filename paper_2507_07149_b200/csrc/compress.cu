@@ -39,7 +39,7 @@ struct TensorDesc {
 };
 
 struct SmemLayout {          // byte offsets into dynamic shared memory
-    uint32_t out0, out_stride, umn, umx, key, cum, grp, total;
+    uint32_t out0, out_stride, umn, umx, key, cum, grp, srt, total;
 };
 
 template <int NT> struct CompressArgs {
@@ -430,7 +430,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     __shared__ uint32_t s_next[8];                               // ticket of window j
     __shared__ uint32_t s_kmin[4], s_kmax[4], s_flag[4];         // per-window exchange: key extremes, "a wait ran out"
     __shared__ uint32_t s_tot[4];                                // packed bytes of window j
-    __shared__ uint32_t s_wtot[NW];
+    __shared__ uint32_t s_wtot[NW], s_coll;
     __shared__ uint32_t s_lost, s_end;                           // s_end: number of windows this CTA packed (set on leaving)
 
     float *const s_umn = reinterpret_cast<float *>(smem + a.lay.umn);    // [2][units]
@@ -438,6 +438,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     uint32_t *const s_key = reinterpret_cast<uint32_t *>(smem + a.lay.key);   // [level][n_max]
     uint32_t *const s_cum = reinterpret_cast<uint32_t *>(smem + a.lay.cum);
     GroupRec *const s_grp = reinterpret_cast<GroupRec *>(smem + a.lay.grp);   // [2][n_max]
+    uint32_t *const s_srt = reinterpret_cast<uint32_t *>(smem + a.lay.srt);   // [2][n_max]: sorted group, its range
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t G = a.G, log2G = a.log2G;
@@ -821,33 +822,128 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             const uint32_t n = n_elems >> log2G;                  // groups in window j
             const Budget bud = budget_of(n);
             const uint64_t g0 = wbase >> log2G;                   // first group of the window in the tensor
-            // -------------------------------------------------------------- general bit choice (owner warps), group records
+            // -------------------------------------------------------------- general bit choice, group records
+            // All compute warps take this branch together.  The greedy of Sec. 3.4.1 accepts the
+            // longest prefix of the candidate raises, sorted by (key descending, level ascending,
+            // group ascending), whose summed cost fits the window's budget.  Within one level the
+            // keys fl(R v_k) are a non-decreasing function of the range R, so one ranking of the
+            // groups by (R descending, group ascending) sorts every level at once; a candidate's
+            // position in the merged order then follows from binary searches in the other levels'
+            // sorted keys.  Only if two different ranges round to the same key (their order would then
+            // be by group index, not by range) does the window fall back to ranking by counting.
+            constexpr uint32_t kBarCompute = 2;                   // hardware barrier of the 16 compute warps
+            constexpr uint32_t kComputeThreads = NW * 32u;
             const uint32_t owners = (n + 31u) >> 5;               // warps that own group records
-            if ((uint32_t)warp < owners) {
-                const uint32_t m = a.m, n_max = a.n_max;
+            const uint32_t m = a.m, n_max = a.n_max, nl = a.m - 1u;
+            const bool mine = (uint32_t)tid < n;
+            uint32_t *const s_Rb = s_cum, *const s_rank = s_cum + n_max, *const s_lvl = s_cum + 2u * n_max;
+            uint32_t *const s_sorted = s_srt, *const s_sR = s_srt + n_max;
+            float mn = 0.0f, Rg = 0.0f;
+            if (mine) {
                 const float *umn = s_umn + (j & 1u) * units, *umx = s_umx + (j & 1u) * units;
-                const bool mine = (uint32_t)tid < n;
-                float mn = 0.0f, Rg = 0.0f;
-                if (mine) {
-                    float mx;
-                    if (G > 256u) {
-                        const uint32_t rr = G >> 8;
-                        mn = umn[tid * rr];
-                        mx = umx[tid * rr];
-                        for (uint32_t k = 1; k < rr; k++) {
-                            mn = fmin2(mn, umn[tid * rr + k]);
-                            mx = fmax2(mx, umx[tid * rr + k]);
-                        }
-                    } else {
-                        mn = umn[tid];
-                        mx = umx[tid];
+                float mx;
+                if (G > 256u) {
+                    const uint32_t rr = G >> 8;
+                    mn = umn[tid * rr];
+                    mx = umx[tid * rr];
+                    for (uint32_t k = 1; k < rr; k++) {
+                        mn = fmin2(mn, umn[tid * rr + k]);
+                        mx = fmax2(mx, umx[tid * rr + k]);
                     }
-                    Rg = __fsub_rn(mx, mn);
-                    if (Rg < 0x1p-118f) Rg = 0.0f;                // degenerate group: constant
+                } else {
+                    mn = umn[tid];
+                    mx = umx[tid];
                 }
-                uint32_t level = bud.ell;
-                bool same = bud.all_max;                          // every group ends at level ell
-                if (!bud.all_max) {
+                Rg = __fsub_rn(mx, mn);
+                if (Rg < 0x1p-118f) Rg = 0.0f;                    // degenerate group: constant
+                s_Rb[tid] = __float_as_uint(Rg);
+                s_rank[tid] = 0u;
+                s_lvl[tid] = 0u;
+            }
+            if (tid == 0) s_coll = 0u;
+            bar_sync(kBarCompute, kComputeThreads);
+
+            // Does every group end at level ell after all?  (every warp works it out for itself)
+            bool same = bud.all_max;
+            if (!bud.all_max && bud.need_sep) {
+                // every raise below level ell sorts ahead of every raise from level ell upward (ties go
+                // to the lower level), they all fit, the next does not
+                same = true;
+                if (bud.ell > 0) {
+                    const float vl = a.v[bud.ell - 1], vh = a.v[bud.ell];
+                    uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+                    for (uint32_t g = lane; g < n; g += 32) {
+                        const float R = __uint_as_float(s_Rb[g]);
+                        kmin = min(kmin, __float_as_uint(__fmul_rn(R, vl)));
+                        kmax = max(kmax, __float_as_uint(__fmul_rn(R, vh)));
+                    }
+                    kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+                    kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+                    same = kmin >= kmax;
+                }
+            }
+            uint32_t level = bud.ell;
+            if (!same) {
+                // (1) rank of every group by (range descending, group ascending): the range list is cut
+                //     into slices so that all threads count, a warp reads one range at a time (broadcast)
+                const uint32_t slices = n >= kComputeThreads ? 1u : kComputeThreads / n;
+                const uint32_t len = (n + slices - 1u) / slices;
+                for (uint32_t it = tid; it < n * slices; it += kComputeThreads) {
+                    const uint32_t g = it % n, sl = it / n;
+                    const uint32_t Rb = s_Rb[g];
+                    const uint32_t h1 = min(n, (sl + 1u) * len);
+                    uint32_t cnt = 0;
+                    for (uint32_t h = sl * len; h < h1; h++) {
+                        const uint32_t Rh = s_Rb[h];
+                        cnt += (Rh > Rb) || (Rh == Rb && h < g);
+                    }
+                    if (cnt) atomicAdd(&s_rank[g], cnt);
+                }
+                bar_sync(kBarCompute, kComputeThreads);
+                if (mine) {
+                    const uint32_t r = s_rank[tid];
+                    s_sorted[r] = (uint32_t)tid;
+                    s_sR[r] = __float_as_uint(Rg);
+                }
+                bar_sync(kBarCompute, kComputeThreads);
+                // (2) keys of every level in sorted order
+                for (uint32_t it = tid; it < n * nl; it += kComputeThreads) {
+                    const uint32_t r = it % n, k = it / n;
+                    s_key[k * n_max + r] = __float_as_uint(__fmul_rn(__uint_as_float(s_sR[r]), a.v[k]));
+                }
+                bar_sync(kBarCompute, kComputeThreads);
+                // (3) two different ranges with the same key?
+                for (uint32_t it = tid; it < (n - 1u) * nl; it += kComputeThreads) {
+                    const uint32_t r = it % (n - 1u), k = it / (n - 1u);
+                    if (s_key[k * n_max + r] == s_key[k * n_max + r + 1u] && s_sR[r] != s_sR[r + 1u]) s_coll = 1u;
+                }
+                bar_sync(kBarCompute, kComputeThreads);
+                if (s_coll == 0u) {
+                    // (4) position of every candidate in the merged order -> accepted or not
+                    for (uint32_t it = tid; it < n * nl; it += kComputeThreads) {
+                        const uint32_t r = it % n, k = it / n;
+                        const uint32_t key = s_key[k * n_max + r];
+                        uint32_t cum = (r + 1u) * a.cost[k];
+                        for (uint32_t k2 = 0; k2 < nl; k2++) {
+                            if (k2 == k) continue;
+                            // number of level-k2 candidates sorting ahead: keys >= key (lower level: ties
+                            // first) or keys > key (higher level); the row is non-increasing
+                            const uint32_t *row = s_key + k2 * n_max;
+                            uint32_t lo_i = 0, hi_i = n;
+                            while (lo_i < hi_i) {
+                                const uint32_t mid = (lo_i + hi_i) >> 1;
+                                const bool ahead = k2 < k ? row[mid] >= key : row[mid] > key;
+                                if (ahead) lo_i = mid + 1u; else hi_i = mid;
+                            }
+                            cum += lo_i * a.cost[k2];
+                        }
+                        if (cum <= bud.rem) atomicAdd(&s_lvl[s_sorted[r]], 1u);
+                    }
+                    bar_sync(kBarCompute, kComputeThreads);
+                    if (mine) level = s_lvl[tid];
+                } else if ((uint32_t)warp < owners) {
+                    // Fallback.  For each candidate (group g, raise k) add up the cost of all candidates
+                    // that sort at or ahead of it; the candidate is accepted iff that total fits.
                     if (mine) {
 #pragma unroll
                         for (int k = 0; k < kMaxLevels - 1; k++) {
@@ -857,49 +953,30 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                     }
                     if (owners > 1) bar_sync(kBarOwners, owners * 32u);
                     else __syncwarp();
-                    if (bud.need_sep) {
-                        // Uniform outcome: every raise below level ell sorts ahead of every raise from
-                        // level ell upward (ties go to the lower level), they all fit, the next does not.
-                        same = true;
-                        if (bud.ell > 0) {
-                            uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
-                            for (uint32_t g = lane; g < n; g += 32) {
-                                kmin = min(kmin, s_key[(bud.ell - 1) * n_max + g]);
-                                kmax = max(kmax, s_key[bud.ell * n_max + g]);
-                            }
-                            kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
-                            kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
-                            same = kmin >= kmax;
+                    const uint32_t items = n * nl * nl;
+                    for (uint32_t it = tid; it < items; it += owners * 32u) {
+                        const uint32_t g = it % n, kk = it / n;
+                        const uint32_t k = kk / nl, k2 = kk % nl;
+                        const uint32_t kg = s_key[k * n_max + g];
+                        const uint32_t *row = s_key + k2 * n_max;
+                        uint32_t cnt = 0;
+                        if (k2 < k) {
+                            for (uint32_t h = 0; h < n; h++) cnt += (row[h] >= kg);
+                        } else if (k2 > k) {
+                            for (uint32_t h = 0; h < n; h++) cnt += (row[h] > kg);
+                        } else {
+                            for (uint32_t h = 0; h < n; h++) cnt += (row[h] > kg) || (row[h] == kg && h <= g);
                         }
+                        atomicAdd(&s_cum[k * n_max + g], cnt * a.cost[k2]);
                     }
-                    if (!same) {
-                        // For each candidate (group g, raise k) add up the cost of all candidates that
-                        // sort at or ahead of it (key descending, level ascending, group ascending);
-                        // the candidate is accepted iff that total fits in the budget.
-                        const uint32_t nl = m - 1;
-                        const uint32_t items = n * nl * nl;
-                        for (uint32_t it = tid; it < items; it += owners * 32u) {
-                            const uint32_t g = it % n, kk = it / n;
-                            const uint32_t k = kk / nl, k2 = kk % nl;
-                            const uint32_t kg = s_key[k * n_max + g];
-                            const uint32_t *row = s_key + k2 * n_max;
-                            uint32_t cnt = 0;
-                            if (k2 < k) {
-                                for (uint32_t h = 0; h < n; h++) cnt += (row[h] >= kg);
-                            } else if (k2 > k) {
-                                for (uint32_t h = 0; h < n; h++) cnt += (row[h] > kg);
-                            } else {
-                                for (uint32_t h = 0; h < n; h++) cnt += (row[h] > kg) || (row[h] == kg && h <= g);
-                            }
-                            atomicAdd(&s_cum[k * n_max + g], cnt * a.cost[k2]);
-                        }
-                        if (owners > 1) bar_sync(kBarOwners, owners * 32u);
-                        else __syncwarp();
-                        level = 0;
-                        if (mine)
-                            for (uint32_t k = 0; k + 1 < m; k++) level += (s_cum[k * n_max + tid] <= bud.rem);
-                    }
+                    if (owners > 1) bar_sync(kBarOwners, owners * 32u);
+                    else __syncwarp();
+                    level = 0;
+                    if (mine)
+                        for (uint32_t k = 0; k + 1 < m; k++) level += (s_cum[k * n_max + tid] <= bud.rem);
                 }
+            }
+            if ((uint32_t)warp < owners) {
                 uint32_t size = 0, b = 0;
                 float inv = 0.0f;
                 if (mine) {
@@ -996,6 +1073,7 @@ static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint
     l.key = at; at += up(4u * (kMaxLevels - 1) * n_max);
     l.cum = at; at += up(4u * (kMaxLevels - 1) * n_max);
     l.grp = at; at += up(2u * 16u * n_max);
+    l.srt = at; at += up(2u * 4u * n_max);
     l.total = at;
     return l;
 }
