@@ -39,14 +39,14 @@ struct TensorDesc {
 };
 
 struct SmemLayout {          // byte offsets into dynamic shared memory
-    uint32_t out0, out_stride, umn, umx, key, cum, grp, srt, total;
+    uint32_t out0, out_stride, umn, umx, key, cum, srt, grp, total;
 };
 
 template <int NT> struct CompressArgs {
     WorkspaceHeader *hdr;
     uint64_t *flags;
     uint32_t total_windows, n_tensors;
-    uint32_t G, log2G, beta_q8, m, nearest, bulk_store, n_max, nbuf;
+    uint32_t G, log2G, beta_q8, m, nearest, bulk_store, n_max;
     uint32_t full_ell, full_rem, full_rem_after;   // budget arithmetic of a full window (n_max groups)
     uint32_t S[kMaxLevels], cost[kMaxLevels];
     float v[kMaxLevels];
@@ -80,7 +80,7 @@ __device__ __forceinline__ void quantize8(const float (&x)[8], float mn, float i
         const float d = __fsub_rn(x[i], mn);
         const float s = __fmaf_rn(d, inv, 256.0f);
         const uint32_t h = (i & 1) ? (o[i >> 1] >> 16) : (o[i >> 1] & 0xFFFFu);
-        const uint32_t t = __float_as_uint(s) * 2u + h;           // mod 2^32; 2*bits(256) = 0x87000000
+        const uint32_t t = (__float_as_uint(s) << 1) + h;         // mod 2^32; 2*bits(256) = 0x87000000
         const int pos = (B * i) & 31;                             // bit position of code i in its word (unrolled: constant)
         uint32_t field;
         if (CLAMP) {
@@ -94,6 +94,28 @@ __device__ __forceinline__ void quantize8(const float (&x)[8], float mn, float i
         if (B == 8 && i >= 4) w1 |= field;
         else w0 |= field;
     }
+}
+
+// The same for a width known only at run time (and possibly different in every lane): the
+// codes are clamped to 2^b - 1, then joined pairwise with multiply-adds by 2^b, 2^2b, 2^4b.
+__device__ __forceinline__ void quantize8_any(const float (&x)[8], float mn, float inv, const uint32_t (&o)[4],
+                                              uint32_t b, uint32_t &w0, uint32_t &w1)
+{
+    const uint32_t m1 = 1u << b, L = m1 - 1u, m2 = m1 * m1;
+    const uint32_t m4 = b == 8u ? 0u : m2 * m2;                   // eight 8-bit codes fill two words
+    uint32_t q[8];
+#pragma unroll
+    for (int i = 0; i < 8; i++) {
+        const float d = __fsub_rn(x[i], mn);
+        const float s = __fmaf_rn(d, inv, 256.0f);
+        const uint32_t h = (i & 1) ? (o[i >> 1] >> 16) : (o[i >> 1] & 0xFFFFu);
+        const uint32_t t = __float_as_uint(s) * 2u + h;
+        q[i] = min((t >> 16) - 0x8700u, L);
+    }
+    const uint32_t q01 = q[1] * m1 + q[0], q23 = q[3] * m1 + q[2], q45 = q[5] * m1 + q[4], q67 = q[7] * m1 + q[6];
+    const uint32_t lo = q23 * m2 + q01, hi = q67 * m2 + q45;
+    w0 = hi * m4 + lo;
+    w1 = hi;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -214,32 +236,17 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity
 }
 
 // Eight consecutive elements of a lane from the staged window (two 16-byte shared loads for
-// 4-byte elements, one for 2-byte elements).  For 4-byte elements a lane owns 32 bytes; the
-// two halves are read in an order that depends on the lane so that each quarter-warp touches
-// all 32 banks.  ORDERED = false leaves the halves as read (enough for min / max).
-template <typename T, bool ORDERED> __device__ __forceinline__ void load8_staged(const unsigned char *chunk, int lane, float (&x)[8]);
+// 4-byte elements, one for 2-byte elements).
+template <typename T> __device__ __forceinline__ void load8_staged(const unsigned char *chunk, int lane, float (&x)[8]);
 
-template <> __device__ __forceinline__ void load8_staged<float, false>(const unsigned char *chunk, int lane, float (&x)[8])
+template <> __device__ __forceinline__ void load8_staged<float>(const unsigned char *chunk, int lane, float (&x)[8])
 {
-    const int odd = (lane >> 2) & 1;
-    const unsigned char *p = chunk + lane * 32;
-    const float4 a = *reinterpret_cast<const float4 *>(p + odd * 16);
-    const float4 b = *reinterpret_cast<const float4 *>(p + (odd ^ 1) * 16);
+    const float4 a = *reinterpret_cast<const float4 *>(chunk + lane * 32);
+    const float4 b = *reinterpret_cast<const float4 *>(chunk + lane * 32 + 16);
     x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
     x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
 }
-template <> __device__ __forceinline__ void load8_staged<float, true>(const unsigned char *chunk, int lane, float (&x)[8])
-{
-    const bool odd = (lane >> 2) & 1;
-    float y[8];
-    load8_staged<float, false>(chunk, lane, y);
-#pragma unroll
-    for (int i = 0; i < 4; i++) {
-        x[i] = odd ? y[i + 4] : y[i];
-        x[i + 4] = odd ? y[i] : y[i + 4];
-    }
-}
-template <bool ORDERED> __device__ __forceinline__ void load8_staged_half(const unsigned char *chunk, int lane, float (&x)[8])
+template <> __device__ __forceinline__ void load8_staged<__half>(const unsigned char *chunk, int lane, float (&x)[8])
 {
     const uint4 v = *reinterpret_cast<const uint4 *>(chunk + lane * 16);
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
@@ -250,7 +257,7 @@ template <bool ORDERED> __device__ __forceinline__ void load8_staged_half(const 
         x[2 * i + 1] = f.y;
     }
 }
-template <bool ORDERED> __device__ __forceinline__ void load8_staged_bf16(const unsigned char *chunk, int lane, float (&x)[8])
+template <> __device__ __forceinline__ void load8_staged<__nv_bfloat16>(const unsigned char *chunk, int lane, float (&x)[8])
 {
     const uint4 v = *reinterpret_cast<const uint4 *>(chunk + lane * 16);
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
@@ -260,43 +267,36 @@ template <bool ORDERED> __device__ __forceinline__ void load8_staged_bf16(const 
         x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
     }
 }
-template <> __device__ __forceinline__ void load8_staged<__half, false>(const unsigned char *c, int l, float (&x)[8]) { load8_staged_half<false>(c, l, x); }
-template <> __device__ __forceinline__ void load8_staged<__half, true>(const unsigned char *c, int l, float (&x)[8]) { load8_staged_half<true>(c, l, x); }
-template <> __device__ __forceinline__ void load8_staged<__nv_bfloat16, false>(const unsigned char *c, int l, float (&x)[8]) { load8_staged_bf16<false>(c, l, x); }
-template <> __device__ __forceinline__ void load8_staged<__nv_bfloat16, true>(const unsigned char *c, int l, float (&x)[8]) { load8_staged_bf16<true>(c, l, x); }
 
 // Staged window -> registers, then min / max per unit of LPU lanes (a full warp uses the
-// redux instruction).  Every lane of a unit ends up with the unit's min / max (lo[c], hi[c]);
-// the unit's first lane also writes them to shared memory for the general bit choice.
-// Chunks past a ragged window's end read stale bytes; their results are never used.
+// redux instruction) written to shared memory.  Chunks past a ragged window's end read
+// stale bytes; their results are never used.
 template <typename T, int CHUNKS, int LPU>
 __device__ __forceinline__ void load_and_reduce(const unsigned char *stage, int warp, int lane, float (&x)[CHUNKS][8],
-                                                float (&lo)[CHUNKS], float (&hi)[CHUNKS], float *s_umn, float *s_umx)
+                                                float *s_umn, float *s_umx)
 {
     constexpr int kChunkBytes = 256 * Elem<T>::kBytes;
 #pragma unroll
-    for (int c = 0; c < CHUNKS; c++) load8_staged<T, false>(stage + (warp * CHUNKS + c) * kChunkBytes, lane, x[c]);
+    for (int c = 0; c < CHUNKS; c++) load8_staged<T>(stage + (warp * CHUNKS + c) * kChunkBytes, lane, x[c]);
 #pragma unroll
     for (int c = 0; c < CHUNKS; c++) {
-        float l = fmin3(fmin3(x[c][0], x[c][1], x[c][2]), fmin3(x[c][3], x[c][4], x[c][5]), fmin2(x[c][6], x[c][7]));
-        float h = fmax3(fmax3(x[c][0], x[c][1], x[c][2]), fmax3(x[c][3], x[c][4], x[c][5]), fmax2(x[c][6], x[c][7]));
+        float lo = fmin3(fmin3(x[c][0], x[c][1], x[c][2]), fmin3(x[c][3], x[c][4], x[c][5]), fmin2(x[c][6], x[c][7]));
+        float hi = fmax3(fmax3(x[c][0], x[c][1], x[c][2]), fmax3(x[c][3], x[c][4], x[c][5]), fmax2(x[c][6], x[c][7]));
         if (LPU == 32) {
-            asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(l) : "f"(l));
-            asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(h) : "f"(h));
+            asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(lo) : "f"(lo));
+            asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(hi) : "f"(hi));
         } else {
 #pragma unroll
             for (int off = 1; off < LPU; off <<= 1) {
-                l = fmin2(l, __shfl_xor_sync(0xFFFFFFFFu, l, off));
-                h = fmax2(h, __shfl_xor_sync(0xFFFFFFFFu, h, off));
+                lo = fmin2(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, off));
+                hi = fmax2(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, off));
             }
         }
         if ((lane & (LPU - 1)) == 0) {
             const int u = (warp * CHUNKS + c) * (32 / LPU) + lane / LPU;
-            s_umn[u] = l;
-            s_umx[u] = h;
+            s_umn[u] = lo;
+            s_umx[u] = hi;
         }
-        lo[c] = l;
-        hi[c] = h;
     }
 }
 
@@ -310,81 +310,45 @@ template <int NT> __device__ __forceinline__ uint32_t find_tensor(const Compress
     return lo;
 }
 
-// One persistent CTA per SM: 16 compute warps plus three service warps, synchronised only through
-// shared-memory mbarriers (every wait on them is bounded) except inside the general bit choice.
-//   s_full[s]  : the bulk copy into stage s has landed (or the control warp has marked the
-//                window behind it as "no more work");
-//   s_cons[s]  : all compute warps have moved stage s into registers and have finished packing
-//                the previous window (16 arrivals);
-//   s_exch     : all compute warps have contributed their part of a window's min / max test
-//                (16 arrivals) -- arrival and wait are split so that the exchange of window
-//                j+1 completes while window j is being quantized;
-//   s_wid      : the group records of a window that needed the general bit choice are ready;
-//   s_ready[b] : the window using packed-bytes buffer b is completely packed (16 arrivals);
-//   s_free[b]  : the packed bytes of the window that used buffer b have left shared memory.
-// Window j uses stage j & 1, packed-bytes buffer j % 3 and slot j & 3 (tickets: j & 7) of the
-// small per-window arrays.  A loader warp owns tickets and bulk copies in; two storer warps
-// alternate over the windows for look-back and bulk stores out.
-constexpr uint32_t kBarOwners = 3;
+// The CTA is 16 compute warps plus one control warp; two CTAs share an SM and cover each
+// other's waits.  Hardware barrier 1 ("stage", owner warps and control warp wait, the rest
+// only arrive): the compute warps have moved the staged window into registers, published its
+// per-unit min / max, and finished the previous window's packed bytes.  Barrier 2 ("widths",
+// compute warps): the owners' verdict on the window is in.  Barrier 3 is private to the warps
+// that own group records; barrier 4 separates the steps of the general bit choice.
+constexpr int kComputeWarps = kWarps;
+constexpr int kCompressThreads = kThreads + 32;
+constexpr uint32_t kBarStage = 1, kBarWidths = 2, kBarOwners = 3, kBarChoice = 4;
 
 __device__ __forceinline__ void bar_sync(uint32_t id, uint32_t threads)
 {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+__device__ __forceinline__ void bar_arrive(uint32_t id, uint32_t threads)
+{
+    __threadfence_block();                                        // this thread's shared-memory writes first
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
 }
 
-// Philox4x32-10 for CHUNKS consecutive counter blocks at once (blk0 + 32 c): the rounds of the
-// independent blocks are interleaved in program order so that their long dependency chains
-// overlap.
-template <typename KEYS, int CHUNKS>
-__device__ __forceinline__ void philox_chunks(uint64_t blk0, const KEYS &keys, uint32_t (&o)[CHUNKS][4])
-{
-    uint32_t c0[CHUNKS], c1[CHUNKS], c2[CHUNKS], c3[CHUNKS];
-#pragma unroll
-    for (int c = 0; c < CHUNKS; c++) {
-        const uint64_t blk = blk0 + 32u * c;
-        c0[c] = (uint32_t)blk;
-        c1[c] = (uint32_t)(blk >> 32);
-        c2[c] = 0u;
-        c3[c] = 0u;
-    }
-#pragma unroll
-    for (int r = 0; r < 10; r++) {
-#pragma unroll
-        for (int c = 0; c < CHUNKS; c++) {
-            const uint64_t p0 = (uint64_t)kPhiloxM0 * c0[c], p1 = (uint64_t)kPhiloxM1 * c2[c];
-            c0[c] = (uint32_t)(p1 >> 32) ^ c1[c] ^ philox_key0(keys, r);
-            c1[c] = (uint32_t)p1;
-            c2[c] = (uint32_t)(p0 >> 32) ^ c3[c] ^ philox_key1(keys, r);
-            c3[c] = (uint32_t)p0;
-        }
-    }
-#pragma unroll
-    for (int c = 0; c < CHUNKS; c++) {
-        o[c][0] = c0[c];
-        o[c][1] = c1[c];
-        o[c][2] = c2[c];
-        o[c][3] = c3[c];
-    }
-}
-
-// Quantize + pack CHUNKS chunks that all have width B, with per-chunk (min, 1/scale) in
-// registers: no per-chunk decisions, packed position computed from the element index alone.
-template <typename KEYS, int CHUNKS, int B, bool CLAMP>
-__device__ __forceinline__ void quantize_uniform(const float (&x)[CHUNKS][8], const float (&mn)[CHUNKS],
-                                                 const float (&inv)[CHUNKS], uint32_t e0, uint64_t blk0, const KEYS &keys,
-                                                 unsigned char *s_out)
+// Quantize + pack one window whose groups all have width B (no clamp needed): no per-chunk
+// decisions, packed position computed from the element index alone.
+template <typename KEYS, int CHUNKS, int B>
+__device__ __forceinline__ void quantize_uniform(const float (&x)[CHUNKS][8], const GroupRec *s_grp, uint32_t log2G,
+                                                 uint32_t e0, uint64_t blk0, const KEYS &keys, unsigned char *s_out)
 {
     unsigned char *const out = s_out + (e0 >> 3) * B;
-    uint32_t o[CHUNKS][4];
-    philox_chunks<KEYS, CHUNKS>(blk0, keys, o);
 #pragma unroll
     for (int c = 0; c < CHUNKS; c++) {
+        const float2 mi = *reinterpret_cast<const float2 *>(&s_grp[(e0 + 256u * c) >> log2G]);   // mn, inv
+        uint32_t o[4];
+        const uint64_t blk = blk0 + 32u * c;
+        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), keys, o);
         uint32_t w0, w1;
-        quantize8<B, CLAMP>(x[c], mn[c], inv[c], o[c], w0, w1);
+        quantize8<B, false>(x[c], mi.x, mi.y, o, w0, w1);
         unsigned char *p = out + 32 * B * c;
         if (B == 1) *p = (unsigned char)w0;
         else if (B == 2) *reinterpret_cast<uint16_t *>(p) = (uint16_t)w0;
@@ -393,17 +357,30 @@ __device__ __forceinline__ void quantize_uniform(const float (&x)[CHUNKS][8], co
     }
 }
 
-template <typename KEYS, int CHUNKS, bool CLAMP>
-__device__ __forceinline__ void quantize_uniform_b(uint32_t b, const float (&x)[CHUNKS][8], const float (&mn)[CHUNKS],
-                                                   const float (&inv)[CHUNKS], uint32_t e0, uint64_t blk0, const KEYS &keys,
+template <typename KEYS, int CHUNKS>
+__device__ __forceinline__ void quantize_uniform_b(uint32_t b, const float (&x)[CHUNKS][8], const GroupRec *s_grp,
+                                                   uint32_t log2G, uint32_t e0, uint64_t blk0, const KEYS &keys,
                                                    unsigned char *s_out)
 {
     switch (b) {
-    case 1: quantize_uniform<KEYS, CHUNKS, 1, CLAMP>(x, mn, inv, e0, blk0, keys, s_out); break;
-    case 2: quantize_uniform<KEYS, CHUNKS, 2, CLAMP>(x, mn, inv, e0, blk0, keys, s_out); break;
-    case 4: quantize_uniform<KEYS, CHUNKS, 4, CLAMP>(x, mn, inv, e0, blk0, keys, s_out); break;
-    default: quantize_uniform<KEYS, CHUNKS, 8, CLAMP>(x, mn, inv, e0, blk0, keys, s_out); break;
+    case 1: quantize_uniform<KEYS, CHUNKS, 1>(x, s_grp, log2G, e0, blk0, keys, s_out); break;
+    case 2: quantize_uniform<KEYS, CHUNKS, 2>(x, s_grp, log2G, e0, blk0, keys, s_out); break;
+    case 4: quantize_uniform<KEYS, CHUNKS, 4>(x, s_grp, log2G, e0, blk0, keys, s_out); break;
+    default: quantize_uniform<KEYS, CHUNKS, 8>(x, s_grp, log2G, e0, blk0, keys, s_out); break;
     }
+}
+
+// Number of entries of a non-increasing row that are > key (OR_EQUAL: >= key).
+template <bool OR_EQUAL> __device__ __forceinline__ uint32_t count_above(const uint32_t *row, uint32_t n, uint32_t key)
+{
+    uint32_t lo = 0, hi = n;
+    while (lo < hi) {
+        const uint32_t mid = (lo + hi) >> 1;
+        const bool ahead = OR_EQUAL ? row[mid] >= key : row[mid] > key;
+        if (ahead) lo = mid + 1u;
+        else hi = mid;
+    }
+    return lo;
 }
 
 // Budget arithmetic of a window of n groups.
@@ -414,42 +391,52 @@ struct Budget {
     bool need_sep;         // the best raise of level ell does not fit: uniform iff the levels separate
 };
 
-// T: element type; CHUNKS: 256-element chunks per compute warp; NW: compute warps; NSTAGE: staged
-// windows per CTA (2: one CTA per SM with a window of look-ahead; 1: two CTAs per SM that cover
-// each other's copy latency); NSTO: storer warps.
-template <typename T, int CHUNKS, int NW, int NSTAGE, int NSTO, bool BATCH>
-__global__ void __launch_bounds__(NW * 32 + 32 + 32 * NSTO, NSTAGE == 1 ? 2 : 1)
+template <typename T, int CHUNKS, bool BATCH>
+__global__ void __launch_bounds__(kCompressThreads, 2)
 compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> a)
 {
-    constexpr int kComputeWarps = NW;
-    constexpr uint32_t WE = NW * 256u * CHUNKS;
-    constexpr uint32_t kStageBytes = WE * Elem<T>::kBytes;
+    constexpr uint32_t WE = kThreads * kLaneElems * CHUNKS;
 
-    extern __shared__ __align__(128) unsigned char smem[];       // [stage 0 | stage 1 | packed x3 | group arrays]
-    __shared__ __align__(8) uint64_t s_full[NSTAGE], s_cons[NSTAGE], s_ready[3], s_free[3], s_exch, s_wid;   // mbarriers
-    __shared__ uint32_t s_next[8];                               // ticket of window j
-    __shared__ uint32_t s_kmin[4], s_kmax[4], s_flag[4];         // per-window exchange: key extremes, "a wait ran out"
-    __shared__ uint32_t s_tot[4];                                // packed bytes of window j
-    __shared__ uint32_t s_wtot[NW], s_coll;
-    __shared__ uint32_t s_lost, s_end;                           // s_end: number of windows this CTA packed (set on leaving)
+    extern __shared__ __align__(128) unsigned char smem[];       // [stage | out0 | out1 | group arrays]
+    __shared__ uint32_t s_wtot[kComputeWarps];
+    __shared__ __align__(8) uint64_t s_full;                     // mbarrier: staged window has landed (or there is none)
+    __shared__ uint32_t s_next;                                  // ticket of the staged window
+    __shared__ uint32_t s_lost;                                  // a staged copy did not land in time
+    __shared__ uint32_t s_tot[2];                                // packed bytes of the window of iteration i (slot i & 1)
+    __shared__ uint32_t s_mode[2];                               // how that window's widths came out (see below)
+    __shared__ uint32_t s_slow[2];                               // a group of that window needs the clamped quantizer
 
-    float *const s_umn = reinterpret_cast<float *>(smem + a.lay.umn);    // [2][units]
+    unsigned char *const s_stage = smem;
+    float *const s_umn = reinterpret_cast<float *>(smem + a.lay.umn);         // [2][units]
     float *const s_umx = reinterpret_cast<float *>(smem + a.lay.umx);
-    uint32_t *const s_key = reinterpret_cast<uint32_t *>(smem + a.lay.key);   // [level][n_max]
-    uint32_t *const s_cum = reinterpret_cast<uint32_t *>(smem + a.lay.cum);
-    GroupRec *const s_grp = reinterpret_cast<GroupRec *>(smem + a.lay.grp);   // [2][n_max]
-    uint32_t *const s_srt = reinterpret_cast<uint32_t *>(smem + a.lay.srt);   // [2][n_max]: sorted group, its range
+    uint32_t *const s_key = reinterpret_cast<uint32_t *>(smem + a.lay.key);   // [level][n_max], in rank order
+    uint32_t *const s_cum = reinterpret_cast<uint32_t *>(smem + a.lay.cum);   // [3][n_max]: range, rank, level
+    uint32_t *const s_srt = reinterpret_cast<uint32_t *>(smem + a.lay.srt);   // [2][n_max]: group of rank r, its range
+    GroupRec *const s_grp = reinterpret_cast<GroupRec *>(smem + a.lay.grp);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t G = a.G, log2G = a.log2G;
 
-    auto record_error = [&](unsigned code, uint32_t window, unsigned site) {
-        if (atomicCAS(&a.hdr->status, 0u, code) == 0u) {
-            a.hdr->fail_window = window;
-            a.hdr->fail_site = site;
+    auto tensor_of = [&](uint32_t gw) -> const TensorDesc & { return a.t[BATCH ? find_tensor(a, gw) : 0u]; };
+    // Control lane: takes a ticket and starts the bulk copy of that window into the stage, or
+    // completes the stage's barrier empty-handed when the windows have run out.
+    auto stage_next = [&]() {
+        const uint32_t t = atomicAdd(&a.hdr->ticket, 1u);
+        s_next = t;                                               // ordered before the barrier's completion
+        if (t < a.total_windows) {
+            const TensorDesc &nd = tensor_of(t);
+            const uint64_t base = (uint64_t)(t - nd.first_window) * WE;
+            const uint64_t left = nd.numel - base;
+            const uint32_t bytes = (uint32_t)(left < WE ? left : WE) * Elem<T>::kBytes;
+            mbar_expect_tx(&s_full, bytes);
+            bulk_load(s_stage, reinterpret_cast<const char *>(nd.in) + base * Elem<T>::kBytes, bytes, &s_full);
+        } else {
+            mbar_arrive(&s_full);
         }
     };
-    auto tensor_of = [&](uint32_t gw) -> const TensorDesc & { return a.t[BATCH ? find_tensor(a, gw) : 0u]; };
+    auto record_error = [&](unsigned code, uint32_t window) {
+        if (atomicCAS(&a.hdr->status, 0u, code) == 0u) a.hdr->fail_window = window;
+    };
     auto budget_of = [&](uint32_t n) {
         Budget b;
         uint32_t rem_after = a.full_rem_after;
@@ -467,382 +454,186 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         return b;
     };
 
-    if (warp == kComputeWarps) {
-        // ============================================================ loader warp
-        // Publishes the ticket of window j and starts its bulk copy into stage j & 1, or completes
-        // the stage's barrier empty-handed when there is no such window.  Round r: once the
-        // compute warps have moved window r into registers, stage r & 1 takes window r+2.
-        auto issue = [&](uint32_t j, uint32_t t) {
-            s_next[j & 7u] = t;
-            uint64_t *bar = &s_full[j % NSTAGE];
-            if (t < a.total_windows) {
-                const TensorDesc &nd = tensor_of(t);
-                const uint64_t base = (uint64_t)(t - nd.first_window) * WE;
-                const uint64_t left = nd.numel - base;
-                const uint32_t bytes = (uint32_t)(left < WE ? left : WE) * Elem<T>::kBytes;
-                mbar_expect_tx(bar, bytes);
-                bulk_load(smem + (j % NSTAGE) * kStageBytes, reinterpret_cast<const char *>(nd.in) + base * Elem<T>::kBytes, bytes, bar);
-            } else {
-                mbar_arrive(bar);
-            }
-        };
-        uint32_t next_w = 0;                                      // next window index to issue
-        uint32_t tk = 0xFFFFFFFFu;                                // its ticket, reserved ahead of time
-        bool more = true;                                         // no "no more work" window issued yet
-        auto issue_next = [&]() {
-            issue(next_w, tk);
-            more = tk < a.total_windows;
-            next_w++;
-            if (more) tk = atomicAdd(&a.hdr->ticket, 1u);         // its latency is off the compute warps' path
-        };
-        if (lane == 0) {
-            for (int k = 0; k < NSTAGE; k++) {
-                mbar_init(&s_full[k], 1);
-                mbar_init(&s_cons[k], kComputeWarps);
-            }
-            for (int k = 0; k < 3; k++) {
-                mbar_init(&s_ready[k], kComputeWarps);
-                mbar_init(&s_free[k], 1);
-            }
-            mbar_init(&s_exch, kComputeWarps);
-            mbar_init(&s_wid, kComputeWarps);
-            s_lost = 0u;
-            s_end = 0xFFFFFFFFu;
-            for (int k = 0; k < 4; k++) {
-                s_kmin[k] = 0xFFFFFFFFu;
-                s_kmax[k] = 0u;
-                s_flag[k] = 0u;
-            }
-            tk = atomicAdd(&a.hdr->ticket, 1u);
-            for (int k = 0; k < NSTAGE && more; k++) issue_next();
-        }
-        __syncthreads();
-        if (lane != 0) return;
-        // Round r: once the compute warps have moved window r into registers, its stage takes
-        // window r + NSTAGE.  Windows 0 .. next_w-1 have been issued, the last of them possibly
-        // as "no more work".
-        for (uint32_t r = 0; more || r + 1u < next_w; r++) {
-            if (!mbar_wait_bounded(&s_cons[r % NSTAGE], (r / NSTAGE) & 1u)) {
-                s_lost = 1u;
-                record_error(DAF_ERR_TIMEOUT, s_next[r & 7u], 2u + 16u * r);
-            }
-            if (s_lost != 0u) {
-                // leaving: windows still held will never be published; copies in flight must land
-                for (uint32_t q = r + 1u; q < next_w; q++) {
-                    const uint32_t t = s_next[q & 7u];
-                    if (t < a.total_windows) {
-                        st_relaxed_u64(a.flags + t, kFlagPoison << kFlagShift);
-                        mbar_wait_bounded(&s_full[q % NSTAGE], (q / NSTAGE) & 1u);
-                    }
-                }
-                if (more && tk < a.total_windows) st_relaxed_u64(a.flags + tk, kFlagPoison << kFlagShift);
-                if (more) {                                       // release anyone still waiting for the next window
-                    tk = 0xFFFFFFFFu;
-                    issue_next();
-                }
-                break;
-            }
-            if (more) issue_next();
-        }
-        return;
+    if (tid == kThreads) {
+        mbar_init(&s_full, 1);
+        s_lost = 0u;
+        s_slow[0] = s_slow[1] = 0u;
+        stage_next();
     }
-    if (warp > kComputeWarps) {
-        // ============================================================ storer warps (taking windows in turn)
-        // For window p: once it is packed, find its byte offset by look-back, publish its inclusive
-        // prefix, send its packed bytes to global memory with one bulk store, free the buffer.
-        __syncthreads();
-        for (uint32_t p = (uint32_t)(warp - kComputeWarps - 1);; p += NSTO) {
-            // s_ready[p % 3] fires when window p is packed -- or when the compute warps have left
-            // their loop without ever reaching a window p (s_end tells which)
-            const bool ok = mbar_wait_bounded(&s_ready[p % 3u], (p / 3u) & 1u);
-            if (ok && p >= s_end) break;
-            const uint32_t p_gw = s_next[p & 7u];
-            if (!ok || s_lost != 0u) {
-                s_lost = 1u;
-                if (lane == 0 && !ok) record_error(DAF_ERR_TIMEOUT, 0u, 8u + 16u * p);
-                if (lane == 0 && ok) st_relaxed_u64(a.flags + p_gw, kFlagPoison << kFlagShift);
+    if (tid < kThreads)
+        for (uint32_t i = (uint32_t)tid; i < 2u * a.n_max; i += kThreads) s_cum[a.n_max + i] = 0u;   // ranks and levels count up from zero
+    __syncthreads();
+
+    if (warp == kComputeWarps) {
+        // ============================================================ control warp
+        // Per window i: wait until the compute warps have consumed stage(i) and finished the
+        // packed bytes of window i-1; start the copy of window i+1; then, off the compute
+        // warps' critical path, find window i-1's byte offset by look-back, publish its
+        // inclusive prefix, and send its packed bytes to global memory.
+        uint32_t gw = s_next;
+        bool have_prev = false;
+        uint32_t p_gw = 0;
+        for (uint32_t iter = 0;; iter++) {
+            const bool valid = gw < a.total_windows;
+            bar_sync(kBarStage, kCompressThreads);
+            const bool lost = s_lost != 0u;
+            uint32_t next = 0xFFFFFFFFu;
+            if (valid && !lost) {
+                if (lane == 0) stage_next();
+                __syncwarp();
+                next = s_next;
+            }
+            if (have_prev) {
+                const TensorDesc &pd = tensor_of(p_gw);
+                const uint32_t p_total = s_tot[(iter & 1u) ^ 1u];
+                const unsigned char *src = smem + a.lay.out0 + ((iter & 1u) ^ 1u) * a.lay.out_stride;
+                uint64_t excl = 0;
+                int state = 1;
+                if (p_gw != pd.first_window) {
+                    state = lookback<kLookDepth>(a.flags, p_gw, pd.first_window, lane, true, &excl);
+                    if (lane == 0)
+                        st_relaxed_u64(a.flags + p_gw, state == 1 ? ((kFlagPrefix << kFlagShift) | (excl + p_total))
+                                                                    : (kFlagPoison << kFlagShift));
+                }
+                const uint32_t pw = p_gw - pd.first_window;
+                bool skip = state != 1;
+                if (!skip) {
+                    if (lane == 0) {
+                        pd.woff[pw] = excl;
+                        if (pw + 1 == pd.n_windows) pd.woff[pw + 1] = excl + p_total;
+                    }
+                    skip = excl + p_total > pd.capacity;
+                }
+                if (skip) {
+                    if (lane == 0) record_error(state == -2 ? DAF_ERR_TIMEOUT : DAF_ERR_CAPACITY, p_gw);
+                } else if (a.bulk_store) {
+                    if (lane == 0 && p_total) {
+                        bulk_store(pd.packed + excl, src, p_total);
+                        bulk_store_wait_read();                   // the buffer is packed into again two windows on
+                    }
+                } else {                                          // groups of 32 / 64: windows are only 4-byte aligned
+                    uint32_t *dst = reinterpret_cast<uint32_t *>(pd.packed + excl);
+                    const uint32_t *s32 = reinterpret_cast<const uint32_t *>(src);
+                    for (uint32_t i = lane; i < (p_total >> 2); i += 32) dst[i] = s32[i];
+                }
+            }
+            if (!valid) break;
+            if (lost) {
+                if (lane == 0) {
+                    record_error(DAF_ERR_TIMEOUT, gw);
+                    st_relaxed_u64(a.flags + gw, kFlagPoison << kFlagShift);
+                    mbar_wait_bounded(&s_full, iter & 1u);        // one more bounded chance for the lost copy
+                }
                 break;
             }
-            const TensorDesc &pd = tensor_of(p_gw);
-            const uint32_t p_total = s_tot[p & 3u];
-            const unsigned char *src = smem + a.lay.out0 + (p % 3u) * a.lay.out_stride;
-            uint64_t excl = 0;
-            int state = 1;
-            if (p_gw != pd.first_window) {
-                state = lookback<kLookDepth>(a.flags, p_gw, pd.first_window, lane, true, &excl);
-                if (lane == 0)
-                    st_relaxed_u64(a.flags + p_gw, state == 1 ? ((kFlagPrefix << kFlagShift) | (excl + p_total))
-                                                                : (kFlagPoison << kFlagShift));
-            }
-            const uint32_t pw = p_gw - pd.first_window;
-            bool skip = state != 1;
-            if (!skip) {
-                if (lane == 0) {
-                    pd.woff[pw] = excl;
-                    if (pw + 1 == pd.n_windows) pd.woff[pw + 1] = excl + p_total;
-                }
-                skip = excl + p_total > pd.capacity;
-            }
-            if (skip) {
-                if (lane == 0)
-                    record_error(state == -2 ? DAF_ERR_TIMEOUT : DAF_ERR_CAPACITY, p_gw, state == 1 ? 5u : (state == -2 ? 3u : 4u));
-            } else if (a.bulk_store) {
-                if (lane == 0 && p_total) {
-                    bulk_store(pd.packed + excl, src, p_total);
-                    bulk_store_wait_read();
-                }
-            } else {                                              // groups of 32 / 64: windows are only 4-byte aligned
-                uint32_t *dst = reinterpret_cast<uint32_t *>(pd.packed + excl);
-                const uint32_t *s32 = reinterpret_cast<const uint32_t *>(src);
-                for (uint32_t k = lane; k < (p_total >> 2); k += 32) dst[k] = s32[k];
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&s_free[p % 3u]);          // the buffer may be rewritten from now on
+            have_prev = true;
+            p_gw = gw;
+            gw = next;
         }
         if (lane == 0) bulk_store_wait_all();
         return;
     }
 
     // ================================================================ compute warps
-    __syncthreads();                                              // barriers initialised by the control warp
     const uint32_t e0 = (uint32_t)(warp * CHUNKS * 256 + lane * 8);    // this lane's first element of chunk 0
-    const uint32_t lpu = (G < 256u ? G : 256u) >> 3;              // lanes per unit
     const uint32_t units = WE >> (G < 256u ? log2G : 8u);         // units per window
-    // Launch-wide facts about full windows (the ragged last window of a tensor always takes the
-    // general path): can the quick uniform-width decision apply, and with which numbers?
-    const Budget fb = budget_of(a.n_max);
-    const bool fast_launch = G <= 256u * CHUNKS && !a.nearest && (fb.all_max || fb.need_sep);
-    const bool test_sep = fast_launch && fb.need_sep && fb.ell > 0;
-    const uint32_t fast_b = a.S[fb.ell];
-    const float fast_L = (float)((1u << fast_b) - 1u);
-    const float v_lo = a.v[fb.ell > 0 ? fb.ell - 1 : 0], v_hi = a.v[fb.ell];
-    // lane k of a unit looks after chunk k's group in the uniform case
-    const int uk = lane & (int)(lpu - 1u), usb = lane - uk;
-    const uint32_t unit_elem = (uint32_t)((warp * CHUNKS + uk) * 256 + usb * 8);   // first element of that unit
-    const bool meta_lane = uk < CHUNKS && (unit_elem & (G - 1u)) == 0u;            // the unit opens a group
-
-    // the window being quantized (registers) and how
-    float x[CHUNKS][8];
-    float q_mn[CHUNKS], q_inv[CHUNKS];                            // uniform windows: per-chunk min and 1/scale
-    uint32_t q_b = 0;                                             // uniform windows: the width; 0 = use the group records
-    uint32_t q_gw = 0, q_elems = 0;
-    uint32_t n_generic = 0;                                       // windows that took the general bit choice so far
-    uint32_t n_packed = 0;                                        // windows 0 .. n_packed-1 are packed
-    bool my_lost = false;
-
-    uint32_t j = 0;
-    for (;; j++) {
-        // ---------------------------------------------------------------- window j has landed (or there is none)
-        if (!mbar_wait_bounded(&s_full[j % NSTAGE], (j / NSTAGE) & 1u)) {
-            my_lost = true;
+    const uint32_t n_max = a.n_max, nl = a.m - 1u;
+    for (uint32_t iter = 0;; iter++) {
+        // ---------------------------------------------------------------- the staged window has landed (or there is none)
+        bool lost = false;
+        if (!mbar_wait_bounded(&s_full, iter & 1u)) {
             s_lost = 1u;
-            if (lane == 0) record_error(DAF_ERR_TIMEOUT, 0u, 1u + 16u * j);
+            lost = true;
         }
-        const uint32_t gw = my_lost ? 0xFFFFFFFFu : s_next[j & 7u];
-        const bool valid = gw < a.total_windows;
-        const unsigned char *stage = smem + (j % NSTAGE) * kStageBytes;
-
-        // ---------------------------------------------------------------- min / max of window j, contribution to its exchange
-        const TensorDesc &td = tensor_of(valid ? gw : 0u);
+        const uint32_t gw = lost ? 0u : s_next;
+        if (!lost && gw >= a.total_windows) break;
+        unsigned char *const s_out = smem + a.lay.out0 + (iter & 1u) * a.lay.out_stride;
+        const TensorDesc &td = tensor_of(gw);
         const uint32_t w = gw - td.first_window;
-        const bool full = (uint64_t)(w + 1u) * WE <= td.numel;
-        const bool fast_ok = fast_launch && full;
-        float lo[CHUNKS], hi[CHUNKS];
-        if (valid) {
-            float y[CHUNKS][8];                                   // transient: only the min / max are kept
-            float *umn = s_umn + (j & 1u) * units, *umx = s_umx + (j & 1u) * units;
-            if (lpu == 32u) load_and_reduce<T, CHUNKS, 32>(stage, warp, lane, y, lo, hi, umn, umx);
-            else if (lpu == 16u) load_and_reduce<T, CHUNKS, 16>(stage, warp, lane, y, lo, hi, umn, umx);
-            else if (lpu == 8u) load_and_reduce<T, CHUNKS, 8>(stage, warp, lane, y, lo, hi, umn, umx);
-            else load_and_reduce<T, CHUNKS, 4>(stage, warp, lane, y, lo, hi, umn, umx);
-            if (fast_ok) {
-                // groups of 512 / 1024 span 2 / 4 chunks of this warp
-                if (G == 512u) {
-#pragma unroll
-                    for (int c = 0; c + 1 < CHUNKS; c += 2) {
-                        lo[c] = lo[c + 1] = fmin2(lo[c], lo[c + 1]);
-                        hi[c] = hi[c + 1] = fmax2(hi[c], hi[c + 1]);
-                    }
-                } else if (G == 1024u && CHUNKS == 4) {
-                    const float l = fmin2(fmin2(lo[0], lo[1]), fmin2(lo[2], lo[3]));
-                    const float h = fmax2(fmax2(hi[0], hi[1]), fmax2(hi[2], hi[3]));
-#pragma unroll
-                    for (int c = 0; c < CHUNKS; c++) {
-                        lo[c] = l;
-                        hi[c] = h;
-                    }
-                }
-                // Contribution to the window's exchange: the separation test of the uniform outcome
-                // (min over groups of the key of the last raise taken, max over groups of the key of
-                // the first raise not taken) and "some range is so large that 1/scale is not a normal
-                // number" (bit 1 of the flag word: such windows take the careful general path).
-                uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
-                float rmax = 0.0f;
-#pragma unroll
-                for (int c = 0; c < CHUNKS; c++) {
-                    float R = __fsub_rn(hi[c], lo[c]);
-                    if (R < 0x1p-118f) R = 0.0f;                  // degenerate group: constant
-                    rmax = fmax2(rmax, R);
-                    if (test_sep) {
-                        kmin = min(kmin, __float_as_uint(__fmul_rn(R, v_lo)));
-                        kmax = max(kmax, __float_as_uint(__fmul_rn(R, v_hi)));
-                    }
-                }
-                if (lpu != 32u) {
-                    if (test_sep) {
-                        kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
-                        kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
-                    }
-                    rmax = __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(rmax)));   // rmax >= 0
-                }
-                if (lane == 0) {
-                    if (test_sep) {
-                        atomicMin(&s_kmin[j & 3u], kmin);
-                        atomicMax(&s_kmax[j & 3u], kmax);
-                    }
-                    if (!(rmax < 0x1p126f)) atomicOr(&s_flag[j & 3u], 2u);
-                }
-            }
-            if (lane == 0 && s_lost != 0u) atomicOr(&s_flag[j & 3u], 1u);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&s_exch);
-        }
+        const uint64_t wbase = (uint64_t)w * WE;
+        const uint64_t left = td.numel - wbase;
+        const uint32_t n_elems = left < WE ? (uint32_t)left : WE;
+        const uint32_t n = n_elems >> log2G;                      // groups in this window
+        float *const umn = s_umn + (iter & 1u) * units, *const umx = s_umx + (iter & 1u) * units;
 
-        // ---------------------------------------------------------------- quantize + pack window j-1 (registers -> shared)
-        if (j > 0) {
-            unsigned char *const s_out = smem + a.lay.out0 + ((j - 1u) % 3u) * a.lay.out_stride;
-            if (j > 3u && !mbar_wait_bounded(&s_free[(j - 1u) % 3u], (((j - 1u) / 3u) - 1u) & 1u)) {
-                s_lost = 1u;                                      // the buffer's previous window never left: give up
-                if (lane == 0) record_error(DAF_ERR_TIMEOUT, q_gw, 9u + 16u * j);
-                break;
-            }
-            const TensorDesc &qd = tensor_of(q_gw);
-            const uint64_t blk0 = ((qd.elem_base >> 3) + (uint64_t)(q_gw - qd.first_window) * (WE / 8u)) + (e0 >> 3);
-            if (q_b != 0u) {
-                if (BATCH) {
-                    const PhiloxSeedKeys sk{(uint32_t)qd.seed, (uint32_t)(qd.seed >> 32)};
-                    quantize_uniform_b<PhiloxSeedKeys, CHUNKS, false>(q_b, x, q_mn, q_inv, e0, blk0, sk, s_out);
-                } else {
-                    quantize_uniform_b<PhiloxKeys, CHUNKS, false>(q_b, x, q_mn, q_inv, e0, blk0, a.keys, s_out);
-                }
-            } else {
-                const GroupRec *grp = s_grp + ((j - 1u) & 1u) * a.n_max;
-#pragma unroll
-                for (int c = 0; c < CHUNKS; c++) {
-                    const uint32_t e = e0 + 256u * c;
-                    const GroupRec rec = grp[e >> log2G];
-                    uint32_t o[4];
-                    if (a.nearest) {
-                        o[0] = o[1] = o[2] = o[3] = 0x80008000u;   // every 16-bit lane = 2 * 2^14
-                    } else {
-                        const uint64_t blk = blk0 + 32u * c;
-                        if (BATCH) {
-                            const PhiloxSeedKeys sk{(uint32_t)qd.seed, (uint32_t)(qd.seed >> 32)};
-                            philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), sk, o);
-                        } else {
-                            philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), a.keys, o);
-                        }
-                    }
-                    uint32_t w0, w1;
-                    unsigned char *p = s_out + rec.off + ((e & (G - 1u)) >> 3) * rec.b;
-                    if (e < q_elems) {
-                        switch (rec.b) {
-                        case 1: quantize8<1, true>(x[c], rec.mn, rec.inv, o, w0, w1); *p = (unsigned char)w0; break;
-                        case 2: quantize8<2, true>(x[c], rec.mn, rec.inv, o, w0, w1); *reinterpret_cast<uint16_t *>(p) = (uint16_t)w0; break;
-                        case 4: quantize8<4, true>(x[c], rec.mn, rec.inv, o, w0, w1); *reinterpret_cast<uint32_t *>(p) = w0; break;
-                        default:
-                            quantize8<8, true>(x[c], rec.mn, rec.inv, o, w0, w1);
-                            if (G >= 64u) {
-                                *reinterpret_cast<uint2 *>(p) = make_uint2(w0, w1);
-                            } else {                               // G = 32: groups are only 4-byte aligned
-                                reinterpret_cast<uint32_t *>(p)[0] = w0;
-                                reinterpret_cast<uint32_t *>(p)[1] = w1;
-                            }
-                            break;
-                        }
-                    }
-                }
-            }
-            if (a.bulk_store) fence_async_shared();               // packed bytes visible to the bulk store issued later
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&s_ready[(j - 1u) % 3u]);  // this warp's share of window j-1 is packed
-            n_packed = j;
-        }
-        if (!valid) break;
-
-        // ---------------------------------------------------------------- the exchange of window j is complete: widths
-        if (!mbar_wait_bounded(&s_exch, j & 1u)) {
-            s_lost = 1u;
-            if (lane == 0) record_error(DAF_ERR_TIMEOUT, gw, 6u + 16u * j);
-            break;
-        }
-        const uint32_t flag = s_flag[j & 3u];
-        if (flag & 1u) break;                                     // some warp ran out of patience: all leave together
-        if (tid == 0) {                                           // recycle the slots two windows ahead
-            s_kmin[(j + 2u) & 3u] = 0xFFFFFFFFu;
-            s_kmax[(j + 2u) & 3u] = 0u;
-            s_flag[(j + 2u) & 3u] = 0u;
-        }
-        const bool uniform = fast_ok && flag == 0u && (!test_sep || s_kmin[j & 3u] >= s_kmax[j & 3u]);
-        if (uniform) {
-            // -------------------------------------------------------------- every group gets width S[ell]
-            // lane k of a unit works out (scale, 1/scale) of chunk k's group, then the unit shares them
-            float Rk = 0.0f, mnk = 0.0f;
-#pragma unroll
-            for (int c = 0; c < CHUNKS; c++)
-                if (uk == c) {
-                    Rk = __fsub_rn(hi[c], lo[c]);
-                    mnk = lo[c];
-                }
-            if (Rk < 0x1p-118f) Rk = 0.0f;                        // degenerate group: constant
-            const float scale_k = Rk > 0.0f ? __fdiv_rn(Rk, fast_L) : 0.0f;
-            const float inv_k = Rk > 0.0f ? __fdiv_rn(fast_L, Rk) : 0.0f;
-            if (meta_lane) {
-                const uint64_t g = (((uint64_t)w * WE) >> log2G) + (unit_elem >> log2G);
-                td.bits[g] = (uint8_t)fast_b;
-                td.mn[g] = mnk;
-                td.scale[g] = scale_k;
-            }
-#pragma unroll
-            for (int c = 0; c < CHUNKS; c++) {
-                q_inv[c] = __shfl_sync(0xFFFFFFFFu, inv_k, usb + c);
-                q_mn[c] = lo[c];
-            }
-            q_b = fast_b;
-            if (tid == 0) {
-                const uint32_t total = a.n_max * (G >> 3) * fast_b;
-                const bool first = (w == 0u);
-                st_relaxed_u64(a.flags + gw, ((first ? kFlagPrefix : kFlagAggregate) << kFlagShift) | total);
-                s_tot[j & 3u] = total;
-            }
-        } else {
-            const uint64_t wbase = (uint64_t)w * WE;
-            const uint64_t left = td.numel - wbase;
-            const uint32_t n_elems = left < WE ? (uint32_t)left : WE;
-            const uint32_t n = n_elems >> log2G;                  // groups in window j
-            const Budget bud = budget_of(n);
-            const uint64_t g0 = wbase >> log2G;                   // first group of the window in the tensor
-            // -------------------------------------------------------------- general bit choice, group records
-            // All compute warps take this branch together.  The greedy of Sec. 3.4.1 accepts the
-            // longest prefix of the candidate raises, sorted by (key descending, level ascending,
-            // group ascending), whose summed cost fits the window's budget.  Within one level the
-            // keys fl(R v_k) are a non-decreasing function of the range R, so one ranking of the
-            // groups by (R descending, group ascending) sorts every level at once; a candidate's
-            // position in the merged order then follows from binary searches in the other levels'
-            // sorted keys.  Only if two different ranges round to the same key (their order would then
-            // be by group index, not by range) does the window fall back to ranking by counting.
-            constexpr uint32_t kBarCompute = 2;                   // hardware barrier of the 16 compute warps
-            constexpr uint32_t kComputeThreads = NW * 32u;
-            const uint32_t owners = (n + 31u) >> 5;               // warps that own group records
-            const uint32_t m = a.m, n_max = a.n_max, nl = a.m - 1u;
-            const bool mine = (uint32_t)tid < n;
-            uint32_t *const s_Rb = s_cum, *const s_rank = s_cum + n_max, *const s_lvl = s_cum + 2u * n_max;
-            uint32_t *const s_sorted = s_srt, *const s_sR = s_srt + n_max;
-            float mn = 0.0f, Rg = 0.0f;
+        // ---------------------------------------------------------------- staged window -> registers, unit min / max
+        float x[CHUNKS][8];
+        if (G >= 256u) load_and_reduce<T, CHUNKS, 32>(s_stage, warp, lane, x, umn, umx);
+        else if (G == 128u) load_and_reduce<T, CHUNKS, 16>(s_stage, warp, lane, x, umn, umx);
+        else if (G == 64u) load_and_reduce<T, CHUNKS, 8>(s_stage, warp, lane, x, umn, umx);
+        else load_and_reduce<T, CHUNKS, 4>(s_stage, warp, lane, x, umn, umx);
+        // ---------------------------------------------------------------- widths, first try: one width for all
+        // The warps that own group records (thread g: group g) test whether every group ends at
+        // level ell: every raise below level ell must sort ahead of every raise from level ell
+        // upward (ties go to the lower level); they all fit and the next does not.  If so they
+        // write the records at once; otherwise all compute warps share the general choice below.
+        const Budget bud = budget_of(n);
+        const uint64_t g0 = wbase >> log2G;                       // first group of the window in the tensor
+        const uint32_t owners = (n + 31u) >> 5;
+        const bool owner = (uint32_t)warp < owners, mine = (uint32_t)tid < n;
+        const bool big = G > 256u;                                // a group spans several 256-element units
+        float mn = 0.0f, Rg = 0.0f;
+        // Owner threads: records, metadata, window total.  level_of: this thread's level.
+        auto write_records = [&](uint32_t level, bool uniform_b) {
+            uint32_t size = 0, b = 0;
+            float inv = 0.0f;
             if (mine) {
-                const float *umn = s_umn + (j & 1u) * units, *umx = s_umx + (j & 1u) * units;
+                b = a.S[level];
+                const float Lf = (float)((1u << b) - 1u);
+                const float scale = Rg > 0.0f ? __fdiv_rn(Rg, Lf) : 0.0f;
+                inv = Rg > 0.0f ? __fdiv_rn(Lf, Rg) : 0.0f;
+                // 1/scale not a normal number: codes may need the clamp, take the careful quantizer
+                if (Rg > 0.0f && inv < 0x1p-126f) s_slow[iter & 1u] = 1u;
+                td.bits[g0 + tid] = (uint8_t)b;
+                td.mn[g0 + tid] = mn;
+                td.scale[g0 + tid] = scale;
+                size = (G >> 3) * b;
+            }
+            uint32_t total, off;
+            if (uniform_b) {
+                off = (uint32_t)tid * size;
+                total = n * (G >> 3) * a.S[level];
+            } else {
+                // byte offset of each group inside the window: exclusive scan of the sizes
+                uint32_t incl = size, before = 0;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                    if (lane >= o) incl += y;
+                }
+                total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                if (owners > 1) {
+                    if (lane == 0) s_wtot[warp] = total;
+                    bar_sync(kBarOwners, owners * 32u);
+                    total = 0;
+                    for (uint32_t k = 0; k < owners; k++) {
+                        const uint32_t t = s_wtot[k];
+                        if (k < (uint32_t)warp) before += t;
+                        total += t;
+                    }
+                }
+                off = before + incl - size;
+            }
+            if (mine) {
+                GroupRec rec;
+                rec.mn = mn;
+                rec.inv = inv;
+                rec.b = b;
+                rec.off = off;
+                s_grp[tid] = rec;
+            }
+            if (tid == 0) {
+                // the window's byte count is known: publish it at once
+                st_relaxed_u64(a.flags + gw, ((w == 0u ? kFlagPrefix : kFlagAggregate) << kFlagShift) | total);
+                s_tot[iter & 1u] = total;
+            }
+        };
+        if (owner) {
+            bar_sync(kBarStage, kCompressThreads);                // every unit's min / max is visible; the stage is free
+            if (tid == 0) s_slow[(iter & 1u) ^ 1u] = 0u;          // reset the flag of the next window
+            if (mine) {
                 float mx;
-                if (G > 256u) {
+                if (big) {
                     const uint32_t rr = G >> 8;
                     mn = umn[tid * rr];
                     mx = umx[tid * rr];
@@ -856,236 +647,199 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 }
                 Rg = __fsub_rn(mx, mn);
                 if (Rg < 0x1p-118f) Rg = 0.0f;                    // degenerate group: constant
-                s_Rb[tid] = __float_as_uint(Rg);
-                s_rank[tid] = 0u;
-                s_lvl[tid] = 0u;
             }
-            if (tid == 0) s_coll = 0u;
-            bar_sync(kBarCompute, kComputeThreads);
-
-            // Does every group end at level ell after all?  (every warp works it out for itself)
-            bool same = bud.all_max;
-            if (!bud.all_max && bud.need_sep) {
-                // every raise below level ell sorts ahead of every raise from level ell upward (ties go
-                // to the lower level), they all fit, the next does not
-                same = true;
-                if (bud.ell > 0) {
-                    const float vl = a.v[bud.ell - 1], vh = a.v[bud.ell];
-                    uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+            bool uniform = bud.all_max || bud.need_sep;
+            if (bud.need_sep && bud.ell > 0) {
+                // each owner warp evaluates the test over all groups itself
+                const float vl = a.v[bud.ell - 1], vh = a.v[bud.ell];
+                uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+                if (owners == 1) {
+                    if (mine) {
+                        kmin = __float_as_uint(__fmul_rn(Rg, vl));
+                        kmax = __float_as_uint(__fmul_rn(Rg, vh));
+                    }
+                } else {                                          // groups of at most 256: one unit per group
                     for (uint32_t g = lane; g < n; g += 32) {
-                        const float R = __uint_as_float(s_Rb[g]);
+                        float R = __fsub_rn(umx[g], umn[g]);
+                        if (R < 0x1p-118f) R = 0.0f;
                         kmin = min(kmin, __float_as_uint(__fmul_rn(R, vl)));
                         kmax = max(kmax, __float_as_uint(__fmul_rn(R, vh)));
                     }
-                    kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
-                    kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
-                    same = kmin >= kmax;
                 }
+                kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+                kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+                uniform = kmin >= kmax;
             }
-            uint32_t level = bud.ell;
-            if (!same) {
-                // (1) rank of every group by (range descending, group ascending): the range list is cut
-                //     into slices so that all threads count, a warp reads one range at a time (broadcast)
-                const uint32_t slices = n >= kComputeThreads ? 1u : kComputeThreads / n;
-                const uint32_t len = (n + slices - 1u) / slices;
-                for (uint32_t it = tid; it < n * slices; it += kComputeThreads) {
-                    const uint32_t g = it % n, sl = it / n;
+            if (s_lost == 0u) {
+                if (uniform) write_records(bud.ell, true);
+                if (tid == 0) s_mode[iter & 1u] = !uniform ? 0u : (n_elems == WE && !a.nearest) ? 1u + a.S[bud.ell] : 1u;
+            }
+        } else {
+            bar_arrive(kBarStage, kCompressThreads);
+        }
+        bar_sync(kBarWidths, kThreads);                           // records (or the news that there are none yet) visible
+        if (s_lost != 0u) break;
+        const uint32_t mode = s_mode[iter & 1u];                  // 0: general choice needed; 1: records; 1 + b: one width b
+        const uint64_t blk0 = ((td.elem_base + wbase) >> 3) + (e0 >> 3);
+
+        if (mode == 0u) {
+            // -------------------------------------------------------------- general bit choice
+            // The greedy of Sec. 3.4.1 accepts the longest prefix of the candidate raises, sorted by
+            // (key descending, level ascending, group ascending), whose summed cost fits the window's
+            // budget.  Within one level the keys fl(R v_k) are a non-decreasing function of the range
+            // R, so one ranking of the groups by (R descending, group ascending) sorts every level at
+            // once.  All compute threads count ranks; the owner of a group files its keys in rank
+            // order; then every thread places one candidate in the merged order by binary searches
+            // in the levels' sorted keys and accepts it if everything up to and including it fits.
+            uint32_t *const s_Rb = s_cum, *const s_rank = s_cum + n_max, *const s_lvl = s_cum + 2u * n_max;
+            uint32_t *const s_sorted = s_srt, *const s_sR = s_srt + n_max;
+            if (mine) s_Rb[tid] = __float_as_uint(Rg);            // the ranges, side by side
+            bar_sync(kBarChoice, kThreads);
+            const bool pow2 = (n & (n - 1u)) == 0u;
+            const uint32_t sh = 31u - (uint32_t)__clz(n);
+            // (1) rank of every group by (range descending, group ascending).  Thread (g, slice)
+            //     counts the groups of its slice that sort ahead of g; a warp's lanes share the slice,
+            //     so its loads are broadcasts.
+            {
+                const uint32_t slices = (uint32_t)kThreads / n;   // n <= 512
+                const uint32_t g = pow2 ? (uint32_t)tid & (n - 1u) : (uint32_t)tid % n;
+                const uint32_t sl = pow2 ? (uint32_t)tid >> sh : (uint32_t)tid / n;
+                if (sl < slices) {
+                    const uint32_t len = (n + slices - 1u) / slices;
+                    const uint32_t h0 = sl * len, h1 = min(n, h0 + len);
                     const uint32_t Rb = s_Rb[g];
-                    const uint32_t h1 = min(n, (sl + 1u) * len);
                     uint32_t cnt = 0;
-                    for (uint32_t h = sl * len; h < h1; h++) {
+#pragma unroll 4
+                    for (uint32_t h = h0; h < h1; h++) {
                         const uint32_t Rh = s_Rb[h];
                         cnt += (Rh > Rb) || (Rh == Rb && h < g);
                     }
                     if (cnt) atomicAdd(&s_rank[g], cnt);
                 }
-                bar_sync(kBarCompute, kComputeThreads);
-                if (mine) {
-                    const uint32_t r = s_rank[tid];
-                    s_sorted[r] = (uint32_t)tid;
-                    s_sR[r] = __float_as_uint(Rg);
-                }
-                bar_sync(kBarCompute, kComputeThreads);
-                // (2) keys of every level in sorted order
-                for (uint32_t it = tid; it < n * nl; it += kComputeThreads) {
-                    const uint32_t r = it % n, k = it / n;
-                    s_key[k * n_max + r] = __float_as_uint(__fmul_rn(__uint_as_float(s_sR[r]), a.v[k]));
-                }
-                bar_sync(kBarCompute, kComputeThreads);
-                // (3) two different ranges with the same key?
-                for (uint32_t it = tid; it < (n - 1u) * nl; it += kComputeThreads) {
-                    const uint32_t r = it % (n - 1u), k = it / (n - 1u);
-                    if (s_key[k * n_max + r] == s_key[k * n_max + r + 1u] && s_sR[r] != s_sR[r + 1u]) s_coll = 1u;
-                }
-                bar_sync(kBarCompute, kComputeThreads);
-                if (s_coll == 0u) {
-                    // (4) position of every candidate in the merged order -> accepted or not
-                    for (uint32_t it = tid; it < n * nl; it += kComputeThreads) {
-                        const uint32_t r = it % n, k = it / n;
-                        const uint32_t key = s_key[k * n_max + r];
-                        uint32_t cum = (r + 1u) * a.cost[k];
-                        for (uint32_t k2 = 0; k2 < nl; k2++) {
-                            if (k2 == k) continue;
-                            // number of level-k2 candidates sorting ahead: keys >= key (lower level: ties
-                            // first) or keys > key (higher level); the row is non-increasing
-                            const uint32_t *row = s_key + k2 * n_max;
-                            uint32_t lo_i = 0, hi_i = n;
-                            while (lo_i < hi_i) {
-                                const uint32_t mid = (lo_i + hi_i) >> 1;
-                                const bool ahead = k2 < k ? row[mid] >= key : row[mid] > key;
-                                if (ahead) lo_i = mid + 1u; else hi_i = mid;
-                            }
-                            cum += lo_i * a.cost[k2];
-                        }
-                        if (cum <= bud.rem) atomicAdd(&s_lvl[s_sorted[r]], 1u);
-                    }
-                    bar_sync(kBarCompute, kComputeThreads);
-                    if (mine) level = s_lvl[tid];
-                } else if ((uint32_t)warp < owners) {
-                    // Fallback.  For each candidate (group g, raise k) add up the cost of all candidates
-                    // that sort at or ahead of it; the candidate is accepted iff that total fits.
-                    if (mine) {
-#pragma unroll
-                        for (int k = 0; k < kMaxLevels - 1; k++) {
-                            s_key[k * n_max + tid] = __float_as_uint(__fmul_rn(Rg, a.v[k]));
-                            s_cum[k * n_max + tid] = 0u;
-                        }
-                    }
-                    if (owners > 1) bar_sync(kBarOwners, owners * 32u);
-                    else __syncwarp();
-                    const uint32_t items = n * nl * nl;
-                    for (uint32_t it = tid; it < items; it += owners * 32u) {
-                        const uint32_t g = it % n, kk = it / n;
-                        const uint32_t k = kk / nl, k2 = kk % nl;
-                        const uint32_t kg = s_key[k * n_max + g];
-                        const uint32_t *row = s_key + k2 * n_max;
-                        uint32_t cnt = 0;
-                        if (k2 < k) {
-                            for (uint32_t h = 0; h < n; h++) cnt += (row[h] >= kg);
-                        } else if (k2 > k) {
-                            for (uint32_t h = 0; h < n; h++) cnt += (row[h] > kg);
-                        } else {
-                            for (uint32_t h = 0; h < n; h++) cnt += (row[h] > kg) || (row[h] == kg && h <= g);
-                        }
-                        atomicAdd(&s_cum[k * n_max + g], cnt * a.cost[k2]);
-                    }
-                    if (owners > 1) bar_sync(kBarOwners, owners * 32u);
-                    else __syncwarp();
-                    level = 0;
-                    if (mine)
-                        for (uint32_t k = 0; k + 1 < m; k++) level += (s_cum[k * n_max + tid] <= bud.rem);
-                }
             }
-            if ((uint32_t)warp < owners) {
-                uint32_t size = 0, b = 0;
-                float inv = 0.0f;
-                if (mine) {
-                    b = a.S[level];
-                    const float Lf = (float)((1u << b) - 1u);
-                    const float scale = Rg > 0.0f ? __fdiv_rn(Rg, Lf) : 0.0f;
-                    inv = Rg > 0.0f ? __fdiv_rn(Lf, Rg) : 0.0f;
-                    td.bits[g0 + tid] = (uint8_t)b;
-                    td.mn[g0 + tid] = mn;
-                    td.scale[g0 + tid] = scale;
-                    size = (G >> 3) * b;
-                }
-                // byte offset of each group inside the window: exclusive scan of the sizes
-                uint32_t incl = size;
-#pragma unroll
-                for (int off = 1; off < 32; off <<= 1) {
-                    const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-                    if (lane >= off) incl += y;
-                }
-                uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31), before = 0;
-                if (owners > 1) {
-                    if (lane == 0) s_wtot[warp] = total;
-                    bar_sync(kBarOwners, owners * 32u);
-                    total = 0;
-                    for (uint32_t k = 0; k < owners; k++) {
-                        const uint32_t t = s_wtot[k];
-                        if (k < (uint32_t)warp) before += t;
-                        total += t;
+            bar_sync(kBarChoice, kThreads);
+            // (2) keys of every level, filed in rank order
+            if (mine) {
+                const uint32_t r = s_rank[tid];
+                s_rank[tid] = 0u;                                 // zero again for the next window that ranks
+                s_sorted[r] = (uint32_t)tid;
+                s_sR[r] = __float_as_uint(Rg);
+                for (uint32_t k = 0; k < nl; k++) s_key[k * n_max + r] = __float_as_uint(__fmul_rn(Rg, a.v[k]));
+            }
+            bar_sync(kBarChoice, kThreads);
+            // (3) candidate (rank r, raise k): summed cost of everything sorting at or ahead of it
+            for (uint32_t it = (uint32_t)tid; it < n * nl; it += kThreads) {
+                const uint32_t r = pow2 ? it & (n - 1u) : it % n;
+                const uint32_t k = pow2 ? it >> sh : it / n;
+                const uint32_t *row = s_key + k * n_max;
+                const uint32_t K = row[r], g = s_sorted[r];
+                // same level: by rank, unless groups of different ranges share the key K (then the
+                // group index decides among them, not the range)
+                uint32_t ahead = r + 1u;
+                const bool head = r == 0u || row[r - 1u] != K, tail = r + 1u == n || row[r + 1u] != K;
+                if (!(head && tail)) {
+                    const uint32_t first = count_above<false>(row, n, K), end = count_above<true>(row, n, K);
+                    if (s_sR[first] != s_sR[end - 1u]) {
+                        ahead = first;
+                        for (uint32_t pos = first; pos < end; pos++) ahead += (s_sorted[pos] <= g);
                     }
-                    bar_sync(kBarOwners, owners * 32u);           // s_wtot may be rewritten by the next general window
                 }
+                uint32_t cum = ahead * a.cost[k];
+                for (uint32_t k2 = 0; k2 < nl; k2++) {            // other levels: ties go to the lower level
+                    if (k2 == k) continue;
+                    const uint32_t *row2 = s_key + k2 * n_max;
+                    cum += (k2 < k ? count_above<true>(row2, n, K) : count_above<false>(row2, n, K)) * a.cost[k2];
+                }
+                if (cum <= bud.rem) atomicAdd(&s_lvl[g], 1u);
+            }
+            bar_sync(kBarChoice, kThreads);
+            if (owner) {
+                uint32_t level = 0;
                 if (mine) {
-                    GroupRec rec;
-                    rec.mn = mn;
-                    rec.inv = inv;
-                    rec.b = b;
-                    rec.off = before + incl - size;
-                    s_grp[(j & 1u) * n_max + tid] = rec;
+                    level = s_lvl[tid];
+                    s_lvl[tid] = 0u;                              // zero again for the next window that ranks
                 }
-                if (tid == 0) {
-                    const bool first = (gw == td.first_window);
-                    st_relaxed_u64(a.flags + gw, ((first ? kFlagPrefix : kFlagAggregate) << kFlagShift) | total);
-                    s_tot[j & 3u] = total;
-                }
+                write_records(level, false);
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&s_wid);
-            if (!mbar_wait_bounded(&s_wid, n_generic & 1u)) {     // group records visible to all compute warps
-                s_lost = 1u;
-                if (lane == 0) record_error(DAF_ERR_TIMEOUT, gw, 7u + 16u * j);
-                break;
-            }
-            n_generic++;
-            q_b = 0u;
-            q_elems = n_elems;
+            bar_sync(kBarChoice, kThreads);                       // group records visible to all compute warps
         }
-        q_gw = gw;
 
-        // ---------------------------------------------------------------- window j: stage -> registers, stage released
-        {
-            constexpr int kChunkBytes = 256 * Elem<T>::kBytes;
+        if (mode >= 2u && s_slow[iter & 1u] == 0u) {
+            // -------------------------------------------------------------- quantize + pack, one width, no clamp needed
+            if (BATCH) {
+                const PhiloxSeedKeys sk{(uint32_t)td.seed, (uint32_t)(td.seed >> 32)};
+                quantize_uniform_b<PhiloxSeedKeys, CHUNKS>(mode - 1u, x, s_grp, log2G, e0, blk0, sk, s_out);
+            } else {
+                quantize_uniform_b<PhiloxKeys, CHUNKS>(mode - 1u, x, s_grp, log2G, e0, blk0, a.keys, s_out);
+            }
+        } else {
+            // -------------------------------------------------------------- quantize + pack with per-group widths
 #pragma unroll
-            for (int c = 0; c < CHUNKS; c++) load8_staged<T, true>(stage + (warp * CHUNKS + c) * kChunkBytes, lane, x[c]);
+            for (int c = 0; c < CHUNKS; c++) {
+                const uint32_t e = e0 + 256u * c;
+                const GroupRec rec = s_grp[e >> log2G];
+                uint32_t o[4];
+                if (a.nearest) {
+                    o[0] = o[1] = o[2] = o[3] = 0x80008000u;       // every 16-bit lane = 2 * 2^14
+                } else {
+                    const uint64_t blk = blk0 + 32u * c;
+                    if (BATCH) {
+                        const PhiloxSeedKeys sk{(uint32_t)td.seed, (uint32_t)(td.seed >> 32)};
+                        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), sk, o);
+                    } else {
+                        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), a.keys, o);
+                    }
+                }
+                uint32_t w0, w1;
+                quantize8_any(x[c], rec.mn, rec.inv, o, rec.b, w0, w1);
+                unsigned char *p = s_out + rec.off + ((e & (G - 1u)) >> 3) * rec.b;
+                if (e < n_elems) {
+                    if (rec.b == 1u) {
+                        *p = (unsigned char)w0;
+                    } else if (rec.b == 2u) {
+                        *reinterpret_cast<uint16_t *>(p) = (uint16_t)w0;
+                    } else if (rec.b == 4u) {
+                        *reinterpret_cast<uint32_t *>(p) = w0;
+                    } else if (G >= 64u) {
+                        *reinterpret_cast<uint2 *>(p) = make_uint2(w0, w1);
+                    } else {                                       // G = 32: groups are only 4-byte aligned
+                        reinterpret_cast<uint32_t *>(p)[0] = w0;
+                        reinterpret_cast<uint32_t *>(p)[1] = w1;
+                    }
+                }
+            }
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&s_cons[j % NSTAGE]);          // stage consumed
+        if (a.bulk_store) fence_async_shared();                   // packed bytes visible to the bulk store issued later
     }
-    // Out of the loop with windows 0 .. n_packed-1 packed: wake the storer warps, which wait for the
-    // windows from n_packed on.  The wake-up goes through the same barriers as a packed
-    // window, so it honours the same rule: never before the buffer's previous window has left.
-    if (tid == 0) s_end = n_packed;
-    for (uint32_t q = n_packed; q < n_packed + NSTO; q++)
-        if (q >= 3u) mbar_wait_bounded(&s_free[q % 3u], ((q / 3u) - 1u) & 1u);
-    __syncwarp();
-    if (lane == 0)
-        for (uint32_t q = n_packed; q < n_packed + NSTO; q++) mbar_arrive(&s_ready[q % 3u]);
+    bar_arrive(kBarStage, kCompressThreads);                      // the last window's packed bytes are complete
 }
 
 // ------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------
 // Shared-memory carve-up for one launch configuration.
-static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint32_t window_cap_bytes, uint32_t nstage)
+static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint32_t window_cap_bytes)
 {
     auto up = [](uint32_t v) { return (v + 127u) & ~127u; };
     const uint32_t n_max = we / G, units = we / (G < 256u ? G : 256u);
     SmemLayout l;
-    uint32_t at = nstage * up(we * elem_bytes);                   // the stages
+    uint32_t at = up(we * elem_bytes);
     l.out0 = at;
     l.out_stride = up(window_cap_bytes < 16u ? 16u : window_cap_bytes);
-    at += 3u * l.out_stride;                                      // three packed-bytes buffers
+    at += 2u * l.out_stride;
     l.umn = at; at += up(2u * 4u * units);
     l.umx = at; at += up(2u * 4u * units);
     l.key = at; at += up(4u * (kMaxLevels - 1) * n_max);
-    l.cum = at; at += up(4u * (kMaxLevels - 1) * n_max);
-    l.grp = at; at += up(2u * 16u * n_max);
+    l.cum = at; at += up(3u * 4u * n_max);
     l.srt = at; at += up(2u * 4u * n_max);
+    l.grp = at; at += up(16u * n_max);
     l.total = at;
     return l;
 }
 
-// Staged windows per CTA.  Two stages and one CTA per SM measured faster on B200 than one stage
-// and two CTAs per SM (which leaves 56 registers per thread and spills).
-constexpr uint32_t kStages = 2, kStorers = 2;
-
-template <typename T, int CHUNKS, int NW, int NSTAGE, int NSTO, bool BATCH>
+template <typename T, int CHUNKS, bool BATCH>
 static cudaError_t launch(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
-    constexpr int kBlock = NW * 32 + 32 + 32 * NSTO;
     static int sms = 0, smem_set = 0, cached_smem = -1, cached_ctas = 0;   // per instantiation, current device
     const int smem = (int)args.lay.total;
     cudaError_t e = cudaSuccess;
@@ -1096,33 +850,31 @@ static cudaError_t launch(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, c
         if (e != cudaSuccess) return e;
     }
     if (smem > smem_set) {
-        e = cudaFuncSetAttribute(compress_kernel<T, CHUNKS, NW, NSTAGE, NSTO, BATCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        e = cudaFuncSetAttribute(compress_kernel<T, CHUNKS, BATCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         smem_set = smem;
     }
     if (smem != cached_smem) {
         int per_sm = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel<T, CHUNKS, NW, NSTAGE, NSTO, BATCH>, kBlock, smem);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel<T, CHUNKS, BATCH>, kCompressThreads, smem);
         if (e != cudaSuccess) return e;
         cached_smem = smem;
         cached_ctas = sms * (per_sm > 0 ? per_sm : 1);
     }
     const uint32_t grid = args.total_windows < (uint32_t)cached_ctas ? args.total_windows : (uint32_t)cached_ctas;
-    compress_kernel<T, CHUNKS, NW, NSTAGE, NSTO, BATCH><<<grid, kBlock, smem, stream>>>(args);
+    compress_kernel<T, CHUNKS, BATCH><<<grid, kCompressThreads, smem, stream>>>(args);
     return cudaGetLastError();
 }
 
-// `chunks4k` = window_elems / 4096: the window is spread over 16 compute warps (a CTA holds at
-// most 1024 threads, and the service warps take some of its 32 warp slots).
 template <bool BATCH>
-static cudaError_t dispatch(uint32_t dtype, uint32_t chunks4k, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
+static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
                             cudaStream_t stream)
 {
-#define DAF_CASE(T)                                                                     \
-    switch (chunks4k) {                                                                 \
-    case 1: return launch<T, 1, 16, kStages, kStorers, BATCH>(args, stream);            \
-    case 2: return launch<T, 2, 16, kStages, kStorers, BATCH>(args, stream);            \
-    default: return launch<T, 4, 16, kStages, kStorers, BATCH>(args, stream);           \
+#define DAF_CASE(T)                                                     \
+    switch (chunks) {                                                   \
+    case 1: return launch<T, 1, BATCH>(args, stream);                   \
+    case 2: return launch<T, 2, BATCH>(args, stream);                   \
+    default: return launch<T, 4, BATCH>(args, stream);                  \
     }
     if (dtype == DAF_F32) { DAF_CASE(float) }
     if (dtype == DAF_F16) { DAF_CASE(__half) }
@@ -1149,8 +901,7 @@ template <int NT> static void fill_common(CompressArgs<NT> &a, const Plan &pl, c
         while (a.full_ell + 1 < pl.m && (pl.S[a.full_ell + 1] - pl.S[0]) * n <= a.full_rem) a.full_ell++;
         a.full_rem_after = a.full_rem - (pl.S[a.full_ell] - pl.S[0]) * n;
     }
-    a.nbuf = 3;
-    a.lay = make_layout(pl.We, elem_bytes, pl.G, (uint32_t)((((uint64_t)pl.beta_q8 * pl.W) >> 8) * pl.G / 8), kStages);
+    a.lay = make_layout(pl.We, elem_bytes, pl.G, (uint32_t)((((uint64_t)pl.beta_q8 * pl.W) >> 8) * pl.G / 8));
     for (int k = 0; k < kMaxLevels; k++) {
         a.S[k] = pl.S[k];
         a.cost[k] = pl.cost[k];
