@@ -124,7 +124,7 @@ __device__ __forceinline__ void quantize8_any(const float (&x)[8], float mn, flo
 // exclusive prefix was found (*excl), 0 when a needed descriptor is still empty and `block`
 // is false, -1 on a poisoned predecessor, -2 when the bounded wait ran out.
 // ------------------------------------------------------------------------------------------
-constexpr int kLookDepth = 16;
+constexpr int kLookDepth = 4;
 
 template <int DEPTH>
 __device__ __forceinline__ int lookback(const uint64_t *flags, uint32_t gw, uint32_t first, int lane, bool block,
