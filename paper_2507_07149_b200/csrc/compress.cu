@@ -241,10 +241,13 @@ template <typename T> __device__ __forceinline__ void load8_staged(const unsigne
 
 template <> __device__ __forceinline__ void load8_staged<float>(const unsigned char *chunk, int lane, float (&x)[8])
 {
-    const float4 a = *reinterpret_cast<const float4 *>(chunk + lane * 32);
-    const float4 b = *reinterpret_cast<const float4 *>(chunk + lane * 32 + 16);
-    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
-    x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+    // a lane owns 32 bytes; which half it reads first depends on the lane, so that each
+    // quarter-warp touches all 32 banks
+    const int odd = (lane >> 2) & 1;
+    const float4 a = *reinterpret_cast<const float4 *>(chunk + lane * 32 + 16 * odd);
+    const float4 b = *reinterpret_cast<const float4 *>(chunk + lane * 32 + 16 * (odd ^ 1));
+    x[0] = odd ? b.x : a.x; x[1] = odd ? b.y : a.y; x[2] = odd ? b.z : a.z; x[3] = odd ? b.w : a.w;
+    x[4] = odd ? a.x : b.x; x[5] = odd ? a.y : b.y; x[6] = odd ? a.z : b.z; x[7] = odd ? a.w : b.w;
 }
 template <> __device__ __forceinline__ void load8_staged<__half>(const unsigned char *chunk, int lane, float (&x)[8])
 {
@@ -317,7 +320,7 @@ template <int NT> __device__ __forceinline__ uint32_t find_tensor(const Compress
 // compute warps): the owners' verdict on the window is in.  Barrier 3 is private to the warps
 // that own group records; barrier 4 separates the steps of the general bit choice.
 constexpr int kComputeWarps = kWarps;
-constexpr int kCompressThreads = kThreads + 32;
+constexpr int kCompressThreads = kThreads + 64;
 constexpr uint32_t kBarStage = 1, kBarWidths = 2, kBarOwners = 3, kBarChoice = 4;
 
 __device__ __forceinline__ void bar_sync(uint32_t id, uint32_t threads)
@@ -400,7 +403,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     extern __shared__ __align__(128) unsigned char smem[];       // [stage | out0 | out1 | group arrays]
     __shared__ uint32_t s_wtot[kComputeWarps];
     __shared__ __align__(8) uint64_t s_full;                     // mbarrier: staged window has landed (or there is none)
-    __shared__ uint32_t s_next;                                  // ticket of the staged window
+    __shared__ uint32_t s_next[2];                               // ticket of the window of iteration i (slot i & 1)
     __shared__ uint32_t s_lost;                                  // a staged copy did not land in time
     __shared__ uint32_t s_tot[2];                                // packed bytes of the window of iteration i (slot i & 1)
     __shared__ uint32_t s_mode[2];                               // how that window's widths came out (see below)
@@ -418,11 +421,11 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     const uint32_t G = a.G, log2G = a.log2G;
 
     auto tensor_of = [&](uint32_t gw) -> const TensorDesc & { return a.t[BATCH ? find_tensor(a, gw) : 0u]; };
-    // Control lane: takes a ticket and starts the bulk copy of that window into the stage, or
+    // Control lane: draws a ticket; starts the bulk copy of that window into the stage, or
     // completes the stage's barrier empty-handed when the windows have run out.
-    auto stage_next = [&]() {
-        const uint32_t t = atomicAdd(&a.hdr->ticket, 1u);
-        s_next = t;                                               // ordered before the barrier's completion
+    auto draw_ticket = [&]() -> uint32_t { return atomicAdd(&a.hdr->ticket, 1u); };
+    auto stage_window = [&](uint32_t t, uint32_t iter) {
+        s_next[iter & 1u] = t;                                    // ordered before the barrier's completion
         if (t < a.total_windows) {
             const TensorDesc &nd = tensor_of(t);
             const uint64_t base = (uint64_t)(t - nd.first_window) * WE;
@@ -458,30 +461,119 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         mbar_init(&s_full, 1);
         s_lost = 0u;
         s_slow[0] = s_slow[1] = 0u;
-        stage_next();
+        stage_window(draw_ticket(), 0u);
     }
     if (tid < kThreads)
         for (uint32_t i = (uint32_t)tid; i < 2u * a.n_max; i += kThreads) s_cum[a.n_max + i] = 0u;   // ranks and levels count up from zero
     __syncthreads();
 
+    // With at most 64 groups per window (groups of 256 elements or more) a warp of its own, which
+    // holds no window data, settles the windows whose groups all end at the same width: lane l
+    // looks after groups l and l + 32.  See the compute warps' own version below for the test.
+    const bool ctl_widths = a.n_max <= 64u;
+    const uint32_t stage_threads = ctl_widths ? kCompressThreads : kThreads + 32;   // who meets at the "stage" barrier
+    auto uniform_widths = [&](uint32_t gw, uint32_t iter) {
+        const TensorDesc &td = tensor_of(gw);
+        const uint32_t w = gw - td.first_window;
+        const uint64_t wbase = (uint64_t)w * WE;
+        const uint64_t left = td.numel - wbase;
+        const uint32_t n_elems = left < WE ? (uint32_t)left : WE;
+        const uint32_t n = n_elems >> log2G, rr = G >> 8;
+        const uint64_t g0 = wbase >> log2G;
+        const uint32_t units = WE >> 8;
+        const float *umn = s_umn + (iter & 1u) * units, *umx = s_umx + (iter & 1u) * units;
+        const Budget bud = budget_of(n);
+        const float vl = a.v[bud.ell > 0 ? bud.ell - 1 : 0], vh = a.v[bud.ell];
+        float mn[2], R[2];
+        uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+#pragma unroll
+        for (int q = 0; q < 2; q++) {
+            const uint32_t g = (uint32_t)lane + 32u * q;
+            mn[q] = R[q] = 0.0f;
+            if (g < n) {
+                float lo = umn[g * rr], hi = umx[g * rr];
+                for (uint32_t k = 1; k < rr; k++) {
+                    lo = fmin2(lo, umn[g * rr + k]);
+                    hi = fmax2(hi, umx[g * rr + k]);
+                }
+                float Rg = __fsub_rn(hi, lo);
+                if (Rg < 0x1p-118f) Rg = 0.0f;                    // degenerate group: constant
+                mn[q] = lo;
+                R[q] = Rg;
+                kmin = min(kmin, __float_as_uint(__fmul_rn(Rg, vl)));
+                kmax = max(kmax, __float_as_uint(__fmul_rn(Rg, vh)));
+            }
+        }
+        bool same = bud.all_max || bud.need_sep;
+        if (bud.need_sep && bud.ell > 0) {
+            kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+            kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+            same = kmin >= kmax;
+        }
+        if (lane == 0) s_slow[(iter & 1u) ^ 1u] = 0u;             // reset the flag of the next window
+        if (same) {
+            const uint32_t b = a.S[bud.ell], size = (G >> 3) * b;
+            const float Lf = (float)((1u << b) - 1u);
+#pragma unroll
+            for (int q = 0; q < 2; q++) {
+                const uint32_t g = (uint32_t)lane + 32u * q;
+                if (g < n) {
+                    const float scale = R[q] > 0.0f ? __fdiv_rn(R[q], Lf) : 0.0f;
+                    const float inv = R[q] > 0.0f ? __fdiv_rn(Lf, R[q]) : 0.0f;
+                    // 1/scale not a normal number: codes may need the clamp, take the careful quantizer
+                    if (R[q] > 0.0f && inv < 0x1p-126f) s_slow[iter & 1u] = 1u;
+                    GroupRec rec;
+                    rec.mn = mn[q];
+                    rec.inv = inv;
+                    rec.b = b;
+                    rec.off = g * size;
+                    s_grp[g] = rec;
+                    td.bits[g0 + g] = (uint8_t)b;
+                    td.mn[g0 + g] = mn[q];
+                    td.scale[g0 + g] = scale;
+                }
+            }
+            if (lane == 0) {
+                // the window's byte count is known: publish it at once
+                const uint32_t total = n * size;
+                st_relaxed_u64(a.flags + gw, ((w == 0u ? kFlagPrefix : kFlagAggregate) << kFlagShift) | total);
+                s_tot[iter & 1u] = total;
+            }
+        }
+        if (lane == 0) s_mode[iter & 1u] = !same ? 0u : (n_elems == WE && !a.nearest) ? 1u + a.S[bud.ell] : 1u;
+    };
+
+    if (warp == kComputeWarps + 1) {
+        // ============================================================ widths warp
+        if (!ctl_widths) return;
+        for (uint32_t iter = 0;; iter++) {
+            bar_sync(kBarStage, stage_threads);                   // every unit's min / max is visible
+            const uint32_t gw = s_next[iter & 1u];
+            if (gw >= a.total_windows) break;
+            if (s_lost == 0u) uniform_widths(gw, iter);
+            bar_arrive(kBarWidths, kThreads + 32);                // the verdict on the window is in
+            if (s_lost != 0u) break;
+        }
+        return;
+    }
     if (warp == kComputeWarps) {
         // ============================================================ control warp
         // Per window i: wait until the compute warps have consumed stage(i) and finished the
         // packed bytes of window i-1; start the copy of window i+1; then, off the compute
         // warps' critical path, find window i-1's byte offset by look-back, publish its
         // inclusive prefix, and send its packed bytes to global memory.
-        uint32_t gw = s_next;
+        uint32_t gw = s_next[0];
         bool have_prev = false;
         uint32_t p_gw = 0;
         for (uint32_t iter = 0;; iter++) {
             const bool valid = gw < a.total_windows;
-            bar_sync(kBarStage, kCompressThreads);
+            bar_sync(kBarStage, stage_threads);
             const bool lost = s_lost != 0u;
             uint32_t next = 0xFFFFFFFFu;
             if (valid && !lost) {
-                if (lane == 0) stage_next();
+                if (lane == 0) stage_window(draw_ticket(), iter + 1u);
                 __syncwarp();
-                next = s_next;
+                next = s_next[(iter + 1u) & 1u];
             }
             if (have_prev) {
                 const TensorDesc &pd = tensor_of(p_gw);
@@ -545,7 +637,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             s_lost = 1u;
             lost = true;
         }
-        const uint32_t gw = lost ? 0u : s_next;
+        const uint32_t gw = lost ? 0u : s_next[iter & 1u];
         if (!lost && gw >= a.total_windows) break;
         unsigned char *const s_out = smem + a.lay.out0 + (iter & 1u) * a.lay.out_stride;
         const TensorDesc &td = tensor_of(gw);
@@ -628,9 +720,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 s_tot[iter & 1u] = total;
             }
         };
-        if (owner) {
-            bar_sync(kBarStage, kCompressThreads);                // every unit's min / max is visible; the stage is free
-            if (tid == 0) s_slow[(iter & 1u) ^ 1u] = 0u;          // reset the flag of the next window
+        auto own_range = [&]() {
             if (mine) {
                 float mx;
                 if (big) {
@@ -648,36 +738,39 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 Rg = __fsub_rn(mx, mn);
                 if (Rg < 0x1p-118f) Rg = 0.0f;                    // degenerate group: constant
             }
-            bool uniform = bud.all_max || bud.need_sep;
-            if (bud.need_sep && bud.ell > 0) {
-                // each owner warp evaluates the test over all groups itself
-                const float vl = a.v[bud.ell - 1], vh = a.v[bud.ell];
-                uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
-                if (owners == 1) {
-                    if (mine) {
-                        kmin = __float_as_uint(__fmul_rn(Rg, vl));
-                        kmax = __float_as_uint(__fmul_rn(Rg, vh));
-                    }
-                } else {                                          // groups of at most 256: one unit per group
+        };
+        if (ctl_widths) {
+            bar_arrive(kBarStage, stage_threads);              // unit min / max out, stage consumed, last window packed
+            bar_sync(kBarWidths, kThreads + 32);                  // the widths warp's verdict (and records) visible
+        } else {
+            if (owner) {
+                bar_sync(kBarStage, stage_threads);            // every unit's min / max is visible; the stage is free
+                if (tid == 0) s_slow[(iter & 1u) ^ 1u] = 0u;      // reset the flag of the next window
+                own_range();
+                bool uniform = bud.all_max || bud.need_sep;
+                if (bud.need_sep && bud.ell > 0) {
+                    // each owner warp evaluates the test over all groups itself (a unit is a group here)
+                    const float vl = a.v[bud.ell - 1], vh = a.v[bud.ell];
+                    uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
                     for (uint32_t g = lane; g < n; g += 32) {
                         float R = __fsub_rn(umx[g], umn[g]);
                         if (R < 0x1p-118f) R = 0.0f;
                         kmin = min(kmin, __float_as_uint(__fmul_rn(R, vl)));
                         kmax = max(kmax, __float_as_uint(__fmul_rn(R, vh)));
                     }
+                    kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+                    kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+                    uniform = kmin >= kmax;
                 }
-                kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
-                kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
-                uniform = kmin >= kmax;
+                if (s_lost == 0u) {
+                    if (uniform) write_records(bud.ell, true);
+                    if (tid == 0) s_mode[iter & 1u] = !uniform ? 0u : (n_elems == WE && !a.nearest) ? 1u + a.S[bud.ell] : 1u;
+                }
+            } else {
+                bar_arrive(kBarStage, stage_threads);
             }
-            if (s_lost == 0u) {
-                if (uniform) write_records(bud.ell, true);
-                if (tid == 0) s_mode[iter & 1u] = !uniform ? 0u : (n_elems == WE && !a.nearest) ? 1u + a.S[bud.ell] : 1u;
-            }
-        } else {
-            bar_arrive(kBarStage, kCompressThreads);
+            bar_sync(kBarWidths, kThreads);                       // records (or the news that there are none yet) visible
         }
-        bar_sync(kBarWidths, kThreads);                           // records (or the news that there are none yet) visible
         if (s_lost != 0u) break;
         const uint32_t mode = s_mode[iter & 1u];                  // 0: general choice needed; 1: records; 1 + b: one width b
         const uint64_t blk0 = ((td.elem_base + wbase) >> 3) + (e0 >> 3);
@@ -693,6 +786,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             // in the levels' sorted keys and accepts it if everything up to and including it fits.
             uint32_t *const s_Rb = s_cum, *const s_rank = s_cum + n_max, *const s_lvl = s_cum + 2u * n_max;
             uint32_t *const s_sorted = s_srt, *const s_sR = s_srt + n_max;
+            if (ctl_widths) own_range();
             if (mine) s_Rb[tid] = __float_as_uint(Rg);            // the ranges, side by side
             bar_sync(kBarChoice, kThreads);
             const bool pow2 = (n & (n - 1u)) == 0u;
@@ -811,7 +905,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         }
         if (a.bulk_store) fence_async_shared();                   // packed bytes visible to the bulk store issued later
     }
-    bar_arrive(kBarStage, kCompressThreads);                      // the last window's packed bytes are complete
+    bar_arrive(kBarStage, stage_threads);                      // the last window's packed bytes are complete
 }
 
 // ------------------------------------------------------------------------------------------
