@@ -1,0 +1,126 @@
+"""Times compress / decompress on the five benchmark workloads and the group-size x budget sweep.
+
+    python -m paper_2507_07149_b200.sweep [--configs 1,2,3,4,5] [--sweep] [--steps K] [--scale S]
+
+Workloads 1-4 are sets of tensors: each set goes through ONE batched call (daf_compress_batch /
+daf_decompress_batch) when it has at most DAF_BATCH_MAX tensors.  Inputs are the seeded synthetic
+tensors of ``workloads.py``, resident in device memory before the timed region; times are CUDA
+events around K back-to-back calls (after 3 warm-up calls).  ``--scale S`` divides the batch
+dimension (or the element count of workload 5) by S for a quick look.  One markdown table row
+per workload is printed: element count, input bytes, packed bytes, compress and decompress
+time, and for each the algorithmic throughput: (tensor bytes + packed bytes + 9 bytes of
+metadata per group + 8 per window) / time, the figure the roofline fractions are quoted on.
+"""
+from __future__ import annotations
+
+import argparse
+
+import numpy as np
+
+
+def _device_tensor(torch, wl, cfg, ti, spec):
+    tdt = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.int16}[spec.dtype]
+    h = torch.empty(spec.numel, dtype=tdt, pin_memory=True)
+    wl.generate(cfg, ti, spec, out=h.numpy().view(wl.np_dtype(spec.dtype)))
+    if spec.dtype == "bf16":
+        h = h.view(torch.bfloat16)
+    return h.cuda()
+
+
+def _time(torch, fn, steps):
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
+def run_set(torch, daf, wl, w, xs, steps):
+    """(compress ms, decompress ms, packed bytes) for the tensors xs of workload w."""
+    params = [daf.make_params(daf.dtype_code(x), x.numel(), w.group_size, w.widths, w.bit_budget, seed=t.philox_seed)
+              for x, t in zip(xs, w.tensors)]
+    outs = [daf.alloc_outputs(p, xs[0].device) for p in params]
+    ys = [torch.empty_like(x) for x in xs]
+    if len(xs) == 1:
+        p, x, c, y = params[0], xs[0], outs[0], ys[0]
+
+        def comp():
+            daf.daf_compress(p, x, c.packed, c.sizes.packed_capacity, c.bits, c.min, c.scale, c.window_offsets,
+                             c.workspace, c.sizes.workspace)
+
+        def dec():
+            daf.daf_decompress(p, c.packed, c.bits, c.min, c.scale, c.window_offsets, y)
+
+        status = lambda: daf.daf_poll_status(c.workspace)
+    else:
+        assert len(xs) <= daf.BATCH_MAX
+        ws_bytes = daf.daf_batch_workspace(params)
+        ws = torch.empty(ws_bytes, dtype=torch.uint8, device=xs[0].device)
+
+        def comp():
+            daf.daf_compress_batch(params, xs, [o.packed for o in outs], [o.sizes.packed_capacity for o in outs],
+                                   [o.bits for o in outs], [o.min for o in outs], [o.scale for o in outs],
+                                   [o.window_offsets for o in outs], ws, ws_bytes)
+
+        def dec():
+            daf.daf_decompress_batch(params, [o.packed for o in outs], [o.bits for o in outs], [o.min for o in outs],
+                                     [o.scale for o in outs], [o.window_offsets for o in outs], ys)
+
+        status = lambda: daf.daf_poll_status(ws)
+    t_c = _time(torch, comp, steps)
+    assert status() == daf.OK, status()
+    t_d = _time(torch, dec, steps)
+    packed = sum(o.packed_bytes() for o in outs)
+    meta = sum(9 * (x.numel() // w.group_size) + 8 * (o.sizes.n_windows + 1) for x, o in zip(xs, outs))
+    return t_c, t_d, packed, meta
+
+
+def row(name, numel, nbytes, packed, meta, t_c, t_d):
+    alg = nbytes + packed + meta
+    return (f"| {name} | {numel} | {nbytes / 2**30:.3f} | {packed / 2**30:.3f} | {t_c:.4f} | {alg / t_c / 1e6:.0f} | "
+            f"{t_d:.4f} | {alg / t_d / 1e6:.0f} |")
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--configs", default="1,2,3,4,5")
+    ap.add_argument("--sweep", action="store_true", help="also the 16 (group size, budget) points of workload 5")
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--scale", type=int, default=1)
+    args = ap.parse_args()
+
+    import torch
+    import paper_2507_07149_b200 as daf
+    from paper_2507_07149_b200 import workloads as wl
+
+    daf.lib()
+    print("| workload | elements | tensor GiB | packed GiB | compress ms | compress GB/s | decompress ms | decompress GB/s |")
+    print("|---|---|---|---|---|---|---|---|")
+    S = args.scale
+    for cfg in [int(c) for c in args.configs.split(",")]:
+        kw = {}
+        if cfg in (2, 3, 4) and S > 1:
+            kw["batch"] = max(1, {2: 64, 3: 128, 4: 64}[cfg] // S)
+        if cfg == 5:
+            kw["numel"] = (1 << 30) // S
+        w = wl.workload(cfg, **kw)
+        xs = [_device_tensor(torch, wl, cfg, i, t) for i, t in enumerate(w.tensors)]
+        t_c, t_d, packed, meta = run_set(torch, daf, wl, w, xs, args.steps)
+        print(row(w.name, w.numel, w.nbytes, packed, meta, t_c, t_d), flush=True)
+        if cfg == 5 and args.sweep:
+            for G in wl.SWEEP_GROUPS:
+                for beta in wl.SWEEP_BUDGETS:
+                    ws = wl.workload(5, numel=kw["numel"], group_size=G, bit_budget=beta)
+                    t_c, t_d, packed, meta = run_set(torch, daf, wl, ws, xs, args.steps)
+                    print(row(ws.name, ws.numel, ws.nbytes, packed, meta, t_c, t_d), flush=True)
+        del xs
+        torch.cuda.empty_cache()
+
+
+if __name__ == "__main__":
+    main()
