@@ -15,7 +15,6 @@ from __future__ import annotations
 
 import argparse
 
-import numpy as np
 
 
 def _device_tensor(torch, wl, cfg, ti, spec):

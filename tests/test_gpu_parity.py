@@ -154,6 +154,48 @@ def test_heavy_ties_relu6_saturation():
         assert_decompress_parity(c, ref, "f16", f"ties/{beta}")
 
 
+@pytest.mark.parametrize("G", [64, 256, 1024])
+def test_different_ranges_with_equal_keys(G):
+    """Ranges that are neighbouring floats: several of them round to the same importance key, so
+    the order among those raises is by group index, not by range, and the budget's cut falls
+    inside such runs for some of the budgets."""
+    rng = np.random.default_rng(G + 17)
+    W, n_win = 16384 // G, 3
+    n_groups = W * n_win + 3                                     # ragged last window
+    base = np.float32(3.99)                                      # R v stays in (or one above) the binade of R: keys coarser than ranges
+    steps = rng.integers(0, 6, n_groups)                         # ranges base * (1 + j ulp), j = 0..5, in random order
+    R = (np.full(n_groups, base, np.float32).view(np.uint32) + steps.astype(np.uint32)).view(np.float32)
+    far = rng.random(n_groups) < 0.15                            # some groups far away, so that levels mix
+    R = np.where(far, R * np.float32(2.0) ** rng.integers(-6, 7, n_groups).astype(np.float32), R).astype(np.float32)
+    a = np.zeros((n_groups, G), np.float32)
+    a[:, 1] = R                                                  # min 0, max R: the range is R exactly
+    a[:, 2:] = rng.random((n_groups, G - 2), dtype=np.float32) * R[:, None] * np.float32(0.999)
+    collided = False
+    for b_lo, b_hi in ((1, 2), (2, 4), (4, 8)):
+        v = oracle.raise_factor(b_lo, b_hi)
+        keys = (R * v).astype(np.float32)
+        for w in range(n_win):
+            k, r = keys[w * W:(w + 1) * W], R[w * W:(w + 1) * W]
+            order = np.argsort(k, kind="stable")
+            same_key = k[order][1:] == k[order][:-1]
+            collided |= bool(np.any(same_key & (r[order][1:] != r[order][:-1])))
+    assert collided, "the construction no longer produces equal keys from different ranges"
+    for beta in (1.25, 1.5, 2.5, 3.0, 3.5, 5.0, 6.0):
+        x, c, ref = assert_compress_parity(a, "f32", G, (1, 2, 4, 8), beta, seed=5, label=f"collide/G{G}/{beta}")
+        assert_decompress_parity(c, ref, "f32", f"collide/G{G}/{beta}")
+
+
+@pytest.mark.parametrize("G,n_last", [(32, 5), (64, 37), (128, 100), (256, 63), (512, 1), (2048, 3)])
+def test_ragged_last_window_takes_the_general_choice(G, n_last):
+    """A last window with a group count that is not a power of two, with mixed widths."""
+    rng = np.random.default_rng(G * 7 + n_last)
+    n = 16384 * 2 + G * n_last
+    a = (rng.standard_normal(n) * np.repeat(10.0 ** rng.uniform(-2, 2, n // G), G)).astype(np.float32)
+    for widths, beta in (((1, 2, 4, 8), 3.0), ((2, 4, 8), 4.0), ((1, 2, 4, 8), 4.0)):
+        x, c, ref = assert_compress_parity(a, "f32", G, widths, beta, seed=11, label=f"ragged/G{G}/{widths}/{beta}")
+        assert_decompress_parity(c, ref, "f32", f"ragged/G{G}")
+
+
 @pytest.mark.parametrize("We", [4096, 8192, 16384])
 @pytest.mark.parametrize("rounding", [daf.ROUND_STOCHASTIC, daf.ROUND_NEAREST])
 def test_window_sizes_rounding_modes_and_shards(We, rounding):
