@@ -73,26 +73,47 @@ __device__ __forceinline__ void quantize8(const float (&x)[8], float mn, float i
                                           uint32_t &w0, uint32_t &w1)
 {
     constexpr uint32_t L = (1u << B) - 1u;
-    w0 = 0u;
-    w1 = 0u;
+    uint32_t t[8];
 #pragma unroll
     for (int i = 0; i < 8; i++) {
         const float d = __fsub_rn(x[i], mn);
         const float s = __fmaf_rn(d, inv, 256.0f);
         const uint32_t h = (i & 1) ? (o[i >> 1] >> 16) : (o[i >> 1] & 0xFFFFu);
-        const uint32_t t = (__float_as_uint(s) << 1) + h;         // mod 2^32; 2*bits(256) = 0x87000000
-        const int pos = (B * i) & 31;                             // bit position of code i in its word (unrolled: constant)
-        uint32_t field;
-        if (CLAMP) {
-            field = min((t >> 16) - 0x8700u, L) << pos;
-        } else {
-            // the code is the B-bit field of t at bit 16 (never above L when 1/scale is a normal
-            // number): move it to its place and mask, without materialising it
-            const uint32_t moved = pos < 16 ? (t >> (16 - pos)) : (pos == 16 ? t : (t << (pos - 16)));
-            field = moved & (L << pos);
+        t[i] = __float_as_uint(s) * 2u + h;                       // mod 2^32; 2*bits(256) = 0x87000000
+    }
+    if (CLAMP) {
+        w0 = 0u;
+        w1 = 0u;
+#pragma unroll
+        for (int i = 0; i < 8; i++) {
+            const int pos = (B * i) & 31;                         // bit position of code i in its word (unrolled: constant)
+            const uint32_t field = min((t[i] >> 16) - 0x8700u, L) << pos;
+            if (B == 8 && i >= 4) w1 |= field;
+            else w0 |= field;
         }
-        if (B == 8 && i >= 4) w1 |= field;
-        else w0 |= field;
+    } else {
+        // The code never exceeds L when 1/scale is a normal number, so byte 2 of t is the code
+        // itself (bits 16+B .. 23 are zero).  Byte permutes gather the eight code bytes; widths
+        // below 8 then close the gaps: 4-bit codes by interleaving two words of nibbles, 2- and
+        // 1-bit codes by a multiplication that lines the four fields of a word up in its top byte.
+        if (B == 4) {
+            // bytes (c0, c2, c4, c6) and (c1, c3, c5, c7): the odd codes become the high nibbles
+            const uint32_t ev = __byte_perm(__byte_perm(t[0], t[2], 0x0062), __byte_perm(t[4], t[6], 0x0062), 0x5410);
+            const uint32_t od = __byte_perm(__byte_perm(t[1], t[3], 0x0062), __byte_perm(t[5], t[7], 0x0062), 0x5410);
+            w0 = od * 16u + ev;
+            w1 = 0u;
+        } else {
+            const uint32_t c0123 = __byte_perm(__byte_perm(t[0], t[1], 0x0062), __byte_perm(t[2], t[3], 0x0062), 0x5410);
+            const uint32_t c4567 = __byte_perm(__byte_perm(t[4], t[5], 0x0062), __byte_perm(t[6], t[7], 0x0062), 0x5410);
+            if (B == 8) {
+                w0 = c0123;
+                w1 = c4567;
+            } else {
+                constexpr uint32_t M = B == 2 ? 0x01041040u : 0x01020408u;   // field i of a word moves up by 24 - (8 - B) i bits
+                w0 = (((c4567 * M) >> 24) << (4 * B)) | ((c0123 * M) >> 24);
+                w1 = 0u;
+            }
+        }
     }
 }
 
