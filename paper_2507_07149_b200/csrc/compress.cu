@@ -316,11 +316,11 @@ __device__ __forceinline__ void load_and_reduce(const unsigned char *stage, int 
                 hi = fmax2(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, off));
             }
         }
-        if ((lane & (LPU - 1)) == 0) {
-            const int u = (warp * CHUNKS + c) * (32 / LPU) + lane / LPU;
-            s_umn[u] = lo;
-            s_umx[u] = hi;
-        }
+        // every lane of a unit holds the unit's result and stores it (same address, same value):
+        // cheaper than a divergent branch around the store
+        const int u = (warp * CHUNKS + c) * (32 / LPU) + lane / LPU;
+        s_umn[u] = lo;
+        s_umx[u] = hi;
     }
 }
 
