@@ -415,7 +415,9 @@ struct Budget {
     bool need_sep;         // the best raise of level ell does not fit: uniform iff the levels separate
 };
 
-template <typename T, int CHUNKS, bool BATCH>
+// WIDTHS: at most 64 groups per window (groups of 256 elements or more), the widths warp settles
+// uniform windows; otherwise the compute warps that own group records do.
+template <typename T, int CHUNKS, bool BATCH, bool WIDTHS>
 __global__ void __launch_bounds__(kCompressThreads, 2)
 compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> a)
 {
@@ -491,7 +493,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     // With at most 64 groups per window (groups of 256 elements or more) a warp of its own, which
     // holds no window data, settles the windows whose groups all end at the same width: lane l
     // looks after groups l and l + 32.  See the compute warps' own version below for the test.
-    const bool ctl_widths = a.n_max <= 64u;
+    constexpr bool ctl_widths = WIDTHS;
     const uint32_t stage_threads = ctl_widths ? kCompressThreads : kThreads + 32;   // who meets at the "stage" barrier
     auto uniform_widths = [&](uint32_t gw, uint32_t iter) {
         const TensorDesc &td = tensor_of(gw);
@@ -952,7 +954,7 @@ static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint
     return l;
 }
 
-template <typename T, int CHUNKS, bool BATCH>
+template <typename T, int CHUNKS, bool BATCH, bool WIDTHS>
 static cudaError_t launch(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
     static int sms = 0, smem_set = 0, cached_smem = -1, cached_ctas = 0;   // per instantiation, current device
@@ -965,19 +967,19 @@ static cudaError_t launch(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, c
         if (e != cudaSuccess) return e;
     }
     if (smem > smem_set) {
-        e = cudaFuncSetAttribute(compress_kernel<T, CHUNKS, BATCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        e = cudaFuncSetAttribute(compress_kernel<T, CHUNKS, BATCH, WIDTHS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         smem_set = smem;
     }
     if (smem != cached_smem) {
         int per_sm = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel<T, CHUNKS, BATCH>, kCompressThreads, smem);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel<T, CHUNKS, BATCH, WIDTHS>, kCompressThreads, smem);
         if (e != cudaSuccess) return e;
         cached_smem = smem;
         cached_ctas = sms * (per_sm > 0 ? per_sm : 1);
     }
     const uint32_t grid = args.total_windows < (uint32_t)cached_ctas ? args.total_windows : (uint32_t)cached_ctas;
-    compress_kernel<T, CHUNKS, BATCH><<<grid, kCompressThreads, smem, stream>>>(args);
+    compress_kernel<T, CHUNKS, BATCH, WIDTHS><<<grid, kCompressThreads, smem, stream>>>(args);
     return cudaGetLastError();
 }
 
@@ -985,12 +987,13 @@ template <bool BATCH>
 static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
                             cudaStream_t stream)
 {
-#define DAF_CASE(T)                                                     \
-    switch (chunks) {                                                   \
-    case 1: return launch<T, 1, BATCH>(args, stream);                   \
-    case 2: return launch<T, 2, BATCH>(args, stream);                   \
-    default: return launch<T, 4, BATCH>(args, stream);                  \
+#define DAF_CASE(T)                                                                     \
+    switch (chunks) {                                                                   \
+    case 1: return widths ? launch<T, 1, BATCH, true>(args, stream) : launch<T, 1, BATCH, false>(args, stream);   \
+    case 2: return widths ? launch<T, 2, BATCH, true>(args, stream) : launch<T, 2, BATCH, false>(args, stream);   \
+    default: return widths ? launch<T, 4, BATCH, true>(args, stream) : launch<T, 4, BATCH, false>(args, stream);  \
     }
+    const bool widths = args.n_max <= 64u;                        // few enough groups for the widths warp
     if (dtype == DAF_F32) { DAF_CASE(float) }
     if (dtype == DAF_F16) { DAF_CASE(__half) }
     DAF_CASE(__nv_bfloat16)
