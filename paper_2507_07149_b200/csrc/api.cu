@@ -51,7 +51,7 @@ daf_status make_plan(const daf_params *p, Plan *pl)
     pl->n_windows = (pl->n_groups + pl->W - 1) / pl->W;
     const uint64_t full = pl->n_groups / pl->W, last = pl->n_groups % pl->W;
     pl->capacity = full * ((((uint64_t)pl->beta_q8 * pl->W) >> 8) * G / 8) + (((uint64_t)pl->beta_q8 * last) >> 8) * G / 8;
-    pl->workspace = sizeof(WorkspaceHeader) + 8ull * pl->n_windows;
+    pl->workspace = sizeof(WorkspaceHeader) + 16ull * pl->n_windows;
     return DAF_OK;
 }
 

@@ -16,15 +16,18 @@ constexpr int kMaxGroups = 512;        // groups per window at G = 32, window 16
 constexpr int kMaxLevels = 4;          // widths {1,2,4,8}
 
 // ---------------------------------------------------------------------------------------------
-// Workspace layout: a 256-byte header followed by one 64-bit look-back descriptor per window.
-// The header and the descriptors are zeroed by a memset enqueued ahead of the kernel.
+// Workspace layout: a 256-byte header followed by two arrays of one 64-bit look-back descriptor
+// per window (one array for the quick kernel, one for the full kernel that runs if the quick one
+// gives up).  The header and the descriptors are zeroed by a memset enqueued ahead of the kernels.
 // ---------------------------------------------------------------------------------------------
 struct WorkspaceHeader {
     unsigned int status;        // daf_status recorded by the device (0 = OK)
     unsigned int ticket;        // next window to hand out
     unsigned int fail_window;   // first window that recorded an error (diagnostic)
     unsigned int fail_site;     // which wait or check recorded it (diagnostic)
-    unsigned int pad[60];
+    unsigned int retry;         // the quick kernel met a window it does not handle: the full kernel must run
+    unsigned int ticket2;       // next window to hand out in the full kernel
+    unsigned int pad[58];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
 

@@ -44,7 +44,9 @@ struct SmemLayout {          // byte offsets into dynamic shared memory
 
 template <int NT> struct CompressArgs {
     WorkspaceHeader *hdr;
-    uint64_t *flags;
+    uint64_t *flags;          // window descriptors of the quick kernel
+    uint64_t *flags2;         // ... of the full kernel
+    uint32_t gated;           // the full kernel runs only if the quick one asked for it
     uint32_t total_windows, n_tensors;
     uint32_t G, log2G, beta_q8, m, nearest, bulk_store, n_max;
     uint32_t full_ell, full_rem, full_rem_after;   // budget arithmetic of a full window (n_max groups)
@@ -417,7 +419,12 @@ struct Budget {
 
 // WIDTHS: at most 64 groups per window (groups of 256 elements or more), the widths warp settles
 // uniform windows; otherwise the compute warps that own group records do.
-template <typename T, int CHUNKS, bool BATCH, bool WIDTHS>
+// FULL: the complete kernel.  The quick kernel (FULL = false) is the same code without the
+// general bit choice and the clamped per-group quantizer, whose presence costs the common path
+// registers; when it meets a window that needs either, it raises hdr->retry, stops the hand-out
+// of windows and leaves, and the full kernel, enqueued behind it, redoes the call.  Otherwise
+// the full kernel finds hdr->retry clear and returns at once.
+template <typename T, int CHUNKS, bool BATCH, bool WIDTHS, bool FULL>
 __global__ void __launch_bounds__(kCompressThreads, 2)
 compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> a)
 {
@@ -428,6 +435,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     __shared__ __align__(8) uint64_t s_full;                     // mbarrier: staged window has landed (or there is none)
     __shared__ uint32_t s_next[2];                               // ticket of the window of iteration i (slot i & 1)
     __shared__ uint32_t s_lost;                                  // a staged copy did not land in time
+    __shared__ uint32_t s_abort;                                 // quick kernel: this CTA met a window it does not handle
     __shared__ uint32_t s_tot[2];                                // packed bytes of the window of iteration i (slot i & 1)
     __shared__ uint32_t s_mode[2];                               // how that window's widths came out (see below)
     __shared__ uint32_t s_slow[2];                               // a group of that window needs the clamped quantizer
@@ -442,11 +450,14 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t G = a.G, log2G = a.log2G;
+    uint64_t *const flags = FULL ? a.flags2 : a.flags;            // each kernel has its own descriptors and tickets
+    unsigned int *const ticket = FULL ? &a.hdr->ticket2 : &a.hdr->ticket;
+    if (FULL && a.gated != 0u && *reinterpret_cast<volatile unsigned int *>(&a.hdr->retry) == 0u) return;   // nothing to redo
 
     auto tensor_of = [&](uint32_t gw) -> const TensorDesc & { return a.t[BATCH ? find_tensor(a, gw) : 0u]; };
     // Control lane: draws a ticket; starts the bulk copy of that window into the stage, or
     // completes the stage's barrier empty-handed when the windows have run out.
-    auto draw_ticket = [&]() -> uint32_t { return atomicAdd(&a.hdr->ticket, 1u); };
+    auto draw_ticket = [&]() -> uint32_t { return atomicAdd(ticket, 1u); };
     auto stage_window = [&](uint32_t t, uint32_t iter) {
         s_next[iter & 1u] = t;                                    // ordered before the barrier's completion
         if (t < a.total_windows) {
@@ -483,6 +494,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     if (tid == kThreads) {
         mbar_init(&s_full, 1);
         s_lost = 0u;
+        s_abort = 0u;
         s_slow[0] = s_slow[1] = 0u;
         stage_window(draw_ticket(), 0u);
     }
@@ -559,11 +571,11 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             if (lane == 0) {
                 // the window's byte count is known: publish it at once
                 const uint32_t total = n * size;
-                st_relaxed_u64(a.flags + gw, ((w == 0u ? kFlagPrefix : kFlagAggregate) << kFlagShift) | total);
+                st_relaxed_u64(flags + gw, ((w == 0u ? kFlagPrefix : kFlagAggregate) << kFlagShift) | total);
                 s_tot[iter & 1u] = total;
             }
         }
-        if (lane == 0) s_mode[iter & 1u] = !same ? 0u : (n_elems == WE && !a.nearest) ? 1u + a.S[bud.ell] : 1u;
+        if (lane == 0) s_mode[iter & 1u] = !same ? 0u : !a.nearest ? 1u + a.S[bud.ell] : 1u;
     };
 
     if (warp == kComputeWarps + 1) {
@@ -572,7 +584,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         for (uint32_t iter = 0;; iter++) {
             bar_sync(kBarStage, stage_threads);                   // every unit's min / max is visible
             const uint32_t gw = s_next[iter & 1u];
-            if (gw >= a.total_windows) break;
+            if (gw >= a.total_windows || s_abort != 0u) break;
             if (s_lost == 0u) uniform_widths(gw, iter);
             bar_arrive(kBarWidths, kThreads + 32);                // the verdict on the window is in
             if (s_lost != 0u) break;
@@ -591,6 +603,15 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         for (uint32_t iter = 0;; iter++) {
             const bool valid = gw < a.total_windows;
             bar_sync(kBarStage, stage_threads);
+            if (!FULL && s_abort != 0u) {
+                // the compute warps have left (the window of the last iteration was not packed): see the
+                // copy in flight land before the shared memory goes away
+                if (valid && lane == 0) {
+                    mbar_wait_bounded(&s_full, iter & 1u);
+                    st_relaxed_u64(flags + gw, kFlagPoison << kFlagShift);   // the staged window is abandoned too
+                }
+                break;
+            }
             const bool lost = s_lost != 0u;
             uint32_t next = 0xFFFFFFFFu;
             if (valid && !lost) {
@@ -605,9 +626,9 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 uint64_t excl = 0;
                 int state = 1;
                 if (p_gw != pd.first_window) {
-                    state = lookback<kLookDepth>(a.flags, p_gw, pd.first_window, lane, true, &excl);
+                    state = lookback<kLookDepth>(flags, p_gw, pd.first_window, lane, true, &excl);
                     if (lane == 0)
-                        st_relaxed_u64(a.flags + p_gw, state == 1 ? ((kFlagPrefix << kFlagShift) | (excl + p_total))
+                        st_relaxed_u64(flags + p_gw, state == 1 ? ((kFlagPrefix << kFlagShift) | (excl + p_total))
                                                                     : (kFlagPoison << kFlagShift));
                 }
                 const uint32_t pw = p_gw - pd.first_window;
@@ -620,7 +641,9 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                     skip = excl + p_total > pd.capacity;
                 }
                 if (skip) {
-                    if (lane == 0) record_error(state == -2 ? DAF_ERR_TIMEOUT : DAF_ERR_CAPACITY, p_gw);
+                    // (a poisoned predecessor in the quick kernel is a window some CTA gave up on: the full
+                    // kernel redoes the call, nothing to report; a failed copy reports itself)
+                    if (lane == 0 && state != -1) record_error(state == -2 ? DAF_ERR_TIMEOUT : DAF_ERR_CAPACITY, p_gw);
                 } else if (a.bulk_store) {
                     if (lane == 0 && p_total) {
                         bulk_store(pd.packed + excl, src, p_total);
@@ -636,7 +659,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             if (lost) {
                 if (lane == 0) {
                     record_error(DAF_ERR_TIMEOUT, gw);
-                    st_relaxed_u64(a.flags + gw, kFlagPoison << kFlagShift);
+                    st_relaxed_u64(flags + gw, kFlagPoison << kFlagShift);
                     mbar_wait_bounded(&s_full, iter & 1u);        // one more bounded chance for the lost copy
                 }
                 break;
@@ -739,7 +762,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             }
             if (tid == 0) {
                 // the window's byte count is known: publish it at once
-                st_relaxed_u64(a.flags + gw, ((w == 0u ? kFlagPrefix : kFlagAggregate) << kFlagShift) | total);
+                st_relaxed_u64(flags + gw, ((w == 0u ? kFlagPrefix : kFlagAggregate) << kFlagShift) | total);
                 s_tot[iter & 1u] = total;
             }
         };
@@ -787,7 +810,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 }
                 if (s_lost == 0u) {
                     if (uniform) write_records(bud.ell, true);
-                    if (tid == 0) s_mode[iter & 1u] = !uniform ? 0u : (n_elems == WE && !a.nearest) ? 1u + a.S[bud.ell] : 1u;
+                    if (tid == 0) s_mode[iter & 1u] = !uniform ? 0u : !a.nearest ? 1u + a.S[bud.ell] : 1u;
                 }
             } else {
                 bar_arrive(kBarStage, stage_threads);
@@ -798,7 +821,20 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         const uint32_t mode = s_mode[iter & 1u];                  // 0: general choice needed; 1: records; 1 + b: one width b
         const uint64_t blk0 = ((td.elem_base + wbase) >> 3) + (e0 >> 3);
 
-        if (mode == 0u) {
+        const bool quick = mode >= 2u && s_slow[iter & 1u] == 0u; // one width, no clamp needed
+        if (!FULL && !quick) {
+            // ---------------------------------------------------------------- the quick kernel gives up
+            // No more windows are handed out (every later ticket is out of range), this window is
+            // marked abandoned for the look-back of its successors, and the CTA leaves.
+            if (tid == 0) {
+                atomicExch(&a.hdr->retry, 1u);
+                atomicOr(ticket, 0x80000000u);
+                st_relaxed_u64(flags + gw, kFlagPoison << kFlagShift);
+                s_abort = 1u;
+            }
+            break;
+        }
+        if (FULL && mode == 0u) {
             // -------------------------------------------------------------- general bit choice
             // The greedy of Sec. 3.4.1 accepts the longest prefix of the candidate raises, sorted by
             // (key descending, level ascending, group ascending), whose summed cost fits the window's
@@ -881,7 +917,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             bar_sync(kBarChoice, kThreads);                       // group records visible to all compute warps
         }
 
-        if (mode >= 2u && s_slow[iter & 1u] == 0u) {
+        if (quick) {
             // -------------------------------------------------------------- quantize + pack, one width, no clamp needed
             if (BATCH) {
                 const PhiloxSeedKeys sk{(uint32_t)td.seed, (uint32_t)(td.seed >> 32)};
@@ -889,7 +925,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             } else {
                 quantize_uniform_b<PhiloxKeys, CHUNKS>(mode - 1u, x, s_grp, log2G, e0, blk0, a.keys, s_out);
             }
-        } else {
+        } else if (FULL) {
             // -------------------------------------------------------------- quantize + pack with per-group widths
 #pragma unroll
             for (int c = 0; c < CHUNKS; c++) {
@@ -954,7 +990,7 @@ static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint
     return l;
 }
 
-template <typename T, int CHUNKS, bool BATCH, bool WIDTHS>
+template <typename T, int CHUNKS, bool BATCH, bool WIDTHS, bool FULL>
 static cudaError_t launch(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
     static int sms = 0, smem_set = 0, cached_smem = -1, cached_ctas = 0;   // per instantiation, current device
@@ -967,37 +1003,57 @@ static cudaError_t launch(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, c
         if (e != cudaSuccess) return e;
     }
     if (smem > smem_set) {
-        e = cudaFuncSetAttribute(compress_kernel<T, CHUNKS, BATCH, WIDTHS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        e = cudaFuncSetAttribute(compress_kernel<T, CHUNKS, BATCH, WIDTHS, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         smem_set = smem;
     }
     if (smem != cached_smem) {
         int per_sm = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel<T, CHUNKS, BATCH, WIDTHS>, kCompressThreads, smem);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel<T, CHUNKS, BATCH, WIDTHS, FULL>, kCompressThreads, smem);
         if (e != cudaSuccess) return e;
         cached_smem = smem;
         cached_ctas = sms * (per_sm > 0 ? per_sm : 1);
     }
     const uint32_t grid = args.total_windows < (uint32_t)cached_ctas ? args.total_windows : (uint32_t)cached_ctas;
-    compress_kernel<T, CHUNKS, BATCH, WIDTHS><<<grid, kCompressThreads, smem, stream>>>(args);
+    compress_kernel<T, CHUNKS, BATCH, WIDTHS, FULL><<<grid, kCompressThreads, smem, stream>>>(args);
     return cudaGetLastError();
 }
 
-template <bool BATCH>
-static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
-                            cudaStream_t stream)
+template <bool BATCH, bool FULL>
+static cudaError_t dispatch_one(uint32_t dtype, uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
+                                cudaStream_t stream)
 {
 #define DAF_CASE(T)                                                                     \
     switch (chunks) {                                                                   \
-    case 1: return widths ? launch<T, 1, BATCH, true>(args, stream) : launch<T, 1, BATCH, false>(args, stream);   \
-    case 2: return widths ? launch<T, 2, BATCH, true>(args, stream) : launch<T, 2, BATCH, false>(args, stream);   \
-    default: return widths ? launch<T, 4, BATCH, true>(args, stream) : launch<T, 4, BATCH, false>(args, stream);  \
+    case 1: return widths ? launch<T, 1, BATCH, true, FULL>(args, stream) : launch<T, 1, BATCH, false, FULL>(args, stream);   \
+    case 2: return widths ? launch<T, 2, BATCH, true, FULL>(args, stream) : launch<T, 2, BATCH, false, FULL>(args, stream);   \
+    default: return widths ? launch<T, 4, BATCH, true, FULL>(args, stream) : launch<T, 4, BATCH, false, FULL>(args, stream);  \
     }
     const bool widths = args.n_max <= 64u;                        // few enough groups for the widths warp
     if (dtype == DAF_F32) { DAF_CASE(float) }
     if (dtype == DAF_F16) { DAF_CASE(__half) }
     DAF_CASE(__nv_bfloat16)
 #undef DAF_CASE
+}
+
+// One call = the quick kernel followed by the full kernel, which returns at once unless the
+// quick one asked for it.  When the parameters rule out windows of one width (a budget that
+// no single width meets exactly and that leaves room for raises, or round-to-nearest), only
+// the full kernel is launched.
+template <bool BATCH>
+static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
+                            cudaStream_t stream)
+{
+    const bool all_max = args.full_ell + 1 == args.m;
+    const bool need_sep = !all_max && args.full_rem_after < args.cost[args.full_ell];
+    const bool try_quick = !args.nearest && (all_max || need_sep);
+    args.flags2 = args.flags + args.total_windows;
+    args.gated = try_quick ? 1u : 0u;
+    if (try_quick) {
+        const cudaError_t e = dispatch_one<BATCH, false>(dtype, chunks, args, stream);
+        if (e != cudaSuccess) return e;
+    }
+    return dispatch_one<BATCH, true>(dtype, chunks, args, stream);
 }
 
 template <int NT> static void fill_common(CompressArgs<NT> &a, const Plan &pl, const daf_params *p, void *ws)
@@ -1067,7 +1123,7 @@ extern "C" daf_status daf_compress(const daf_params *params, const void *d_in, v
 // only a handle: the address a kernel can use comes from cudaGetSymbolAddress, looked up once
 // per device with that device current.
 // ------------------------------------------------------------------------------------------
-static __device__ __align__(256) unsigned char g_static_scratch[sizeof(WorkspaceHeader) + 8ull * DAF_STATIC_MAX_WINDOWS];
+static __device__ __align__(256) unsigned char g_static_scratch[sizeof(WorkspaceHeader) + 16ull * DAF_STATIC_MAX_WINDOWS];
 
 extern "C" daf_status daf_compress_static(const daf_params *params, const void *d_in, void *d_packed,
                                           uint64_t packed_capacity, uint8_t *d_bits, float *d_min, float *d_scale,
@@ -1120,7 +1176,7 @@ extern "C" uint64_t daf_batch_workspace(uint32_t n, const daf_params *params)
         if (make_plan(&params[i], &pl) != DAF_OK) return 0;
         windows += pl.n_windows;
     }
-    return sizeof(WorkspaceHeader) + 8ull * windows;
+    return sizeof(WorkspaceHeader) + 16ull * windows;
 }
 
 extern "C" daf_status daf_compress_batch(uint32_t n, const daf_params *params, const void *const *d_in,
@@ -1159,7 +1215,7 @@ extern "C" daf_status daf_compress_batch(uint32_t n, const daf_params *params, c
         windows += pl.n_windows;
     }
     a.total_windows = (uint32_t)windows;
-    const uint64_t need = sizeof(WorkspaceHeader) + 8ull * windows;
+    const uint64_t need = sizeof(WorkspaceHeader) + 16ull * windows;
     if (workspace_bytes < need) return DAF_ERR_CAPACITY;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(d_workspace, 0, need, s) != cudaSuccess) return DAF_ERR_CUDA;
