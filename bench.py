@@ -31,7 +31,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per element seen by ncu (dram__bytes_read.sum + dram__bytes_write.sum) for one launch
 # on a 2^27-element fp32 slice of this workload (G = 256, budget 4): profiles/*_cfg5_G256_b4.md.
 # Traffic grows in proportion to the element count, so it is scaled to the launch being timed.
-NCU_TRAFFIC_BYTES_PER_ELEM = {"compress": 598.52e6 / (1 << 27), "decompress": 549.83e6 / (1 << 27)}
+NCU_TRAFFIC_BYTES_PER_ELEM = {"compress": 597.71e6 / (1 << 27), "decompress": 549.83e6 / (1 << 27)}
 
 
 def parse():
@@ -344,7 +344,7 @@ def run_cuda(args):
                            "l2": "inputs (4 GiB) far exceed the 126 MB L2; no flush needed"},
                 "compress_gbs": nbytes / (t_c.mean() * 1e-3) / 1e9, "decompress_gbs": nbytes / (t_d.mean() * 1e-3) / 1e9,
                 "compress_ms": float(t_c.mean()), "decompress_ms": float(t_d.mean()),
-                "clocks": clocks, "e2e": e2e, "gpu_launches": 2 * K, "roofline": roofline, "roofline_other": roofline_other,
+                "clocks": clocks, "e2e": e2e, "gpu_launches": 3 * K, "roofline": roofline, "roofline_other": roofline_other,
                 "cpu_baseline": cpu,
                 "parity": parity}
         print(json.dumps(line))

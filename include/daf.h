@@ -95,9 +95,12 @@ daf_status daf_sizes(const daf_params *params, uint64_t *n_groups, uint64_t *n_w
  *   d_window_offsets out: n_windows + 1 uint64
  *   d_workspace          : workspace_bytes of scratch, contents irrelevant on entry; also
  *                          holds the device status word afterwards (see daf_poll_status)
- * One fused kernel reads the input once.  If the packed output of a window would pass
- * packed_capacity, nothing of that window is stored and the status word becomes
- * DAF_ERR_CAPACITY.  Inputs must be finite; behaviour on NaN / Inf is unspecified but
+ * A fused kernel reads the input once.  (The call enqueues a quick kernel, which handles
+ * windows whose groups all end at the same width, and behind it the full kernel, which does
+ * nothing unless the quick one met a window it does not handle; then it redoes the call.
+ * Every output is final when the call's work on the stream is done.)  If the packed output
+ * of a window would pass packed_capacity, nothing of that window is stored and the status
+ * word becomes DAF_ERR_CAPACITY.  Inputs must be finite; behaviour on NaN / Inf is unspecified but
  * memory safe.  Calls sharing a workspace must not overlap on the GPU.
  */
 daf_status daf_compress(const daf_params *params, const void *d_in, void *d_packed,
@@ -165,8 +168,8 @@ daf_status daf_decompress_batch(uint32_t n, const daf_params *params, const void
  * for a workspace tensor would re-enter it; paths that cannot afford the device-wide
  * synchronisation an allocation may imply.  For them the scratch of the compress kernel (the
  * 256-byte header with ticket and status word, and one 64-bit look-back descriptor per window)
- * lives in a fixed array inside the library's device image: DAF_STATIC_MAX_WINDOWS descriptors,
- * 512.25 KiB, held by every GPU that loads the library until the process exits.
+ * lives in a fixed array inside the library's device image: two descriptors per window up to DAF_STATIC_MAX_WINDOWS,
+ * 1 MiB + 256 B, held by every GPU that loads the library until the process exits.
  *
  * Arguments as for daf_compress, minus the workspace.  d_status (device, 4-byte aligned, may be
  * NULL) receives the device status word (a daf_status) once the stream reaches that point.
