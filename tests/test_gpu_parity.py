@@ -185,6 +185,34 @@ def test_different_ranges_with_equal_keys(G):
         assert_decompress_parity(c, ref, "f32", f"collide/G{G}/{beta}")
 
 
+@pytest.mark.parametrize("dtype,G", [("f32", 256), ("f32", 64), ("bf16", 128), ("f32", 4096)])
+def test_a_few_mixed_windows_among_many_uniform_ones(dtype, G):
+    """Most windows end with one width for all groups (the quick kernel's case); a few windows far
+    into the tensor have groups of very different ranges, one has a range that needs the clamp, and
+    the last window is ragged: the call must come out the same whichever kernel finishes it."""
+    rng = np.random.default_rng(G + len(dtype))
+    n_win = 600                                                  # more windows than resident CTAs
+    n = 16384 * n_win + G * 3
+    a32 = rng.standard_normal(n).astype(np.float32)
+    for wdw in (301, 302, 577):                                  # mixed ranges: the general bit choice
+        lo = wdw * 16384
+        scale = 10.0 ** rng.uniform(-3, 3, 16384 // G)
+        a32[lo:lo + 16384] *= np.repeat(scale, G).astype(np.float32)
+    if dtype == "f32":
+        a32[450 * 16384] = np.float32(1.5e38)                      # 1/scale is not a normal number there
+        a32[450 * 16384 + 1] = np.float32(-1.5e38)
+    a = a32 if dtype == "f32" else wl.f32_to_bf16_bits(a32)
+    for beta in (4.0, 2.0):
+        x, c, ref = assert_compress_parity(a, dtype, G, (1, 2, 4, 8), beta, seed=21, label=f"few-mixed/{dtype}/G{G}/{beta}")
+        assert len(np.unique(ref.bits)) >= 2
+        assert_decompress_parity(c, ref, dtype, f"few-mixed/{dtype}/G{G}/{beta}")
+    # and a tensor that never leaves the quick kernel, right after one that did, on fresh outputs
+    u = rng.standard_normal(16384 * 40).astype(np.float32)
+    u = u if dtype == "f32" else wl.f32_to_bf16_bits(u)
+    x, c, ref = assert_compress_parity(u, dtype, G, (1, 2, 4, 8), 4.0, seed=22, label=f"all-uniform/{dtype}/G{G}")
+    assert_decompress_parity(c, ref, dtype, f"all-uniform/{dtype}/G{G}")
+
+
 @pytest.mark.parametrize("G,n_last", [(32, 5), (64, 37), (128, 100), (256, 63), (512, 1), (2048, 3)])
 def test_ragged_last_window_takes_the_general_choice(G, n_last):
     """A last window with a group count that is not a power of two, with mixed widths."""
