@@ -507,7 +507,8 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     // looks after groups l and l + 32.  See the compute warps' own version below for the test.
     constexpr bool ctl_widths = WIDTHS;
     const uint32_t stage_threads = ctl_widths ? kCompressThreads : kThreads + 32;   // who meets at the "stage" barrier
-    auto uniform_widths = [&](uint32_t gw, uint32_t iter) {
+    auto uniform_widths = [&](uint32_t gw, uint32_t iter, bool &arrived) {
+        arrived = false;
         const TensorDesc &td = tensor_of(gw);
         const uint32_t w = gw - td.first_window;
         const uint64_t wbase = (uint64_t)w * WE;
@@ -553,7 +554,6 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             for (int q = 0; q < 2; q++) {
                 const uint32_t g = (uint32_t)lane + 32u * q;
                 if (g < n) {
-                    const float scale = R[q] > 0.0f ? __fdiv_rn(R[q], Lf) : 0.0f;
                     const float inv = R[q] > 0.0f ? __fdiv_rn(Lf, R[q]) : 0.0f;
                     // 1/scale not a normal number: codes may need the clamp, take the careful quantizer
                     if (R[q] > 0.0f && inv < 0x1p-126f) s_slow[iter & 1u] = 1u;
@@ -563,9 +563,6 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                     rec.b = b;
                     rec.off = g * size;
                     s_grp[g] = rec;
-                    td.bits[g0 + g] = (uint8_t)b;
-                    td.mn[g0 + g] = mn[q];
-                    td.scale[g0 + g] = scale;
                 }
             }
             if (lane == 0) {
@@ -576,6 +573,21 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             }
         }
         if (lane == 0) s_mode[iter & 1u] = !same ? 0u : !a.nearest ? 1u + a.S[bud.ell] : 1u;
+        if (!same) return;
+        // the compute warps have what they need: let them go, then write the groups' metadata
+        bar_arrive(kBarWidths, kThreads + 32);
+        arrived = true;
+        const uint32_t b = a.S[bud.ell];
+        const float Lf = (float)((1u << b) - 1u);
+#pragma unroll
+        for (int q = 0; q < 2; q++) {
+            const uint32_t g = (uint32_t)lane + 32u * q;
+            if (g < n) {
+                td.bits[g0 + g] = (uint8_t)b;
+                td.mn[g0 + g] = mn[q];
+                td.scale[g0 + g] = R[q] > 0.0f ? __fdiv_rn(R[q], Lf) : 0.0f;
+            }
+        }
     };
 
     if (warp == kComputeWarps + 1) {
@@ -585,8 +597,9 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             bar_sync(kBarStage, stage_threads);                   // every unit's min / max is visible
             const uint32_t gw = s_next[iter & 1u];
             if (gw >= a.total_windows || s_abort != 0u) break;
-            if (s_lost == 0u) uniform_widths(gw, iter);
-            bar_arrive(kBarWidths, kThreads + 32);                // the verdict on the window is in
+            bool arrived = false;
+            if (s_lost == 0u) uniform_widths(gw, iter, arrived);
+            if (!arrived) bar_arrive(kBarWidths, kThreads + 32);  // the verdict on the window is in
             if (s_lost != 0u) break;
         }
         return;
