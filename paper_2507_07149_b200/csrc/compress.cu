@@ -439,6 +439,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     __shared__ uint32_t s_tot[2];                                // packed bytes of the window of iteration i (slot i & 1)
     __shared__ uint32_t s_mode[2];                               // how that window's widths came out (see below)
     __shared__ uint32_t s_slow[2];                               // a group of that window needs the clamped quantizer
+    __shared__ uint32_t s_kmin[2], s_kmax[2];                    // separation test of that window: key extremes over the owner warps
 
     unsigned char *const s_stage = smem;
     float *const s_umn = reinterpret_cast<float *>(smem + a.lay.umn);         // [2][units]
@@ -496,6 +497,8 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         s_lost = 0u;
         s_abort = 0u;
         s_slow[0] = s_slow[1] = 0u;
+        s_kmin[0] = s_kmin[1] = 0xFFFFFFFFu;
+        s_kmax[0] = s_kmax[1] = 0u;
         stage_window(draw_ticket(), 0u);
     }
     if (tid < kThreads)
@@ -804,21 +807,31 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         } else {
             if (owner) {
                 bar_sync(kBarStage, stage_threads);            // every unit's min / max is visible; the stage is free
-                if (tid == 0) s_slow[(iter & 1u) ^ 1u] = 0u;      // reset the flag of the next window
+                if (tid == 0) {                                   // reset the next window's slots
+                    s_slow[(iter & 1u) ^ 1u] = 0u;
+                    s_kmin[(iter & 1u) ^ 1u] = 0xFFFFFFFFu;
+                    s_kmax[(iter & 1u) ^ 1u] = 0u;
+                }
                 own_range();
                 bool uniform = bud.all_max || bud.need_sep;
                 if (bud.need_sep && bud.ell > 0) {
-                    // each owner warp evaluates the test over all groups itself (a unit is a group here)
-                    const float vl = a.v[bud.ell - 1], vh = a.v[bud.ell];
+                    // each owner warp puts in the key extremes of its own groups; the owners meet once
                     uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
-                    for (uint32_t g = lane; g < n; g += 32) {
-                        float R = __fsub_rn(umx[g], umn[g]);
-                        if (R < 0x1p-118f) R = 0.0f;
-                        kmin = min(kmin, __float_as_uint(__fmul_rn(R, vl)));
-                        kmax = max(kmax, __float_as_uint(__fmul_rn(R, vh)));
+                    if (mine) {
+                        kmin = __float_as_uint(__fmul_rn(Rg, a.v[bud.ell - 1]));
+                        kmax = __float_as_uint(__fmul_rn(Rg, a.v[bud.ell]));
                     }
                     kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
                     kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+                    if (owners > 1) {
+                        if (lane == 0) {
+                            atomicMin(&s_kmin[iter & 1u], kmin);
+                            atomicMax(&s_kmax[iter & 1u], kmax);
+                        }
+                        bar_sync(kBarOwners, owners * 32u);
+                        kmin = s_kmin[iter & 1u];
+                        kmax = s_kmax[iter & 1u];
+                    }
                     uniform = kmin >= kmax;
                 }
                 if (s_lost == 0u) {
