@@ -4,8 +4,9 @@
 
 Workloads 1-4 are sets of tensors: each set goes through ONE batched call (daf_compress_batch /
 daf_decompress_batch) when it has at most DAF_BATCH_MAX tensors.  Inputs are the seeded synthetic
-tensors of ``workloads.py``, resident in device memory before the timed region; times are CUDA
-events around K back-to-back calls (after 3 warm-up calls).  ``--scale S`` divides the batch
+tensors of ``workloads.py``, resident in device memory before the timed region; the time of a call
+is the median over K repetitions (after 3 warm-up calls), each bracketed by CUDA events; sets of
+less than 512 MiB have the L2 flushed between repetitions.  ``--scale S`` divides the batch
 dimension (or the element count of workload 5) by S for a quick look.  One markdown table row
 per workload is printed: element count, input bytes, packed bytes, compress and decompress
 time, and for each the algorithmic throughput: (tensor bytes + packed bytes + 9 bytes of
@@ -14,6 +15,8 @@ metadata per group + 8 per window) / time, the figure the roofline fractions are
 from __future__ import annotations
 
 import argparse
+
+import numpy as np
 
 
 
@@ -26,17 +29,28 @@ def _device_tensor(torch, wl, cfg, ti, spec):
     return h.cuda()
 
 
-def _time(torch, fn, steps):
+_FLUSH = None
+
+
+def _time(torch, fn, steps, flush):
+    """Median over `steps` repetitions, each bracketed by its own pair of CUDA events.  With `flush`
+    (working sets that would otherwise sit in the 126 MB L2) a 256 MiB buffer is overwritten
+    between repetitions, outside the timed interval."""
+    global _FLUSH
+    if flush and _FLUSH is None:
+        _FLUSH = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     for _ in range(3):
         fn()
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for e0, e1 in ev:
+        if flush:
+            _FLUSH.fill_(1)
+        e0.record()
         fn()
-    e1.record()
+        e1.record()
     torch.cuda.synchronize()
-    return e0.elapsed_time(e1) / steps
+    return float(np.median([e0.elapsed_time(e1) for e0, e1 in ev]))
 
 
 def run_set(torch, daf, wl, w, xs, steps):
@@ -71,9 +85,10 @@ def run_set(torch, daf, wl, w, xs, steps):
                                      [o.scale for o in outs], [o.window_offsets for o in outs], ys)
 
         status = lambda: daf.daf_poll_status(ws)
-    t_c = _time(torch, comp, steps)
+    flush = sum(x.numel() * x.element_size() for x in xs) < (512 << 20)
+    t_c = _time(torch, comp, steps, flush)
     assert status() == daf.OK, status()
-    t_d = _time(torch, dec, steps)
+    t_d = _time(torch, dec, steps, flush)
     packed = sum(o.packed_bytes() for o in outs)
     meta = sum(9 * (x.numel() // w.group_size) + 8 * (o.sizes.n_windows + 1) for x, o in zip(xs, outs))
     return t_c, t_d, packed, meta
@@ -89,7 +104,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", default="1,2,3,4,5")
     ap.add_argument("--sweep", action="store_true", help="also the 16 (group size, budget) points of workload 5")
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--scale", type=int, default=1)
     args = ap.parse_args()
 
