@@ -728,19 +728,26 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         const bool big = G > 256u;                                // a group spans several 256-element units
         float mn = 0.0f, Rg = 0.0f;
         // Owner threads: records, metadata, window total.  level_of: this thread's level.
+        // (the group's metadata is written by write_metadata: at once, or after the other warps have
+        // been let go when they wait for nothing but the records)
+        auto write_metadata = [&](uint32_t level) {
+            if (mine) {
+                const uint32_t b = a.S[level];
+                const float Lf = (float)((1u << b) - 1u);
+                td.bits[g0 + tid] = (uint8_t)b;
+                td.mn[g0 + tid] = mn;
+                td.scale[g0 + tid] = Rg > 0.0f ? __fdiv_rn(Rg, Lf) : 0.0f;
+            }
+        };
         auto write_records = [&](uint32_t level, bool uniform_b) {
             uint32_t size = 0, b = 0;
             float inv = 0.0f;
             if (mine) {
                 b = a.S[level];
                 const float Lf = (float)((1u << b) - 1u);
-                const float scale = Rg > 0.0f ? __fdiv_rn(Rg, Lf) : 0.0f;
                 inv = Rg > 0.0f ? __fdiv_rn(Lf, Rg) : 0.0f;
                 // 1/scale not a normal number: codes may need the clamp, take the careful quantizer
                 if (Rg > 0.0f && inv < 0x1p-126f) s_slow[iter & 1u] = 1u;
-                td.bits[g0 + tid] = (uint8_t)b;
-                td.mn[g0 + tid] = mn;
-                td.scale[g0 + tid] = scale;
                 size = (G >> 3) * b;
             }
             uint32_t total, off;
@@ -842,6 +849,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 bar_arrive(kBarStage, stage_threads);
             }
             bar_sync(kBarWidths, kThreads);                       // records (or the news that there are none yet) visible
+            if (owner && s_lost == 0u && s_mode[iter & 1u] != 0u) write_metadata(bud.ell);
         }
         if (s_lost != 0u) break;
         const uint32_t mode = s_mode[iter & 1u];                  // 0: general choice needed; 1: records; 1 + b: one width b
@@ -939,6 +947,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                     s_lvl[tid] = 0u;                              // zero again for the next window that ranks
                 }
                 write_records(level, false);
+                write_metadata(level);
             }
             bar_sync(kBarChoice, kThreads);                       // group records visible to all compute warps
         }
