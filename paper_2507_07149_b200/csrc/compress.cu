@@ -1,24 +1,30 @@
-// Fused compress kernel: one persistent CTA processes one window (window_elems elements) at a
-// time and reads the input from HBM exactly once.
+// Fused compress kernel: a persistent CTA (two per SM) processes one window (window_elems
+// elements) at a time and reads the input from HBM exactly once.
 //
 //   - the next window is staged into shared memory by one bulk asynchronous copy (TMA,
 //     completion on an mbarrier) while the current one is processed;
 //   - staged window -> registers (8 consecutive elements per lane and chunk), per-group
 //     min / max (3-input min/max, warp redux or segmented shuffles);
-//   - per-window greedy bit-width choice (Sec. 3.4.1 of the paper: importance per bit);
+//   - per-window greedy bit-width choice (Sec. 3.4.1 of the paper: importance per bit): a quick
+//     test recognises windows whose groups all end at the same width; the general case ranks
+//     the groups once and merges the levels' sorted keys by binary search;
 //   - intra-window exclusive scan of the group byte lengths; the window's byte count is
 //     published at once in a 64-bit descriptor;
 //   - Eq. 1 quantization with stochastic rounding (Philox4x32-10, 16 bits per element, the
 //     float -> uint step done with the power-of-two offset of Eq. 5) and lane-local LSB-first
 //     packing into a shared-memory buffer;
 //   - the window's device-wide byte offset comes from a bounded decoupled look-back over the
-//     descriptors, resolved opportunistically after the quantize pass and otherwise one
-//     window later, so that no CTA waits for its neighbours; the packed window then leaves
-//     shared memory as one bulk asynchronous store.
+//     descriptors, done one window later by a warp of its own, so that the compute warps never
+//     wait for other CTAs; the packed window then leaves shared memory as one bulk asynchronous
+//     store.
 //
 // Windows are handed out by an atomic ticket, so every window with a smaller index than the
 // one a CTA holds is owned by a running (or finished) CTA and the look-back always makes
 // progress; every wait is bounded all the same.
+//
+// The kernel is compiled in two forms (template flag FULL): a quick one for calls whose
+// windows all end with one width and need no clamp, and the full one, which runs behind it
+// only if the quick one gave up (see compress_kernel).
 #include "common.cuh"
 
 namespace daf {
