@@ -511,7 +511,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         for (uint32_t i = (uint32_t)tid; i < 2u * a.n_max; i += kThreads) s_cum[a.n_max + i] = 0u;   // ranks and levels count up from zero
     __syncthreads();
 
-    // With at most 64 groups per window (groups of 256 elements or more) a warp of its own, which
+    // With at most 64 groups per window (groups of 256 elements or more at the default window) a warp of its own, which
     // holds no window data, settles the windows whose groups all end at the same width: lane l
     // looks after groups l and l + 32.  See the compute warps' own version below for the test.
     constexpr bool ctl_widths = WIDTHS;
@@ -523,9 +523,10 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         const uint64_t wbase = (uint64_t)w * WE;
         const uint64_t left = td.numel - wbase;
         const uint32_t n_elems = left < WE ? (uint32_t)left : WE;
-        const uint32_t n = n_elems >> log2G, rr = G >> 8;
+        const uint32_t n = n_elems >> log2G;
+        const uint32_t rr = G > 256u ? G >> 8 : 1u;               // units per group (a unit: one group, at most 256 elements)
         const uint64_t g0 = wbase >> log2G;
-        const uint32_t units = WE >> 8;
+        const uint32_t units = WE >> (G < 256u ? log2G : 8u);
         const float *umn = s_umn + (iter & 1u) * units, *umx = s_umx + (iter & 1u) * units;
         const Budget bud = budget_of(n);
         const float vl = a.v[bud.ell > 0 ? bud.ell - 1 : 0], vh = a.v[bud.ell];

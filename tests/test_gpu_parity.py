@@ -345,6 +345,34 @@ def test_outputs_have_intact_guard_bands():
     assert np.array_equal(bufs["out"][1].cpu().numpy().view(np.uint16), oracle.decompress(ref).view(np.uint16))
 
 
+@pytest.mark.parametrize("case", range(48))
+def test_seeded_random_configurations(case):
+    """Group size, window size, widths, budget, type, rounding, length and value mix drawn from a
+    seed: uniform stretches, stretches of mixed ranges, constant groups and a ragged end in one tensor."""
+    rng = np.random.default_rng(1000 + case)
+    dtype = ("f32", "f16", "bf16")[case % 3]
+    We = int(rng.choice([4096, 8192, 16384]))
+    G = int(rng.choice([g for g in (32, 64, 128, 256, 512, 1024, 2048, 4096) if g <= We]))
+    widths = tuple(sorted(rng.choice([1, 2, 4, 8], size=int(rng.integers(1, 5)), replace=False).tolist()))
+    beta = float(rng.choice([min(widths), min(widths) + 0.5, 2.0, 3.0, 4.0, 8.0]))
+    beta = max(beta, float(min(widths)))
+    n_groups = int(rng.integers(1, 40 * We // G + 2))
+    x = rng.standard_normal((n_groups, G)).astype(np.float32)
+    kind = rng.random(n_groups)
+    scale = np.where(kind < 0.25, 10.0 ** rng.uniform(-3, 3, n_groups), 1.0).astype(np.float32)   # mixed ranges
+    x *= scale[:, None]
+    x[kind > 0.95] = np.float32(rng.standard_normal())                                            # constant groups
+    if case % 5 == 0:
+        x = np.abs(x)                                                                                # one-sided (ReLU-like)
+    a = x.reshape(-1)
+    a = a if dtype == "f32" else (a.astype(np.float16) if dtype == "f16" else wl.f32_to_bf16_bits(a))
+    rounding = daf.ROUND_NEAREST if case % 7 == 3 else daf.ROUND_STOCHASTIC
+    label = f"random/{case}/{dtype}/G{G}/We{We}/{widths}/{beta}"
+    xd, c, ref = assert_compress_parity(a, dtype, G, widths, beta, window_elems=We, rounding=rounding,
+                                        seed=case * 7919 + 1, label=label)
+    assert_decompress_parity(c, ref, dtype, label)
+
+
 # ------------------------------------------------------------------ batched calls
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_batched_calls_equal_single_calls(dtype):
