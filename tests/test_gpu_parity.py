@@ -409,3 +409,44 @@ def test_batched_calls_equal_single_calls(dtype):
         got = to_host(ys[i], dtype)
         assert np.array_equal(got.view(np.uint32 if dtype == "f32" else np.uint16),
                               want.view(np.uint32 if dtype == "f32" else np.uint16)), i
+
+
+@pytest.mark.parametrize("G,beta,mixed", [(256, 4.0, None), (256, 4.0, 3), (64, 2.0, 1), (1024, 4.0, 4), (4096, 8.0, None), (128, 4.0, 0)])
+def test_batched_calls_through_the_quick_and_the_full_kernel(G, beta, mixed):
+    """A set of tensors with ragged ends in one batched call; `mixed` names a tensor with groups of very
+    different ranges (the quick kernel gives up there and the full kernel redoes the whole set)."""
+    rng = np.random.default_rng(G + (mixed or 0))
+    widths = (1, 2, 4, 8)
+    sizes = [16384 * 7 + G, 16384 * 3, G * 2, 16384 * 21 + G * 5, 16384 * 2]
+    arrays = []
+    for i, n in enumerate(sizes):
+        a32 = rng.standard_normal(n).astype(np.float32)
+        if mixed == i:
+            a32 *= np.repeat(10.0 ** rng.uniform(-3, 3, n // G), G).astype(np.float32)
+        arrays.append(a32)
+    xs = [to_device(a, "f32") for a in arrays]
+    params = [daf.make_params(daf.F32, a.size, G, widths, beta, seed=500 + i) for i, a in enumerate(arrays)]
+    outs = [daf.alloc_outputs(p, "cuda") for p in params]
+    ws_bytes = daf.daf_batch_workspace(params)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    for _ in range(2):                                           # the second call reuses the workspace as it was left
+        daf.daf_compress_batch(params, xs, [o.packed for o in outs], [o.sizes.packed_capacity for o in outs],
+                               [o.bits for o in outs], [o.min for o in outs], [o.scale for o in outs],
+                               [o.window_offsets for o in outs], ws, ws_bytes)
+        assert daf.daf_poll_status(ws) == daf.OK
+    ys = [torch.empty_like(x) for x in xs]
+    daf.daf_decompress_batch(params, [o.packed for o in outs], [o.bits for o in outs], [o.min for o in outs],
+                             [o.scale for o in outs], [o.window_offsets for o in outs], ys)
+    torch.cuda.synchronize()
+    for i, a in enumerate(arrays):
+        ref = oracle.compress(a, G, widths, beta, seed=500 + i)
+        o = outs[i]
+        assert np.array_equal(o.bits.cpu().numpy(), ref.bits), i
+        assert np.array_equal(o.window_offsets.cpu().numpy().view(np.uint64), ref.window_offsets), i
+        assert np.array_equal(o.packed[: ref.packed.size].cpu().numpy(), ref.packed), i
+        assert np.array_equal(o.min.cpu().numpy().view(np.uint32), ref.mn.view(np.uint32)), i
+        assert np.array_equal(o.scale.cpu().numpy().view(np.uint32), ref.scale.view(np.uint32)), i
+        d = np.abs(ys[i].cpu().numpy().view(np.int32).astype(np.int64) - oracle.decompress(ref).view(np.int32).astype(np.int64))
+        assert d.max() <= 1, (i, int(d.max()))
+    if mixed is not None:
+        assert len(np.unique(oracle.compress(arrays[mixed], G, widths, beta, seed=500 + mixed).bits)) >= 2
