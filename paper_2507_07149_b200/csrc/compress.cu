@@ -582,8 +582,144 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 s_tot[iter & 1u] = total;
             }
         }
-        if (lane == 0) s_mode[iter & 1u] = !same ? 0u : !a.nearest ? 1u + a.S[bud.ell] : 1u;
-        if (!same) return;
+        if (!same) {
+            if (!FULL) {
+                if (lane == 0) s_mode[iter & 1u] = 0u;            // the quick kernel gives up on this window
+                return;
+            }
+            // ------------------------------------------------------------ general bit choice, by this warp alone
+            // The greedy of Sec. 3.4.1 accepts the longest prefix of the candidate raises, sorted by
+            // (key descending, level ascending, group ascending), whose summed cost fits what the
+            // window has left.  F(t), the cost of all raises with key >= t, falls as t grows, so the
+            // prefix is: every raise with a key above Kp, the largest t with F(t) > rem, and then
+            // the raises with key Kp in order while they fit.  Each lane holds the six keys of its
+            // two groups; one warp reduction gives F(t) and N(t), the number of raises with key >= t.
+            // The interval that holds Kp starts as the keys' common leading bits and is halved bit by
+            // bit; as soon as a single raise is left in it, its key is Kp.
+            const uint32_t nl = a.m - 1u;
+            uint32_t key[2][3], cw[2][3];                         // cw: cost in the low half, 1 in the high half
+            uint32_t hi = 0u, lo = 0xFFFFFFFFu;
+#pragma unroll
+            for (int q = 0; q < 2; q++)
+#pragma unroll
+                for (int k = 0; k < 3; k++) {
+                    const bool on = (uint32_t)k < nl && (uint32_t)lane + 32u * q < n;
+                    key[q][k] = on ? __float_as_uint(__fmul_rn(R[q], a.v[k])) : 0u;
+                    cw[q][k] = on ? a.cost[k] | 0x10000u : 0u;    // 0: not a candidate
+                    if (on) {
+                        hi = max(hi, key[q][k]);
+                        lo = min(lo, key[q][k]);
+                    }
+                }
+            hi = __reduce_max_sync(0xFFFFFFFFu, hi);
+            lo = __reduce_min_sync(0xFFFFFFFFu, lo);
+            auto from = [&](uint32_t t) {                         // F(t) | N(t) << 16
+                uint32_t f = 0;
+#pragma unroll
+                for (int q = 0; q < 2; q++)
+#pragma unroll
+                    for (int k = 0; k < 3; k++) f += key[q][k] >= t ? cw[q][k] : 0u;
+                return __reduce_add_sync(0xFFFFFFFFu, f);
+            };
+            uint32_t Kp = 0u, at_lo = from(0u), at_hi;            // F | N at the two ends of the interval
+            if ((at_lo & 0xFFFFu) > bud.rem) {
+                const uint32_t diff = hi ^ lo;
+                int bit = diff != 0u ? 31 - __clz(diff) : -1;     // the interval is [Kp, Kp + 2^(bit+1))
+                Kp = diff != 0u ? hi & ~((2u << bit) - 1u) : hi;
+                at_hi = 0u;
+                while (bit >= 0 && (at_lo >> 16) - (at_hi >> 16) > 1u) {
+                    const uint32_t t = Kp | (1u << bit);
+                    const uint32_t e = from(t);
+                    if ((e & 0xFFFFu) > bud.rem) {
+                        Kp = t;
+                        at_lo = e;
+                    } else {
+                        at_hi = e;
+                    }
+                    bit--;
+                }
+                if (bit >= 0) {                                   // one raise left in the interval: Kp is its key
+                    const uint32_t sh = (uint32_t)bit + 1u;
+                    uint32_t only = 0u;
+#pragma unroll
+                    for (int q = 0; q < 2; q++)
+#pragma unroll
+                        for (int k = 0; k < 3; k++)
+                            if (cw[q][k] != 0u && (sh >= 32u || (key[q][k] >> sh) == (Kp >> sh))) only = key[q][k];
+                    Kp = __reduce_max_sync(0xFFFFFFFFu, only);
+                }
+            } else {
+                at_hi = from(1u);                                 // every raise fits (Kp = 0)
+            }
+            uint32_t left = bud.rem - (at_hi & 0xFFFFu);          // after every raise with a key above Kp
+            uint32_t lvl[2] = {0u, 0u};
+            bool open = true;                                     // no raise has been turned down yet
+            const uint32_t below = (1u << lane) - 1u;
+#pragma unroll
+            for (int k = 0; k < 3; k++)
+#pragma unroll
+                for (int q = 0; q < 2; q++) {
+                    const bool on = cw[q][k] != 0u, tie = on && key[q][k] == Kp;
+                    const uint32_t ties = __ballot_sync(0xFFFFFFFFu, tie);
+                    uint32_t fit = 0u;
+                    if (ties != 0u && open) {
+                        const uint32_t cnt = (uint32_t)__popc(ties);
+                        fit = min(cnt, left / a.cost[k]);
+                        left -= fit * a.cost[k];
+                        open = fit == cnt;                        // the walk stops at the first raise that does not fit
+                    }
+                    lvl[q] += on && (key[q][k] > Kp || (tie && (uint32_t)__popc(ties & below) < fit));
+                }
+            // records: width, 1/scale, byte offset (exclusive scan of the sizes, both groups of a lane in one word)
+            uint32_t bq[2], size[2];
+#pragma unroll
+            for (int q = 0; q < 2; q++) {
+                bq[q] = a.S[lvl[q]];
+                size[q] = (uint32_t)lane + 32u * q < n ? (G >> 3) * bq[q] : 0u;
+            }
+            uint32_t incl = size[0] | (size[1] << 16);
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (lane >= o) incl += y;
+            }
+            const uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            const uint32_t total = (tot & 0xFFFFu) + (tot >> 16);
+#pragma unroll
+            for (int q = 0; q < 2; q++) {
+                const uint32_t g = (uint32_t)lane + 32u * q;
+                if (g < n) {
+                    const float Lf = (float)((1u << bq[q]) - 1u);
+                    const float inv = R[q] > 0.0f ? __fdiv_rn(Lf, R[q]) : 0.0f;
+                    if (R[q] > 0.0f && inv < 0x1p-126f) s_slow[iter & 1u] = 1u;
+                    GroupRec rec;
+                    rec.mn = mn[q];
+                    rec.inv = inv;
+                    rec.b = bq[q];
+                    rec.off = q == 0 ? (incl & 0xFFFFu) - size[0] : (tot & 0xFFFFu) + (incl >> 16) - size[1];
+                    s_grp[g] = rec;
+                }
+            }
+            if (lane == 0) {
+                st_relaxed_u64(flags + gw, ((w == 0u ? kFlagPrefix : kFlagAggregate) << kFlagShift) | total);
+                s_tot[iter & 1u] = total;
+                s_mode[iter & 1u] = 1u;                           // per-group records
+            }
+            bar_arrive(kBarWidths, kThreads + 32);
+            arrived = true;
+#pragma unroll
+            for (int q = 0; q < 2; q++) {
+                const uint32_t g = (uint32_t)lane + 32u * q;
+                if (g < n) {
+                    const float Lf = (float)((1u << bq[q]) - 1u);
+                    td.bits[g0 + g] = (uint8_t)bq[q];
+                    td.mn[g0 + g] = mn[q];
+                    td.scale[g0 + g] = R[q] > 0.0f ? __fdiv_rn(R[q], Lf) : 0.0f;
+                }
+            }
+            return;
+        }
+        if (lane == 0) s_mode[iter & 1u] = !a.nearest ? 1u + a.S[bud.ell] : 1u;
         // the compute warps have what they need: let them go, then write the groups' metadata
         bar_arrive(kBarWidths, kThreads + 32);
         arrived = true;
@@ -875,8 +1011,8 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             }
             break;
         }
-        if (FULL && mode == 0u) {
-            // -------------------------------------------------------------- general bit choice
+        if (FULL && !ctl_widths && mode == 0u) {
+            // -------------------------------------------------------------- general bit choice (more than 64 groups)
             // The greedy of Sec. 3.4.1 accepts the longest prefix of the candidate raises, sorted by
             // (key descending, level ascending, group ascending), whose summed cost fits the window's
             // budget.  Within one level the keys fl(R v_k) are a non-decreasing function of the range
@@ -886,7 +1022,6 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             // in the levels' sorted keys and accepts it if everything up to and including it fits.
             uint32_t *const s_Rb = s_cum, *const s_rank = s_cum + n_max, *const s_lvl = s_cum + 2u * n_max;
             uint32_t *const s_sorted = s_srt, *const s_sR = s_srt + n_max;
-            if (ctl_widths) own_range();
             if (mine) s_Rb[tid] = __float_as_uint(Rg);            // the ranges, side by side
             bar_sync(kBarChoice, kThreads);
             const bool pow2 = (n & (n - 1u)) == 0u;
