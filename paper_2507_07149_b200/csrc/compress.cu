@@ -415,6 +415,87 @@ template <bool OR_EQUAL> __device__ __forceinline__ uint32_t count_above(const u
     return lo;
 }
 
+// ------------------------------------------------------------------------------------------
+// The greedy of Sec. 3.4.1 on one warp.  Every lane holds NK candidate raises (key, cw = cost
+// | 1 << 16, or cw = 0 for "no candidate"); slot s of lane l sorts, among equal keys, before
+// slot s' > s of any lane and before slot s of lane l' > l.  Accepted is the longest prefix,
+// in the order (key descending, then that order), whose summed cost is at most rem; take[s]
+// says whether this lane's slot s is in it.  F(t), the cost of all raises with key >= t, falls
+// as t grows, so the prefix is every raise with a key above Kp, the largest t with F(t) > rem,
+// and then the raises with key Kp in order while they fit.  One warp reduction gives F(t) and
+// N(t), the number of raises with key >= t; the interval that holds Kp starts from the keys'
+// common leading bits (BOUNDS: the caller passes the largest and the smallest key) and is
+// halved bit by bit; as soon as a single raise is left in it, its key is Kp.
+// ------------------------------------------------------------------------------------------
+template <int NK, bool BOUNDS>
+__device__ __forceinline__ void accept_prefix(const uint32_t (&key)[NK], const uint32_t (&cw)[NK],
+                                              const uint32_t (&slot_cost)[NK], uint32_t rem, uint32_t hi, uint32_t lo,
+                                              int lane, bool (&take)[NK])
+{
+    if (!BOUNDS) {
+        hi = 0u;
+        lo = 0xFFFFFFFFu;
+#pragma unroll
+        for (int s = 0; s < NK; s++)
+            if (cw[s] != 0u) {
+                hi = max(hi, key[s]);
+                lo = min(lo, key[s]);
+            }
+        hi = __reduce_max_sync(0xFFFFFFFFu, hi);
+        lo = __reduce_min_sync(0xFFFFFFFFu, lo);
+    }
+    auto from = [&](uint32_t t) {                                 // F(t) | N(t) << 16
+        uint32_t f = 0;
+#pragma unroll
+        for (int s = 0; s < NK; s++) f += key[s] >= t ? cw[s] : 0u;
+        return __reduce_add_sync(0xFFFFFFFFu, f);
+    };
+    uint32_t Kp = 0u, at_lo = from(0u), at_hi;                    // F | N at the two ends of the interval
+    if ((at_lo & 0xFFFFu) > rem) {
+        const uint32_t diff = hi ^ lo;
+        int bit = diff != 0u ? 31 - __clz(diff) : -1;             // the interval is [Kp, Kp + 2^(bit+1))
+        Kp = diff != 0u ? hi & ~((2u << bit) - 1u) : hi;
+        at_hi = 0u;
+        while (bit >= 0 && (at_lo >> 16) - (at_hi >> 16) > 1u) {
+            const uint32_t t = Kp | (1u << bit);
+            const uint32_t e = from(t);
+            if ((e & 0xFFFFu) > rem) {
+                Kp = t;
+                at_lo = e;
+            } else {
+                at_hi = e;
+            }
+            bit--;
+        }
+        if (bit >= 0) {                                           // one raise left in the interval: Kp is its key
+            const uint32_t sh = (uint32_t)bit + 1u;
+            uint32_t only = 0u;
+#pragma unroll
+            for (int s = 0; s < NK; s++)
+                if (cw[s] != 0u && (sh >= 32u || (key[s] >> sh) == (Kp >> sh))) only = key[s];
+            Kp = __reduce_max_sync(0xFFFFFFFFu, only);
+        }
+    } else {
+        at_hi = from(1u);                                         // every raise fits (Kp = 0)
+    }
+    uint32_t left = rem - (at_hi & 0xFFFFu);                      // after every raise with a key above Kp
+    bool open = true;                                             // no raise has been turned down yet
+    const uint32_t below = (1u << lane) - 1u;
+#pragma unroll
+    for (int s = 0; s < NK; s++) {
+        const bool on = cw[s] != 0u, tie = on && key[s] == Kp;
+        const uint32_t ties = __ballot_sync(0xFFFFFFFFu, tie);
+        uint32_t fit = 0u;
+        if (ties != 0u && open) {
+            const uint32_t cnt = (uint32_t)__popc(ties);
+            fit = min(cnt, left / slot_cost[s]);
+            left -= fit * slot_cost[s];
+            open = fit == cnt;                                    // the walk stops at the first raise that does not fit
+        }
+        take[s] = on && (key[s] > Kp || (tie && (uint32_t)__popc(ties & below) < fit));
+    }
+}
+
 // Budget arithmetic of a window of n groups.
 struct Budget {
     uint32_t ell;          // largest level every group can be raised to
@@ -588,88 +669,54 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 return;
             }
             // ------------------------------------------------------------ general bit choice, by this warp alone
-            // The greedy of Sec. 3.4.1 accepts the longest prefix of the candidate raises, sorted by
-            // (key descending, level ascending, group ascending), whose summed cost fits what the
-            // window has left.  F(t), the cost of all raises with key >= t, falls as t grows, so the
-            // prefix is: every raise with a key above Kp, the largest t with F(t) > rem, and then
-            // the raises with key Kp in order while they fit.  Each lane holds the six keys of its
-            // two groups; one warp reduction gives F(t) and N(t), the number of raises with key >= t.
-            // The interval that holds Kp starts as the keys' common leading bits and is halved bit by
-            // bit; as soon as a single raise is left in it, its key is Kp.
+            // Lane l holds the keys fl(R v_k) of groups l and l + 32.  If every raise below level ell
+            // sorts ahead of every raise of level ell, and every raise above it behind, the accepted
+            // prefix is: all raises below ell (they fit by the definition of ell) and then raises of
+            // level ell alone, so only those two keys per lane enter the search; otherwise all six do.
             const uint32_t nl = a.m - 1u;
-            uint32_t key[2][3], cw[2][3];                         // cw: cost in the low half, 1 in the high half
-            uint32_t hi = 0u, lo = 0xFFFFFFFFu;
-#pragma unroll
-            for (int q = 0; q < 2; q++)
-#pragma unroll
-                for (int k = 0; k < 3; k++) {
-                    const bool on = (uint32_t)k < nl && (uint32_t)lane + 32u * q < n;
-                    key[q][k] = on ? __float_as_uint(__fmul_rn(R[q], a.v[k])) : 0u;
-                    cw[q][k] = on ? a.cost[k] | 0x10000u : 0u;    // 0: not a candidate
-                    if (on) {
-                        hi = max(hi, key[q][k]);
-                        lo = min(lo, key[q][k]);
-                    }
-                }
-            hi = __reduce_max_sync(0xFFFFFFFFu, hi);
-            lo = __reduce_min_sync(0xFFFFFFFFu, lo);
-            auto from = [&](uint32_t t) {                         // F(t) | N(t) << 16
-                uint32_t f = 0;
-#pragma unroll
-                for (int q = 0; q < 2; q++)
-#pragma unroll
-                    for (int k = 0; k < 3; k++) f += key[q][k] >= t ? cw[q][k] : 0u;
-                return __reduce_add_sync(0xFFFFFFFFu, f);
-            };
-            uint32_t Kp = 0u, at_lo = from(0u), at_hi;            // F | N at the two ends of the interval
-            if ((at_lo & 0xFFFFu) > bud.rem) {
-                const uint32_t diff = hi ^ lo;
-                int bit = diff != 0u ? 31 - __clz(diff) : -1;     // the interval is [Kp, Kp + 2^(bit+1))
-                Kp = diff != 0u ? hi & ~((2u << bit) - 1u) : hi;
-                at_hi = 0u;
-                while (bit >= 0 && (at_lo >> 16) - (at_hi >> 16) > 1u) {
-                    const uint32_t t = Kp | (1u << bit);
-                    const uint32_t e = from(t);
-                    if ((e & 0xFFFFu) > bud.rem) {
-                        Kp = t;
-                        at_lo = e;
-                    } else {
-                        at_hi = e;
-                    }
-                    bit--;
-                }
-                if (bit >= 0) {                                   // one raise left in the interval: Kp is its key
-                    const uint32_t sh = (uint32_t)bit + 1u;
-                    uint32_t only = 0u;
-#pragma unroll
-                    for (int q = 0; q < 2; q++)
-#pragma unroll
-                        for (int k = 0; k < 3; k++)
-                            if (cw[q][k] != 0u && (sh >= 32u || (key[q][k] >> sh) == (Kp >> sh))) only = key[q][k];
-                    Kp = __reduce_max_sync(0xFFFFFFFFu, only);
-                }
-            } else {
-                at_hi = from(1u);                                 // every raise fits (Kp = 0)
-            }
-            uint32_t left = bud.rem - (at_hi & 0xFFFFu);          // after every raise with a key above Kp
-            uint32_t lvl[2] = {0u, 0u};
-            bool open = true;                                     // no raise has been turned down yet
-            const uint32_t below = (1u << lane) - 1u;
+            uint32_t key[6], cw[6], slot_cost[6];                 // slot 2k + q: raise k of group lane + 32 q
+            uint32_t up_min = 0xFFFFFFFFu, dn_max = 0u, my_min = 0xFFFFFFFFu, my_max = 0u;
 #pragma unroll
             for (int k = 0; k < 3; k++)
 #pragma unroll
                 for (int q = 0; q < 2; q++) {
-                    const bool on = cw[q][k] != 0u, tie = on && key[q][k] == Kp;
-                    const uint32_t ties = __ballot_sync(0xFFFFFFFFu, tie);
-                    uint32_t fit = 0u;
-                    if (ties != 0u && open) {
-                        const uint32_t cnt = (uint32_t)__popc(ties);
-                        fit = min(cnt, left / a.cost[k]);
-                        left -= fit * a.cost[k];
-                        open = fit == cnt;                        // the walk stops at the first raise that does not fit
+                    const bool on = (uint32_t)k < nl && (uint32_t)lane + 32u * q < n;
+                    const uint32_t kk = on ? __float_as_uint(__fmul_rn(R[q], a.v[k])) : 0u;
+                    key[2 * k + q] = kk;
+                    cw[2 * k + q] = on ? a.cost[k] | 0x10000u : 0u;   // cost in the low half, 1 in the high half; 0: no candidate
+                    slot_cost[2 * k + q] = a.cost[k];
+                    if (on) {
+                        if ((uint32_t)k < bud.ell) up_min = min(up_min, kk);
+                        else if ((uint32_t)k > bud.ell) dn_max = max(dn_max, kk);
+                        else {
+                            my_min = min(my_min, kk);
+                            my_max = max(my_max, kk);
+                        }
                     }
-                    lvl[q] += on && (key[q][k] > Kp || (tie && (uint32_t)__popc(ties & below) < fit));
                 }
+            up_min = __reduce_min_sync(0xFFFFFFFFu, up_min);
+            dn_max = __reduce_max_sync(0xFFFFFFFFu, dn_max);
+            my_min = __reduce_min_sync(0xFFFFFFFFu, my_min);
+            my_max = __reduce_max_sync(0xFFFFFFFFu, my_max);
+            uint32_t lvl[2];
+            if (up_min >= my_max && dn_max <= my_min) {           // ties go to the lower level: >= and <= are enough
+                uint32_t key2[2], cw2[2], cost2[2];
+                bool take[2];
+#pragma unroll
+                for (int q = 0; q < 2; q++) {
+                    key2[q] = bud.ell == 0u ? key[q] : bud.ell == 1u ? key[2 + q] : key[4 + q];
+                    cw2[q] = bud.ell == 0u ? cw[q] : bud.ell == 1u ? cw[2 + q] : cw[4 + q];
+                    cost2[q] = a.cost[bud.ell];
+                }
+                accept_prefix<2, true>(key2, cw2, cost2, bud.rem - (a.S[bud.ell] - a.S[0]) * n, my_max, my_min, lane, take);
+                lvl[0] = bud.ell + take[0];
+                lvl[1] = bud.ell + take[1];
+            } else {
+                bool take[6];
+                accept_prefix<6, false>(key, cw, slot_cost, bud.rem, 0u, 0u, lane, take);
+                lvl[0] = (uint32_t)take[0] + take[2] + take[4];
+                lvl[1] = (uint32_t)take[1] + take[3] + take[5];
+            }
             // records: width, 1/scale, byte offset (exclusive scan of the sizes, both groups of a lane in one word)
             uint32_t bq[2], size[2];
 #pragma unroll
@@ -1104,6 +1151,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             }
         } else if (FULL) {
             // -------------------------------------------------------------- quantize + pack with per-group widths
+            const bool one_width_per_chunk = G >= 256u && s_slow[iter & 1u] == 0u;
 #pragma unroll
             for (int c = 0; c < CHUNKS; c++) {
                 const uint32_t e = e0 + 256u * c;
@@ -1121,7 +1169,16 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                     }
                 }
                 uint32_t w0, w1;
-                quantize8_any(x[c], rec.mn, rec.inv, o, rec.b, w0, w1);
+                if (one_width_per_chunk) {                        // the warp's chunk lies in one group: no clamp, fixed-width packing
+                    switch (rec.b) {
+                    case 1: quantize8<1, false>(x[c], rec.mn, rec.inv, o, w0, w1); break;
+                    case 2: quantize8<2, false>(x[c], rec.mn, rec.inv, o, w0, w1); break;
+                    case 4: quantize8<4, false>(x[c], rec.mn, rec.inv, o, w0, w1); break;
+                    default: quantize8<8, false>(x[c], rec.mn, rec.inv, o, w0, w1); break;
+                    }
+                } else {
+                    quantize8_any(x[c], rec.mn, rec.inv, o, rec.b, w0, w1);
+                }
                 unsigned char *p = s_out + rec.off + ((e & (G - 1u)) >> 3) * rec.b;
                 if (e < n_elems) {
                     if (rec.b == 1u) {
