@@ -45,7 +45,7 @@ struct TensorDesc {
 };
 
 struct SmemLayout {          // byte offsets into dynamic shared memory
-    uint32_t out0, out_stride, umn, umx, key, cum, srt, grp, total;
+    uint32_t out0, out_stride, umn, umx, sel, grp, total;
 };
 
 template <int NT> struct CompressArgs {
@@ -351,6 +351,7 @@ template <int NT> __device__ __forceinline__ uint32_t find_tensor(const Compress
 constexpr int kComputeWarps = kWarps;
 constexpr int kCompressThreads = kThreads + 64;
 constexpr uint32_t kBarStage = 1, kBarWidths = 2, kBarOwners = 3, kBarChoice = 4;
+constexpr int kSelWords = 180;                                // shared words of the general bit choice with more than 64 groups
 
 __device__ __forceinline__ void bar_sync(uint32_t id, uint32_t threads)
 {
@@ -400,19 +401,6 @@ __device__ __forceinline__ void quantize_uniform_b(uint32_t b, const float (&x)[
     case 4: quantize_uniform<KEYS, CHUNKS, 4>(x, s_grp, log2G, e0, blk0, keys, s_out); break;
     default: quantize_uniform<KEYS, CHUNKS, 8>(x, s_grp, log2G, e0, blk0, keys, s_out); break;
     }
-}
-
-// Number of entries of a non-increasing row that are > key (OR_EQUAL: >= key).
-template <bool OR_EQUAL> __device__ __forceinline__ uint32_t count_above(const uint32_t *row, uint32_t n, uint32_t key)
-{
-    uint32_t lo = 0, hi = n;
-    while (lo < hi) {
-        const uint32_t mid = (lo + hi) >> 1;
-        const bool ahead = OR_EQUAL ? row[mid] >= key : row[mid] > key;
-        if (ahead) lo = mid + 1u;
-        else hi = mid;
-    }
-    return lo;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -531,9 +519,8 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     unsigned char *const s_stage = smem;
     float *const s_umn = reinterpret_cast<float *>(smem + a.lay.umn);         // [2][units]
     float *const s_umx = reinterpret_cast<float *>(smem + a.lay.umx);
-    uint32_t *const s_key = reinterpret_cast<uint32_t *>(smem + a.lay.key);   // [level][n_max], in rank order
-    uint32_t *const s_cum = reinterpret_cast<uint32_t *>(smem + a.lay.cum);   // [3][n_max]: range, rank, level
-    uint32_t *const s_srt = reinterpret_cast<uint32_t *>(smem + a.lay.srt);   // [2][n_max]: group of rank r, its range
+    // general bit choice with more than 64 groups: [8][16] bins, largest / smallest key, sum of all, the last key, [3][16] ties
+    uint32_t *const s_sel = reinterpret_cast<uint32_t *>(smem + a.lay.sel);
     GroupRec *const s_grp = reinterpret_cast<GroupRec *>(smem + a.lay.grp);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -588,8 +575,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         s_kmax[0] = s_kmax[1] = 0u;
         stage_window(draw_ticket(), 0u);
     }
-    if (tid < kThreads)
-        for (uint32_t i = (uint32_t)tid; i < 2u * a.n_max; i += kThreads) s_cum[a.n_max + i] = 0u;   // ranks and levels count up from zero
+    if (FULL && !WIDTHS && tid < kSelWords) s_sel[tid] = tid == 129 ? 0xFFFFFFFFu : 0u;   // rest state of the choice's counters
     __syncthreads();
 
     // With at most 64 groups per window (groups of 256 elements or more at the default window) a warp of its own, which
@@ -1062,83 +1048,121 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             // -------------------------------------------------------------- general bit choice (more than 64 groups)
             // The greedy of Sec. 3.4.1 accepts the longest prefix of the candidate raises, sorted by
             // (key descending, level ascending, group ascending), whose summed cost fits the window's
-            // budget.  Within one level the keys fl(R v_k) are a non-decreasing function of the range
-            // R, so one ranking of the groups by (R descending, group ascending) sorts every level at
-            // once.  All compute threads count ranks; the owner of a group files its keys in rank
-            // order; then every thread places one candidate in the merged order by binary searches
-            // in the levels' sorted keys and accepts it if everything up to and including it fits.
-            uint32_t *const s_Rb = s_cum, *const s_rank = s_cum + n_max, *const s_lvl = s_cum + 2u * n_max;
-            uint32_t *const s_sorted = s_srt, *const s_sR = s_srt + n_max;
-            if (mine) s_Rb[tid] = __float_as_uint(Rg);            // the ranges, side by side
+            // budget.  F(t), the cost of all raises with key >= t, falls as t grows, so the prefix is
+            // every raise with a key above Kp, the largest t with F(t) > rem, and then the raises with
+            // key Kp in order while they fit.  Thread g holds the keys of group g; Kp is found four bits
+            // at a time from the top (below the keys' common leading bits): the raises whose key lies in
+            // the interval that still holds Kp are counted into sixteen bins by the next four bits
+            // (cost and number), one meeting per step, and every warp reads off the bin that holds Kp.
+            // As soon as a single raise is left in the interval, its key is Kp.
+            uint32_t *const H = s_sel, *const s_hi = s_sel + 128, *const s_lo = s_sel + 129, *const s_all = s_sel + 130;
+            uint32_t *const s_only = s_sel + 131, *const s_tie = s_sel + 132;
+            uint32_t key[3], cwk[3];                              // cwk: cost | 1 << 16, or 0 for "no candidate"
+            uint32_t whi = 0u, wlo = 0xFFFFFFFFu, wall = 0u;
+#pragma unroll
+            for (int k = 0; k < 3; k++) {
+                const bool on = mine && (uint32_t)k < nl;
+                key[k] = on ? __float_as_uint(__fmul_rn(Rg, a.v[k])) : 0u;
+                cwk[k] = on ? a.cost[k] | 0x10000u : 0u;
+                if (on) {
+                    whi = max(whi, key[k]);
+                    wlo = min(wlo, key[k]);
+                    wall += cwk[k];
+                }
+            }
+            whi = __reduce_max_sync(0xFFFFFFFFu, whi);
+            wlo = __reduce_min_sync(0xFFFFFFFFu, wlo);
+            wall = __reduce_add_sync(0xFFFFFFFFu, wall);
+            if (lane == 0 && wall != 0u) {
+                atomicMax(s_hi, whi);
+                atomicMin(s_lo, wlo);
+                atomicAdd(s_all, wall);
+            }
             bar_sync(kBarChoice, kThreads);
-            const bool pow2 = (n & (n - 1u)) == 0u;
-            const uint32_t sh = 31u - (uint32_t)__clz(n);
-            // (1) rank of every group by (range descending, group ascending).  Thread (g, slice)
-            //     counts the groups of its slice that sort ahead of g; a warp's lanes share the slice,
-            //     so its loads are broadcasts.
-            {
-                const uint32_t slices = (uint32_t)kThreads / n;   // n <= 512
-                const uint32_t g = pow2 ? (uint32_t)tid & (n - 1u) : (uint32_t)tid % n;
-                const uint32_t sl = pow2 ? (uint32_t)tid >> sh : (uint32_t)tid / n;
-                if (sl < slices) {
-                    const uint32_t len = (n + slices - 1u) / slices;
-                    const uint32_t h0 = sl * len, h1 = min(n, h0 + len);
-                    const uint32_t Rb = s_Rb[g];
-                    uint32_t cnt = 0;
-#pragma unroll 4
-                    for (uint32_t h = h0; h < h1; h++) {
-                        const uint32_t Rh = s_Rb[h];
-                        cnt += (Rh > Rb) || (Rh == Rb && h < g);
+            const uint32_t hi = *s_hi, lo = *s_lo, all = *s_all;
+            const uint32_t below = (1u << lane) - 1u;
+            uint32_t Kp = hi, above = 0u, ties = all >> 16;       // above: F | N << 16 of the raises beyond the interval
+            const bool take_all = (all & 0xFFFFu) <= bud.rem;     // every raise fits
+            if (!take_all && hi != lo) {
+                uint32_t sh = (31u - (uint32_t)__clz(hi ^ lo)) & ~3u;   // the four bits sh .. sh + 3 come next
+                Kp = sh >= 28u ? 0u : (hi >> (sh + 4u)) << (sh + 4u);
+                for (uint32_t j = 0;; j++) {
+                    uint32_t *const Hj = H + 16u * j;
+#pragma unroll
+                    for (int k = 0; k < 3; k++) {
+                        const bool m = cwk[k] != 0u && (sh >= 28u || ((key[k] ^ Kp) >> (sh + 4u)) == 0u);
+                        const uint32_t d = (key[k] >> sh) & 15u;
+                        const uint32_t act = __ballot_sync(0xFFFFFFFFu, m);
+                        if (act != 0u) {
+                            const int leader = __ffs(act) - 1;
+                            const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, d, leader);
+                            if (__all_sync(0xFFFFFFFFu, !m || d == d0)) {   // one bin for the whole warp: one atomic
+                                const uint32_t sum = __reduce_add_sync(0xFFFFFFFFu, m ? cwk[k] : 0u);
+                                if (lane == leader) atomicAdd(&Hj[d0], sum);
+                            } else if (m) {
+                                atomicAdd(&Hj[d], cwk[k]);
+                            }
+                        }
                     }
-                    if (cnt) atomicAdd(&s_rank[g], cnt);
+                    bar_sync(kBarChoice, kThreads);
+                    const uint32_t h = lane < 16 ? Hj[lane] : 0u;
+                    uint32_t S = h;                               // lanes 0..15: bins lane .. 15 summed
+#pragma unroll
+                    for (int o = 1; o < 16; o <<= 1) S += __shfl_down_sync(0xFFFFFFFFu, S, o);
+                    const uint32_t over = __ballot_sync(0xFFFFFFFFu, ((above + S) & 0xFFFFu) > bud.rem) & 0xFFFFu;
+                    const uint32_t dstar = 31u - (uint32_t)__clz(over | 1u);   // bin 0 always qualifies
+                    above += __shfl_sync(0xFFFFFFFFu, S, (int)(dstar + 1u));   // lane 16 holds 0
+                    ties = __shfl_sync(0xFFFFFFFFu, h, (int)dstar) >> 16;
+                    Kp |= dstar << sh;
+                    if (ties == 1u || sh == 0u) break;
+                    sh -= 4u;
+                }
+                if (sh != 0u) {                                   // one raise left in [Kp, Kp + 2^sh): Kp is its key
+#pragma unroll
+                    for (int k = 0; k < 3; k++)
+                        if (cwk[k] != 0u && ((key[k] ^ Kp) >> sh) == 0u) *s_only = key[k];
+                    bar_sync(kBarChoice, kThreads);
+                    Kp = *s_only;
                 }
             }
-            bar_sync(kBarChoice, kThreads);
-            // (2) keys of every level, filed in rank order
-            if (mine) {
-                const uint32_t r = s_rank[tid];
-                s_rank[tid] = 0u;                                 // zero again for the next window that ranks
-                s_sorted[r] = (uint32_t)tid;
-                s_sR[r] = __float_as_uint(Rg);
-                for (uint32_t k = 0; k < nl; k++) s_key[k * n_max + r] = __float_as_uint(__fmul_rn(Rg, a.v[k]));
-            }
-            bar_sync(kBarChoice, kThreads);
-            // (3) candidate (rank r, raise k): summed cost of everything sorting at or ahead of it
-            for (uint32_t it = (uint32_t)tid; it < n * nl; it += kThreads) {
-                const uint32_t r = pow2 ? it & (n - 1u) : it % n;
-                const uint32_t k = pow2 ? it >> sh : it / n;
-                const uint32_t *row = s_key + k * n_max;
-                const uint32_t K = row[r], g = s_sorted[r];
-                // same level: by rank, unless groups of different ranges share the key K (then the
-                // group index decides among them, not the range)
-                uint32_t ahead = r + 1u;
-                const bool head = r == 0u || row[r - 1u] != K, tail = r + 1u == n || row[r + 1u] != K;
-                if (!(head && tail)) {
-                    const uint32_t first = count_above<false>(row, n, K), end = count_above<true>(row, n, K);
-                    if (s_sR[first] != s_sR[end - 1u]) {
-                        ahead = first;
-                        for (uint32_t pos = first; pos < end; pos++) ahead += (s_sorted[pos] <= g);
+            const uint32_t left = bud.rem - (above & 0xFFFFu);    // after every raise with a key above Kp
+            uint32_t level = 0;
+            if (take_all) {
+                level = mine ? nl : 0u;
+            } else if (ties <= 1u) {
+#pragma unroll
+                for (int k = 0; k < 3; k++)
+                    if (cwk[k] != 0u) level += key[k] > Kp || (key[k] == Kp && a.cost[k] <= left);
+            } else {
+                // several raises share the key Kp: they are accepted level by level, group by group, while they fit
+                uint32_t tb[3];
+#pragma unroll
+                for (int k = 0; k < 3; k++) {
+                    tb[k] = __ballot_sync(0xFFFFFFFFu, cwk[k] != 0u && key[k] == Kp);
+                    if (lane == 0) s_tie[16 * k + warp] = (uint32_t)__popc(tb[k]);
+                }
+                bar_sync(kBarChoice, kThreads);
+#pragma unroll
+                for (int k = 0; k < 3; k++) {
+                    if (cwk[k] == 0u) continue;
+                    if (key[k] > Kp) {
+                        level++;
+                    } else if (key[k] == Kp) {
+                        uint32_t cum = 0;
+                        for (int k2 = 0; k2 < k; k2++)
+                            for (int wp = 0; wp < kComputeWarps; wp++) cum += s_tie[16 * k2 + wp] * a.cost[k2];
+                        for (int wp = 0; wp < warp; wp++) cum += s_tie[16 * k + wp] * a.cost[k];
+                        cum += ((uint32_t)__popc(tb[k] & below) + 1u) * a.cost[k];
+                        level += cum <= left;
                     }
                 }
-                uint32_t cum = ahead * a.cost[k];
-                for (uint32_t k2 = 0; k2 < nl; k2++) {            // other levels: ties go to the lower level
-                    if (k2 == k) continue;
-                    const uint32_t *row2 = s_key + k2 * n_max;
-                    cum += (k2 < k ? count_above<true>(row2, n, K) : count_above<false>(row2, n, K)) * a.cost[k2];
-                }
-                if (cum <= bud.rem) atomicAdd(&s_lvl[g], 1u);
             }
-            bar_sync(kBarChoice, kThreads);
             if (owner) {
-                uint32_t level = 0;
-                if (mine) {
-                    level = s_lvl[tid];
-                    s_lvl[tid] = 0u;                              // zero again for the next window that ranks
-                }
                 write_records(level, false);
                 write_metadata(level);
             }
             bar_sync(kBarChoice, kThreads);                       // group records visible to all compute warps
+            if (tid < kSelWords) s_sel[tid] = tid == 129 ? 0xFFFFFFFFu : 0u;   // the counters go back to their rest state
         }
 
         if (quick) {
@@ -1216,9 +1240,7 @@ static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint
     at += 2u * l.out_stride;
     l.umn = at; at += up(2u * 4u * units);
     l.umx = at; at += up(2u * 4u * units);
-    l.key = at; at += up(4u * (kMaxLevels - 1) * n_max);
-    l.cum = at; at += up(3u * 4u * n_max);
-    l.srt = at; at += up(2u * 4u * n_max);
+    l.sel = at; at += n_max > 64u ? up(4u * kSelWords) : 0u;
     l.grp = at; at += up(16u * n_max);
     l.total = at;
     return l;
