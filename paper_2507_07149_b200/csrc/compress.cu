@@ -1053,8 +1053,9 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             // key Kp in order while they fit.  Thread g holds the keys of group g; Kp is found four bits
             // at a time from the top (below the keys' common leading bits): the raises whose key lies in
             // the interval that still holds Kp are counted into sixteen bins by the next four bits
-            // (cost and number), one meeting per step, and every warp reads off the bin that holds Kp.
-            // As soon as a single raise is left in the interval, its key is Kp.
+            // (cost and number), one meeting of the owner warps per step, and each of them reads off the
+            // bin that holds Kp.  As soon as a single raise is left in the interval, its key is Kp.
+            if (owner) {                                          // the warps that own group records; the others wait below
             uint32_t *const H = s_sel, *const s_hi = s_sel + 128, *const s_lo = s_sel + 129, *const s_all = s_sel + 130;
             uint32_t *const s_only = s_sel + 131, *const s_tie = s_sel + 132;
             uint32_t key[3], cwk[3];                              // cwk: cost | 1 << 16, or 0 for "no candidate"
@@ -1078,7 +1079,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 atomicMin(s_lo, wlo);
                 atomicAdd(s_all, wall);
             }
-            bar_sync(kBarChoice, kThreads);
+            bar_sync(kBarOwners, owners * 32u);
             const uint32_t hi = *s_hi, lo = *s_lo, all = *s_all;
             const uint32_t below = (1u << lane) - 1u;
             uint32_t Kp = hi, above = 0u, ties = all >> 16;       // above: F | N << 16 of the raises beyond the interval
@@ -1104,7 +1105,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                             }
                         }
                     }
-                    bar_sync(kBarChoice, kThreads);
+                    bar_sync(kBarOwners, owners * 32u);
                     const uint32_t h = lane < 16 ? Hj[lane] : 0u;
                     uint32_t S = h;                               // lanes 0..15: bins lane .. 15 summed
 #pragma unroll
@@ -1121,7 +1122,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
 #pragma unroll
                     for (int k = 0; k < 3; k++)
                         if (cwk[k] != 0u && ((key[k] ^ Kp) >> sh) == 0u) *s_only = key[k];
-                    bar_sync(kBarChoice, kThreads);
+                    bar_sync(kBarOwners, owners * 32u);
                     Kp = *s_only;
                 }
             }
@@ -1141,7 +1142,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                     tb[k] = __ballot_sync(0xFFFFFFFFu, cwk[k] != 0u && key[k] == Kp);
                     if (lane == 0) s_tie[16 * k + warp] = (uint32_t)__popc(tb[k]);
                 }
-                bar_sync(kBarChoice, kThreads);
+                bar_sync(kBarOwners, owners * 32u);
 #pragma unroll
                 for (int k = 0; k < 3; k++) {
                     if (cwk[k] == 0u) continue;
@@ -1157,9 +1158,8 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                     }
                 }
             }
-            if (owner) {
-                write_records(level, false);
-                write_metadata(level);
+            write_records(level, false);
+            write_metadata(level);
             }
             bar_sync(kBarChoice, kThreads);                       // group records visible to all compute warps
             if (tid < kSelWords) s_sel[tid] = tid == 129 ? 0xFFFFFFFFu : 0u;   // the counters go back to their rest state
