@@ -25,6 +25,8 @@
 // The kernel is compiled in two forms (template flag FULL): a quick one for calls whose
 // windows all end with one width and need no clamp, and the full one, which runs behind it
 // only if the quick one gave up (see compress_kernel).
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace daf {
@@ -351,6 +353,7 @@ template <int NT> __device__ __forceinline__ uint32_t find_tensor(const Compress
 constexpr int kComputeWarps = kWarps;
 constexpr int kCompressThreads = kThreads + 64;
 constexpr uint32_t kBarStage = 1, kBarWidths = 2, kBarOwners = 3, kBarChoice = 4;
+constexpr uint32_t kQuickMinWindows = 512;                      // calls of fewer windows go to the full kernel alone
 constexpr int kSelWords = 180;                                // shared words of the general bit choice with more than 64 groups
 
 __device__ __forceinline__ void bar_sync(uint32_t id, uint32_t threads)
@@ -1296,13 +1299,22 @@ static cudaError_t dispatch_one(uint32_t dtype, uint32_t chunks, const CompressA
 // quick one asked for it.  When the parameters rule out windows of one width (a budget that
 // no single width meets exactly and that leaves room for raises, or round-to-nearest), only
 // the full kernel is launched.
+// Calls of at most this many windows skip the quick kernel (DAF_QUICK_MIN_WINDOWS in the environment overrides it).
+static uint32_t quick_min_windows()
+{
+    const char *e = std::getenv("DAF_QUICK_MIN_WINDOWS");
+    return e && *e ? (uint32_t)std::strtoul(e, nullptr, 10) : kQuickMinWindows;
+}
+
 template <bool BATCH>
 static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
                             cudaStream_t stream)
 {
     const bool all_max = args.full_ell + 1 == args.m;
     const bool need_sep = !all_max && args.full_rem_after < args.cost[args.full_ell];
-    const bool try_quick = !args.nearest && (all_max || need_sep);
+    // The quick kernel pays when there are many windows per CTA; a small call is launch-bound, and one
+    // launch of the full kernel is cheaper than the pair.
+    const bool try_quick = !args.nearest && (all_max || need_sep) && args.total_windows > quick_min_windows();
     args.flags2 = args.flags + args.total_windows;
     args.gated = try_quick ? 1u : 0u;
     if (try_quick) {

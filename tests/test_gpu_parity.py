@@ -349,6 +349,23 @@ def test_outputs_have_intact_guard_bands():
 def test_seeded_random_configurations(case):
     """Group size, window size, widths, budget, type, rounding, length and value mix drawn from a
     seed: uniform stretches, stretches of mixed ranges, constant groups and a ragged end in one tensor."""
+    _random_configuration(case)
+
+
+@pytest.mark.parametrize("case", range(0, 48, 2))
+def test_seeded_random_configurations_full_kernel_alone(case, default_quick_limit):
+    """The same with the library's default limit: calls this small skip the quick kernel."""
+    _random_configuration(case)
+
+
+def test_small_uniform_call_full_kernel_alone(default_quick_limit):
+    a = _gen(1, 0, wl.workload(1).tensors[0])[: 16384 * 9 + 2048]
+    x, c, ref = assert_compress_parity(a, "f32", 256, (1, 2, 4, 8), 4.0, seed=5, label="small/full-only")
+    assert set(np.unique(ref.bits)) == {4}
+    assert_decompress_parity(c, ref, "f32", "small/full-only")
+
+
+def _random_configuration(case):
     rng = np.random.default_rng(1000 + case)
     dtype = ("f32", "f16", "bf16")[case % 3]
     We = int(rng.choice([4096, 8192, 16384]))
