@@ -6,8 +6,9 @@
 //   - staged window -> registers (8 consecutive elements per lane and chunk), per-group
 //     min / max (3-input min/max, warp redux or segmented shuffles);
 //   - per-window greedy bit-width choice (Sec. 3.4.1 of the paper: importance per bit): a quick
-//     test recognises windows whose groups all end at the same width; the general case ranks
-//     the groups once and merges the levels' sorted keys by binary search;
+//     test recognises windows whose groups all end at the same width; the general case finds
+//     the key at which the accepted prefix of the sorted raises ends without sorting them (a
+//     bitwise search by one warp for up to 64 groups, a radix select by the owner warps above);
 //   - intra-window exclusive scan of the group byte lengths; the window's byte count is
 //     published at once in a 64-bit descriptor;
 //   - Eq. 1 quantization with stochastic rounding (Philox4x32-10, 16 bits per element, the
