@@ -92,26 +92,34 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, const Ke
     o[0] = c0; o[1] = c1; o[2] = c2; o[3] = c3;
 }
 
-// Round keys formed on the fly from a seed held in registers (used when the seed is not a
-// kernel-wide constant).
-struct PhiloxSeedKeys {
-    uint32_t lo, hi;
+// Round keys laid out in shared memory as {k0[r], k1[r]} pairs, r = 0 .. 9 (two rounds per
+// 16-byte load): for kernels that serve tensors with different seeds.
+struct PhiloxSharedKeys {
+    const uint4 *pairs;
 };
-__device__ __forceinline__ uint32_t philox_key0(const PhiloxKeys &k, int r) { return k.k0[r]; }
-__device__ __forceinline__ uint32_t philox_key1(const PhiloxKeys &k, int r) { return k.k1[r]; }
-__device__ __forceinline__ uint32_t philox_key0(const PhiloxSeedKeys &k, int r) { return k.lo + (uint32_t)r * kPhiloxW0; }
-__device__ __forceinline__ uint32_t philox_key1(const PhiloxSeedKeys &k, int r) { return k.hi + (uint32_t)r * kPhiloxW1; }
+__device__ __forceinline__ void philox_store_round_keys(uint32_t *pairs, uint64_t seed, int r)
+{
+    pairs[2 * r] = (uint32_t)seed + (uint32_t)r * kPhiloxW0;
+    pairs[2 * r + 1] = (uint32_t)(seed >> 32) + (uint32_t)r * kPhiloxW1;
+}
 template <>
-__device__ __forceinline__ void philox4x32_10<PhiloxSeedKeys>(uint32_t c0, uint32_t c1, const PhiloxSeedKeys &s,
-                                                               uint32_t (&o)[4])
+__device__ __forceinline__ void philox4x32_10<PhiloxSharedKeys>(uint32_t c0, uint32_t c1, const PhiloxSharedKeys &s,
+                                                                 uint32_t (&o)[4])
 {
     uint32_t c2 = 0u, c3 = 0u;
 #pragma unroll
-    for (int r = 0; r < 10; r++) {
-        const uint64_t p0 = (uint64_t)kPhiloxM0 * c0, p1 = (uint64_t)kPhiloxM1 * c2;
-        c0 = (uint32_t)(p1 >> 32) ^ c1 ^ (s.lo + (uint32_t)r * kPhiloxW0);
+    for (int i = 0; i < 5; i++) {
+        const uint4 k = s.pairs[i];
+        uint64_t p0 = (uint64_t)kPhiloxM0 * c0, p1 = (uint64_t)kPhiloxM1 * c2;
+        c0 = (uint32_t)(p1 >> 32) ^ c1 ^ k.x;
         c1 = (uint32_t)p1;
-        c2 = (uint32_t)(p0 >> 32) ^ c3 ^ (s.hi + (uint32_t)r * kPhiloxW1);
+        c2 = (uint32_t)(p0 >> 32) ^ c3 ^ k.y;
+        c3 = (uint32_t)p0;
+        p0 = (uint64_t)kPhiloxM0 * c0;
+        p1 = (uint64_t)kPhiloxM1 * c2;
+        c0 = (uint32_t)(p1 >> 32) ^ c1 ^ k.z;
+        c1 = (uint32_t)p1;
+        c2 = (uint32_t)(p0 >> 32) ^ c3 ^ k.w;
         c3 = (uint32_t)p0;
     }
     o[0] = c0; o[1] = c1; o[2] = c2; o[3] = c3;

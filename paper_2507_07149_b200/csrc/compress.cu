@@ -515,6 +515,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     __shared__ uint32_t s_next[2];                               // ticket of the window of iteration i (slot i & 1)
     __shared__ uint32_t s_lost;                                  // a staged copy did not land in time
     __shared__ uint32_t s_abort;                                 // quick kernel: this CTA met a window it does not handle
+    __shared__ __align__(16) uint32_t s_rkeys[2][20];            // batched calls: Philox round keys of the window's tensor
     __shared__ uint32_t s_tot[2];                                // packed bytes of the window of iteration i (slot i & 1)
     __shared__ uint32_t s_mode[2];                               // how that window's widths came out (see below)
     __shared__ uint32_t s_slow[2];                               // a group of that window needs the clamped quantizer
@@ -590,6 +591,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     auto uniform_widths = [&](uint32_t gw, uint32_t iter, bool &arrived) {
         arrived = false;
         const TensorDesc &td = tensor_of(gw);
+        if (BATCH && lane < 10) philox_store_round_keys(s_rkeys[iter & 1u], td.seed, lane);
         const uint32_t w = gw - td.first_window;
         const uint64_t wbase = (uint64_t)w * WE;
         const uint64_t left = td.numel - wbase;
@@ -994,6 +996,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         } else {
             if (owner) {
                 bar_sync(kBarStage, stage_threads);            // every unit's min / max is visible; the stage is free
+                if (BATCH && tid < 10) philox_store_round_keys(s_rkeys[iter & 1u], td.seed, tid);
                 if (tid == 0) {                                   // reset the next window's slots
                     s_slow[(iter & 1u) ^ 1u] = 0u;
                     s_kmin[(iter & 1u) ^ 1u] = 0xFFFFFFFFu;
@@ -1172,8 +1175,8 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         if (quick) {
             // -------------------------------------------------------------- quantize + pack, one width, no clamp needed
             if (BATCH) {
-                const PhiloxSeedKeys sk{(uint32_t)td.seed, (uint32_t)(td.seed >> 32)};
-                quantize_uniform_b<PhiloxSeedKeys, CHUNKS>(mode - 1u, x, s_grp, log2G, e0, blk0, sk, s_out);
+                const PhiloxSharedKeys sk{reinterpret_cast<const uint4 *>(s_rkeys[iter & 1u])};
+                quantize_uniform_b<PhiloxSharedKeys, CHUNKS>(mode - 1u, x, s_grp, log2G, e0, blk0, sk, s_out);
             } else {
                 quantize_uniform_b<PhiloxKeys, CHUNKS>(mode - 1u, x, s_grp, log2G, e0, blk0, a.keys, s_out);
             }
@@ -1190,7 +1193,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 } else {
                     const uint64_t blk = blk0 + 32u * c;
                     if (BATCH) {
-                        const PhiloxSeedKeys sk{(uint32_t)td.seed, (uint32_t)(td.seed >> 32)};
+                        const PhiloxSharedKeys sk{reinterpret_cast<const uint4 *>(s_rkeys[iter & 1u])};
                         philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), sk, o);
                     } else {
                         philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), a.keys, o);
