@@ -1182,12 +1182,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
             }
         } else if (FULL) {
             // -------------------------------------------------------------- quantize + pack with per-group widths
-            const bool one_width_per_chunk = G >= 256u && s_slow[iter & 1u] == 0u;
-#pragma unroll
-            for (int c = 0; c < CHUNKS; c++) {
-                const uint32_t e = e0 + 256u * c;
-                const GroupRec rec = s_grp[e >> log2G];
-                uint32_t o[4];
+            auto draw = [&](int c, uint32_t (&o)[4]) {
                 if (a.nearest) {
                     o[0] = o[1] = o[2] = o[3] = 0x80008000u;       // every 16-bit lane = 2 * 2^14
                 } else {
@@ -1199,30 +1194,58 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                         philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), a.keys, o);
                     }
                 }
-                uint32_t w0, w1;
-                if (one_width_per_chunk) {                        // the warp's chunk lies in one group: no clamp, fixed-width packing
+            };
+            if (G >= 256u && s_slow[iter & 1u] == 0u) {
+                // a warp's chunk lies in one group: no clamp, fixed-width packing, 8-byte aligned stores
+#pragma unroll
+                for (int c = 0; c < CHUNKS; c++) {
+                    const uint32_t e = e0 + 256u * c;
+                    if (e >= n_elems) break;                      // ragged last window: whole chunks are missing
+                    const GroupRec rec = s_grp[e >> log2G];
+                    uint32_t o[4], w0, w1;
+                    draw(c, o);
+                    unsigned char *p = s_out + rec.off + ((e & (G - 1u)) >> 3) * rec.b;
                     switch (rec.b) {
-                    case 1: quantize8<1, false>(x[c], rec.mn, rec.inv, o, w0, w1); break;
-                    case 2: quantize8<2, false>(x[c], rec.mn, rec.inv, o, w0, w1); break;
-                    case 4: quantize8<4, false>(x[c], rec.mn, rec.inv, o, w0, w1); break;
-                    default: quantize8<8, false>(x[c], rec.mn, rec.inv, o, w0, w1); break;
-                    }
-                } else {
-                    quantize8_any(x[c], rec.mn, rec.inv, o, rec.b, w0, w1);
-                }
-                unsigned char *p = s_out + rec.off + ((e & (G - 1u)) >> 3) * rec.b;
-                if (e < n_elems) {
-                    if (rec.b == 1u) {
+                    case 1:
+                        quantize8<1, false>(x[c], rec.mn, rec.inv, o, w0, w1);
                         *p = (unsigned char)w0;
-                    } else if (rec.b == 2u) {
+                        break;
+                    case 2:
+                        quantize8<2, false>(x[c], rec.mn, rec.inv, o, w0, w1);
                         *reinterpret_cast<uint16_t *>(p) = (uint16_t)w0;
-                    } else if (rec.b == 4u) {
+                        break;
+                    case 4:
+                        quantize8<4, false>(x[c], rec.mn, rec.inv, o, w0, w1);
                         *reinterpret_cast<uint32_t *>(p) = w0;
-                    } else if (G >= 64u) {
+                        break;
+                    default:
+                        quantize8<8, false>(x[c], rec.mn, rec.inv, o, w0, w1);
                         *reinterpret_cast<uint2 *>(p) = make_uint2(w0, w1);
-                    } else {                                       // G = 32: groups are only 4-byte aligned
-                        reinterpret_cast<uint32_t *>(p)[0] = w0;
-                        reinterpret_cast<uint32_t *>(p)[1] = w1;
+                        break;
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int c = 0; c < CHUNKS; c++) {
+                    const uint32_t e = e0 + 256u * c;
+                    const GroupRec rec = s_grp[e >> log2G];
+                    uint32_t o[4], w0, w1;
+                    draw(c, o);
+                    quantize8_any(x[c], rec.mn, rec.inv, o, rec.b, w0, w1);
+                    unsigned char *p = s_out + rec.off + ((e & (G - 1u)) >> 3) * rec.b;
+                    if (e < n_elems) {
+                        if (rec.b == 1u) {
+                            *p = (unsigned char)w0;
+                        } else if (rec.b == 2u) {
+                            *reinterpret_cast<uint16_t *>(p) = (uint16_t)w0;
+                        } else if (rec.b == 4u) {
+                            *reinterpret_cast<uint32_t *>(p) = w0;
+                        } else if (G >= 64u) {
+                            *reinterpret_cast<uint2 *>(p) = make_uint2(w0, w1);
+                        } else {                                   // G = 32: groups are only 4-byte aligned
+                            reinterpret_cast<uint32_t *>(p)[0] = w0;
+                            reinterpret_cast<uint32_t *>(p)[1] = w1;
+                        }
                     }
                 }
             }
