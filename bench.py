@@ -31,7 +31,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per element seen by ncu (dram__bytes_read.sum + dram__bytes_write.sum) for one launch
 # on a 2^27-element fp32 slice of this workload (G = 256, budget 4): profiles/*_cfg5_G256_b4.md.
 # Traffic grows in proportion to the element count, so it is scaled to the launch being timed.
-NCU_TRAFFIC_BYTES_PER_ELEM = {"compress": 596.52e6 / (1 << 27), "decompress": 549.83e6 / (1 << 27)}
+NCU_TRAFFIC_BYTES_PER_ELEM = {"compress": 599.04e6 / (1 << 27), "decompress": 549.83e6 / (1 << 27)}
 
 
 def parse():
