@@ -78,28 +78,31 @@ decompress_kernel(const __grid_constant__ DecompressArgs<BATCH ? DAF_BATCH_MAX :
     const uint32_t n = n_elems >> log2G;
     const uint64_t g0 = wbase >> log2G;
 
-    // group records: width, min, scale and the group's byte offset inside the window
-    uint32_t b = 0, size = 0;
+    const uint64_t window_offset = td.woff[w];                    // asked for now, needed after the two meetings below
+    // group records: width, min, scale and the group's byte offset inside the window; built by the
+    // warps whose threads map to groups (thread g: group g), the others only meet them
+    const bool owner = (uint32_t)(warp * 32) < n;
+    uint32_t b = 0, size = 0, incl = 0;
     float mn = 0.0f, scale = 0.0f;
-    if ((uint32_t)tid < n) {
-        b = td.bits[g0 + tid];
-        mn = td.mn[g0 + tid];
-        scale = td.scale[g0 + tid];
-        size = (G >> 3) * b;
-    }
-    uint32_t incl = size;
+    if (owner) {
+        if ((uint32_t)tid < n) {
+            b = td.bits[g0 + tid];
+            mn = td.mn[g0 + tid];
+            scale = td.scale[g0 + tid];
+            size = (G >> 3) * b;
+        }
+        incl = size;
 #pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        uint32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-        if (lane >= off) incl += y;
+        for (int off = 1; off < 32; off <<= 1) {
+            uint32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+            if (lane >= off) incl += y;
+        }
+        if (lane == 31) s_wtot[warp] = incl;
     }
-    if (lane == 31) s_wtot[warp] = incl;
     __syncthreads();
-    uint32_t before = 0;
-#pragma unroll
-    for (int i = 0; i < kWarps; i++)
-        if (i < warp) before += s_wtot[i];
     if ((uint32_t)tid < n) {
+        uint32_t before = 0;
+        for (int i = 0; i < warp; i++) before += s_wtot[i];
         DecRec rec;
         rec.mn = mn;
         rec.scale = scale;
@@ -109,7 +112,7 @@ decompress_kernel(const __grid_constant__ DecompressArgs<BATCH ? DAF_BATCH_MAX :
     }
     __syncthreads();
 
-    const uint8_t *src = td.packed + td.woff[w];
+    const uint8_t *src = td.packed + window_offset;
     char *out = reinterpret_cast<char *>(td.out) + wbase * Elem<T>::kBytes;
 #pragma unroll
     for (int c = 0; c < CHUNKS; c++) {
