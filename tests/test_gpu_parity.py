@@ -467,3 +467,60 @@ def test_batched_calls_through_the_quick_and_the_full_kernel(G, beta, mixed):
         assert d.max() <= 1, (i, int(d.max()))
     if mixed is not None:
         assert len(np.unique(oracle.compress(arrays[mixed], G, widths, beta, seed=500 + mixed).bits)) >= 2
+
+
+def test_batched_calls_replayed_from_a_cuda_graph():
+    """The calls only enqueue work (a memset and kernels), so a layer list can be captured once and
+    replayed: compress + decompress of three tensors captured in a CUDA graph, replayed on new contents."""
+    rng = np.random.default_rng(77)
+    G, widths, beta = 256, (1, 2, 4, 8), 4.0
+    sizes = [16384 * 40 + G * 3, 16384 * 6, 16384 * 13 + G]
+    xs = [torch.empty(n, dtype=torch.float32, device="cuda") for n in sizes]
+    params = [daf.make_params(daf.F32, n, G, widths, beta, seed=900 + i) for i, n in enumerate(sizes)]
+    outs = [daf.alloc_outputs(p, "cuda") for p in params]
+    ys = [torch.empty_like(x) for x in xs]
+    ws_bytes = daf.daf_batch_workspace(params)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+
+    def step():
+        daf.daf_compress_batch(params, xs, [o.packed for o in outs], [o.sizes.packed_capacity for o in outs],
+                               [o.bits for o in outs], [o.min for o in outs], [o.scale for o in outs],
+                               [o.window_offsets for o in outs], ws, ws_bytes)
+        daf.daf_decompress_batch(params, [o.packed for o in outs], [o.bits for o in outs], [o.min for o in outs],
+                                 [o.scale for o in outs], [o.window_offsets for o in outs], ys)
+
+    def fill(mixed):
+        arrays = []
+        for i, (x, n) in enumerate(zip(xs, sizes)):
+            a = rng.standard_normal(n).astype(np.float32)
+            if i == mixed:
+                a *= np.repeat(10.0 ** rng.uniform(-2, 2, n // G), G).astype(np.float32)
+            x.copy_(torch.from_numpy(a))
+            arrays.append(a)
+        return arrays
+
+    fill(None)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()                                                   # first call outside the capture (one-time set-up)
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for mixed in (None, 1):                                      # uniform windows only, then a tensor the quick kernel gives up on
+        arrays = fill(mixed)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert daf.daf_poll_status(ws) == daf.OK
+        for i, a in enumerate(arrays):
+            ref = oracle.compress(a, G, widths, beta, seed=900 + i)
+            o = outs[i]
+            assert np.array_equal(o.bits.cpu().numpy(), ref.bits), (mixed, i)
+            assert np.array_equal(o.window_offsets.cpu().numpy().view(np.uint64), ref.window_offsets), (mixed, i)
+            assert np.array_equal(o.packed[: ref.packed.size].cpu().numpy(), ref.packed), (mixed, i)
+            d = np.abs(ys[i].cpu().numpy().view(np.int32).astype(np.int64)
+                       - oracle.decompress(ref).view(np.int32).astype(np.int64))
+            assert d.max() <= 1, (mixed, i, int(d.max()))
+        if mixed is not None:
+            assert len(np.unique(oracle.compress(arrays[mixed], G, widths, beta, seed=900 + mixed).bits)) >= 2
