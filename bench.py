@@ -277,7 +277,7 @@ def run_cuda(args):
         oracle.build()
         We = 16384
         n_w = c.sizes.n_windows
-        pick = sorted(set([0, n_w - 1] + list(np.random.default_rng(0).integers(0, n_w, 6))))
+        pick = sorted(set([0, n_w - 1] + [int(v) for v in np.random.default_rng(0).integers(0, n_w, 256)]))   # first, last, 256 random
         woff = c.window_offsets.cpu().numpy()
         for wi in pick:
             lo, hi = wi * We, min(spec.numel, (wi + 1) * We)

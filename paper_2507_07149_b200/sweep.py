@@ -10,7 +10,8 @@ less than 512 MiB have the L2 flushed between repetitions.  ``--scale S`` divide
 dimension (or the element count of workload 5) by S for a quick look.  One markdown table row
 per workload is printed: element count, input bytes, packed bytes, compress and decompress
 time, and for each the algorithmic throughput: (tensor bytes + packed bytes + 9 bytes of
-metadata per group + 8 per window) / time, the figure the roofline fractions are quoted on.
+metadata per group + 8 per window) / time, the figure the roofline fractions are quoted on;
+for the sets also the times of the same work issued as one call per tensor.
 """
 from __future__ import annotations
 
@@ -91,13 +92,26 @@ def run_set(torch, daf, wl, w, xs, steps):
     t_d = _time(torch, dec, steps, flush)
     packed = sum(o.packed_bytes() for o in outs)
     meta = sum(9 * (x.numel() // w.group_size) + 8 * (o.sizes.n_windows + 1) for x, o in zip(xs, outs))
-    return t_c, t_d, packed, meta
+    per_tensor = None
+    if len(xs) > 1:                                              # the same set as one call per tensor
+        def comp_each():
+            for p, x, c in zip(params, xs, outs):
+                daf.daf_compress(p, x, c.packed, c.sizes.packed_capacity, c.bits, c.min, c.scale, c.window_offsets,
+                                 c.workspace, c.sizes.workspace)
+
+        def dec_each():
+            for p, c, y in zip(params, outs, ys):
+                daf.daf_decompress(p, c.packed, c.bits, c.min, c.scale, c.window_offsets, y)
+
+        per_tensor = (_time(torch, comp_each, steps, flush), _time(torch, dec_each, steps, flush))
+    return t_c, t_d, packed, meta, per_tensor
 
 
-def row(name, numel, nbytes, packed, meta, t_c, t_d):
+def row(name, numel, nbytes, packed, meta, t_c, t_d, per_tensor=None):
     alg = nbytes + packed + meta
+    each = "— | —" if per_tensor is None else f"{per_tensor[0]:.4f} | {per_tensor[1]:.4f}"
     return (f"| {name} | {numel} | {nbytes / 2**30:.3f} | {packed / 2**30:.3f} | {t_c:.4f} | {alg / t_c / 1e6:.0f} | "
-            f"{t_d:.4f} | {alg / t_d / 1e6:.0f} |")
+            f"{t_d:.4f} | {alg / t_d / 1e6:.0f} | {each} |")
 
 
 def main():
@@ -113,8 +127,9 @@ def main():
     from paper_2507_07149_b200 import workloads as wl
 
     daf.lib()
-    print("| workload | elements | tensor GiB | packed GiB | compress ms | compress GB/s | decompress ms | decompress GB/s |")
-    print("|---|---|---|---|---|---|---|---|")
+    print("| workload | elements | tensor GiB | packed GiB | compress ms | compress GB/s | decompress ms | decompress GB/s "
+          "| compress ms, one call per tensor | decompress ms, one call per tensor |")
+    print("|---|---|---|---|---|---|---|---|---|---|")
     S = args.scale
     for cfg in [int(c) for c in args.configs.split(",")]:
         kw = {}
@@ -124,14 +139,14 @@ def main():
             kw["numel"] = (1 << 30) // S
         w = wl.workload(cfg, **kw)
         xs = [_device_tensor(torch, wl, cfg, i, t) for i, t in enumerate(w.tensors)]
-        t_c, t_d, packed, meta = run_set(torch, daf, wl, w, xs, args.steps)
-        print(row(w.name, w.numel, w.nbytes, packed, meta, t_c, t_d), flush=True)
+        t_c, t_d, packed, meta, each = run_set(torch, daf, wl, w, xs, args.steps)
+        print(row(w.name, w.numel, w.nbytes, packed, meta, t_c, t_d, each), flush=True)
         if cfg == 5 and args.sweep:
             for G in wl.SWEEP_GROUPS:
                 for beta in wl.SWEEP_BUDGETS:
                     ws = wl.workload(5, numel=kw["numel"], group_size=G, bit_budget=beta)
-                    t_c, t_d, packed, meta = run_set(torch, daf, wl, ws, xs, args.steps)
-                    print(row(ws.name, ws.numel, ws.nbytes, packed, meta, t_c, t_d), flush=True)
+                    t_c, t_d, packed, meta, each = run_set(torch, daf, wl, ws, xs, args.steps)
+                    print(row(ws.name, ws.numel, ws.nbytes, packed, meta, t_c, t_d, each), flush=True)
         del xs
         torch.cuda.empty_cache()
 
