@@ -623,6 +623,13 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 kmax = max(kmax, __float_as_uint(__fmul_rn(Rg, vh)));
             }
         }
+        // 1/scale for the width all groups would share: the divisions overlap the reductions below
+        float inv_ell[2];
+        {
+            const float Lf = (float)((1u << a.S[bud.ell]) - 1u);
+#pragma unroll
+            for (int q = 0; q < 2; q++) inv_ell[q] = R[q] > 0.0f ? __fdiv_rn(Lf, R[q]) : 0.0f;
+        }
         bool same = bud.all_max || bud.need_sep;
         if (bud.need_sep && bud.ell > 0) {
             kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
@@ -632,12 +639,11 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         if (lane == 0) s_slow[(iter & 1u) ^ 1u] = 0u;             // reset the flag of the next window
         if (same) {
             const uint32_t b = a.S[bud.ell], size = (G >> 3) * b;
-            const float Lf = (float)((1u << b) - 1u);
 #pragma unroll
             for (int q = 0; q < 2; q++) {
                 const uint32_t g = (uint32_t)lane + 32u * q;
                 if (g < n) {
-                    const float inv = R[q] > 0.0f ? __fdiv_rn(Lf, R[q]) : 0.0f;
+                    const float inv = inv_ell[q];
                     // 1/scale not a normal number: codes may need the clamp, take the careful quantizer
                     if (R[q] > 0.0f && inv < 0x1p-126f) s_slow[iter & 1u] = 1u;
                     GroupRec rec;
