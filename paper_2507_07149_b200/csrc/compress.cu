@@ -496,8 +496,9 @@ struct Budget {
     bool need_sep;         // the best raise of level ell does not fit: uniform iff the levels separate
 };
 
-// WIDTHS: at most 64 groups per window (groups of 256 elements or more), the widths warp settles
-// uniform windows; otherwise the compute warps that own group records do.
+// WIDTHS: at most 64 groups per window (groups of 256 elements or more at the default window): the
+// widths warp settles every window, of one width or mixed; otherwise the compute warps that own
+// group records do (mixed windows: radix select on the keys).
 // FULL: the complete kernel.  The quick kernel (FULL = false) is the same code without the
 // general bit choice and the clamped per-group quantizer, whose presence costs the common path
 // registers; when it meets a window that needs either, it raises hdr->retry, stops the hand-out
