@@ -110,6 +110,19 @@ daf_status daf_compress(const daf_params *params, const void *d_in, void *d_pack
                         uint64_t *d_window_offsets, void *d_workspace, uint64_t workspace_bytes,
                         daf_stream stream);
 
+/* Fused producer (Sec. 3.2.3, kernel fusion: the statistics are taken where the activation is
+ * produced, so it crosses HBM once).  Computes act = max(x, +0) element-wise (ReLU; -0 and
+ * negative values give +0), writes it to d_act in the input's type, and compresses act exactly
+ * as daf_compress would: every other output is that of daf_compress(params, d_act, ...).
+ * d_act (device, numel elements, 32-byte aligned) may be d_in itself.  Default window only
+ * (window_elems 0 or 16384; DAF_ERR_UNSUPPORTED otherwise); other arguments, ownership and
+ * errors as for daf_compress.
+ */
+daf_status daf_relu_compress(const daf_params *params, const void *d_in, void *d_act, void *d_packed,
+                             uint64_t packed_capacity, uint8_t *d_bits, float *d_min, float *d_scale,
+                             uint64_t *d_window_offsets, void *d_workspace, uint64_t workspace_bytes,
+                             daf_stream stream);
+
 /*
  * Decompress (Sec. 2.3: stored activations are dequantized to their original precision
  * for the gradient computation): x_hat = fma(code, scale, min), rounded to nearest even

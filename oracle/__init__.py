@@ -103,6 +103,14 @@ def widen(a: np.ndarray, dtype: str | None = None) -> np.ndarray:
 
 
 # ---------------------------------------------------------------- stage functions
+def relu(a: np.ndarray, dtype: str | None = None) -> np.ndarray:
+    """The producer that can be fused in front of the compression (Sec. 3.2.3): x where x > 0, else +0,
+    in the array's own type (bf16 arrays are uint16 bit patterns: negative = sign bit set)."""
+    if dtype == "bf16" or a.dtype == np.uint16:
+        return np.where((a & 0x8000) != 0, np.uint16(0), a).astype(np.uint16)
+    return np.where(a > 0, a, a.dtype.type(0)).astype(a.dtype)
+
+
 def stats(x, G: int):
     x = _c(x, np.float32).reshape(-1)
     ng = x.size // G

@@ -50,6 +50,8 @@ SIGNATURES = {
     "daf_sizes": (ctypes.c_int, [ctypes.POINTER(daf_params), _u64p, _u64p, _u64p, _u64p]),
     "daf_compress": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, ctypes.c_uint64, _vp, _vp, _vp, _vp, _vp,
                                     ctypes.c_uint64, _vp]),
+    "daf_relu_compress": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, _vp, ctypes.c_uint64, _vp, _vp, _vp, _vp, _vp,
+                                         ctypes.c_uint64, _vp]),
     "daf_compress_static": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, ctypes.c_uint64, _vp, _vp, _vp, _vp, _vp, _vp]),
     "daf_decompress": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_uint64, _vp]),
     "daf_group_offsets": (ctypes.c_int, [_vp, ctypes.c_uint64, ctypes.c_uint32, _vp, _vp, ctypes.c_uint64, _vp]),
@@ -145,6 +147,15 @@ def daf_compress(params, d_in, d_packed, packed_capacity, d_bits, d_min, d_scale
     _check(lib().daf_compress(ctypes.byref(params), _ptr(d_in), _ptr(d_packed), packed_capacity, _ptr(d_bits), _ptr(d_min),
                               _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_workspace), workspace_bytes, _stream(stream)),
            "daf_compress")
+
+
+def daf_relu_compress(params, d_in, d_act, d_packed, packed_capacity, d_bits, d_min, d_scale, d_window_offsets, d_workspace,
+                      workspace_bytes, stream=None):
+    """Fused producer: d_act = max(d_in, +0) is written and compressed in one pass (d_act may be d_in)."""
+    _check(lib().daf_relu_compress(ctypes.byref(params), _ptr(d_in), _ptr(d_act), _ptr(d_packed), packed_capacity, _ptr(d_bits),
+                                   _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_workspace), workspace_bytes,
+                                   _stream(stream)),
+           "daf_relu_compress")
 
 
 STATIC_MAX_WINDOWS = 65536
@@ -261,6 +272,24 @@ def compress(x, group_size: int, widths, bit_budget: float, *, window_elems: int
     if check:
         _check(daf_poll_status(c.workspace, stream), "daf_compress (device status)")
     return c
+
+
+def relu_compress(x, group_size: int, widths, bit_budget: float, *, rounding: int = ROUND_STOCHASTIC, seed: int = 0,
+                  elem_index_base: int = 0, inplace: bool = False, out: CompressedTensor | None = None, check: bool = False,
+                  stream=None):
+    """(relu(x), compressed relu(x)) in one pass over x (daf_relu_compress); ``inplace`` overwrites x."""
+    if not x.is_cuda or not x.is_contiguous():
+        raise ValueError("relu_compress expects a contiguous CUDA tensor")
+    params = make_params(dtype_code(x), x.numel(), group_size, widths, bit_budget, rounding=rounding, seed=seed,
+                         elem_index_base=elem_index_base)
+    c = out if out is not None else alloc_outputs(params, x.device, x.shape)
+    c.params = params
+    act = x if inplace else _torch().empty_like(x)
+    daf_relu_compress(params, x, act, c.packed, c.sizes.packed_capacity, c.bits, c.min, c.scale, c.window_offsets,
+                      c.workspace, c.sizes.workspace, stream)
+    if check:
+        _check(daf_poll_status(c.workspace, stream), "daf_relu_compress (device status)")
+    return act, c
 
 
 def decompress(c: CompressedTensor, out=None, stream=None):

@@ -45,6 +45,7 @@ struct TensorDesc {
     uint64_t seed;
     uint32_t first_window;   // index of this tensor's window 0 among all windows of the launch
     uint32_t n_windows;
+    void *act;               // fused producer (daf_relu_compress): where the activation itself goes
 };
 
 struct SmemLayout {          // byte offsets into dynamic shared memory
@@ -306,13 +307,19 @@ template <> __device__ __forceinline__ void load8_staged<__nv_bfloat16>(const un
 // Staged window -> registers, then min / max per unit of LPU lanes (a full warp uses the
 // redux instruction) written to shared memory.  Chunks past a ragged window's end read
 // stale bytes; their results are never used.
-template <typename T, int CHUNKS, int LPU>
+template <typename T, int CHUNKS, int LPU, bool RELU>
 __device__ __forceinline__ void load_and_reduce(const unsigned char *stage, int warp, int lane, float (&x)[CHUNKS][8],
                                                 float *s_umn, float *s_umx)
 {
     constexpr int kChunkBytes = 256 * Elem<T>::kBytes;
 #pragma unroll
     for (int c = 0; c < CHUNKS; c++) load8_staged<T>(stage + (warp * CHUNKS + c) * kChunkBytes, lane, x[c]);
+    if (RELU) {                                                   // fused producer: what is compressed is max(x, +0)
+#pragma unroll
+        for (int c = 0; c < CHUNKS; c++)
+#pragma unroll
+            for (int i = 0; i < 8; i++) x[c][i] = fmaxf(x[c][i], 0.0f);
+    }
 #pragma unroll
     for (int c = 0; c < CHUNKS; c++) {
         float lo = fmin3(fmin3(x[c][0], x[c][1], x[c][2]), fmin3(x[c][3], x[c][4], x[c][5]), fmin2(x[c][6], x[c][7]));
@@ -345,12 +352,13 @@ template <int NT> __device__ __forceinline__ uint32_t find_tensor(const Compress
     return lo;
 }
 
-// The CTA is 16 compute warps plus one control warp; two CTAs share an SM and cover each
-// other's waits.  Hardware barrier 1 ("stage", owner warps and control warp wait, the rest
-// only arrive): the compute warps have moved the staged window into registers, published its
-// per-unit min / max, and finished the previous window's packed bytes.  Barrier 2 ("widths",
-// compute warps): the owners' verdict on the window is in.  Barrier 3 is private to the warps
-// that own group records; barrier 4 separates the steps of the general bit choice.
+// The CTA is 16 compute warps, one control warp and one widths warp; two CTAs share an SM and
+// cover each other's waits.  Hardware barrier 1 ("stage"; the control warp, the widths warp
+// when it is in charge, else the owner warps wait, the rest only arrive): the compute warps have
+// moved the staged window into registers, published its per-unit min / max, and finished the
+// previous window's packed bytes.  Barrier 2 ("widths", compute warps wait): the verdict on the
+// window's widths and the group records are in.  Barrier 3 is private to the warps that own
+// group records (more than 64 groups per window); barrier 4 ends their general bit choice.
 constexpr int kComputeWarps = kWarps;
 constexpr int kCompressThreads = kThreads + 64;
 constexpr uint32_t kBarStage = 1, kBarWidths = 2, kBarOwners = 3, kBarChoice = 4;
@@ -504,7 +512,7 @@ struct Budget {
 // registers; when it meets a window that needs either, it raises hdr->retry, stops the hand-out
 // of windows and leaves, and the full kernel, enqueued behind it, redoes the call.  Otherwise
 // the full kernel finds hdr->retry clear and returns at once.
-template <typename T, int CHUNKS, bool BATCH, bool WIDTHS, bool FULL>
+template <typename T, int CHUNKS, bool BATCH, bool WIDTHS, bool FULL, bool RELU>
 __global__ void __launch_bounds__(kCompressThreads, 2)
 compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> a)
 {
@@ -901,10 +909,20 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
 
         // ---------------------------------------------------------------- staged window -> registers, unit min / max
         float x[CHUNKS][8];
-        if (G >= 256u) load_and_reduce<T, CHUNKS, 32>(s_stage, warp, lane, x, umn, umx);
-        else if (G == 128u) load_and_reduce<T, CHUNKS, 16>(s_stage, warp, lane, x, umn, umx);
-        else if (G == 64u) load_and_reduce<T, CHUNKS, 8>(s_stage, warp, lane, x, umn, umx);
-        else load_and_reduce<T, CHUNKS, 4>(s_stage, warp, lane, x, umn, umx);
+        if (G >= 256u) load_and_reduce<T, CHUNKS, 32, RELU>(s_stage, warp, lane, x, umn, umx);
+        else if (G == 128u) load_and_reduce<T, CHUNKS, 16, RELU>(s_stage, warp, lane, x, umn, umx);
+        else if (G == 64u) load_and_reduce<T, CHUNKS, 8, RELU>(s_stage, warp, lane, x, umn, umx);
+        else load_and_reduce<T, CHUNKS, 4, RELU>(s_stage, warp, lane, x, umn, umx);
+        if (RELU && !lost) {
+            // the activation goes out as it is compressed: one 8-element store per lane and chunk (the
+            // window was staged whole before, so the output may be the input buffer)
+            char *const act = reinterpret_cast<char *>(td.act) + wbase * Elem<T>::kBytes;
+#pragma unroll
+            for (int c = 0; c < CHUNKS; c++) {
+                const uint32_t e = e0 + 256u * c;
+                if (e < n_elems) Elem<T>::store8(act + (size_t)e * Elem<T>::kBytes, x[c]);
+            }
+        }
         // ---------------------------------------------------------------- widths, first try: one width for all
         // The warps that own group records (thread g: group g) test whether every group ends at
         // level ell: every raise below level ell must sort ahead of every raise from level ell
@@ -1283,7 +1301,7 @@ static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint
     return l;
 }
 
-template <typename T, int CHUNKS, bool BATCH, bool WIDTHS, bool FULL>
+template <typename T, int CHUNKS, bool BATCH, bool WIDTHS, bool FULL, bool RELU = false>
 static cudaError_t launch(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
     static int sms = 0, smem_set = 0, cached_smem = -1, cached_ctas = 0;   // per instantiation, current device
@@ -1296,37 +1314,49 @@ static cudaError_t launch(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, c
         if (e != cudaSuccess) return e;
     }
     if (smem > smem_set) {
-        e = cudaFuncSetAttribute(compress_kernel<T, CHUNKS, BATCH, WIDTHS, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        e = cudaFuncSetAttribute(compress_kernel<T, CHUNKS, BATCH, WIDTHS, FULL, RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         smem_set = smem;
     }
     if (smem != cached_smem) {
         int per_sm = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel<T, CHUNKS, BATCH, WIDTHS, FULL>, kCompressThreads, smem);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel<T, CHUNKS, BATCH, WIDTHS, FULL, RELU>, kCompressThreads, smem);
         if (e != cudaSuccess) return e;
         cached_smem = smem;
         cached_ctas = sms * (per_sm > 0 ? per_sm : 1);
     }
     const uint32_t grid = args.total_windows < (uint32_t)cached_ctas ? args.total_windows : (uint32_t)cached_ctas;
-    compress_kernel<T, CHUNKS, BATCH, WIDTHS, FULL><<<grid, kCompressThreads, smem, stream>>>(args);
+    compress_kernel<T, CHUNKS, BATCH, WIDTHS, FULL, RELU><<<grid, kCompressThreads, smem, stream>>>(args);
     return cudaGetLastError();
 }
 
-template <bool BATCH, bool FULL>
+template <bool BATCH, bool FULL, bool RELU>
 static cudaError_t dispatch_one(uint32_t dtype, uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
                                 cudaStream_t stream)
 {
+    const bool widths = args.n_max <= 64u;                        // few enough groups for the widths warp
+    if constexpr (RELU) {                                         // fused producer: single tensor, default window (chunks == 4)
+        static_assert(!BATCH, "the fused producer is compiled for single-tensor launches only");
+        if (dtype == DAF_F32)
+            return widths ? launch<float, 4, false, true, FULL, true>(args, stream)
+                          : launch<float, 4, false, false, FULL, true>(args, stream);
+        if (dtype == DAF_F16)
+            return widths ? launch<__half, 4, false, true, FULL, true>(args, stream)
+                          : launch<__half, 4, false, false, FULL, true>(args, stream);
+        return widths ? launch<__nv_bfloat16, 4, false, true, FULL, true>(args, stream)
+                      : launch<__nv_bfloat16, 4, false, false, FULL, true>(args, stream);
+    } else {
 #define DAF_CASE(T)                                                                     \
     switch (chunks) {                                                                   \
     case 1: return widths ? launch<T, 1, BATCH, true, FULL>(args, stream) : launch<T, 1, BATCH, false, FULL>(args, stream);   \
     case 2: return widths ? launch<T, 2, BATCH, true, FULL>(args, stream) : launch<T, 2, BATCH, false, FULL>(args, stream);   \
     default: return widths ? launch<T, 4, BATCH, true, FULL>(args, stream) : launch<T, 4, BATCH, false, FULL>(args, stream);  \
     }
-    const bool widths = args.n_max <= 64u;                        // few enough groups for the widths warp
     if (dtype == DAF_F32) { DAF_CASE(float) }
     if (dtype == DAF_F16) { DAF_CASE(__half) }
     DAF_CASE(__nv_bfloat16)
 #undef DAF_CASE
+    }
 }
 
 // One call = the quick kernel followed by the full kernel, which returns at once unless the
@@ -1340,7 +1370,7 @@ static uint32_t quick_min_windows()
     return e && *e ? (uint32_t)std::strtoul(e, nullptr, 10) : kQuickMinWindows;
 }
 
-template <bool BATCH>
+template <bool BATCH, bool RELU = false>
 static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
                             cudaStream_t stream)
 {
@@ -1352,10 +1382,10 @@ static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, CompressArgs<BATCH 
     args.flags2 = args.flags + args.total_windows;
     args.gated = try_quick ? 1u : 0u;
     if (try_quick) {
-        const cudaError_t e = dispatch_one<BATCH, false>(dtype, chunks, args, stream);
+        const cudaError_t e = dispatch_one<BATCH, false, RELU>(dtype, chunks, args, stream);
         if (e != cudaSuccess) return e;
     }
-    return dispatch_one<BATCH, true>(dtype, chunks, args, stream);
+    return dispatch_one<BATCH, true, RELU>(dtype, chunks, args, stream);
 }
 
 template <int NT> static void fill_common(CompressArgs<NT> &a, const Plan &pl, const daf_params *p, void *ws)
@@ -1417,6 +1447,36 @@ extern "C" daf_status daf_compress(const daf_params *params, const void *d_in, v
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(d_workspace, 0, pl.workspace, s) != cudaSuccess) return DAF_ERR_CUDA;
     return dispatch<false>(params->dtype, pl.chunks, a, s) == cudaSuccess ? DAF_OK : DAF_ERR_CUDA;
+}
+
+extern "C" daf_status daf_relu_compress(const daf_params *params, const void *d_in, void *d_act, void *d_packed,
+                                        uint64_t packed_capacity, uint8_t *d_bits, float *d_min, float *d_scale,
+                                        uint64_t *d_window_offsets, void *d_workspace, uint64_t workspace_bytes,
+                                        daf_stream stream)
+{
+    Plan pl;
+    daf_status st = make_plan(params, &pl);
+    if (st != DAF_OK) return st;
+    if (!d_in || !d_act || !d_packed || !d_bits || !d_min || !d_scale || !d_window_offsets || !d_workspace)
+        return DAF_ERR_INVALID_ARG;
+    if (!aligned16(d_in) || !aligned16(d_packed) || !aligned16(d_workspace) || (reinterpret_cast<uintptr_t>(d_act) & 31u) ||
+        (reinterpret_cast<uintptr_t>(d_min) & 3u) || (reinterpret_cast<uintptr_t>(d_scale) & 3u) ||
+        (reinterpret_cast<uintptr_t>(d_window_offsets) & 7u))
+        return DAF_ERR_INVALID_ARG;
+    if (workspace_bytes < pl.workspace) return DAF_ERR_CAPACITY;
+    if (pl.n_windows > 0xFFFFFFF0ull || pl.chunks != 4) return DAF_ERR_UNSUPPORTED;   // default window only
+
+    CompressArgs<1> a;
+    fill_common(a, pl, params, d_workspace);
+    a.total_windows = (uint32_t)pl.n_windows;
+    a.n_tensors = 1;
+    a.keys = philox_keys(params->seed);
+    a.t[0] = TensorDesc{d_in, reinterpret_cast<uint8_t *>(d_packed), packed_capacity, d_bits, d_min, d_scale,
+                        d_window_offsets, params->numel, params->elem_index_base, params->seed, 0u,
+                        (uint32_t)pl.n_windows, d_act};
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(d_workspace, 0, pl.workspace, s) != cudaSuccess) return DAF_ERR_CUDA;
+    return dispatch<false, true>(params->dtype, pl.chunks, a, s) == cudaSuccess ? DAF_OK : DAF_ERR_CUDA;
 }
 
 // ------------------------------------------------------------------------------------------

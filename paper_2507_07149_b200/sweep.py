@@ -1,6 +1,6 @@
 """Times compress / decompress on the five benchmark workloads and the group-size x budget sweep.
 
-    python -m paper_2507_07149_b200.sweep [--configs 1,2,3,4,5] [--sweep] [--steps K] [--scale S]
+    python -m paper_2507_07149_b200.sweep [--configs 1,2,3,4,5] [--sweep] [--relu] [--steps K] [--scale S]
 
 Workloads 1-4 are sets of tensors: each set goes through ONE batched call (daf_compress_batch /
 daf_decompress_batch) when it has at most DAF_BATCH_MAX tensors.  Inputs are the seeded synthetic
@@ -120,6 +120,8 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="also the 16 (group size, budget) points of workload 5")
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--scale", type=int, default=1)
+    ap.add_argument("--relu", action="store_true",
+                    help="also the fused producer on workload 5: daf_relu_compress against torch.relu followed by daf_compress")
     args = ap.parse_args()
 
     import torch
@@ -147,6 +149,29 @@ def main():
                     ws = wl.workload(5, numel=kw["numel"], group_size=G, bit_budget=beta)
                     t_c, t_d, packed, meta, each = run_set(torch, daf, wl, ws, xs, args.steps)
                     print(row(ws.name, ws.numel, ws.nbytes, packed, meta, t_c, t_d, each), flush=True)
+        if cfg == 5 and args.relu:
+            x = xs[0]
+            p = daf.make_params(daf.dtype_code(x), x.numel(), w.group_size, w.widths, w.bit_budget, seed=0)
+            c = daf.alloc_outputs(p, x.device)
+            act = torch.empty_like(x)
+
+            def fused():
+                daf.daf_relu_compress(p, x, act, c.packed, c.sizes.packed_capacity, c.bits, c.min, c.scale,
+                                      c.window_offsets, c.workspace, c.sizes.workspace)
+
+            def separate():
+                torch.clamp_min(x, 0, out=act)                    # relu into a preallocated tensor
+                daf.daf_compress(p, act, c.packed, c.sizes.packed_capacity, c.bits, c.min, c.scale, c.window_offsets,
+                                 c.workspace, c.sizes.workspace)
+
+            t_f = _time(torch, fused, args.steps, False)
+            assert daf.daf_poll_status(c.workspace) == daf.OK
+            packed = c.packed_bytes()
+            t_s = _time(torch, separate, args.steps, False)
+            alg = 2 * w.nbytes + packed + 9 * (x.numel() // w.group_size) + 8 * (c.sizes.n_windows + 1)
+            print(f"| {w.name} relu + compress, fused | {w.numel} | {w.nbytes / 2**30:.3f} | {packed / 2**30:.3f} | "
+                  f"{t_f:.4f} | {alg / t_f / 1e6:.0f} | — | — | torch.relu + daf_compress: {t_s:.4f} | — |", flush=True)
+            del act, c
         del xs
         torch.cuda.empty_cache()
 

@@ -1,0 +1,84 @@
+"""GPU: the fused producer daf_relu_compress (Sec. 3.2.3, kernel fusion) against the oracle --
+the activation written out is relu(x) bit for bit, everything else is the compression of it."""
+import numpy as np
+import pytest
+
+import oracle
+import paper_2507_07149_b200 as daf
+from paper_2507_07149_b200 import workloads as wl
+
+from gpu_util import to_device, to_host
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+
+def _input(rng, n, G, dtype, mixed):
+    a = rng.standard_normal(n).astype(np.float32)
+    if mixed:                                                     # a stretch of groups with very different ranges
+        k = n // G
+        s = np.ones(k, np.float32)
+        s[k // 3: 2 * k // 3] = (10.0 ** rng.uniform(-2, 2, 2 * k // 3 - k // 3)).astype(np.float32)
+        a *= np.repeat(s, G)
+    a[::7] = -0.0                                                 # negative zeros must come out as +0
+    if dtype == "f32":
+        return a
+    return a.astype(np.float16) if dtype == "f16" else wl.f32_to_bf16_bits(a)
+
+
+def _check(a, dtype, G, beta, inplace, seed=3):
+    x = to_device(a, dtype)
+    x0 = x.clone()
+    act, c = daf.relu_compress(x, G, (1, 2, 4, 8), beta, seed=seed, inplace=inplace, check=True)
+    y = daf.decompress(c)
+    torch.cuda.synchronize()
+    want_act = oracle.relu(a, dtype)
+    got_act = to_host(act, dtype)
+    assert np.array_equal(got_act.view(np.uint32 if dtype == "f32" else np.uint16),
+                          want_act.view(np.uint32 if dtype == "f32" else np.uint16))
+    if inplace:
+        assert act.data_ptr() == x.data_ptr()
+    else:
+        assert torch.equal(x.view(torch.int16 if dtype != "f32" else torch.int32),
+                           x0.view(torch.int16 if dtype != "f32" else torch.int32))      # the input is left alone
+    ref = oracle.compress(want_act, G, (1, 2, 4, 8), beta, dtype="bf16" if dtype == "bf16" else None, seed=seed)
+    assert np.array_equal(c.bits.cpu().numpy(), ref.bits)
+    assert np.array_equal(c.window_offsets.cpu().numpy().view(np.uint64), ref.window_offsets)
+    assert np.array_equal(c.min.cpu().numpy().view(np.uint32), ref.mn.view(np.uint32))
+    assert np.array_equal(c.scale.cpu().numpy().view(np.uint32), ref.scale.view(np.uint32))
+    assert np.array_equal(c.packed[: ref.packed.size].cpu().numpy(), ref.packed)
+    want = oracle.decompress(ref)
+    got = to_host(y.reshape(-1), dtype)
+    if dtype == "f32":
+        d = np.abs(got.view(np.int32).astype(np.int64) - want.view(np.int32).astype(np.int64))
+        assert d.max() <= 1
+    else:
+        assert np.array_equal(got.view(np.uint16), want.view(np.uint16))
+    return ref
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+@pytest.mark.parametrize("G,beta,mixed", [(256, 4.0, False), (256, 3.0, False), (256, 4.0, True), (64, 2.0, True), (1024, 8.0, False)])
+def test_relu_compress_matches_relu_then_compress(dtype, G, beta, mixed):
+    rng = np.random.default_rng(G + int(beta * 10) + mixed)
+    n = 16384 * 37 + G * 5                                        # several windows per CTA wave is not needed: ragged end
+    ref = _check(_input(rng, n, G, dtype, mixed), dtype, G, beta, inplace=False)
+    if mixed or beta == 3.0:
+        assert len(np.unique(ref.bits)) >= 2
+
+
+@pytest.mark.parametrize("mixed", [False, True])
+def test_relu_compress_in_place(mixed):
+    rng = np.random.default_rng(17 + mixed)
+    n = 16384 * 700 + 256 * 9                                     # more windows than CTAs: every CTA stages several windows
+    _check(_input(rng, n, 256, "f32", mixed), "f32", 256, 4.0, inplace=True)
+
+
+def test_relu_compress_rejects_other_windows():
+    x = torch.zeros(1 << 16, device="cuda")
+    p = daf.make_params(daf.F32, x.numel(), 256, (1, 2, 4, 8), 4.0, window_elems=4096)
+    c = daf.alloc_outputs(p, "cuda")
+    with pytest.raises(daf.DafError) as e:
+        daf.daf_relu_compress(p, x, x, c.packed, c.sizes.packed_capacity, c.bits, c.min, c.scale, c.window_offsets,
+                              c.workspace, c.sizes.workspace)
+    assert e.value.status == daf.ERR_UNSUPPORTED

@@ -477,3 +477,13 @@ def test_compress_argument_checks():
         oracle.compress(x, 64, [4], 4.0)           # numel not a multiple of the group size
     with pytest.raises(oracle.OracleError):
         oracle.compress(x, 32, [4], 3.0)           # budget below the smallest width
+
+
+def test_relu_by_hand():
+    """The producer fused in front of the compression (Sec. 3.2.3): negatives and -0 give +0."""
+    a = np.array([-1.5, -0.0, 0.0, 2.5, -1e-30, 1e-30], np.float32)
+    want = np.array([0.0, 0.0, 0.0, 2.5, 0.0, 1e-30], np.float32)
+    assert np.array_equal(oracle.relu(a).view(np.uint32), want.view(np.uint32))
+    assert np.array_equal(oracle.relu(a.astype(np.float16)).view(np.uint16), want.astype(np.float16).view(np.uint16))
+    b = np.array([0xBFC0, 0x8000, 0x0000, 0x4020, 0x8001], np.uint16)          # bf16 -1.5, -0, +0, 2.5, a negative subnormal
+    assert np.array_equal(oracle.relu(b, "bf16"), np.array([0, 0, 0, 0x4020, 0], np.uint16))
