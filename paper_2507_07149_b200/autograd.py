@@ -81,3 +81,47 @@ class saved_activation_compression(torch.autograd.graph.saved_tensors_hooks):
         if not isinstance(s, _Saved):
             return s
         return decompress(s.c).view(s.shape)
+
+
+class _ReluSavedCompressed(torch.autograd.Function):
+    """ReLU whose output is written and compressed in one pass (daf_relu_compress); the backward pass
+    restores the saved output from the packed form and masks the gradient with it."""
+
+    @staticmethod
+    def forward(ctx, x, module):
+        from . import relu_compress
+        act, c = relu_compress(x.contiguous(), module.group_size, module.widths, module.bit_budget, rounding=module.rounding,
+                               seed=module.seed, elem_index_base=module._next_index, check=module.trim)
+        module._next_index += (x.numel() + 7) & ~7
+        if module.trim:
+            c.packed = c.packed[:max(c.packed_bytes(), 16)].clone()
+            c.workspace = None
+        ctx.saved = c
+        ctx.shape = x.shape
+        return act.view(x.shape)
+
+    @staticmethod
+    def backward(ctx, grad_out):
+        y = decompress(ctx.saved).view(ctx.shape)
+        return grad_out * (y > 0).to(grad_out.dtype), None
+
+
+class CompressedReLU(torch.nn.Module):
+    """ReLU layer that keeps its output for the backward pass in compressed form only, produced by the
+    fused kernel (the activation crosses device memory once: read x, write relu(x) and its packed form).
+    Inputs that do not qualify (see ``saved_activation_compression``) go through ``torch.relu``."""
+
+    def __init__(self, group_size: int = 256, widths=(1, 2, 4, 8), bit_budget: float = 4.0, *, seed: int = 0,
+                 rounding: int = ROUND_STOCHASTIC, min_numel: int = 16384, trim: bool = True):
+        super().__init__()
+        self.group_size, self.widths, self.bit_budget = int(group_size), tuple(widths), float(bit_budget)
+        self.seed, self.rounding, self.min_numel, self.trim = int(seed), int(rounding), int(min_numel), bool(trim)
+        self._next_index = 0
+
+    def reseed(self, seed: int) -> None:
+        self.seed, self._next_index = int(seed), 0
+
+    def forward(self, x):
+        ok = (x.is_cuda and x.dtype in _DTYPES and x.numel() >= self.min_numel and x.numel() % self.group_size == 0
+              and torch.is_grad_enabled() and x.requires_grad)
+        return _ReluSavedCompressed.apply(x, self) if ok else torch.relu(x)

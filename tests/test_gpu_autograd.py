@@ -112,3 +112,28 @@ def test_small_cnn_trains_on_compressed_activations():
     assert np.mean(base[-5:]) < 0.3 * base[0]
     assert np.mean(comp[-5:]) < 0.3 * comp[0]                  # trains as well, within noise
     assert abs(np.mean(comp[-5:]) - np.mean(base[-5:])) < 0.25 * base[0]
+
+
+def test_compressed_relu_layer_masks_with_the_restored_output():
+    """CompressedReLU: forward = relu(x) exactly; backward = grad * (restored output > 0), the restored
+    output being what the oracle decodes from the compression of relu(x)."""
+    from paper_2507_07149_b200.autograd import CompressedReLU
+    daf.lib()
+    rng = np.random.default_rng(23)
+    n, G, beta, seed = 16384 * 9 + 512, 256, 2.0, 41
+    a = rng.standard_normal(n).astype(np.float32)
+    gw = rng.standard_normal(n).astype(np.float32)
+    x = torch.from_numpy(a).cuda().requires_grad_(True)
+    layer = CompressedReLU(group_size=G, bit_budget=beta, seed=seed, min_numel=1024)
+    y = layer(x)
+    assert np.array_equal(y.detach().cpu().numpy().view(np.uint32), oracle.relu(a).view(np.uint32))
+    (y * torch.from_numpy(gw).cuda()).sum().backward()
+    ref = oracle.compress(oracle.relu(a), G, (1, 2, 4, 8), beta, seed=seed)
+    restored = oracle.decompress(ref)
+    want = gw * (restored > 0)
+    assert np.array_equal(x.grad.cpu().numpy(), want.astype(np.float32))
+    assert 0 < int((restored > 0).sum()) < int((a > 0).sum())     # at 2 bits some small positives are restored as 0
+    # a small or ragged input takes the plain path
+    small = torch.randn(100, device="cuda", requires_grad=True)
+    layer(small).sum().backward()
+    assert torch.equal(small.grad, (small.detach() > 0).float())
