@@ -127,12 +127,23 @@ daf_status daf_relu_compress(const daf_params *params, const void *d_in, void *d
  * Decompress (Sec. 2.3: stored activations are dequantized to their original precision
  * for the gradient computation): x_hat = fma(code, scale, min), rounded to nearest even
  * into params->dtype.  Inputs are the outputs of daf_compress for the same params;
- * d_out receives numel elements.  The workspace is not used by this version and may be NULL.
+ * d_out receives numel elements; it must be 32-byte aligned for DAF_F32 (a lane stores eight
+ * elements at once), 16-byte aligned otherwise.  The workspace is not used by this version and may be NULL.
  */
 daf_status daf_decompress(const daf_params *params, const void *d_packed, const uint8_t *d_bits,
                           const float *d_min, const float *d_scale,
                           const uint64_t *d_window_offsets, void *d_out, void *d_workspace,
                           uint64_t workspace_bytes, daf_stream stream);
+
+/* Fused consumer (Sec. 3.2.3): the backward pass of a ReLU whose output was stored compressed.
+ * d_grad_in[i] = d_grad_out[i] where the restored activation (exactly what daf_decompress would
+ * store, in params->dtype) is > 0, else +0; the restored activation itself is never written.
+ * d_grad_out, d_grad_in: device, numel elements of params->dtype, aligned like d_out of
+ * daf_decompress; they may be the same buffer.  Other arguments and errors as for daf_decompress.
+ */
+daf_status daf_decompress_relu_grad(const daf_params *params, const void *d_packed, const uint8_t *d_bits,
+                                    const float *d_min, const float *d_scale, const uint64_t *d_window_offsets,
+                                    const void *d_grad_out, void *d_grad_in, daf_stream stream);
 
 /*
  * Device-wide exclusive prefix sum of the group byte lengths G*b_g/8 ("layout

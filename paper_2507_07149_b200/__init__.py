@@ -54,6 +54,7 @@ SIGNATURES = {
                                          ctypes.c_uint64, _vp]),
     "daf_compress_static": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, ctypes.c_uint64, _vp, _vp, _vp, _vp, _vp, _vp]),
     "daf_decompress": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_uint64, _vp]),
+    "daf_decompress_relu_grad": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "daf_group_offsets": (ctypes.c_int, [_vp, ctypes.c_uint64, ctypes.c_uint32, _vp, _vp, ctypes.c_uint64, _vp]),
     "daf_group_offsets_workspace": (ctypes.c_uint64, [ctypes.c_uint64]),
     "daf_poll_status": (ctypes.c_int, [_vp, _vp]),
@@ -169,6 +170,13 @@ def daf_compress_static(params, d_in, d_packed, packed_capacity, d_bits, d_min, 
     _check(lib().daf_compress_static(ctypes.byref(params), _ptr(d_in), _ptr(d_packed), packed_capacity, _ptr(d_bits),
                                      _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_status), _stream(stream)),
            "daf_compress_static")
+
+
+def daf_decompress_relu_grad(params, d_packed, d_bits, d_min, d_scale, d_window_offsets, d_grad_out, d_grad_in, stream=None):
+    """Fused consumer: d_grad_in = d_grad_out where the restored activation is > 0, else 0 (may be in place)."""
+    _check(lib().daf_decompress_relu_grad(ctypes.byref(params), _ptr(d_packed), _ptr(d_bits), _ptr(d_min), _ptr(d_scale),
+                                          _ptr(d_window_offsets), _ptr(d_grad_out), _ptr(d_grad_in), _stream(stream)),
+           "daf_decompress_relu_grad")
 
 
 def daf_decompress(params, d_packed, d_bits, d_min, d_scale, d_window_offsets, d_out, d_workspace=None,
@@ -298,6 +306,17 @@ def decompress(c: CompressedTensor, out=None, stream=None):
     if out is None:
         out = torch.empty(c.shape, dtype=dt, device=c.packed.device)
     daf_decompress(c.params, c.packed, c.bits, c.min, c.scale, c.window_offsets, out, None, 0, stream)
+    return out
+
+
+def relu_grad(c: CompressedTensor, grad_out, out=None, stream=None):
+    """Gradient of a ReLU from its compressed output: grad_out where the restored output is > 0."""
+    torch = _torch()
+    if not grad_out.is_contiguous():
+        grad_out = grad_out.contiguous()
+    if out is None:
+        out = torch.empty_like(grad_out)
+    daf_decompress_relu_grad(c.params, c.packed, c.bits, c.min, c.scale, c.window_offsets, grad_out, out, stream)
     return out
 
 

@@ -85,7 +85,8 @@ class saved_activation_compression(torch.autograd.graph.saved_tensors_hooks):
 
 class _ReluSavedCompressed(torch.autograd.Function):
     """ReLU whose output is written and compressed in one pass (daf_relu_compress); the backward pass
-    restores the saved output from the packed form and masks the gradient with it."""
+    masks the gradient with the output restored from the packed form (daf_decompress_relu_grad: the
+    restored output is never written)."""
 
     @staticmethod
     def forward(ctx, x, module):
@@ -102,8 +103,12 @@ class _ReluSavedCompressed(torch.autograd.Function):
 
     @staticmethod
     def backward(ctx, grad_out):
-        y = decompress(ctx.saved).view(ctx.shape)
-        return grad_out * (y > 0).to(grad_out.dtype), None
+        from . import relu_grad
+        c = ctx.saved
+        if grad_out.dtype != {0: torch.float32, 1: torch.float16, 2: torch.bfloat16}[int(c.params.dtype)]:
+            y = decompress(c).view(ctx.shape)                     # gradient in another type: mask in torch
+            return grad_out * (y > 0).to(grad_out.dtype), None
+        return relu_grad(c, grad_out.reshape(-1)).view(ctx.shape), None   # one pass: packed + gradient in, gradient out
 
 
 class CompressedReLU(torch.nn.Module):

@@ -20,6 +20,7 @@ struct DecTensor {
     uint64_t numel;
     uint32_t first_window;
     uint32_t n_windows;
+    const void *grad;        // fused consumer (daf_decompress_relu_grad): the incoming gradient
 };
 
 template <int NT> struct DecompressArgs {
@@ -49,7 +50,15 @@ template <int B> __device__ __forceinline__ void decode8(uint32_t w0, uint32_t w
     }
 }
 
-template <typename T, int CHUNKS, bool BATCH>
+// The restored value as it would be stored in type T (round to nearest even), back in binary32.
+template <typename T> __device__ __forceinline__ float as_stored(float y);
+template <> __device__ __forceinline__ float as_stored<float>(float y) { return y; }
+template <> __device__ __forceinline__ float as_stored<__half>(float y) { return __half2float(__float2half_rn(y)); }
+template <> __device__ __forceinline__ float as_stored<__nv_bfloat16>(float y) { return __bfloat162float(__float2bfloat16_rn(y)); }
+
+// MASK: fused consumer.  Instead of the restored activation the kernel stores the gradient of a
+// ReLU that produced it: the incoming gradient where the restored value is positive, else +0.
+template <typename T, int CHUNKS, bool BATCH, bool MASK>
 __global__ void __launch_bounds__(kThreads)
 decompress_kernel(const __grid_constant__ DecompressArgs<BATCH ? DAF_BATCH_MAX : 1> a)
 {
@@ -139,26 +148,32 @@ decompress_kernel(const __grid_constant__ DecompressArgs<BATCH ? DAF_BATCH_MAX :
             break;
         }
         }
+        if (MASK) {
+            float g[8];
+            Elem<T>::load8(reinterpret_cast<const char *>(td.grad) + (wbase + e) * Elem<T>::kBytes, g);
+#pragma unroll
+            for (int i = 0; i < 8; i++) y[i] = as_stored<T>(y[i]) > 0.0f ? g[i] : 0.0f;
+        }
         Elem<T>::store8(out + (size_t)e * Elem<T>::kBytes, y);
     }
 }
 
-template <typename T, int CHUNKS, bool BATCH>
+template <typename T, int CHUNKS, bool BATCH, bool MASK>
 static cudaError_t launch(const DecompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
-    decompress_kernel<T, CHUNKS, BATCH><<<args.total_windows, kThreads, 0, stream>>>(args);
+    decompress_kernel<T, CHUNKS, BATCH, MASK><<<args.total_windows, kThreads, 0, stream>>>(args);
     return cudaGetLastError();
 }
 
-template <bool BATCH>
+template <bool BATCH, bool MASK = false>
 static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, const DecompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
                             cudaStream_t stream)
 {
 #define DAF_CASE(T)                                                     \
     switch (chunks) {                                                   \
-    case 1: return launch<T, 1, BATCH>(args, stream);                   \
-    case 2: return launch<T, 2, BATCH>(args, stream);                   \
-    default: return launch<T, 4, BATCH>(args, stream);                  \
+    case 1: return launch<T, 1, BATCH, MASK>(args, stream);             \
+    case 2: return launch<T, 2, BATCH, MASK>(args, stream);             \
+    default: return launch<T, 4, BATCH, MASK>(args, stream);            \
     }
     if (dtype == DAF_F32) { DAF_CASE(float) }
     if (dtype == DAF_F16) { DAF_CASE(__half) }
@@ -169,10 +184,11 @@ static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, const DecompressArg
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 static daf_status check_ptrs(const void *packed, const uint8_t *bits, const float *mn, const float *scale,
-                             const uint64_t *woff, const void *out)
+                             const uint64_t *woff, const void *out, uint32_t dtype)
 {
     if (!packed || !bits || !mn || !scale || !woff || !out) return DAF_ERR_INVALID_ARG;
-    if (!aligned16(packed) || !aligned16(out) || (reinterpret_cast<uintptr_t>(mn) & 3u) ||
+    const uintptr_t out_mask = dtype == DAF_F32 ? 31u : 15u;      // a lane stores its 8 elements at once
+    if (!aligned16(packed) || (reinterpret_cast<uintptr_t>(out) & out_mask) || (reinterpret_cast<uintptr_t>(mn) & 3u) ||
         (reinterpret_cast<uintptr_t>(scale) & 3u) || (reinterpret_cast<uintptr_t>(woff) & 7u))
         return DAF_ERR_INVALID_ARG;
     return DAF_OK;
@@ -191,7 +207,7 @@ extern "C" daf_status daf_decompress(const daf_params *params, const void *d_pac
     Plan pl;
     daf_status st = make_plan(params, &pl);
     if (st != DAF_OK) return st;
-    st = check_ptrs(d_packed, d_bits, d_min, d_scale, d_window_offsets, d_out);
+    st = check_ptrs(d_packed, d_bits, d_min, d_scale, d_window_offsets, d_out, params->dtype);
     if (st != DAF_OK) return st;
     if (pl.n_windows > 0x7FFFFFFFull) return DAF_ERR_UNSUPPORTED;
     DecompressArgs<1> a;
@@ -203,6 +219,29 @@ extern "C" daf_status daf_decompress(const daf_params *params, const void *d_pac
                        params->numel, 0u, (uint32_t)pl.n_windows};
     return dispatch<false>(params->dtype, pl.chunks, a, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? DAF_OK
                                                                                                                  : DAF_ERR_CUDA;
+}
+
+extern "C" daf_status daf_decompress_relu_grad(const daf_params *params, const void *d_packed, const uint8_t *d_bits,
+                                               const float *d_min, const float *d_scale, const uint64_t *d_window_offsets,
+                                               const void *d_grad_out, void *d_grad_in, daf_stream stream)
+{
+    Plan pl;
+    daf_status st = make_plan(params, &pl);
+    if (st != DAF_OK) return st;
+    st = check_ptrs(d_packed, d_bits, d_min, d_scale, d_window_offsets, d_grad_in, params->dtype);
+    if (st != DAF_OK) return st;
+    if (!d_grad_out || (reinterpret_cast<uintptr_t>(d_grad_out) & (params->dtype == DAF_F32 ? 31u : 15u))) return DAF_ERR_INVALID_ARG;
+    if (pl.n_windows > 0x7FFFFFFFull) return DAF_ERR_UNSUPPORTED;
+    DecompressArgs<1> a;
+    a.total_windows = (uint32_t)pl.n_windows;
+    a.n_tensors = 1;
+    a.G = pl.G;
+    a.log2G = pl.log2G;
+    a.t[0] = DecTensor{reinterpret_cast<const uint8_t *>(d_packed), d_bits, d_min, d_scale, d_window_offsets, d_grad_in,
+                       params->numel, 0u, (uint32_t)pl.n_windows, d_grad_out};
+    return dispatch<false, true>(params->dtype, pl.chunks, a, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? DAF_OK
+               : DAF_ERR_CUDA;
 }
 
 extern "C" daf_status daf_decompress_batch(uint32_t n, const daf_params *params, const void *const *d_packed,
@@ -225,7 +264,7 @@ extern "C" daf_status daf_decompress_batch(uint32_t n, const daf_params *params,
         st = make_plan(&params[i], &pl);
         if (st != DAF_OK) return st;
         if (params[i].dtype != params[0].dtype || pl.G != pl0.G || pl.We != pl0.We) return DAF_ERR_INVALID_ARG;
-        st = check_ptrs(d_packed[i], d_bits[i], d_min[i], d_scale[i], d_window_offsets[i], d_out[i]);
+        st = check_ptrs(d_packed[i], d_bits[i], d_min[i], d_scale[i], d_window_offsets[i], d_out[i], params[i].dtype);
         if (st != DAF_OK) return st;
         if (windows + pl.n_windows > 0x7FFFFFFFull) return DAF_ERR_UNSUPPORTED;
         a.t[i] = DecTensor{reinterpret_cast<const uint8_t *>(d_packed[i]), d_bits[i], d_min[i], d_scale[i],

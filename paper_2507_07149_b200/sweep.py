@@ -171,7 +171,22 @@ def main():
             alg = 2 * w.nbytes + packed + 9 * (x.numel() // w.group_size) + 8 * (c.sizes.n_windows + 1)
             print(f"| {w.name} relu + compress, fused | {w.numel} | {w.nbytes / 2**30:.3f} | {packed / 2**30:.3f} | "
                   f"{t_f:.4f} | {alg / t_f / 1e6:.0f} | — | — | torch.relu + daf_compress: {t_s:.4f} | — |", flush=True)
-            del act, c
+            g = torch.randn_like(x)
+            gi = torch.empty_like(x)
+
+            def fused_back():
+                daf.daf_decompress_relu_grad(p, c.packed, c.bits, c.min, c.scale, c.window_offsets, g, gi)
+
+            def separate_back():
+                daf.daf_decompress(p, c.packed, c.bits, c.min, c.scale, c.window_offsets, act)
+                torch.ops.aten.threshold_backward.grad_input(g, act, 0.0, grad_input=gi)   # the ReLU backward kernel of torch
+
+            t_fb = _time(torch, fused_back, args.steps, False)
+            t_sb = _time(torch, separate_back, args.steps, False)
+            print(f"| {w.name} ReLU gradient from the packed output, fused | {w.numel} | {w.nbytes / 2**30:.3f} | "
+                  f"{packed / 2**30:.3f} | — | — | {t_fb:.4f} | {alg / t_fb / 1e6:.0f} | — | daf_decompress + the ReLU backward kernel of torch: {t_sb:.4f} |",
+                  flush=True)
+            del act, c, g, gi
         del xs
         torch.cuda.empty_cache()
 

@@ -82,3 +82,51 @@ def test_relu_compress_rejects_other_windows():
         daf.daf_relu_compress(p, x, x, c.packed, c.sizes.packed_capacity, c.bits, c.min, c.scale, c.window_offsets,
                               c.workspace, c.sizes.workspace)
     assert e.value.status == daf.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+@pytest.mark.parametrize("G,beta,mixed,We", [(256, 2.0, False, 16384), (128, 3.0, True, 16384), (64, 1.0, True, 4096)])
+def test_relu_grad_from_the_packed_output(dtype, G, beta, mixed, We):
+    """daf_decompress_relu_grad = grad where the restored activation (in its own type) is > 0."""
+    rng = np.random.default_rng(G + int(beta))
+    n = We * 11 + G * 3
+    a = oracle.relu(_input(rng, n, G, dtype, mixed), dtype)
+    if dtype != "bf16":
+        a[G * 5: G * 6] *= a.dtype.type(1e-7 if dtype == "f16" else 1e-40)     # a group that restores to (sub)normal dust
+    g32 = rng.standard_normal(n).astype(np.float32)
+    g = g32 if dtype == "f32" else (g32.astype(np.float16) if dtype == "f16" else wl.f32_to_bf16_bits(g32))
+    x = to_device(a, dtype)
+    code = {"f32": daf.F32, "f16": daf.F16, "bf16": daf.BF16}[dtype]
+    p = daf.make_params(code, n, G, (1, 2, 4, 8), beta, window_elems=We, seed=9)
+    c = daf.alloc_outputs(p, "cuda")
+    daf.daf_compress(p, x, c.packed, c.sizes.packed_capacity, c.bits, c.min, c.scale, c.window_offsets, c.workspace,
+                     c.sizes.workspace)
+    gd = to_device(g, dtype)
+    out = daf.relu_grad(c, gd)
+    torch.cuda.synchronize()
+    ref = oracle.compress(a, G, (1, 2, 4, 8), beta, dtype="bf16" if dtype == "bf16" else None, window_elems=We, seed=9)
+    restored = oracle.decompress(ref)
+    if dtype == "bf16":
+        positive = (restored != 0) & ((restored & 0x8000) == 0)
+        want = np.where(positive, g, np.uint16(0)).astype(np.uint16)
+    else:
+        want = np.where(restored > 0, g, g.dtype.type(0)).astype(g.dtype)
+    got = to_host(out, dtype)
+    view = np.uint32 if dtype == "f32" else np.uint16
+    assert np.array_equal(got.view(view), want.view(view))
+    assert 0 < int((want.view(view) != 0).sum()) < n
+    # in place
+    daf.daf_decompress_relu_grad(p, c.packed, c.bits, c.min, c.scale, c.window_offsets, gd, gd)
+    torch.cuda.synchronize()
+    assert np.array_equal(to_host(gd, dtype).view(view), want.view(view))
+
+
+def test_fp32_outputs_must_be_32_byte_aligned():
+    x = torch.randn(1 << 16, device="cuda")
+    c = daf.compress(x, 256, (1, 2, 4, 8), 4.0)
+    buf = torch.empty((1 << 16) + 8, device="cuda")
+    with pytest.raises(daf.DafError) as e:
+        daf.daf_decompress(c.params, c.packed, c.bits, c.min, c.scale, c.window_offsets, buf[4:4 + (1 << 16)])
+    assert e.value.status == daf.ERR_INVALID_ARG
+    daf.daf_decompress(c.params, c.packed, c.bits, c.min, c.scale, c.window_offsets, buf[8:8 + (1 << 16)])
+    torch.cuda.synchronize()
