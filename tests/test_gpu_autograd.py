@@ -79,12 +79,12 @@ def test_ineligible_tensors_pass_through():
     assert torch.equal(w.grad, 2 * w.detach()) and torch.equal(small.grad, 2 * small.detach())
 
 
-def _train(ctx_factory, steps=100):
+def _train(ctx_factory, steps=100, relu=torch.nn.ReLU):
     import contextlib
     torch.manual_seed(0)
     net = torch.nn.Sequential(
-        torch.nn.Conv2d(3, 16, 3, padding=1), torch.nn.ReLU(),
-        torch.nn.Conv2d(16, 32, 3, padding=1), torch.nn.ReLU(),
+        torch.nn.Conv2d(3, 16, 3, padding=1), relu(),
+        torch.nn.Conv2d(16, 32, 3, padding=1), relu(),
         torch.nn.AdaptiveAvgPool2d(4), torch.nn.Flatten(), torch.nn.Linear(512, 10)).cuda()
     opt = torch.optim.SGD(net.parameters(), lr=0.05, momentum=0.9)
     g = torch.Generator(device="cuda").manual_seed(1)
@@ -137,3 +137,14 @@ def test_compressed_relu_layer_masks_with_the_restored_output():
     small = torch.randn(100, device="cuda", requires_grad=True)
     layer(small).sum().backward()
     assert torch.equal(small.grad, (small.detach() > 0).float())
+
+
+def test_small_cnn_trains_with_compressed_relu_layers():
+    """The same network with its ReLUs replaced by CompressedReLU (fused producer forward, fused consumer backward)."""
+    from paper_2507_07149_b200.autograd import CompressedReLU
+    daf.lib()
+    base, _ = _train(None)
+    comp, _ = _train(None, relu=lambda: CompressedReLU(group_size=256, bit_budget=4.0, seed=7))
+    assert np.mean(base[-5:]) < 0.3 * base[0]
+    assert np.mean(comp[-5:]) < 0.3 * comp[0]
+    assert abs(np.mean(comp[-5:]) - np.mean(base[-5:])) < 0.25 * base[0]
