@@ -524,3 +524,43 @@ def test_batched_calls_replayed_from_a_cuda_graph():
             assert d.max() <= 1, (mixed, i, int(d.max()))
         if mixed is not None:
             assert len(np.unique(oracle.compress(arrays[mixed], G, widths, beta, seed=900 + mixed).bits)) >= 2
+
+
+@pytest.mark.parametrize("G", [64, 256])
+def test_non_finite_inputs_stay_inside_the_buffers(G):
+    """NaN / Inf inputs: results unspecified, but nothing may be written outside the caller's buffers and
+    the calls must complete (widths come from integer budget arithmetic whatever the keys are)."""
+    rng = np.random.default_rng(G)
+    n = 16384 * 6 + G * 3
+    a = (rng.standard_normal(n) * np.repeat(10.0 ** rng.uniform(-2, 2, n // G), G)).astype(np.float32)
+    bad = rng.integers(0, n, 400)
+    a[bad[:150]] = np.nan
+    a[bad[150:250]] = np.inf
+    a[bad[250:350]] = -np.inf
+    a[G * 40: G * 41] = np.nan                                   # a whole group of NaN
+    a[G * 50: G * 51] = np.inf                                   # ... and of +Inf
+    x = to_device(a, "f32")
+    pad = 512
+    for beta in (2.0, 3.0, 4.0):
+        p = daf.make_params(daf.F32, n, G, (1, 2, 4, 8), beta, seed=2)
+        sz = daf.daf_sizes(p)
+
+        def guarded(nbytes):
+            t = torch.full((nbytes + 2 * pad,), 0xA5, dtype=torch.uint8, device="cuda")
+            return t, t[pad: pad + nbytes]
+
+        bufs = {k: guarded(nb) for k, nb in (("packed", sz.packed_capacity), ("bits", sz.n_groups), ("mn", 4 * sz.n_groups),
+                                             ("scale", 4 * sz.n_groups), ("woff", 8 * (sz.n_windows + 1)), ("out", 4 * n))}
+        ws = torch.empty(sz.workspace, dtype=torch.uint8, device="cuda")
+        daf.daf_compress(p, x, bufs["packed"][1], sz.packed_capacity, bufs["bits"][1], bufs["mn"][1], bufs["scale"][1],
+                         bufs["woff"][1], ws, sz.workspace)
+        assert daf.daf_poll_status(ws) == daf.OK
+        bits = bufs["bits"][1].cpu().numpy()
+        assert set(np.unique(bits)) <= {1, 2, 4, 8}
+        woff = bufs["woff"][1].cpu().numpy().view(np.uint64)
+        assert int(woff[-1]) == int(bits.astype(np.int64).sum()) * G // 8 <= sz.packed_capacity
+        daf.daf_decompress(p, bufs["packed"][1], bufs["bits"][1], bufs["mn"][1], bufs["scale"][1], bufs["woff"][1],
+                           bufs["out"][1])
+        torch.cuda.synchronize()
+        for name, (full, inner) in bufs.items():
+            assert bool((full[:pad] == 0xA5).all()) and bool((full[pad + inner.numel():] == 0xA5).all()), (beta, name)
