@@ -1220,8 +1220,9 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                     }
                 }
             };
-            if (G >= 256u && s_slow[iter & 1u] == 0u) {
-                // a warp's chunk lies in one group: no clamp, fixed-width packing, 8-byte aligned stores
+            if (G >= 64u && s_slow[iter & 1u] == 0u) {
+                // no clamp needed: fixed-width packing chosen by the lane's width, 8-byte aligned stores.  With
+                // G >= 256 a warp's chunk lies in one group; below, the warp splits by width (mostly into one part)
 #pragma unroll
                 for (int c = 0; c < CHUNKS; c++) {
                     const uint32_t e = e0 + 256u * c;
