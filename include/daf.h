@@ -98,7 +98,7 @@ daf_status daf_sizes(const daf_params *params, uint64_t *n_groups, uint64_t *n_w
  * A fused kernel reads the input once.  (The call enqueues a quick kernel, which handles
  * windows whose groups all end at the same width, and behind it the full kernel, which does
  * nothing unless the quick one met a window it does not handle; then it redoes the call.
- * A call of at most 512 windows is launch-bound and goes to the full kernel alone; the
+ * A call of at most 4096 windows goes to the full kernel alone (one launch is then cheaper than the pair); the
  * environment variable DAF_QUICK_MIN_WINDOWS, read at every call, overrides that number.
  * Every output is final when the call's work on the stream is done.)  If the packed output
  * of a window would pass packed_capacity, nothing of that window is stored and the status

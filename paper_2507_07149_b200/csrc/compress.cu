@@ -362,7 +362,7 @@ template <int NT> __device__ __forceinline__ uint32_t find_tensor(const Compress
 constexpr int kComputeWarps = kWarps;
 constexpr int kCompressThreads = kThreads + 64;
 constexpr uint32_t kBarStage = 1, kBarWidths = 2, kBarOwners = 3, kBarChoice = 4;
-constexpr uint32_t kQuickMinWindows = 512;                      // calls of fewer windows go to the full kernel alone
+constexpr uint32_t kQuickMinWindows = 4096;                     // calls of at most this many windows go to the full kernel alone (measured break-even)
 constexpr int kSelWords = 180;                                // shared words of the general bit choice with more than 64 groups
 
 __device__ __forceinline__ void bar_sync(uint32_t id, uint32_t threads)
