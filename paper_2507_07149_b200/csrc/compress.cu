@@ -157,7 +157,7 @@ __device__ __forceinline__ void quantize8_any(const float (&x)[8], float mn, flo
 // exclusive prefix was found (*excl), 0 when a needed descriptor is still empty and `block`
 // is false, -1 on a poisoned predecessor, -2 when the bounded wait ran out.
 // ------------------------------------------------------------------------------------------
-constexpr int kLookDepth = 4;                                 // halved in the kernels with a widths warp (measured: 0.6 % faster there, 1.8 % slower in the others)
+constexpr int kLookDepth = 4;                                 // measured: 2 is 5 % slower with groups of 1024 elements, 8 is 13 % slower everywhere
 
 template <int DEPTH>
 __device__ __forceinline__ int lookback(const uint64_t *flags, uint32_t gw, uint32_t first, int lane, bool block,
@@ -839,7 +839,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 uint64_t excl = 0;
                 int state = 1;
                 if (p_gw != pd.first_window) {
-                    state = lookback<WIDTHS ? kLookDepth / 2 : kLookDepth>(flags, p_gw, pd.first_window, lane, true, &excl);
+                    state = lookback<kLookDepth>(flags, p_gw, pd.first_window, lane, true, &excl);
                     if (lane == 0)
                         st_relaxed_u64(flags + p_gw, state == 1 ? ((kFlagPrefix << kFlagShift) | (excl + p_total))
                                                                     : (kFlagPoison << kFlagShift));
