@@ -108,3 +108,24 @@ def test_pool_first_fit_and_eviction():
     with pytest.raises(daf.DafError):
         pool.free(12345)
     pool.close()
+
+
+def test_training_integration_leaves_cpu_tensors_alone():
+    """Host logic of the autograd integration: what does not qualify (here: CPU tensors) never reaches the
+    library and is saved / computed as usual."""
+    torch = pytest.importorskip("torch")
+    from paper_2507_07149_b200.autograd import CompressedReLU, saved_activation_compression
+    x = torch.randn(1 << 15, requires_grad=True)
+    ctx = saved_activation_compression(min_numel=1024)
+    with ctx:
+        y = x.pow(2).sum()
+    y.backward()
+    assert ctx.stats["tensors"] == 0 and ctx.stats["passed_through"] >= 1
+    assert torch.equal(x.grad, 2 * x.detach())
+    layer = CompressedReLU(min_numel=1024)
+    z = torch.randn(1 << 15, requires_grad=True)
+    layer(z).sum().backward()
+    assert torch.equal(z.grad, (z.detach() > 0).float())
+    ctx.reseed(5)
+    layer.reseed(5)
+    assert ctx.seed == 5 and layer.seed == 5 and ctx._next_index == 0 and layer._next_index == 0
