@@ -564,3 +564,25 @@ def test_non_finite_inputs_stay_inside_the_buffers(G):
         torch.cuda.synchronize()
         for name, (full, inner) in bufs.items():
             assert bool((full[:pad] == 0xA5).all()) and bool((full[pad + inner.numel():] == 0xA5).all()), (beta, name)
+
+
+@pytest.mark.parametrize("case", range(36))
+def test_seeded_tie_heavy_configurations(case):
+    """Few distinct ranges per window (integer-valued data): candidate raises collide on the same key all the
+    time, so the order among equal keys (level, then group) decides most widths."""
+    rng = np.random.default_rng(50000 + case)
+    dtype = ("f32", "f16", "bf16")[case % 3]
+    We = int(rng.choice([4096, 8192, 16384]))
+    G = int(rng.choice([g for g in (32, 64, 128, 256, 512, 1024) if g <= We]))
+    widths = tuple(sorted(rng.choice([1, 2, 4, 8], size=int(rng.integers(2, 5)), replace=False).tolist()))
+    beta = min(float(min(widths) + rng.choice([0.25, 0.5, 1.0, 1.5, 2.0, 3.0])), 8.0)
+    n_groups = int(rng.integers(1, 8 * We // G + 2))
+    x = rng.integers(0, int(rng.integers(2, 7)), size=(n_groups, G)).astype(np.float32)
+    x *= rng.choice([1.0, 2.0, 0.5, 3.0], size=(n_groups, 1)).astype(np.float32)
+    if case % 4 == 0:
+        x[rng.random(n_groups) < 0.3] = 1.0                       # constant groups
+    a = x.reshape(-1)
+    a = a if dtype == "f32" else (a.astype(np.float16) if dtype == "f16" else wl.f32_to_bf16_bits(a))
+    label = f"ties/{case}/{dtype}/G{G}/We{We}/{widths}/{beta}"
+    xd, c, ref = assert_compress_parity(a, dtype, G, widths, beta, window_elems=We, seed=case, label=label)
+    assert_decompress_parity(c, ref, dtype, label)
