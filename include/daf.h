@@ -68,11 +68,26 @@ typedef struct daf_params {
     uint32_t width_mask;      /* bit b set <=> width b allowed; non-empty subset of {1,2,4,8}       */
     float    bit_budget;      /* average bits per element per window; floor(budget*256)/256 is used */
     uint32_t rounding;        /* daf_round                                                          */
-    uint32_t reserved;        /* must be 0                                                          */
+    uint32_t flags;           /* 0, or DAF_FLAG_* values or'ed together (launch policy, diagnostics) */
     uint64_t seed;            /* Philox key                                                         */
     uint64_t elem_index_base; /* global index of element 0 (a multiple of 8); 0 unless the tensor
                                  is a shard of a larger one compressed with the same seed          */
 } daf_params;
+
+/* daf_params.flags.  None of them changes a result.
+ *   DAF_FLAG_STREAM_ALWAYS / _NEVER : daf_compress first runs a streaming kernel that assumes windows
+ *       of one width (see daf_compress) unless the call is small or the parameters rule such windows
+ *       out; ALWAYS drops the size rule, NEVER goes to the general kernel directly (e.g. for data known
+ *       to mix widths).  Giving both is an error.
+ *   DAF_FLAG_KEEP_WORKSPACE : diagnostic.  The workspace is not cleared on entry: the caller has
+ *       prepared it (all zero, except what a test of the failure paths has planted there).
+ *   DAF_FLAG_POLL_LIMIT(n)  : diagnostic.  Bounded device-side waits give up after n polls
+ *       (1 <= n < 2^24) instead of the default 2^20.
+ */
+#define DAF_FLAG_STREAM_ALWAYS  0x1u
+#define DAF_FLAG_STREAM_NEVER   0x2u
+#define DAF_FLAG_KEEP_WORKSPACE 0x4u
+#define DAF_FLAG_POLL_LIMIT(n)  ((uint32_t)(n) << 8)
 
 /*
  * Sizes that follow from the parameters (host only, launches nothing).

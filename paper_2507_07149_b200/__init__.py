@@ -17,6 +17,18 @@ LIB_PATH = os.path.join(_HERE, "libdaf.so")
 OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_BUDGET, ERR_CAPACITY, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED = range(8)
 F32, F16, BF16 = 0, 1, 2
 ROUND_STOCHASTIC, ROUND_NEAREST = 0, 1
+FLAG_STREAM_ALWAYS, FLAG_STREAM_NEVER, FLAG_KEEP_WORKSPACE = 1, 2, 4
+
+
+# daf_params.flags used by make_params when the caller gives none (the GPU tests set FLAG_STREAM_ALWAYS here so
+# that their small tensors still go through both compress kernels).
+DEFAULT_FLAGS = 0
+
+
+def flag_poll_limit(n: int) -> int:
+    """daf_params.flags value that makes bounded device-side waits give up after n polls (diagnostic)."""
+    return int(n) << 8
+
 BATCH_MAX = 64
 DEFAULT_WINDOW = 16384
 
@@ -24,7 +36,7 @@ DEFAULT_WINDOW = 16384
 class daf_params(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_uint32), ("dtype", ctypes.c_uint32), ("numel", ctypes.c_uint64),
                 ("group_size", ctypes.c_uint32), ("window_elems", ctypes.c_uint32), ("width_mask", ctypes.c_uint32),
-                ("bit_budget", ctypes.c_float), ("rounding", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
+                ("bit_budget", ctypes.c_float), ("rounding", ctypes.c_uint32), ("flags", ctypes.c_uint32),
                 ("seed", ctypes.c_uint64), ("elem_index_base", ctypes.c_uint64)]
 
 
@@ -102,9 +114,12 @@ def width_mask(widths) -> int:
 
 
 def make_params(dtype: int, numel: int, group_size: int, widths, bit_budget: float, *, window_elems: int = 0,
-                rounding: int = ROUND_STOCHASTIC, seed: int = 0, elem_index_base: int = 0) -> daf_params:
+                rounding: int = ROUND_STOCHASTIC, seed: int = 0, elem_index_base: int = 0,
+                flags: int | None = None) -> daf_params:
+    if flags is None:
+        flags = DEFAULT_FLAGS
     return daf_params(ctypes.sizeof(daf_params), dtype, numel, group_size, window_elems, width_mask(widths),
-                      bit_budget, rounding, 0, seed, elem_index_base)
+                      bit_budget, rounding, flags, seed, elem_index_base)
 
 
 @dataclass
@@ -266,13 +281,13 @@ def alloc_outputs(params: daf_params, device, shape=None) -> CompressedTensor:
 
 
 def compress(x, group_size: int, widths, bit_budget: float, *, window_elems: int = 0, rounding: int = ROUND_STOCHASTIC,
-             seed: int = 0, elem_index_base: int = 0, out: CompressedTensor | None = None, check: bool = False,
-             stream=None) -> CompressedTensor:
+             seed: int = 0, elem_index_base: int = 0, flags: int | None = None, out: CompressedTensor | None = None,
+             check: bool = False, stream=None) -> CompressedTensor:
     """Allocate outputs with torch (unless given) and call daf_compress on the current stream."""
     if not x.is_cuda or not x.is_contiguous():
         raise ValueError("compress expects a contiguous CUDA tensor")
     params = make_params(dtype_code(x), x.numel(), group_size, widths, bit_budget, window_elems=window_elems,
-                         rounding=rounding, seed=seed, elem_index_base=elem_index_base)
+                         rounding=rounding, seed=seed, elem_index_base=elem_index_base, flags=flags)
     c = out if out is not None else alloc_outputs(params, x.device, x.shape)
     c.params = params
     daf_compress(params, x, c.packed, c.sizes.packed_capacity, c.bits, c.min, c.scale, c.window_offsets, c.workspace,
@@ -283,13 +298,13 @@ def compress(x, group_size: int, widths, bit_budget: float, *, window_elems: int
 
 
 def relu_compress(x, group_size: int, widths, bit_budget: float, *, rounding: int = ROUND_STOCHASTIC, seed: int = 0,
-                  elem_index_base: int = 0, inplace: bool = False, out: CompressedTensor | None = None, check: bool = False,
-                  stream=None):
+                  elem_index_base: int = 0, flags: int | None = None, inplace: bool = False, out: CompressedTensor | None = None,
+                  check: bool = False, stream=None):
     """(relu(x), compressed relu(x)) in one pass over x (daf_relu_compress); ``inplace`` overwrites x."""
     if not x.is_cuda or not x.is_contiguous():
         raise ValueError("relu_compress expects a contiguous CUDA tensor")
     params = make_params(dtype_code(x), x.numel(), group_size, widths, bit_budget, rounding=rounding, seed=seed,
-                         elem_index_base=elem_index_base)
+                         elem_index_base=elem_index_base, flags=flags)
     c = out if out is not None else alloc_outputs(params, x.device, x.shape)
     c.params = params
     act = x if inplace else _torch().empty_like(x)

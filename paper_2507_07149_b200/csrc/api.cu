@@ -3,8 +3,35 @@
 #include <string.h>
 
 #include "common.cuh"
+#include "launch_cache.hpp"
 
 namespace daf {
+
+cudaError_t persistent_ctas(const void *kernel, int threads, int dyn_smem, int *ctas)
+{
+    static LaunchCache cache;
+    int device = 0;
+    cudaError_t e = cudaGetDevice(&device);
+    if (e != cudaSuccess) return e;
+    const int err = cache.get(kernel, device, dyn_smem, ctas, [&](int *value) -> int {
+        int sms = 0, per_sm = 0, optin = 0;
+        cudaError_t q = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+        // the limit on dynamic shared memory is a property of the kernel on this device: raised to all the
+        // device offers, so that later requests of any size find it high enough
+        if (q == cudaSuccess && dyn_smem > 48 * 1024) {
+            cudaFuncAttributes fa;
+            q = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+            if (q == cudaSuccess) q = cudaFuncGetAttributes(&fa, kernel);
+            if (q == cudaSuccess)   // static and dynamic shared memory share the device's limit
+                q = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - (int)fa.sharedSizeBytes);
+        }
+        if (q == cudaSuccess) q = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, (size_t)dyn_smem);
+        if (q != cudaSuccess) return (int)q;
+        *value = sms * (per_sm > 0 ? per_sm : 1);
+        return 0;
+    });
+    return (cudaError_t)err;
+}
 
 static bool is_pow2(uint32_t v) { return v && !(v & (v - 1)); }
 
@@ -20,8 +47,9 @@ static float raise_factor(uint32_t lo, uint32_t hi)
 
 daf_status make_plan(const daf_params *p, Plan *pl)
 {
-    if (!p || p->struct_size != sizeof(daf_params) || p->reserved != 0) return DAF_ERR_INVALID_ARG;
+    if (!p || p->struct_size != sizeof(daf_params) || (p->flags & 0xF8u) != 0) return DAF_ERR_INVALID_ARG;
     if (p->dtype > DAF_BF16 || p->rounding > DAF_ROUND_NEAREST) return DAF_ERR_INVALID_ARG;
+    if ((p->flags & DAF_FLAG_STREAM_ALWAYS) && (p->flags & DAF_FLAG_STREAM_NEVER)) return DAF_ERR_INVALID_ARG;
     const uint32_t We = p->window_elems ? p->window_elems : 16384u;
     const uint32_t G = p->group_size;
     if (!is_pow2(G) || G < 32u) return DAF_ERR_INVALID_ARG;

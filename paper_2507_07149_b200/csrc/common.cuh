@@ -139,6 +139,13 @@ template <> struct Elem<float> {
                      : "=f"(x[0]), "=f"(x[1]), "=f"(x[2]), "=f"(x[3]), "=f"(x[4]), "=f"(x[5]), "=f"(x[6]), "=f"(x[7])
                      : "l"(p));
     }
+    // the same load, but the line stays in L1 for a second reader on this multiprocessor
+    static __device__ __forceinline__ void load8_keep(const void *p, float (&x)[8])
+    {
+        asm volatile("ld.global.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=f"(x[0]), "=f"(x[1]), "=f"(x[2]), "=f"(x[3]), "=f"(x[4]), "=f"(x[5]), "=f"(x[6]), "=f"(x[7])
+                     : "l"(p));
+    }
     static __device__ __forceinline__ void store8(void *p, const float (&x)[8])
     {
         asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(x[0]), "f"(x[1]), "f"(x[2]),
@@ -158,6 +165,18 @@ template <> struct Elem<__half> {
         for (int i = 0; i < 4; i++) {
             __half2 h = *reinterpret_cast<const __half2 *>(&w[i]);
             float2 f = __half22float2(h);
+            x[2 * i] = f.x;
+            x[2 * i + 1] = f.y;
+        }
+    }
+    static __device__ __forceinline__ void load8_keep(const void *p, float (&x)[8])
+    {
+        uint4 v;
+        asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
             x[2 * i] = f.x;
             x[2 * i + 1] = f.y;
         }
@@ -184,6 +203,17 @@ template <> struct Elem<__nv_bfloat16> {
 #pragma unroll
         for (int i = 0; i < 4; i++) {
             x[2 * i] = __uint_as_float(w[i] << 16);              // bfloat16 is the top half of binary32
+            x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+    }
+    static __device__ __forceinline__ void load8_keep(const void *p, float (&x)[8])
+    {
+        uint4 v;
+        asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+            x[2 * i] = __uint_as_float(w[i] << 16);
             x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
         }
     }
@@ -237,5 +267,11 @@ struct Plan {
 };
 
 daf_status make_plan(const daf_params *p, Plan *plan);
+
+// Grid of a persistent kernel on the current device: multiprocessors x resident CTAs per
+// multiprocessor for `threads` threads and `dyn_smem` bytes of dynamic shared memory (the kernel's
+// limit on dynamic shared memory is raised first when it has to be).  Both are properties of a
+// (kernel, device) pair and are remembered per pair; safe to call from several host threads.
+cudaError_t persistent_ctas(const void *kernel, int threads, int dyn_smem, int *ctas);
 
 }  // namespace daf

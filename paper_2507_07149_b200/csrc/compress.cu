@@ -26,130 +26,9 @@
 // The kernel is compiled in two forms (template flag FULL): a quick one for calls whose
 // windows all end with one width and need no clamp, and the full one, which runs behind it
 // only if the quick one gave up (see compress_kernel).
-#include <cstdlib>
-
-#include "common.cuh"
+#include "compress_shared.cuh"
 
 namespace daf {
-
-struct TensorDesc {
-    const void *in;
-    uint8_t *packed;
-    uint64_t capacity;
-    uint8_t *bits;
-    float *mn;
-    float *scale;
-    uint64_t *woff;
-    uint64_t numel;
-    uint64_t elem_base;
-    uint64_t seed;
-    uint32_t first_window;   // index of this tensor's window 0 among all windows of the launch
-    uint32_t n_windows;
-    void *act;               // fused producer (daf_relu_compress): where the activation itself goes
-};
-
-struct SmemLayout {          // byte offsets into dynamic shared memory
-    uint32_t out0, out_stride, umn, umx, sel, grp, total;
-};
-
-template <int NT> struct CompressArgs {
-    WorkspaceHeader *hdr;
-    uint64_t *flags;          // window descriptors of the quick kernel
-    uint64_t *flags2;         // ... of the full kernel
-    uint32_t gated;           // the full kernel runs only if the quick one asked for it
-    uint32_t total_windows, n_tensors;
-    uint32_t G, log2G, beta_q8, m, nearest, bulk_store, n_max;
-    uint32_t full_ell, full_rem, full_rem_after;   // budget arithmetic of a full window (n_max groups)
-    uint32_t S[kMaxLevels], cost[kMaxLevels];
-    float v[kMaxLevels];
-    SmemLayout lay;
-    PhiloxKeys keys;          // round keys of tensor 0 (single-tensor launches)
-    TensorDesc t[NT];
-};
-
-struct GroupRec {             // what the quantize pass needs per group (one 16-byte shared load)
-    float mn, inv;
-    uint32_t b, off;
-};
-
-// ------------------------------------------------------------------------------------------
-// Eight codes of width B from eight values; o[] holds eight 16-bit random lanes (two per word).
-// s = fma(x - mn, inv, 256) lies in [256, 512) where one ulp is 2^-15, so its mantissa field
-// is the fixed-point quotient; adding a 15-bit random offset r15 and dropping 15 bits rounds
-// stochastically (r15 = 2^14: round half up).  With h = 2*r15 + (one more random bit),
-// (fixed + r15) >> 15 == (2*bits(s) + h - 2*bits(256)) >> 16, which needs one add, one shift
-// and one fused subtract-and-clamp per element.
-// ------------------------------------------------------------------------------------------
-template <int B, bool CLAMP>
-__device__ __forceinline__ void quantize8(const float (&x)[8], float mn, float inv, const uint32_t (&o)[4],
-                                          uint32_t &w0, uint32_t &w1)
-{
-    constexpr uint32_t L = (1u << B) - 1u;
-    uint32_t t[8];
-#pragma unroll
-    for (int i = 0; i < 8; i++) {
-        const float d = __fsub_rn(x[i], mn);
-        const float s = __fmaf_rn(d, inv, 256.0f);
-        const uint32_t h = (i & 1) ? (o[i >> 1] >> 16) : (o[i >> 1] & 0xFFFFu);
-        t[i] = __float_as_uint(s) * 2u + h;                       // mod 2^32; 2*bits(256) = 0x87000000
-    }
-    if (CLAMP) {
-        w0 = 0u;
-        w1 = 0u;
-#pragma unroll
-        for (int i = 0; i < 8; i++) {
-            const int pos = (B * i) & 31;                         // bit position of code i in its word (unrolled: constant)
-            const uint32_t field = min((t[i] >> 16) - 0x8700u, L) << pos;
-            if (B == 8 && i >= 4) w1 |= field;
-            else w0 |= field;
-        }
-    } else {
-        // The code never exceeds L when 1/scale is a normal number, so byte 2 of t is the code
-        // itself (bits 16+B .. 23 are zero).  Byte permutes gather the eight code bytes; widths
-        // below 8 then close the gaps: 4-bit codes by interleaving two words of nibbles, 2- and
-        // 1-bit codes by a multiplication that lines the four fields of a word up in its top byte.
-        if (B == 4) {
-            // bytes (c0, c2, c4, c6) and (c1, c3, c5, c7): the odd codes become the high nibbles
-            const uint32_t ev = __byte_perm(__byte_perm(t[0], t[2], 0x0062), __byte_perm(t[4], t[6], 0x0062), 0x5410);
-            const uint32_t od = __byte_perm(__byte_perm(t[1], t[3], 0x0062), __byte_perm(t[5], t[7], 0x0062), 0x5410);
-            w0 = od * 16u + ev;
-            w1 = 0u;
-        } else {
-            const uint32_t c0123 = __byte_perm(__byte_perm(t[0], t[1], 0x0062), __byte_perm(t[2], t[3], 0x0062), 0x5410);
-            const uint32_t c4567 = __byte_perm(__byte_perm(t[4], t[5], 0x0062), __byte_perm(t[6], t[7], 0x0062), 0x5410);
-            if (B == 8) {
-                w0 = c0123;
-                w1 = c4567;
-            } else {
-                constexpr uint32_t M = B == 2 ? 0x01041040u : 0x01020408u;   // field i of a word moves up by 24 - (8 - B) i bits
-                w0 = (((c4567 * M) >> 24) << (4 * B)) | ((c0123 * M) >> 24);
-                w1 = 0u;
-            }
-        }
-    }
-}
-
-// The same for a width known only at run time (and possibly different in every lane): the
-// codes are clamped to 2^b - 1, then joined pairwise with multiply-adds by 2^b, 2^2b, 2^4b.
-__device__ __forceinline__ void quantize8_any(const float (&x)[8], float mn, float inv, const uint32_t (&o)[4],
-                                              uint32_t b, uint32_t &w0, uint32_t &w1)
-{
-    const uint32_t m1 = 1u << b, L = m1 - 1u, m2 = m1 * m1;
-    const uint32_t m4 = b == 8u ? 0u : m2 * m2;                   // eight 8-bit codes fill two words
-    uint32_t q[8];
-#pragma unroll
-    for (int i = 0; i < 8; i++) {
-        const float d = __fsub_rn(x[i], mn);
-        const float s = __fmaf_rn(d, inv, 256.0f);
-        const uint32_t h = (i & 1) ? (o[i >> 1] >> 16) : (o[i >> 1] & 0xFFFFu);
-        const uint32_t t = __float_as_uint(s) * 2u + h;
-        q[i] = min((t >> 16) - 0x8700u, L);
-    }
-    const uint32_t q01 = q[1] * m1 + q[0], q23 = q[3] * m1 + q[2], q45 = q[5] * m1 + q[4], q67 = q[7] * m1 + q[6];
-    const uint32_t lo = q23 * m2 + q01, hi = q67 * m2 + q45;
-    w0 = hi * m4 + lo;
-    w1 = hi;
-}
 
 // ------------------------------------------------------------------------------------------
 // Decoupled look-back over the window descriptors, executed by one full warp.  Each round
@@ -161,7 +40,7 @@ constexpr int kLookDepth = 4;                                 // measured: 2 is 
 
 template <int DEPTH>
 __device__ __forceinline__ int lookback(const uint64_t *flags, uint32_t gw, uint32_t first, int lane, bool block,
-                                        uint64_t *excl_out)
+                                        unsigned limit, uint64_t *excl_out)
 {
     uint64_t excl = 0;
     int64_t idx = (int64_t)gw - 1 - lane;                         // lane's nearest predecessor of this round
@@ -190,7 +69,7 @@ __device__ __forceinline__ int lookback(const uint64_t *flags, uint32_t gw, uint
             }
             if (ready) break;
             if (!block) return 0;
-            if (++polls > kMaxPolls) return -2;
+            if (++polls > limit) return -2;
             __nanosleep(64);
         }
         // accumulate up to and including the first prefix; a poisoned predecessor fails the window
@@ -261,9 +140,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 }
 // Returns false if the copy did not land within the poll budget (try_wait itself blocks for a
 // hardware-defined interval, so the loop turns slowly).
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, unsigned limit)
 {
-    for (unsigned polls = 0; polls < kMaxPolls; polls++)
+    for (unsigned polls = 0; polls < limit; polls++)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
@@ -362,7 +241,6 @@ template <int NT> __device__ __forceinline__ uint32_t find_tensor(const Compress
 constexpr int kComputeWarps = kWarps;
 constexpr int kCompressThreads = kThreads + 64;
 constexpr uint32_t kBarStage = 1, kBarWidths = 2, kBarOwners = 3, kBarChoice = 4;
-constexpr uint32_t kQuickMinWindows = 4096;                     // calls of at most this many windows go to the full kernel alone (measured break-even)
 constexpr int kSelWords = 180;                                // shared words of the general bit choice with more than 64 groups
 
 __device__ __forceinline__ void bar_sync(uint32_t id, uint32_t threads)
@@ -820,7 +698,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 // the compute warps have left (the window of the last iteration was not packed): see the
                 // copy in flight land before the shared memory goes away
                 if (valid && lane == 0) {
-                    mbar_wait_bounded(&s_full, iter & 1u);
+                    mbar_wait_bounded(&s_full, iter & 1u, a.poll_limit);
                     st_relaxed_u64(flags + gw, kFlagPoison << kFlagShift);   // the staged window is abandoned too
                 }
                 break;
@@ -839,7 +717,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 uint64_t excl = 0;
                 int state = 1;
                 if (p_gw != pd.first_window) {
-                    state = lookback<kLookDepth>(flags, p_gw, pd.first_window, lane, true, &excl);
+                    state = lookback<kLookDepth>(flags, p_gw, pd.first_window, lane, true, a.poll_limit, &excl);
                     if (lane == 0)
                         st_relaxed_u64(flags + p_gw, state == 1 ? ((kFlagPrefix << kFlagShift) | (excl + p_total))
                                                                     : (kFlagPoison << kFlagShift));
@@ -873,7 +751,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 if (lane == 0) {
                     record_error(DAF_ERR_TIMEOUT, gw);
                     st_relaxed_u64(flags + gw, kFlagPoison << kFlagShift);
-                    mbar_wait_bounded(&s_full, iter & 1u);        // one more bounded chance for the lost copy
+                    mbar_wait_bounded(&s_full, iter & 1u, a.poll_limit);        // one more bounded chance for the lost copy
                 }
                 break;
             }
@@ -892,7 +770,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     for (uint32_t iter = 0;; iter++) {
         // ---------------------------------------------------------------- the staged window has landed (or there is none)
         bool lost = false;
-        if (!mbar_wait_bounded(&s_full, iter & 1u)) {
+        if (!mbar_wait_bounded(&s_full, iter & 1u, a.poll_limit)) {
             s_lost = 1u;
             lost = true;
         }
@@ -1305,28 +1183,12 @@ static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint
 template <typename T, int CHUNKS, bool BATCH, bool WIDTHS, bool FULL, bool RELU = false>
 static cudaError_t launch(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
-    static int sms = 0, smem_set = 0, cached_smem = -1, cached_ctas = 0;   // per instantiation, current device
     const int smem = (int)args.lay.total;
-    cudaError_t e = cudaSuccess;
-    if (sms == 0) {
-        int dev = 0;
-        e = cudaGetDevice(&dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
-    }
-    if (smem > smem_set) {
-        e = cudaFuncSetAttribute(compress_kernel<T, CHUNKS, BATCH, WIDTHS, FULL, RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return e;
-        smem_set = smem;
-    }
-    if (smem != cached_smem) {
-        int per_sm = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel<T, CHUNKS, BATCH, WIDTHS, FULL, RELU>, kCompressThreads, smem);
-        if (e != cudaSuccess) return e;
-        cached_smem = smem;
-        cached_ctas = sms * (per_sm > 0 ? per_sm : 1);
-    }
-    const uint32_t grid = args.total_windows < (uint32_t)cached_ctas ? args.total_windows : (uint32_t)cached_ctas;
+    int ctas = 0;
+    const cudaError_t e = persistent_ctas(reinterpret_cast<const void *>(&compress_kernel<T, CHUNKS, BATCH, WIDTHS, FULL, RELU>),
+                                          kCompressThreads, smem, &ctas);
+    if (e != cudaSuccess) return e;
+    const uint32_t grid = args.total_windows < (uint32_t)ctas ? args.total_windows : (uint32_t)ctas;
     compress_kernel<T, CHUNKS, BATCH, WIDTHS, FULL, RELU><<<grid, kCompressThreads, smem, stream>>>(args);
     return cudaGetLastError();
 }
@@ -1360,30 +1222,43 @@ static cudaError_t dispatch_one(uint32_t dtype, uint32_t chunks, const CompressA
     }
 }
 
-// One call = the quick kernel followed by the full kernel, which returns at once unless the
-// quick one asked for it.  When the parameters rule out windows of one width (a budget that
-// no single width meets exactly and that leaves room for raises, or round-to-nearest), only
-// the full kernel is launched.
-// Calls of at most this many windows skip the quick kernel (DAF_QUICK_MIN_WINDOWS in the environment overrides it).
-static uint32_t quick_min_windows()
+// Packed size of tensor t if every window ends with one width (what the streaming kernel assumes).
+template <int NT> static uint64_t one_width_total(const CompressArgs<NT> &a, const TensorDesc &t, uint32_t we)
 {
-    const char *e = std::getenv("DAF_QUICK_MIN_WINDOWS");
-    return e && *e ? (uint32_t)std::strtoul(e, nullptr, 10) : kQuickMinWindows;
+    const uint64_t full_bytes = (uint64_t)(we >> 3) * a.S[a.full_ell];
+    const uint64_t last_elems = t.numel - (uint64_t)(t.n_windows - 1u) * we;
+    uint32_t ell = a.full_ell;
+    if (last_elems != we) {                                       // ragged last window: its own budget arithmetic
+        const uint64_t n = last_elems >> a.log2G;
+        const uint64_t rem = (((uint64_t)a.beta_q8 * n) >> 8) - (uint64_t)a.S[0] * n;
+        ell = 0;
+        while (ell + 1 < a.m && (uint64_t)(a.S[ell + 1] - a.S[0]) * n <= rem) ell++;
+    }
+    return (uint64_t)(t.n_windows - 1u) * full_bytes + (last_elems >> 3) * a.S[ell];
 }
 
+// One call = the streaming kernel, which assumes that every window ends with one width, followed
+// by the general kernel, which returns at once unless the streaming one asked for it.  When the
+// parameters rule out windows of one width (a budget that no single width meets exactly and that
+// leaves room for raises, or round-to-nearest), when the packed buffer could not hold such a result
+// (the general kernel then reports the overflow window by window), or when the call is small (it is
+// launch-bound, and one launch is cheaper than two), only the general kernel is launched.
+constexpr uint32_t kStreamMinWindows = 4096;                     // measured break-even
+
 template <bool BATCH, bool RELU = false>
-static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
+static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, uint32_t flags, CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
                             cudaStream_t stream)
 {
     const bool all_max = args.full_ell + 1 == args.m;
     const bool need_sep = !all_max && args.full_rem_after < args.cost[args.full_ell];
-    // The quick kernel pays when there are many windows per CTA; a small call is launch-bound, and one
-    // launch of the full kernel is cheaper than the pair.
-    const bool try_quick = !args.nearest && (all_max || need_sep) && args.total_windows > quick_min_windows();
+    bool try_stream = !args.nearest && (all_max || need_sep) && !(flags & DAF_FLAG_STREAM_NEVER) &&
+                      (args.total_windows > kStreamMinWindows || (flags & DAF_FLAG_STREAM_ALWAYS));
+    for (uint32_t i = 0; try_stream && i < args.n_tensors; i++)
+        try_stream = one_width_total(args, args.t[i], chunks * 4096u) <= args.t[i].capacity;
     args.flags2 = args.flags + args.total_windows;
-    args.gated = try_quick ? 1u : 0u;
-    if (try_quick) {
-        const cudaError_t e = dispatch_one<BATCH, false, RELU>(dtype, chunks, args, stream);
+    args.gated = try_stream ? 1u : 0u;
+    if (try_stream) {
+        const cudaError_t e = dispatch_stream<BATCH, RELU>(dtype, chunks, args, stream);
         if (e != cudaSuccess) return e;
     }
     return dispatch_one<BATCH, true, RELU>(dtype, chunks, args, stream);
@@ -1398,6 +1273,7 @@ template <int NT> static void fill_common(CompressArgs<NT> &a, const Plan &pl, c
     a.beta_q8 = pl.beta_q8;
     a.m = pl.m;
     a.nearest = p->rounding == DAF_ROUND_NEAREST;
+    a.poll_limit = (p->flags >> 8) ? (p->flags >> 8) : kMaxPolls;
     a.bulk_store = pl.G >= 128u;                                  // every group is then a multiple of 16 bytes
     a.n_max = pl.We / pl.G;
     const uint32_t elem_bytes = p->dtype == DAF_F32 ? 4u : 2u;
@@ -1407,6 +1283,7 @@ template <int NT> static void fill_common(CompressArgs<NT> &a, const Plan &pl, c
         a.full_ell = 0;
         while (a.full_ell + 1 < pl.m && (pl.S[a.full_ell + 1] - pl.S[0]) * n <= a.full_rem) a.full_ell++;
         a.full_rem_after = a.full_rem - (pl.S[a.full_ell] - pl.S[0]) * n;
+        a.full_test = a.full_ell + 1 < pl.m && a.full_rem_after < pl.cost[a.full_ell] && a.full_ell > 0;
     }
     a.lay = make_layout(pl.We, elem_bytes, pl.G, (uint32_t)((((uint64_t)pl.beta_q8 * pl.W) >> 8) * pl.G / 8));
     for (int k = 0; k < kMaxLevels; k++) {
@@ -1446,8 +1323,8 @@ extern "C" daf_status daf_compress(const daf_params *params, const void *d_in, v
                         d_window_offsets, params->numel, params->elem_index_base, params->seed, 0u,
                         (uint32_t)pl.n_windows};
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    if (cudaMemsetAsync(d_workspace, 0, pl.workspace, s) != cudaSuccess) return DAF_ERR_CUDA;
-    return dispatch<false>(params->dtype, pl.chunks, a, s) == cudaSuccess ? DAF_OK : DAF_ERR_CUDA;
+    if (!(params->flags & DAF_FLAG_KEEP_WORKSPACE) && cudaMemsetAsync(d_workspace, 0, pl.workspace, s) != cudaSuccess) return DAF_ERR_CUDA;
+    return dispatch<false>(params->dtype, pl.chunks, params->flags, a, s) == cudaSuccess ? DAF_OK : DAF_ERR_CUDA;
 }
 
 extern "C" daf_status daf_relu_compress(const daf_params *params, const void *d_in, void *d_act, void *d_packed,
@@ -1476,8 +1353,8 @@ extern "C" daf_status daf_relu_compress(const daf_params *params, const void *d_
                         d_window_offsets, params->numel, params->elem_index_base, params->seed, 0u,
                         (uint32_t)pl.n_windows, d_act};
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    if (cudaMemsetAsync(d_workspace, 0, pl.workspace, s) != cudaSuccess) return DAF_ERR_CUDA;
-    return dispatch<false, true>(params->dtype, pl.chunks, a, s) == cudaSuccess ? DAF_OK : DAF_ERR_CUDA;
+    if (!(params->flags & DAF_FLAG_KEEP_WORKSPACE) && cudaMemsetAsync(d_workspace, 0, pl.workspace, s) != cudaSuccess) return DAF_ERR_CUDA;
+    return dispatch<false, true>(params->dtype, pl.chunks, params->flags, a, s) == cudaSuccess ? DAF_OK : DAF_ERR_CUDA;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1525,7 +1402,7 @@ extern "C" daf_status daf_compress_static(const daf_params *params, const void *
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     // header (ticket, status) and this call's descriptors must start at zero: the array keeps the last call's contents
     if (cudaMemsetAsync(scratch, 0, pl.workspace, s) != cudaSuccess) return DAF_ERR_CUDA;
-    if (dispatch<false>(params->dtype, pl.chunks, a, s) != cudaSuccess) return DAF_ERR_CUDA;
+    if (dispatch<false>(params->dtype, pl.chunks, params->flags, a, s) != cudaSuccess) return DAF_ERR_CUDA;
     if (d_status && cudaMemcpyAsync(d_status, scratch, sizeof(uint32_t), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
         return DAF_ERR_CUDA;
     return DAF_OK;
@@ -1565,7 +1442,7 @@ extern "C" daf_status daf_compress_batch(uint32_t n, const daf_params *params, c
         st = make_plan(p, &pl);
         if (st != DAF_OK) return st;
         if (p->dtype != params[0].dtype || pl.G != pl0.G || pl.We != pl0.We || p->width_mask != params[0].width_mask ||
-            pl.beta_q8 != pl0.beta_q8 || p->rounding != params[0].rounding)
+            pl.beta_q8 != pl0.beta_q8 || p->rounding != params[0].rounding || p->flags != params[0].flags)
             return DAF_ERR_INVALID_ARG;
         if (!d_in[i] || !d_packed[i] || !d_bits[i] || !d_min[i] || !d_scale[i] || !d_window_offsets[i] || !aligned16(d_in[i]) ||
             !aligned16(d_packed[i]) || (reinterpret_cast<uintptr_t>(d_min[i]) & 3u) ||
@@ -1581,6 +1458,6 @@ extern "C" daf_status daf_compress_batch(uint32_t n, const daf_params *params, c
     const uint64_t need = sizeof(WorkspaceHeader) + 16ull * windows;
     if (workspace_bytes < need) return DAF_ERR_CAPACITY;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    if (cudaMemsetAsync(d_workspace, 0, need, s) != cudaSuccess) return DAF_ERR_CUDA;
-    return dispatch<true>(params[0].dtype, pl0.chunks, a, s) == cudaSuccess ? DAF_OK : DAF_ERR_CUDA;
+    if (!(params[0].flags & DAF_FLAG_KEEP_WORKSPACE) && cudaMemsetAsync(d_workspace, 0, need, s) != cudaSuccess) return DAF_ERR_CUDA;
+    return dispatch<true>(params[0].dtype, pl0.chunks, params[0].flags, a, s) == cudaSuccess ? DAF_OK : DAF_ERR_CUDA;
 }

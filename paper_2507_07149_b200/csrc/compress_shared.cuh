@@ -1,0 +1,143 @@
+// Argument structures and the lane-local quantize-and-pack routines shared by the compress kernels
+// (the streaming kernel for windows of one width and the window-synchronous general kernel).
+#pragma once
+#include "common.cuh"
+
+namespace daf {
+
+struct TensorDesc {
+    const void *in;
+    uint8_t *packed;
+    uint64_t capacity;
+    uint8_t *bits;
+    float *mn;
+    float *scale;
+    uint64_t *woff;
+    uint64_t numel;
+    uint64_t elem_base;
+    uint64_t seed;
+    uint32_t first_window;   // index of this tensor's window 0 among all windows of the launch
+    uint32_t n_windows;
+    void *act;               // fused producer (daf_relu_compress): where the activation itself goes
+};
+
+struct SmemLayout {          // byte offsets into dynamic shared memory
+    uint32_t out0, out_stride, umn, umx, sel, grp, total;
+};
+
+template <int NT> struct CompressArgs {
+    WorkspaceHeader *hdr;
+    uint64_t *flags;          // window descriptors of the quick kernel
+    uint64_t *flags2;         // ... of the full kernel
+    uint32_t gated;           // the full kernel runs only if the quick one asked for it
+    uint32_t poll_limit;      // polls after which a bounded wait gives up
+    uint32_t total_windows, n_tensors;
+    uint32_t G, log2G, beta_q8, m, nearest, bulk_store, n_max;
+    uint32_t full_ell, full_rem, full_rem_after;   // budget arithmetic of a full window (n_max groups)
+    uint32_t full_test;       // ... whose groups share a width only if the keys of the levels around full_ell separate
+    uint32_t S[kMaxLevels], cost[kMaxLevels];
+    float v[kMaxLevels];
+    SmemLayout lay;
+    PhiloxKeys keys;          // round keys of tensor 0 (single-tensor launches)
+    TensorDesc t[NT];
+};
+
+// The streaming kernel for calls whose windows all end with one width (compress_stream.cuh; one
+// translation unit per element type).
+template <typename T, bool BATCH, bool RELU>
+cudaError_t dispatch_stream_t(uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream);
+
+template <bool BATCH, bool RELU>
+inline cudaError_t dispatch_stream(uint32_t dtype, uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
+                                   cudaStream_t stream)
+{
+    if (dtype == DAF_F32) return dispatch_stream_t<float, BATCH, RELU>(chunks, args, stream);
+    if (dtype == DAF_F16) return dispatch_stream_t<__half, BATCH, RELU>(chunks, args, stream);
+    return dispatch_stream_t<__nv_bfloat16, BATCH, RELU>(chunks, args, stream);
+}
+
+struct GroupRec {             // what the quantize pass needs per group (one 16-byte shared load)
+    float mn, inv;
+    uint32_t b, off;
+};
+
+// ------------------------------------------------------------------------------------------
+// Eight codes of width B from eight values; o[] holds eight 16-bit random lanes (two per word).
+// s = fma(x - mn, inv, 256) lies in [256, 512) where one ulp is 2^-15, so its mantissa field
+// is the fixed-point quotient; adding a 15-bit random offset r15 and dropping 15 bits rounds
+// stochastically (r15 = 2^14: round half up).  With h = 2*r15 + (one more random bit),
+// (fixed + r15) >> 15 == (2*bits(s) + h - 2*bits(256)) >> 16, which needs one add, one shift
+// and one fused subtract-and-clamp per element.
+// ------------------------------------------------------------------------------------------
+template <int B, bool CLAMP>
+__device__ __forceinline__ void quantize8(const float (&x)[8], float mn, float inv, const uint32_t (&o)[4],
+                                          uint32_t &w0, uint32_t &w1)
+{
+    constexpr uint32_t L = (1u << B) - 1u;
+    uint32_t t[8];
+#pragma unroll
+    for (int i = 0; i < 8; i++) {
+        const float d = __fsub_rn(x[i], mn);
+        const float s = __fmaf_rn(d, inv, 256.0f);
+        const uint32_t h = (i & 1) ? (o[i >> 1] >> 16) : (o[i >> 1] & 0xFFFFu);
+        t[i] = __float_as_uint(s) * 2u + h;                       // mod 2^32; 2*bits(256) = 0x87000000
+    }
+    if (CLAMP) {
+        w0 = 0u;
+        w1 = 0u;
+#pragma unroll
+        for (int i = 0; i < 8; i++) {
+            const int pos = (B * i) & 31;                         // bit position of code i in its word (unrolled: constant)
+            const uint32_t field = min((t[i] >> 16) - 0x8700u, L) << pos;
+            if (B == 8 && i >= 4) w1 |= field;
+            else w0 |= field;
+        }
+    } else {
+        // The code never exceeds L when 1/scale is a normal number, so byte 2 of t is the code
+        // itself (bits 16+B .. 23 are zero).  Byte permutes gather the eight code bytes; widths
+        // below 8 then close the gaps: 4-bit codes by interleaving two words of nibbles, 2- and
+        // 1-bit codes by a multiplication that lines the four fields of a word up in its top byte.
+        if (B == 4) {
+            // bytes (c0, c2, c4, c6) and (c1, c3, c5, c7): the odd codes become the high nibbles
+            const uint32_t ev = __byte_perm(__byte_perm(t[0], t[2], 0x0062), __byte_perm(t[4], t[6], 0x0062), 0x5410);
+            const uint32_t od = __byte_perm(__byte_perm(t[1], t[3], 0x0062), __byte_perm(t[5], t[7], 0x0062), 0x5410);
+            w0 = od * 16u + ev;
+            w1 = 0u;
+        } else {
+            const uint32_t c0123 = __byte_perm(__byte_perm(t[0], t[1], 0x0062), __byte_perm(t[2], t[3], 0x0062), 0x5410);
+            const uint32_t c4567 = __byte_perm(__byte_perm(t[4], t[5], 0x0062), __byte_perm(t[6], t[7], 0x0062), 0x5410);
+            if (B == 8) {
+                w0 = c0123;
+                w1 = c4567;
+            } else {
+                constexpr uint32_t M = B == 2 ? 0x01041040u : 0x01020408u;   // field i of a word moves up by 24 - (8 - B) i bits
+                w0 = (((c4567 * M) >> 24) << (4 * B)) | ((c0123 * M) >> 24);
+                w1 = 0u;
+            }
+        }
+    }
+}
+
+// The same for a width known only at run time (and possibly different in every lane): the
+// codes are clamped to 2^b - 1, then joined pairwise with multiply-adds by 2^b, 2^2b, 2^4b.
+__device__ __forceinline__ void quantize8_any(const float (&x)[8], float mn, float inv, const uint32_t (&o)[4],
+                                              uint32_t b, uint32_t &w0, uint32_t &w1)
+{
+    const uint32_t m1 = 1u << b, L = m1 - 1u, m2 = m1 * m1;
+    const uint32_t m4 = b == 8u ? 0u : m2 * m2;                   // eight 8-bit codes fill two words
+    uint32_t q[8];
+#pragma unroll
+    for (int i = 0; i < 8; i++) {
+        const float d = __fsub_rn(x[i], mn);
+        const float s = __fmaf_rn(d, inv, 256.0f);
+        const uint32_t h = (i & 1) ? (o[i >> 1] >> 16) : (o[i >> 1] & 0xFFFFu);
+        const uint32_t t = __float_as_uint(s) * 2u + h;
+        q[i] = min((t >> 16) - 0x8700u, L);
+    }
+    const uint32_t q01 = q[1] * m1 + q[0], q23 = q[3] * m1 + q[2], q45 = q[5] * m1 + q[4], q67 = q[7] * m1 + q[6];
+    const uint32_t lo = q23 * m2 + q01, hi = q67 * m2 + q45;
+    w0 = hi * m4 + lo;
+    w1 = hi;
+}
+
+}  // namespace daf

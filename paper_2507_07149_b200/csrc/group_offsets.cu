@@ -141,14 +141,8 @@ extern "C" daf_status daf_group_offsets(const uint8_t *d_bits, uint64_t n_groups
     if (ws_bytes < need) return DAF_ERR_CAPACITY;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(d_ws, 0, need, s) != cudaSuccess) return DAF_ERR_CUDA;
-    static int max_ctas = 0;
-    if (max_ctas == 0) {
-        int dev = 0, sms = 0, per_sm = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, group_offsets_kernel, kThreads, 0) != cudaSuccess)
-            return DAF_ERR_CUDA;
-        max_ctas = sms * (per_sm > 0 ? per_sm : 1);
-    }
+    int max_ctas = 0;
+    if (persistent_ctas(reinterpret_cast<const void *>(&group_offsets_kernel), kThreads, 0, &max_ctas) != cudaSuccess) return DAF_ERR_CUDA;
     ScanArgs a;
     a.bits = d_bits;
     a.offsets = d_offsets;

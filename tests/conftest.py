@@ -8,9 +8,11 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
-# Small calls skip the quick kernel by default; the GPU tests are small, so they lower the limit to
-# zero to keep exercising both kernels (tests of the default behaviour unset it again).
-os.environ.setdefault("DAF_QUICK_MIN_WINDOWS", "0")
+# Small calls go to the general compress kernel alone by default; the GPU tests are small, so their
+# parameter blocks ask for the streaming kernel whatever the size (tests of the default policy undo it).
+import paper_2507_07149_b200 as _daf  # noqa: E402
+
+_daf.DEFAULT_FLAGS = _daf.FLAG_STREAM_ALWAYS
 
 
 def pytest_configure(config):
@@ -19,8 +21,8 @@ def pytest_configure(config):
 
 @pytest.fixture
 def default_quick_limit(monkeypatch):
-    """The library's own limit on the windows of a call that goes to the full kernel alone."""
-    monkeypatch.delenv("DAF_QUICK_MIN_WINDOWS", raising=False)
+    """The library's own rule for which calls go to the general kernel alone."""
+    monkeypatch.setattr(_daf, "DEFAULT_FLAGS", 0)
 
 
 @pytest.fixture(scope="session")
