@@ -23,6 +23,10 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", 
               "--fmad=false", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 
 
+# Extra compiler flags for development builds (e.g. -DDAF_STAMPS), read when the library is built.
+NVCC_FLAGS += os.environ.get("DAF_NVCC_EXTRA", "").split()
+
+
 def _nvcc() -> str:
     exe = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
     if not os.path.exists(exe):

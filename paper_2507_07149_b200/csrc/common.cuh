@@ -139,12 +139,10 @@ template <> struct Elem<float> {
                      : "=f"(x[0]), "=f"(x[1]), "=f"(x[2]), "=f"(x[3]), "=f"(x[4]), "=f"(x[5]), "=f"(x[6]), "=f"(x[7])
                      : "l"(p));
     }
-    // the same load, but the line stays in L1 for a second reader on this multiprocessor
-    static __device__ __forceinline__ void load8_keep(const void *p, float (&x)[8])
+    static __device__ __forceinline__ void widen8(const uint4 &v, float (&x)[8])   // 16 bytes = 4 elements
     {
-        asm volatile("ld.global.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                     : "=f"(x[0]), "=f"(x[1]), "=f"(x[2]), "=f"(x[3]), "=f"(x[4]), "=f"(x[5]), "=f"(x[6]), "=f"(x[7])
-                     : "l"(p));
+        x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y); x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
+        x[4] = x[0]; x[5] = x[1]; x[6] = x[2]; x[7] = x[3];
     }
     static __device__ __forceinline__ void store8(void *p, const float (&x)[8])
     {
@@ -169,10 +167,8 @@ template <> struct Elem<__half> {
             x[2 * i + 1] = f.y;
         }
     }
-    static __device__ __forceinline__ void load8_keep(const void *p, float (&x)[8])
+    static __device__ __forceinline__ void widen8(const uint4 &v, float (&x)[8])   // 16 bytes = 8 elements
     {
-        uint4 v;
-        asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int i = 0; i < 4; i++) {
@@ -206,10 +202,8 @@ template <> struct Elem<__nv_bfloat16> {
             x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
         }
     }
-    static __device__ __forceinline__ void load8_keep(const void *p, float (&x)[8])
+    static __device__ __forceinline__ void widen8(const uint4 &v, float (&x)[8])   // 16 bytes = 8 elements
     {
-        uint4 v;
-        asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int i = 0; i < 4; i++) {

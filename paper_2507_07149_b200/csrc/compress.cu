@@ -97,92 +97,6 @@ __device__ __forceinline__ int lookback(const uint64_t *flags, uint32_t gw, uint
     return 1;
 }
 
-// ------------------------------------------------------------------------------------------
-// Bulk asynchronous copies (TMA, non-tensor form) and the mbarrier that signals a landed
-// window.  All waits are bounded.
-// ------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void bulk_load(void *dst_smem, const void *src, uint32_t bytes, uint64_t *bar)
-{
-    asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_addr(dst_smem)),
-                 "l"(src), "r"(bytes), "r"(smem_addr(bar))
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_store(void *dst, const void *src_smem, uint32_t bytes)
-{
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_addr(src_smem)), "r"(bytes)
-                 : "memory");
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-__device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-// Orders this thread's earlier writes to shared memory before later reads by the async proxy.
-__device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok)
-                 : "r"(smem_addr(bar)), "r"(parity)
-                 : "memory");
-    return ok != 0;
-}
-// Returns false if the copy did not land within the poll budget (try_wait itself blocks for a
-// hardware-defined interval, so the loop turns slowly).
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, unsigned limit)
-{
-    for (unsigned polls = 0; polls < limit; polls++)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-
-// Eight consecutive elements of a lane from the staged window (two 16-byte shared loads for
-// 4-byte elements, one for 2-byte elements).
-template <typename T> __device__ __forceinline__ void load8_staged(const unsigned char *chunk, int lane, float (&x)[8]);
-
-template <> __device__ __forceinline__ void load8_staged<float>(const unsigned char *chunk, int lane, float (&x)[8])
-{
-    // a lane owns 32 bytes; which half it reads first depends on the lane, so that each
-    // quarter-warp touches all 32 banks
-    const int odd = (lane >> 2) & 1;
-    const float4 a = *reinterpret_cast<const float4 *>(chunk + lane * 32 + 16 * odd);
-    const float4 b = *reinterpret_cast<const float4 *>(chunk + lane * 32 + 16 * (odd ^ 1));
-    x[0] = odd ? b.x : a.x; x[1] = odd ? b.y : a.y; x[2] = odd ? b.z : a.z; x[3] = odd ? b.w : a.w;
-    x[4] = odd ? a.x : b.x; x[5] = odd ? a.y : b.y; x[6] = odd ? a.z : b.z; x[7] = odd ? a.w : b.w;
-}
-template <> __device__ __forceinline__ void load8_staged<__half>(const unsigned char *chunk, int lane, float (&x)[8])
-{
-    const uint4 v = *reinterpret_cast<const uint4 *>(chunk + lane * 16);
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int i = 0; i < 4; i++) {
-        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
-        x[2 * i] = f.x;
-        x[2 * i + 1] = f.y;
-    }
-}
-template <> __device__ __forceinline__ void load8_staged<__nv_bfloat16>(const unsigned char *chunk, int lane, float (&x)[8])
-{
-    const uint4 v = *reinterpret_cast<const uint4 *>(chunk + lane * 16);
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int i = 0; i < 4; i++) {
-        x[2 * i] = __uint_as_float(w[i] << 16);
-        x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
-    }
-}
-
 // Staged window -> registers, then min / max per unit of LPU lanes (a full warp uses the
 // redux instruction) written to shared memory.  Chunks past a ragged window's end read
 // stale bytes; their results are never used.
@@ -1222,6 +1136,43 @@ static cudaError_t dispatch_one(uint32_t dtype, uint32_t chunks, const CompressA
     }
 }
 
+// Runs behind the streaming kernel: one thread per window compares the key extremes gathered in
+// the window's word, checks that a ragged last window's budget arithmetic asks for the same
+// single width, and writes the window's offset (and the total behind a tensor's last window).
+template <int NT>
+__global__ void __launch_bounds__(256) verify_stream_kernel(const __grid_constant__ CompressArgs<NT> a, uint32_t we)
+{
+    const uint32_t gw = blockIdx.x * blockDim.x + threadIdx.x;
+    if (gw >= a.total_windows) return;
+    uint32_t lo = 0, hi = a.n_tensors - 1;                        // last tensor whose first window is <= gw
+    while (lo < hi) {
+        const uint32_t mid = (lo + hi + 1) >> 1;
+        if (a.t[mid].first_window <= gw) lo = mid; else hi = mid - 1;
+    }
+    const TensorDesc &td = a.t[lo];
+    const uint32_t w = gw - td.first_window, b = a.S[a.full_ell];
+    const uint64_t wbytes = (uint64_t)(we >> 3) * b;
+    bool ok = true;
+    if (a.full_test != 0u) {
+        const uint64_t word = a.flags[gw];
+        ok = ~(uint32_t)word >= (uint32_t)(word >> 32);
+    }
+    td.woff[w] = (uint64_t)w * wbytes;
+    if (w + 1u == td.n_windows) {
+        const uint64_t n_elems = td.numel - (uint64_t)w * we;
+        if (n_elems != we) {
+            const uint32_t n = (uint32_t)(n_elems >> a.log2G);
+            const uint32_t rem = (uint32_t)((((uint64_t)a.beta_q8 * n) >> 8) - (uint64_t)a.S[0] * n);
+            uint32_t ell = 0;
+            while (ell + 1 < a.m && (a.S[ell + 1] - a.S[0]) * n <= rem) ell++;
+            const uint32_t rem_after = rem - (a.S[ell] - a.S[0]) * n;
+            ok = ok && ell == a.full_ell && (ell + 1 == a.m || rem_after < a.cost[ell]);
+        }
+        td.woff[w + 1u] = (uint64_t)w * wbytes + (n_elems >> 3) * b;
+    }
+    if (!ok) atomicExch(&a.hdr->retry, 1u);
+}
+
 // Packed size of tensor t if every window ends with one width (what the streaming kernel assumes).
 template <int NT> static uint64_t one_width_total(const CompressArgs<NT> &a, const TensorDesc &t, uint32_t we)
 {
@@ -1258,7 +1209,10 @@ static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, uint32_t flags, Com
     args.flags2 = args.flags + args.total_windows;
     args.gated = try_stream ? 1u : 0u;
     if (try_stream) {
-        const cudaError_t e = dispatch_stream<BATCH, RELU>(dtype, chunks, args, stream);
+        cudaError_t e = dispatch_stream<BATCH, RELU>(dtype, chunks, args, stream);
+        if (e != cudaSuccess) return e;
+        verify_stream_kernel<BATCH ? DAF_BATCH_MAX : 1><<<(args.total_windows + 255u) / 256u, 256, 0, stream>>>(args, chunks * 4096u);
+        e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
     return dispatch_one<BATCH, true, RELU>(dtype, chunks, args, stream);
@@ -1284,6 +1238,8 @@ template <int NT> static void fill_common(CompressArgs<NT> &a, const Plan &pl, c
         while (a.full_ell + 1 < pl.m && (pl.S[a.full_ell + 1] - pl.S[0]) * n <= a.full_rem) a.full_ell++;
         a.full_rem_after = a.full_rem - (pl.S[a.full_ell] - pl.S[0]) * n;
         a.full_test = a.full_ell + 1 < pl.m && a.full_rem_after < pl.cost[a.full_ell] && a.full_ell > 0;
+        a.stream_v_lo = pl.v[a.full_ell > 0 ? a.full_ell - 1 : 0];
+        a.stream_v_hi = pl.v[a.full_ell];
     }
     a.lay = make_layout(pl.We, elem_bytes, pl.G, (uint32_t)((((uint64_t)pl.beta_q8 * pl.W) >> 8) * pl.G / 8));
     for (int k = 0; k < kMaxLevels; k++) {

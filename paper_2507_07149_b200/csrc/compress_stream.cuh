@@ -2,90 +2,50 @@
 // a budget that one allowed width meets exactly, ranges within a window close enough that no
 // raise of a higher level sorts ahead of one of a lower level, Sec. 3.4.1 of the paper).
 //
-// One persistent CTA of 32 warps per multiprocessor takes windows blockIdx.x, blockIdx.x +
-// gridDim.x, ...; its warps have two roles and never meet at a CTA-wide barrier:
+// With one width B = S[ell] for every group, the packed position of every code follows from its
+// index, and a warp can take 8 * 32 * CHUNKS consecutive elements (a "strip") from global memory
+// to packed bytes on its own, with no shared memory and no meeting with other warps:
 //
-//   stats warps (NS of them) run ahead.  Per window each reads its share of the 256-element
-//     chunks (32 bytes per lane and load, four loads in flight), reduces them to per-group
-//     min / max (3-input min/max, warp redux or segmented shuffles) and leaves these in the
-//     window's slot of a small ring in shared memory.  The warp that finishes a window last
-//     does the per-group arithmetic for all its groups, one group per lane: range, importance
-//     keys, 1/scale and scale by IEEE division, group records into the slot, metadata to global
-//     memory, and the test that the window really ends with one width.  Then it completes the
-//     slot's "full" barrier.  They also ask for the window two ahead to be brought into L2
-//     (one bulk prefetch per warp), so that HBM latency is paid long before anybody waits.
-//   quantize warps take the CTA's chunks round-robin.  A chunk's 8 elements per lane come from
-//     L1 / L2 (the stats warps had them a moment ago), the group record from the slot; then
-//     Eq. 1 with stochastic rounding (Philox4x32-10, the float -> uint step by the power-of-two
-//     offset of Eq. 5), lane-local LSB-first packing, one coalesced store.  Every chunk done
-//     counts on the slot's "empty" barrier, which frees the slot for the stats warps.
+//   strip -> registers (32 bytes per lane and load, all loads of the strip in flight)
+//   -> per-group min / max (3-input min/max, warp redux or segmented shuffles)
+//   -> range, 1/scale and scale by IEEE division, metadata stores
+//   -> Eq. 1 with stochastic rounding (Philox4x32-10, the float -> uint step by the power-of-two
+//      offset of Eq. 5), lane-local LSB-first packing, coalesced stores.
 //
-// With every window of one width B, the packed position of a code follows from its index, so
-// nothing here depends on another CTA.  If a window fails the test (or a group needs the clamped
-// quantizer, or a ragged last window has a budget that asks for another width), the kernel raises
-// hdr->retry and stops; the general kernel, enqueued behind it, then redoes the call.
+// A CTA takes windows blockIdx.x, blockIdx.x + gridDim.x, ...; its warp w takes strip w of each.
+// That every window really is of one width is an assumption while the strips are processed.
+// Each warp adds the extremes of the importance keys of its groups to the window's word in the
+// workspace (two atomic max); verify_stream_kernel, enqueued behind, compares them window by
+// window, checks the budget arithmetic of ragged last windows and writes the window offsets.  If
+// a test fails anywhere (or a group needs the clamped quantizer), hdr->retry is raised and the
+// general kernel, enqueued behind both, redoes the call; the streaming kernel itself stops as
+// soon as it sees the flag, and raises it itself when the keys of one strip alone do not
+// separate.  Groups larger than a strip are the one case where warps meet: those that
+// share a group exchange their extremes through shared memory at a named barrier of their own.
 //
-// The kernel is a template over the element type, the window size, the width B, batched calls
-// and the fused ReLU; this header is included by one translation unit per element type.
+// The kernel is a template over the element type, the strip length, the width B, the relation
+// of group size and strip (GC: 0 = groups below 256 elements, 1 = groups of whole chunks inside
+// a strip, 2 = groups of one or more strips), batched calls and the fused ReLU; this header is
+// included by one translation unit per element type.
 #pragma once
+#include <type_traits>
+
 #include "compress_shared.cuh"
 
 namespace daf {
 
 namespace stream {
 
-constexpr int kWarpsPerCta = 32, kCtaThreads = 32 * kWarpsPerCta;
-constexpr int kSlots = 4;                                         // windows between the stats warps and the slowest quantize warp
-constexpr int kMaxUnits = 512;                                    // per window: 256-element chunks, or groups when they are smaller
-
-struct Slot {
-    uint64_t full;            // mbarrier: the window's records are complete (one arrival)
-    uint64_t empty;           // mbarrier: every chunk of the window has been quantized (one arrival per chunk)
-    const char *src;          // the window's first element
-    unsigned char *out;       // the window's first packed byte
-    char *act;                // fused ReLU: where the window's activation goes
-    uint64_t blk;             // Philox block of the window's first element
-    uint32_t n_elems;         // elements of the window (a ragged last window has fewer)
-    uint32_t done;            // stats warps that have finished the window
-    uint32_t pad[2];
-    uint32_t rkeys[20];       // Philox round keys of the window's tensor (batched calls)
-    float umn[kMaxUnits], umx[kMaxUnits];
-    float2 rec[kMaxUnits];    // per group: min, 1/scale
-};
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void bar_init(uint64_t *bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void bar_arrive(uint64_t *bar)
-{
-    asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool bar_try_wait(uint64_t *bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cta.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok)
-                 : "r"(smem_u32(bar)), "r"(parity)
-                 : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ uint32_t ld_volatile_shared(const uint32_t *p)
-{
-    return *reinterpret_cast<const volatile uint32_t *>(p);
-}
-__device__ __forceinline__ void st_volatile_shared(uint32_t *p, uint32_t v)
-{
-    *reinterpret_cast<volatile uint32_t *>(p) = v;
-}
 __device__ __forceinline__ uint32_t ld_relaxed_u32(const unsigned int *p)
 {
     uint32_t v;
     asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-
+__device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
 // Lane-local extremes of eight values.
 __device__ __forceinline__ void extremes8(const float (&x)[8], float &lo, float &hi)
 {
@@ -102,7 +62,6 @@ __device__ __forceinline__ float warp_max(float v)
     asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(v) : "f"(v));
     return v;
 }
-
 template <int B> __device__ __forceinline__ void store_packed(unsigned char *p, uint32_t w0, uint32_t w1)
 {
     if (B == 1) *p = (unsigned char)w0;
@@ -111,295 +70,317 @@ template <int B> __device__ __forceinline__ void store_packed(unsigned char *p, 
     else *reinterpret_cast<uint2 *>(p) = make_uint2(w0, w1);
 }
 
+// What a group needs before its elements can be quantized.
+struct Settled {
+    float mn, inv, scale;
+    bool slow;                // 1/scale is not a normal number: the codes may need the clamp, which this kernel does not have
+};
+// Range, 1/scale = L / R and scale = R / L by IEEE division, importance keys of the last raise taken and of the
+// first raise not taken (Sec. 3.4.1).
+template <int B>
+__device__ __forceinline__ Settled settle(float lo, float hi, float v_lo, float v_hi, uint32_t &kmin, uint32_t &kmax)
+{
+    constexpr float Lf = (float)((1u << B) - 1u);
+    const float R0 = __fsub_rn(hi, lo);
+    const bool pos = R0 >= 0x1p-118f;                             // below: degenerate group, treated as constant
+    const float R = pos ? R0 : 0.0f;
+    const float Rd = pos ? R0 : 1.0f;                             // (a constant group divides by one: the division stays on its fast path)
+    Settled s;
+    s.mn = lo;
+    s.inv = pos ? __fdiv_rn(Lf, Rd) : 0.0f;
+    s.scale = pos ? __fdiv_rn(Rd, Lf) : 0.0f;
+    s.slow = pos && s.inv < 0x1p-126f;
+    kmin = min(kmin, __float_as_uint(__fmul_rn(R, v_lo)));
+    kmax = max(kmax, __float_as_uint(__fmul_rn(R, v_hi)));
+    return s;
+}
+
 }  // namespace stream
 
-template <typename T, int WE, int B, int NS, bool BATCH, bool RELU>
-__global__ void __launch_bounds__(stream::kCtaThreads, 1)
+template <typename T, int CHUNKS, int B, int GC, bool BATCH, bool RELU>
+__global__ void __launch_bounds__(kThreads, 2)
 stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> a)
 {
     using namespace stream;
-    constexpr uint32_t CPW = WE / 256u;                           // chunks per window
-    constexpr uint32_t NQ = kWarpsPerCta - NS;                    // quantize warps
-    constexpr uint32_t SHARE = CPW / NS;                          // chunks of a window per stats warp
+    constexpr uint32_t STRIP = 256u * CHUNKS;                     // elements per warp and window
+    constexpr uint32_t WE = kWarps * STRIP;
     constexpr uint32_t EB = Elem<T>::kBytes;
     constexpr uint32_t WBYTES = (WE >> 3) * B;                    // packed bytes of a whole window
-    static_assert(CPW % NS == 0 && SHARE >= 1, "the stats warps share a window's chunks evenly");
-    constexpr int BATCHED = SHARE < 4 ? (int)SHARE : 4;           // loads a stats warp keeps in flight
 
-    __shared__ __align__(16) Slot s_slot[kSlots];
-    __shared__ uint32_t s_abort;                                  // this CTA stops: the call is redone (or a wait ran out)
+    __shared__ float s_ext[2][kWarps][2];                         // strip extremes of groups that span warps
+    __shared__ uint32_t s_stop[2][kWarps];                        // ... and each warp's wish to stop
     __shared__ uint32_t s_first[BATCH ? DAF_BATCH_MAX : 1];       // first window of every tensor
+    __shared__ __align__(16) uint32_t s_rkeys[BATCH ? kWarps : 1][20];   // Philox round keys of the warp's current tensor
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid < kSlots) {
-        bar_init(&s_slot[tid].full, 1u);
-        bar_init(&s_slot[tid].empty, CPW);
-        s_slot[tid].done = 0u;
-    }
-    if (tid == 0) {
-        s_abort = 0u;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
     if (BATCH) {
-        for (uint32_t i = tid; i < DAF_BATCH_MAX; i += kCtaThreads) s_first[i] = i < a.n_tensors ? a.t[i].first_window : 0xFFFFFFFFu;
+        for (uint32_t i = tid; i < DAF_BATCH_MAX; i += kThreads) s_first[i] = i < a.n_tensors ? a.t[i].first_window : 0xFFFFFFFFu;
+        __syncthreads();
     }
-    __syncthreads();
-
     const uint32_t log2G = a.log2G;
-    auto tensor_index = [&](uint32_t gw) -> uint32_t {
-        if (!BATCH) return 0u;
-        const uint32_t n0 = __popc(__ballot_sync(0xFFFFFFFFu, s_first[lane] <= gw));
-        const uint32_t n1 = __popc(__ballot_sync(0xFFFFFFFFu, s_first[lane + 32] <= gw));
-        return n0 + n1 - 1u;
-    };
-    auto give_up = [&]() {                                        // the general kernel redoes the call
-        atomicExch(&a.hdr->retry, 1u);
-        st_volatile_shared(&s_abort, 1u);
-    };
-    // Bounded wait on one of the slots' barriers; false: stop (another warp gave up, or the wait ran out).
-    auto wait = [&](uint64_t *bar, uint32_t parity, uint32_t gw, uint32_t site) -> bool {
-        for (unsigned polls = 0;; polls++) {
-            if (bar_try_wait(bar, parity)) return true;
-            if (ld_volatile_shared(&s_abort) != 0u) return false;
-            if (polls > a.poll_limit) {
-                if (lane == 0 && atomicCAS(&a.hdr->status, 0u, (unsigned)DAF_ERR_TIMEOUT) == 0u) {
-                    a.hdr->fail_window = gw;
-                    a.hdr->fail_site = site;
-                }
-                st_volatile_shared(&s_abort, 1u);
-                return false;
-            }
-        }
-    };
+    const uint32_t strip0 = (uint32_t)warp * STRIP;               // the strip's first element within its window
+    const uint32_t e0 = strip0 + (uint32_t)lane * 8u;             // the lane's first element of chunk 0
+    uint32_t cur_keys = 0xFFFFFFFFu;
+    uint32_t stop = 0u, retry_seen = 0u;
+    uint32_t it = 0;
 
-    if (warp < NS) {
-        // ============================================================ stats warps
-        uint32_t retry_seen = 0u;
-        for (uint32_t it = 0;; it++) {
-            const uint32_t gw = blockIdx.x + it * gridDim.x;
-            if (gw >= a.total_windows) break;
-            if ((retry_seen | ld_volatile_shared(&s_abort)) != 0u) {
-                st_volatile_shared(&s_abort, 1u);                 // the quantize warps stop waiting for this window
-                break;
-            }
-            retry_seen = ld_relaxed_u32(&a.hdr->retry);           // consumed one window later
-            Slot &sl = s_slot[it % kSlots];
-            const uint32_t use = it / kSlots;
-            const uint32_t ti = tensor_index(gw);
-            const TensorDesc &td = a.t[ti];
-            const uint32_t w = BATCH ? gw - td.first_window : gw;
-            uint32_t n_elems = WE;
-            if (w + 1u == td.n_windows) n_elems = (uint32_t)(td.numel - (uint64_t)w * WE);
-            const char *const src = reinterpret_cast<const char *>(td.in) + (uint64_t)w * (WE * EB);
-
-            // ---- the window two ahead is requested into L2 now (this warp's share of it)
-            {
-                const uint32_t gw_p = gw + 2u * gridDim.x;
-                if (gw_p < a.total_windows) {
-                    const TensorDesc &tp = a.t[tensor_index(gw_p)];
-                    const uint64_t at = (uint64_t)(BATCH ? gw_p - tp.first_window : gw_p) * WE + (uint32_t)warp * (SHARE * 256u);
-                    if (lane == 0 && at < tp.numel) {
-                        const uint64_t left = (tp.numel - at) * EB;
-                        const uint32_t bytes = left < SHARE * 256u * EB ? (uint32_t)left : SHARE * 256u * EB;
-                        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<const char *>(tp.in) + at * EB),
-                                     "r"(bytes & ~15u));
-                    }
+    // One strip.  WHOLE: the window has all its elements (no predicates anywhere).
+    auto strip = [&](auto whole_tag, const TensorDesc &td, uint32_t gw, uint32_t w, uint32_t n_elems) {
+        constexpr bool WHOLE = decltype(whole_tag)::value;
+        // ---- the strip's loads go out first
+        float x[CHUNKS][8];
+        {
+            const char *const src = reinterpret_cast<const char *>(td.in) + ((uint64_t)w * WE + e0) * EB;
+#pragma unroll
+            for (int c = 0; c < CHUNKS; c++) {
+                if (WHOLE) {
+                    Elem<T>::load8(src + 256u * EB * c, x[c]);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 8; i++) x[c][i] = 0.0f;
+                    if (e0 + 256u * c < n_elems) Elem<T>::load8(src + 256u * EB * c, x[c]);
                 }
             }
-            // ---- the slot must have been drained by the quantize warps
-            if (use > 0u && !wait(&sl.empty, (use - 1u) & 1u, gw, 8u)) break;
-
-            // ---- this warp's chunks: per-unit min / max into the slot
-            const uint32_t c0 = (uint32_t)warp * SHARE;
-#pragma unroll 1
-            for (uint32_t cb = 0; cb < SHARE; cb += BATCHED) {
-                float x[BATCHED][8];
-#pragma unroll
-                for (int j = 0; j < BATCHED; j++) {
-                    const uint32_t e = (c0 + cb + j) * 256u + (uint32_t)lane * 8u;
-                    if (e < n_elems) {
-                        Elem<T>::load8_keep(src + (size_t)e * EB, x[j]);
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 8; i++) x[j][i] = 0.0f;
-                    }
-                }
-#pragma unroll
-                for (int j = 0; j < BATCHED; j++) {
-                    if (RELU) {
-#pragma unroll
-                        for (int i = 0; i < 8; i++) x[j][i] = fmaxf(x[j][i], 0.0f);
-                    }
-                    float lo, hi;
-                    extremes8(x[j], lo, hi);
-                    const uint32_t c = c0 + cb + j;
-                    if (log2G >= 8u) {
-                        lo = warp_min(lo);
-                        hi = warp_max(hi);
-                        if (lane == 0) {
-                            sl.umn[c] = lo;
-                            sl.umx[c] = hi;
-                        }
-                    } else {
-                        const uint32_t lpu = 1u << (log2G - 3u);  // lanes per group
-                        for (uint32_t off = 1; off < lpu; off <<= 1) {
-                            lo = fmin2(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, off));
-                            hi = fmax2(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, off));
-                        }
-                        if (((uint32_t)lane & (lpu - 1u)) == 0u) {
-                            const uint32_t u = (c << (8u - log2G)) + ((uint32_t)lane >> (log2G - 3u));
-                            sl.umn[u] = lo;
-                            sl.umx[u] = hi;
-                        }
-                    }
-                }
-            }
-            // ---- the warp that finishes the window last settles its groups
-            __syncwarp();
-            uint32_t last = 0u;
-            if (lane == 0) {
-                __threadfence_block();
-                last = atomicAdd(&sl.done, 1u) + 1u == (uint32_t)NS;
-                __threadfence_block();
-            }
-            last = __shfl_sync(0xFFFFFFFFu, last, 0);
-            if (last == 0u) continue;
-
-            const uint32_t n = n_elems >> log2G;                  // groups of the window
-            bool ok = true;
-            if (n_elems != WE) {
-                // ragged last window: its own budget arithmetic must ask for the same single width
-                const uint32_t rem = (uint32_t)((((uint64_t)a.beta_q8 * n) >> 8) - (uint64_t)a.S[0] * n);
-                uint32_t ell = 0;
-                while (ell + 1 < a.m && (a.S[ell + 1] - a.S[0]) * n <= rem) ell++;
-                const uint32_t rem_after = rem - (a.S[ell] - a.S[0]) * n;
-                const bool all_max = ell + 1 == a.m;
-                ok = ell == a.full_ell && (all_max || rem_after < a.cost[ell]);
-            }
-            const float Lf = (float)((1u << B) - 1u);
-            const float v_lo = a.v[a.full_ell > 0u ? a.full_ell - 1u : 0u], v_hi = a.v[a.full_ell];
-            const uint32_t cpg = log2G > 8u ? 1u << (log2G - 8u) : 1u;   // units per group
-            const uint64_t g0 = (uint64_t)w * (WE >> log2G);      // first group of the window in the tensor
-            uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
-            bool slow = false;
-            for (uint32_t g = lane; g < n; g += 32u) {
-                float lo = sl.umn[g * cpg], hi = sl.umx[g * cpg];
-                for (uint32_t j = 1; j < cpg; j++) {
-                    lo = fmin2(lo, sl.umn[g * cpg + j]);
-                    hi = fmax2(hi, sl.umx[g * cpg + j]);
-                }
-                float R = __fsub_rn(hi, lo);
-                if (R < 0x1p-118f) R = 0.0f;                      // degenerate group: constant
-                kmin = min(kmin, __float_as_uint(__fmul_rn(R, v_lo)));
-                kmax = max(kmax, __float_as_uint(__fmul_rn(R, v_hi)));
-                const float inv = R > 0.0f ? __fdiv_rn(Lf, R) : 0.0f;
-                const float scale = R > 0.0f ? __fdiv_rn(R, Lf) : 0.0f;
-                // 1/scale not a normal number: the codes may need the clamp, which this kernel does not have
-                slow |= R > 0.0f && inv < 0x1p-126f;
-                sl.rec[g] = make_float2(lo, inv);
-                td.bits[g0 + g] = (uint8_t)B;
-                td.mn[g0 + g] = lo;
-                td.scale[g0 + g] = scale;
-            }
-            if (a.full_test != 0u) {
-                // every raise below level ell must sort ahead of every raise from level ell upward
-                kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
-                kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
-                ok = ok && kmin >= kmax;
-            }
-            ok = ok && !__any_sync(0xFFFFFFFFu, slow);
-            if (lane < 10 && BATCH) philox_store_round_keys(sl.rkeys, td.seed, lane);
-            if (lane == 0) {
-                if (!ok) give_up();
-                sl.src = src;
-                sl.out = td.packed + (uint64_t)w * WBYTES;
-                sl.act = RELU ? reinterpret_cast<char *>(td.act) + (uint64_t)w * (WE * EB) : nullptr;
-                sl.blk = (td.elem_base >> 3) + (uint64_t)w * (WE >> 3);
-                sl.n_elems = n_elems;
-                sl.done = 0u;
-                td.woff[w] = (uint64_t)w * WBYTES;
-                if (w + 1u == td.n_windows) td.woff[w + 1u] = (uint64_t)w * WBYTES + (uint64_t)(n_elems >> 3) * B;
-            }
-            __syncwarp();
-            if (lane == 0) bar_arrive(&sl.full);                  // (release: the slot's contents are visible to who sees the phase)
         }
-        return;
-    }
-
-    // ================================================================ quantize warps
-    uint32_t cur_it = 0xFFFFFFFFu;
-    const char *src = nullptr;
-    unsigned char *out = nullptr;
-    char *act = nullptr;
-    uint64_t blk0 = 0;
-    uint32_t n_elems = 0;
-    for (uint32_t nseq = (uint32_t)warp - NS;; nseq += NQ) {
-        const uint32_t it = nseq / CPW, c = nseq % CPW;
-        const uint32_t gw = blockIdx.x + it * gridDim.x;
-        if (gw >= a.total_windows) break;
-        Slot &sl = s_slot[it % kSlots];
-        if (it != cur_it) {
-            if (!wait(&sl.full, (it / kSlots) & 1u, gw, 9u)) break;
-            cur_it = it;
-            src = sl.src;
-            out = sl.out;
-            act = sl.act;
-            blk0 = sl.blk;
-            n_elems = sl.n_elems;
-        }
-        const uint32_t e = c * 256u + (uint32_t)lane * 8u;
-        const bool on = e < n_elems;
-        float x[8];
-        if (on) {
-            Elem<T>::load8(src + (size_t)e * EB, x);
-        } else {
-#pragma unroll
-            for (int i = 0; i < 8; i++) x[i] = 0.0f;
-        }
-        const float2 rec = sl.rec[on ? e >> log2G : 0u];
-        uint32_t o[4], w0, w1;
-        const uint64_t blk = blk0 + (e >> 3);
-        if (BATCH) {
-            const PhiloxSharedKeys sk{reinterpret_cast<const uint4 *>(sl.rkeys)};
-            philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), sk, o);
-        } else {
-            philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), a.keys, o);
-        }
+        // ---- meanwhile: has anybody asked to stop?
+        stop |= retry_seen;
+        retry_seen = ld_relaxed_u32(&a.hdr->retry);               // consumed one window later
         if (RELU) {
-            // fused producer: what is compressed (and written out) is max(x, +0); the lane stores what it loaded, so
-            // the output may be the input buffer (the stats warps are done with this window)
+            // fused producer: what is compressed (and written out) is max(x, +0); a lane stores the chunk it loaded, so
+            // the output may be the input buffer
+            char *const act = reinterpret_cast<char *>(td.act) + ((uint64_t)w * WE + e0) * EB;
 #pragma unroll
-            for (int i = 0; i < 8; i++) x[i] = fmaxf(x[i], 0.0f);
-            if (on) Elem<T>::store8(act + (size_t)e * EB, x);
+            for (int c = 0; c < CHUNKS; c++) {
+#pragma unroll
+                for (int i = 0; i < 8; i++) x[c][i] = fmaxf(x[c][i], 0.0f);
+                if (WHOLE || e0 + 256u * c < n_elems) Elem<T>::store8(act + 256u * EB * c, x[c]);
+            }
         }
-        quantize8<B, false>(x, rec.x, rec.y, o, w0, w1);
-        if (on) store_packed<B>(out + (size_t)(e >> 3) * B, w0, w1);
-        __syncwarp();                                             // every lane has read its record
-        if (lane == 0) bar_arrive(&sl.empty);
+
+        const uint64_t blk0 = (td.elem_base >> 3) + (uint64_t)w * (WE >> 3) + (e0 >> 3);
+        unsigned char *const out = td.packed + (uint64_t)w * WBYTES + (size_t)(e0 >> 3) * B;
+        const uint64_t g0 = (uint64_t)w * (WE >> log2G) + (strip0 >> log2G);   // the strip's first group in the tensor
+        uint8_t *const bits_p = td.bits + g0;
+        float *const mn_p = td.mn + g0, *const scale_p = td.scale + g0;
+        uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+        bool slow = false;
+        // Philox + Eq. 1 + pack + store of chunk c with the group's minimum and 1/scale
+        auto quantize = [&](auto chunk_tag, float mn, float inv) {
+            constexpr int c = decltype(chunk_tag)::value;
+            uint32_t o[4], w0, w1;
+            const uint64_t blk = blk0 + 32u * c;
+            if (BATCH) {
+                const PhiloxSharedKeys sk{reinterpret_cast<const uint4 *>(s_rkeys[warp])};
+                philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), sk, o);
+            } else {
+                philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), a.keys, o);
+            }
+            quantize8<B, false>(x[c], mn, inv, o, w0, w1);
+            if (WHOLE || e0 + 256u * c < n_elems) store_packed<B>(out + 32 * B * c, w0, w1);
+        };
+        auto for_chunks = [&](auto f) {                           // f(integral_constant<int, c>) for every chunk of the strip
+            f(std::integral_constant<int, 0>{});
+            if constexpr (CHUNKS > 1) f(std::integral_constant<int, 1>{});
+            if constexpr (CHUNKS > 2) {
+                f(std::integral_constant<int, 2>{});
+                f(std::integral_constant<int, 3>{});
+            }
+        };
+
+        if (GC == 0) {
+            // ---- several groups per chunk: a segmented shuffle leaves every lane with its own group's extremes
+            const uint32_t lpg = 1u << (log2G - 3u);              // lanes per group
+            for_chunks([&](auto ct) {
+                constexpr int c = decltype(ct)::value;
+                float lo, hi;
+                extremes8(x[c], lo, hi);
+                lo = fmin2(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, 1));
+                hi = fmax2(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, 1));
+                lo = fmin2(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, 2));
+                hi = fmax2(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, 2));
+                if (lpg > 4u) {
+                    lo = fmin2(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, 4));
+                    hi = fmax2(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, 4));
+                }
+                if (lpg > 8u) {
+                    lo = fmin2(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, 8));
+                    hi = fmax2(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, 8));
+                }
+                uint32_t k1 = 0xFFFFFFFFu, k2 = 0u;
+                const Settled s = settle<B>(lo, hi, a.stream_v_lo, a.stream_v_hi, k1, k2);
+                if (WHOLE || e0 + 256u * c < n_elems) {           // (groups are whole: the lane's group exists iff its elements do)
+                    kmin = min(kmin, k1);
+                    kmax = max(kmax, k2);
+                    slow |= s.slow;
+                    if (((uint32_t)lane & (lpg - 1u)) == 0u) {
+                        const uint32_t g = (((uint32_t)c << 8) >> log2G) + ((uint32_t)lane >> (log2G - 3u));
+                        bits_p[g] = (uint8_t)B;
+                        mn_p[g] = s.mn;
+                        scale_p[g] = s.scale;
+                    }
+                }
+                quantize(ct, s.mn, s.inv);
+            });
+        } else if (GC == 1 && (CHUNKS == 2 || log2G == 8u)) {
+            // ---- one group per chunk
+            for_chunks([&](auto ct) {
+                constexpr int c = decltype(ct)::value;
+                float lo, hi;
+                extremes8(x[c], lo, hi);
+                lo = warp_min(lo);
+                hi = warp_max(hi);
+                uint32_t k1 = 0xFFFFFFFFu, k2 = 0u;
+                const Settled s = settle<B>(lo, hi, a.stream_v_lo, a.stream_v_hi, k1, k2);
+                if (WHOLE || strip0 + 256u * c < n_elems) {
+                    kmin = min(kmin, k1);
+                    kmax = max(kmax, k2);
+                    slow |= s.slow;
+                    if (lane == 0) {
+                        bits_p[c] = (uint8_t)B;
+                        mn_p[c] = s.mn;
+                        scale_p[c] = s.scale;
+                    }
+                }
+                quantize(ct, s.mn, s.inv);
+            });
+        } else if (GC == 1) {
+            // ---- two chunks per group (strips of four chunks, groups of 512 elements)
+            if constexpr (CHUNKS == 4) {
+                auto pair = [&](auto c_even, auto c_odd) {
+                    constexpr int p = decltype(c_even)::value / 2;
+                    float lo, hi, l2, h2;
+                    extremes8(x[2 * p], lo, hi);
+                    extremes8(x[2 * p + 1], l2, h2);
+                    lo = warp_min(fmin2(lo, l2));
+                    hi = warp_max(fmax2(hi, h2));
+                    uint32_t k1 = 0xFFFFFFFFu, k2 = 0u;
+                    const Settled s = settle<B>(lo, hi, a.stream_v_lo, a.stream_v_hi, k1, k2);
+                    if (WHOLE || strip0 + 512u * p < n_elems) {
+                        kmin = min(kmin, k1);
+                        kmax = max(kmax, k2);
+                        slow |= s.slow;
+                        if (lane == 0) {
+                            bits_p[p] = (uint8_t)B;
+                            mn_p[p] = s.mn;
+                            scale_p[p] = s.scale;
+                        }
+                    }
+                    quantize(c_even, s.mn, s.inv);
+                    quantize(c_odd, s.mn, s.inv);
+                };
+                pair(std::integral_constant<int, 0>{}, std::integral_constant<int, 1>{});
+                pair(std::integral_constant<int, 2>{}, std::integral_constant<int, 3>{});
+            }
+        } else {
+            // ---- the strip lies in one group, which k warps share
+            const uint32_t k = (1u << log2G) / STRIP;
+            float lo, hi;
+            extremes8(x[0], lo, hi);
+#pragma unroll
+            for (int c = 1; c < CHUNKS; c++) {
+                float l2, h2;
+                extremes8(x[c], l2, h2);
+                lo = fmin2(lo, l2);
+                hi = fmax2(hi, h2);
+            }
+            lo = warp_min(lo);
+            hi = warp_max(hi);
+            if (k > 1u) {
+                // exchange the strips' extremes (and the wish to stop, so that the k warps leave together and nobody is
+                // left at the barrier)
+                const uint32_t buf = it & 1u, first = (uint32_t)warp & ~(k - 1u);
+                if (lane == 0) {
+                    s_ext[buf][warp][0] = lo;
+                    s_ext[buf][warp][1] = hi;
+                    s_stop[buf][warp] = stop;
+                }
+                named_bar_sync(1u + first / k, 32u * k);
+                for (uint32_t j = 0; j < k; j++) {
+                    lo = fmin2(lo, s_ext[buf][first + j][0]);
+                    hi = fmax2(hi, s_ext[buf][first + j][1]);
+                    stop |= s_stop[buf][first + j];
+                }
+            }
+            uint32_t k1 = 0xFFFFFFFFu, k2 = 0u;
+            const Settled s = settle<B>(lo, hi, a.stream_v_lo, a.stream_v_hi, k1, k2);
+            if (WHOLE || strip0 < n_elems) {
+                kmin = k1;
+                kmax = k2;
+                slow = s.slow;
+                if (lane == 0 && ((uint32_t)warp & (k - 1u)) == 0u) {
+                    bits_p[0] = (uint8_t)B;
+                    mn_p[0] = s.mn;
+                    scale_p[0] = s.scale;
+                }
+            }
+            for_chunks([&](auto ct) { quantize(ct, s.mn, s.inv); });
+        }
+
+        // ---- this strip's part of the test that the window ends with one width
+        if (GC == 0) {
+            kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+            kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+            slow = __any_sync(0xFFFFFFFFu, slow);
+        }
+        if (lane == 0) {
+            if (a.full_test != 0u) {
+                // every raise below level ell must sort ahead of every raise from level ell upward: the window's word
+                // gathers the smallest key of the former (complemented) and the largest of the latter, for the kernel
+                // that runs behind this one; keys of this strip alone that do not separate settle the matter at once
+                unsigned int *const word = reinterpret_cast<unsigned int *>(a.flags + gw);
+                atomicMax(word, ~kmin);
+                atomicMax(word + 1, kmax);
+                slow |= kmin < kmax;
+            }
+            if (slow) atomicExch(&a.hdr->retry, 1u);              // the general kernel redoes the call
+        }
+    };
+
+    for (uint32_t gw = blockIdx.x; gw < a.total_windows; gw += gridDim.x, it++) {
+        uint32_t ti = 0u;
+        if (BATCH) {
+            const uint32_t n0 = __popc(__ballot_sync(0xFFFFFFFFu, s_first[lane] <= gw));
+            const uint32_t n1 = __popc(__ballot_sync(0xFFFFFFFFu, s_first[lane + 32] <= gw));
+            ti = n0 + n1 - 1u;
+            if (ti != cur_keys) {                                 // round keys of this tensor's seed
+                __syncwarp();
+                if (lane < 10) philox_store_round_keys(s_rkeys[warp], a.t[ti].seed, lane);
+                __syncwarp();
+                cur_keys = ti;
+            }
+        }
+        const TensorDesc &td = a.t[ti];
+        const uint32_t w = BATCH ? gw - td.first_window : gw;
+        uint32_t n_elems = WE;                                    // a ragged last window has fewer (whole groups)
+        if (w + 1u == td.n_windows) n_elems = (uint32_t)(td.numel - (uint64_t)w * WE);
+        if (n_elems == WE) strip(std::true_type{}, td, gw, w, n_elems);
+        else strip(std::false_type{}, td, gw, w, n_elems);
+        if (stop != 0u) break;                                    // (the same decision in all warps that share a group)
     }
 }
 
-template <typename T, int WE, int B, int NS, bool BATCH, bool RELU>
+template <typename T, int CHUNKS, int B, int GC, bool BATCH, bool RELU>
 static cudaError_t launch_stream(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
     int ctas = 0;
-    const cudaError_t e = persistent_ctas(reinterpret_cast<const void *>(&stream_compress_kernel<T, WE, B, NS, BATCH, RELU>),
-                                          stream::kCtaThreads, 0, &ctas);
+    const cudaError_t e = persistent_ctas(reinterpret_cast<const void *>(&stream_compress_kernel<T, CHUNKS, B, GC, BATCH, RELU>),
+                                          kThreads, 0, &ctas);
     if (e != cudaSuccess) return e;
     const uint32_t grid = args.total_windows < (uint32_t)ctas ? args.total_windows : (uint32_t)ctas;
-    stream_compress_kernel<T, WE, B, NS, BATCH, RELU><<<grid, stream::kCtaThreads, 0, stream>>>(args);
+    stream_compress_kernel<T, CHUNKS, B, GC, BATCH, RELU><<<grid, kThreads, 0, stream>>>(args);
     return cudaGetLastError();
 }
 
-template <typename T, int WE, bool BATCH, bool RELU>
-static cudaError_t launch_stream_w(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
+template <typename T, int CHUNKS, bool BATCH, bool RELU>
+static cudaError_t launch_stream_c(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
-    // groups below 256 elements cost the stats warps segmented shuffles and more groups to settle: eight of them
-    const bool many = args.G < 256u;
-#define DAF_CASE(BB)                                                                              \
-    case BB:                                                                                      \
-        return many ? launch_stream<T, WE, BB, 8, BATCH, RELU>(args, stream)                      \
-                    : launch_stream<T, WE, BB, 4, BATCH, RELU>(args, stream);
+    const uint32_t strip = 256u * CHUNKS;
+    const int gc = args.G < 256u ? 0 : args.G < strip ? 1 : 2;
+#define DAF_CASE(BB)                                                                                                 \
+    case BB:                                                                                                         \
+        if (gc == 0) return launch_stream<T, CHUNKS, BB, 0, BATCH, RELU>(args, stream);                              \
+        if constexpr (CHUNKS > 1) { if (gc == 1) return launch_stream<T, CHUNKS, BB, 1, BATCH, RELU>(args, stream); } \
+        return launch_stream<T, CHUNKS, BB, 2, BATCH, RELU>(args, stream);
     switch (args.S[args.full_ell]) {
         DAF_CASE(1)
         DAF_CASE(2)
@@ -410,16 +391,17 @@ static cudaError_t launch_stream_w(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1>
 #undef DAF_CASE
 }
 
-// Launch for element type T: window size from the plan's chunk count, B = the width every whole window ends with.
+// Launch for element type T: strip length from the window size, GC from the group size, B = the
+// width every whole window ends with.
 template <typename T, bool BATCH, bool RELU>
 cudaError_t dispatch_stream_t(uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
     if constexpr (RELU) {                                         // fused producer: single tensor, default window
-        return launch_stream_w<T, 16384, false, true>(args, stream);
+        return launch_stream_c<T, 4, false, true>(args, stream);
     } else {
-        if (chunks == 1) return launch_stream_w<T, 4096, BATCH, false>(args, stream);
-        if (chunks == 2) return launch_stream_w<T, 8192, BATCH, false>(args, stream);
-        return launch_stream_w<T, 16384, BATCH, false>(args, stream);
+        if (chunks == 1) return launch_stream_c<T, 1, BATCH, false>(args, stream);
+        if (chunks == 2) return launch_stream_c<T, 2, BATCH, false>(args, stream);
+        return launch_stream_c<T, 4, BATCH, false>(args, stream);
     }
 }
 
