@@ -70,29 +70,16 @@ template <int B> __device__ __forceinline__ void store_packed(unsigned char *p, 
     else *reinterpret_cast<uint2 *>(p) = make_uint2(w0, w1);
 }
 
-// What a group needs before its elements can be quantized.
-struct Settled {
-    float mn, inv, scale;
-    bool slow;                // 1/scale is not a normal number: the codes may need the clamp, which this kernel does not have
-};
-// Range, 1/scale = L / R and scale = R / L by IEEE division, importance keys of the last raise taken and of the
-// first raise not taken (Sec. 3.4.1).
-template <int B>
-__device__ __forceinline__ Settled settle(float lo, float hi, float v_lo, float v_hi, uint32_t &kmin, uint32_t &kmax)
+// What a group's elements need before they can be quantized: the minimum and 1/scale = L / R (IEEE division).  R comes
+// back as the range the oracle uses (zero for a degenerate group).
+template <int B> __device__ __forceinline__ float inverse_scale(float lo, float hi, float &R)
 {
     constexpr float Lf = (float)((1u << B) - 1u);
     const float R0 = __fsub_rn(hi, lo);
     const bool pos = R0 >= 0x1p-118f;                             // below: degenerate group, treated as constant
-    const float R = pos ? R0 : 0.0f;
-    const float Rd = pos ? R0 : 1.0f;                             // (a constant group divides by one: the division stays on its fast path)
-    Settled s;
-    s.mn = lo;
-    s.inv = pos ? __fdiv_rn(Lf, Rd) : 0.0f;
-    s.scale = pos ? __fdiv_rn(Rd, Lf) : 0.0f;
-    s.slow = pos && s.inv < 0x1p-126f;
-    kmin = min(kmin, __float_as_uint(__fmul_rn(R, v_lo)));
-    kmax = max(kmax, __float_as_uint(__fmul_rn(R, v_hi)));
-    return s;
+    R = pos ? R0 : 0.0f;
+    // (a constant group divides by one: the division stays on its fast path)
+    return pos ? __fdiv_rn(Lf, pos ? R0 : 1.0f) : 0.0f;
 }
 
 }  // namespace stream
@@ -142,6 +129,16 @@ stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MA
                 }
             }
         }
+        // ---- the strip this warp takes next is asked into L2 now, a whole strip's work ahead of its loads (one 128-byte
+        // line per lane; whole windows only: the line must exist)
+#ifndef DAF_PF_DIST
+#define DAF_PF_DIST 1u
+#endif
+        if (WHOLE && gw + DAF_PF_DIST * gridDim.x + 1u < a.total_windows && (uint32_t)lane * 128u < STRIP * EB) {
+            const char *const next = reinterpret_cast<const char *>(td.in) + ((uint64_t)(w + DAF_PF_DIST * gridDim.x) * WE + strip0) * EB;
+            if (!BATCH || w + DAF_PF_DIST * gridDim.x + 1u < td.n_windows)
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(next + (uint32_t)lane * 128u));
+        }
         // ---- meanwhile: has anybody asked to stop?
         stop |= retry_seen;
         retry_seen = ld_relaxed_u32(&a.hdr->retry);               // consumed one window later
@@ -162,8 +159,10 @@ stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MA
         const uint64_t g0 = (uint64_t)w * (WE >> log2G) + (strip0 >> log2G);   // the strip's first group in the tensor
         uint8_t *const bits_p = td.bits + g0;
         float *const mn_p = td.mn + g0, *const scale_p = td.scale + g0;
-        uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
-        bool slow = false;
+        // Each group's (minimum, range) is parked in one lane while the chunks are quantized; afterwards one pass over the
+        // lanes works out the scales and the importance keys and stores the metadata of the whole strip.
+        float p_mn = 0.0f, p_R = 0.0f, inv_min = __int_as_float(0x7f800000);
+        uint32_t p_idx = 0xFFFFFFFFu;                             // the parked group's index within the strip (none yet)
         // Philox + Eq. 1 + pack + store of chunk c with the group's minimum and 1/scale
         auto quantize = [&](auto chunk_tag, float mn, float inv) {
             constexpr int c = decltype(chunk_tag)::value;
@@ -188,8 +187,9 @@ stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MA
         };
 
         if (GC == 0) {
-            // ---- several groups per chunk: a segmented shuffle leaves every lane with its own group's extremes
-            const uint32_t lpg = 1u << (log2G - 3u);              // lanes per group
+            // ---- several groups per chunk: a segmented shuffle leaves every lane with its own group's extremes; the lane
+            // whose position in its group equals the chunk number parks the group
+            const uint32_t lpg = 1u << (log2G - 3u);              // lanes per group (4, 8 or 16)
             for_chunks([&](auto ct) {
                 constexpr int c = decltype(ct)::value;
                 float lo, hi;
@@ -206,71 +206,47 @@ stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MA
                     lo = fmin2(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, 8));
                     hi = fmax2(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, 8));
                 }
-                uint32_t k1 = 0xFFFFFFFFu, k2 = 0u;
-                const Settled s = settle<B>(lo, hi, a.stream_v_lo, a.stream_v_hi, k1, k2);
-                if (WHOLE || e0 + 256u * c < n_elems) {           // (groups are whole: the lane's group exists iff its elements do)
-                    kmin = min(kmin, k1);
-                    kmax = max(kmax, k2);
-                    slow |= s.slow;
-                    if (((uint32_t)lane & (lpg - 1u)) == 0u) {
-                        const uint32_t g = (((uint32_t)c << 8) >> log2G) + ((uint32_t)lane >> (log2G - 3u));
-                        bits_p[g] = (uint8_t)B;
-                        mn_p[g] = s.mn;
-                        scale_p[g] = s.scale;
-                    }
+                float R;
+                const float inv = inverse_scale<B>(lo, hi, R);
+                // (groups are whole: the lane's group exists iff its elements do)
+                if ((WHOLE || e0 + 256u * c < n_elems) && ((uint32_t)lane & (lpg - 1u)) == (uint32_t)c) {
+                    p_mn = lo;
+                    p_R = R;
+                    p_idx = (((uint32_t)c << 8) >> log2G) + ((uint32_t)lane >> (log2G - 3u));
                 }
-                quantize(ct, s.mn, s.inv);
+                if (R > 0.0f) inv_min = fminf(inv_min, inv);
+                quantize(ct, lo, inv);
             });
-        } else if (GC == 1 && (CHUNKS == 2 || log2G == 8u)) {
-            // ---- one group per chunk
+        } else if (GC == 1) {
+            // ---- groups of one chunk, or of two (strips of four chunks, groups of 512 elements): lane j parks group j
+            const bool pairs = CHUNKS == 4 && log2G == 9u;
+            float l_prev = 0.0f, h_prev = 0.0f, mn_pair = 0.0f, inv_pair = 0.0f;
             for_chunks([&](auto ct) {
                 constexpr int c = decltype(ct)::value;
                 float lo, hi;
-                extremes8(x[c], lo, hi);
-                lo = warp_min(lo);
-                hi = warp_max(hi);
-                uint32_t k1 = 0xFFFFFFFFu, k2 = 0u;
-                const Settled s = settle<B>(lo, hi, a.stream_v_lo, a.stream_v_hi, k1, k2);
-                if (WHOLE || strip0 + 256u * c < n_elems) {
-                    kmin = min(kmin, k1);
-                    kmax = max(kmax, k2);
-                    slow |= s.slow;
-                    if (lane == 0) {
-                        bits_p[c] = (uint8_t)B;
-                        mn_p[c] = s.mn;
-                        scale_p[c] = s.scale;
+                if (!pairs || (c & 1) == 0) {
+                    extremes8(x[c], lo, hi);
+                    if (pairs && c + 1 < CHUNKS) {
+                        extremes8(x[(c + 1) % CHUNKS], l_prev, h_prev);
+                        lo = fmin2(lo, l_prev);
+                        hi = fmax2(hi, h_prev);
                     }
+                    lo = warp_min(lo);
+                    hi = warp_max(hi);
+                    float R;
+                    const float inv = inverse_scale<B>(lo, hi, R);
+                    const uint32_t j = pairs ? (uint32_t)c >> 1 : (uint32_t)c;
+                    if ((WHOLE || strip0 + 256u * c < n_elems) && (uint32_t)lane == j) {
+                        p_mn = lo;
+                        p_R = R;
+                        p_idx = j;
+                    }
+                    if (R > 0.0f) inv_min = fminf(inv_min, inv);
+                    mn_pair = lo;
+                    inv_pair = inv;
                 }
-                quantize(ct, s.mn, s.inv);
+                quantize(ct, mn_pair, inv_pair);
             });
-        } else if (GC == 1) {
-            // ---- two chunks per group (strips of four chunks, groups of 512 elements)
-            if constexpr (CHUNKS == 4) {
-                auto pair = [&](auto c_even, auto c_odd) {
-                    constexpr int p = decltype(c_even)::value / 2;
-                    float lo, hi, l2, h2;
-                    extremes8(x[2 * p], lo, hi);
-                    extremes8(x[2 * p + 1], l2, h2);
-                    lo = warp_min(fmin2(lo, l2));
-                    hi = warp_max(fmax2(hi, h2));
-                    uint32_t k1 = 0xFFFFFFFFu, k2 = 0u;
-                    const Settled s = settle<B>(lo, hi, a.stream_v_lo, a.stream_v_hi, k1, k2);
-                    if (WHOLE || strip0 + 512u * p < n_elems) {
-                        kmin = min(kmin, k1);
-                        kmax = max(kmax, k2);
-                        slow |= s.slow;
-                        if (lane == 0) {
-                            bits_p[p] = (uint8_t)B;
-                            mn_p[p] = s.mn;
-                            scale_p[p] = s.scale;
-                        }
-                    }
-                    quantize(c_even, s.mn, s.inv);
-                    quantize(c_odd, s.mn, s.inv);
-                };
-                pair(std::integral_constant<int, 0>{}, std::integral_constant<int, 1>{});
-                pair(std::integral_constant<int, 2>{}, std::integral_constant<int, 3>{});
-            }
         } else {
             // ---- the strip lies in one group, which k warps share
             const uint32_t k = (1u << log2G) / STRIP;
@@ -301,38 +277,47 @@ stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MA
                     stop |= s_stop[buf][first + j];
                 }
             }
-            uint32_t k1 = 0xFFFFFFFFu, k2 = 0u;
-            const Settled s = settle<B>(lo, hi, a.stream_v_lo, a.stream_v_hi, k1, k2);
-            if (WHOLE || strip0 < n_elems) {
-                kmin = k1;
-                kmax = k2;
-                slow = s.slow;
-                if (lane == 0 && ((uint32_t)warp & (k - 1u)) == 0u) {
-                    bits_p[0] = (uint8_t)B;
-                    mn_p[0] = s.mn;
-                    scale_p[0] = s.scale;
-                }
+            float R;
+            const float inv = inverse_scale<B>(lo, hi, R);
+            // the group's first warp parks it (in lane 0) and stores its metadata
+            if ((WHOLE || strip0 < n_elems) && lane == 0 && ((uint32_t)warp & (k - 1u)) == 0u) {
+                p_mn = lo;
+                p_R = R;
+                p_idx = 0u;
             }
-            for_chunks([&](auto ct) { quantize(ct, s.mn, s.inv); });
+            if (R > 0.0f) inv_min = fminf(inv_min, inv);
+            for_chunks([&](auto ct) { quantize(ct, lo, inv); });
         }
 
-        // ---- this strip's part of the test that the window ends with one width
-        if (GC == 0) {
+        // ---- the strip's metadata and its part of the test that the window ends with one width
+        {
+            constexpr float Lf = (float)((1u << B) - 1u);
+            const bool on = p_idx != 0xFFFFFFFFu, pos = p_R > 0.0f;
+            const float scale = pos ? __fdiv_rn(p_R, Lf) : 0.0f;  // (lanes without a group divide zero)
+            // importance keys of the last raise taken and of the first raise not taken (Sec. 3.4.1)
+            uint32_t kmin = on ? __float_as_uint(__fmul_rn(p_R, a.stream_v_lo)) : 0xFFFFFFFFu;
+            uint32_t kmax = on ? __float_as_uint(__fmul_rn(p_R, a.stream_v_hi)) : 0u;
+            if (on) {
+                bits_p[p_idx] = (uint8_t)B;
+                mn_p[p_idx] = p_mn;
+                scale_p[p_idx] = scale;
+            }
             kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
             kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
-            slow = __any_sync(0xFFFFFFFFu, slow);
-        }
-        if (lane == 0) {
-            if (a.full_test != 0u) {
-                // every raise below level ell must sort ahead of every raise from level ell upward: the window's word
-                // gathers the smallest key of the former (complemented) and the largest of the latter, for the kernel
-                // that runs behind this one; keys of this strip alone that do not separate settle the matter at once
-                unsigned int *const word = reinterpret_cast<unsigned int *>(a.flags + gw);
-                atomicMax(word, ~kmin);
-                atomicMax(word + 1, kmax);
-                slow |= kmin < kmax;
+            // 1/scale not a normal number: the codes may need the clamp, which this kernel does not have
+            bool give_up = __any_sync(0xFFFFFFFFu, inv_min < 0x1p-126f);
+            if (lane == 0) {
+                if (a.full_test != 0u) {
+                    // every raise below level ell must sort ahead of every raise from level ell upward: the window's
+                    // word gathers the smallest key of the former (complemented) and the largest of the latter, for the
+                    // kernel that runs behind this one; keys of this strip alone that do not separate settle the matter
+                    unsigned int *const word = reinterpret_cast<unsigned int *>(a.flags + gw);
+                    atomicMax(word, ~kmin);
+                    atomicMax(word + 1, kmax);
+                    give_up |= kmin < kmax;
+                }
+                if (give_up) atomicExch(&a.hdr->retry, 1u);       // the general kernel redoes the call
             }
-            if (slow) atomicExch(&a.hdr->retry, 1u);              // the general kernel redoes the call
         }
     };
 
