@@ -139,6 +139,13 @@ template <> struct Elem<float> {
                      : "=f"(x[0]), "=f"(x[1]), "=f"(x[2]), "=f"(x[3]), "=f"(x[4]), "=f"(x[5]), "=f"(x[6]), "=f"(x[7])
                      : "l"(p));
     }
+    // the same load, but the line may stay in L1 for a second reader on this multiprocessor
+    static __device__ __forceinline__ void load8_keep(const void *p, float (&x)[8])
+    {
+        asm volatile("ld.global.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=f"(x[0]), "=f"(x[1]), "=f"(x[2]), "=f"(x[3]), "=f"(x[4]), "=f"(x[5]), "=f"(x[6]), "=f"(x[7])
+                     : "l"(p));
+    }
     static __device__ __forceinline__ void widen8(const uint4 &v, float (&x)[8])   // 16 bytes = 4 elements
     {
         x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y); x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
@@ -166,6 +173,12 @@ template <> struct Elem<__half> {
             x[2 * i] = f.x;
             x[2 * i + 1] = f.y;
         }
+    }
+    static __device__ __forceinline__ void load8_keep(const void *p, float (&x)[8])
+    {
+        uint4 v;
+        asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+        widen8(v, x);
     }
     static __device__ __forceinline__ void widen8(const uint4 &v, float (&x)[8])   // 16 bytes = 8 elements
     {
@@ -201,6 +214,12 @@ template <> struct Elem<__nv_bfloat16> {
             x[2 * i] = __uint_as_float(w[i] << 16);              // bfloat16 is the top half of binary32
             x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
         }
+    }
+    static __device__ __forceinline__ void load8_keep(const void *p, float (&x)[8])
+    {
+        uint4 v;
+        asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+        widen8(v, x);
     }
     static __device__ __forceinline__ void widen8(const uint4 &v, float (&x)[8])   // 16 bytes = 8 elements
     {

@@ -1,0 +1,6 @@
+// The general compress kernel for bf16 inputs (see compress_general.cuh).
+#include "compress_general.cuh"
+
+namespace daf {
+DAF_INSTANTIATE_GENERAL(__nv_bfloat16)
+}

@@ -21,24 +21,19 @@ struct TensorDesc {
     void *act;               // fused producer (daf_relu_compress): where the activation itself goes
 };
 
-struct SmemLayout {          // byte offsets into dynamic shared memory
-    uint32_t out0, out_stride, umn, umx, sel, grp, total;
-};
-
 template <int NT> struct CompressArgs {
     WorkspaceHeader *hdr;
-    uint64_t *flags;          // window descriptors of the quick kernel
-    uint64_t *flags2;         // ... of the full kernel
-    uint32_t gated;           // the full kernel runs only if the quick one asked for it
+    uint64_t *flags;          // per window: key extremes gathered by the streaming kernel
+    uint64_t *flags2;         // per window: look-back descriptor of the general kernel
+    uint32_t gated;           // the general kernel runs only if the streaming one (or its verifier) asked for it
     uint32_t poll_limit;      // polls after which a bounded wait gives up
     uint32_t total_windows, n_tensors;
-    uint32_t G, log2G, beta_q8, m, nearest, bulk_store, n_max;
+    uint32_t G, log2G, beta_q8, m, nearest, n_max;
     uint32_t full_ell, full_rem, full_rem_after;   // budget arithmetic of a full window (n_max groups)
     uint32_t full_test;       // ... whose groups share a width only if the keys of the levels around full_ell separate
     float stream_v_lo, stream_v_hi;   // importance factors of the raise into level full_ell and of the raise out of it
     uint32_t S[kMaxLevels], cost[kMaxLevels];
     float v[kMaxLevels];
-    SmemLayout lay;
     PhiloxKeys keys;          // round keys of tensor 0 (single-tensor launches)
     TensorDesc t[NT];
 };
@@ -129,10 +124,90 @@ template <> __device__ __forceinline__ void load8_staged<__nv_bfloat16>(const un
     }
 }
 
+// ------------------------------------------------------------------------------------------
+// Decoupled look-back over the window descriptors, executed by one full warp.  Each round
+// inspects DEPTH * 32 predecessors with all loads in flight at once.  Returns 1 when the
+// exclusive prefix was found (*excl), 0 when a needed descriptor is still empty and `block`
+// is false, -1 on a poisoned predecessor, -2 when the bounded wait ran out.
+// ------------------------------------------------------------------------------------------
+constexpr int kLookDepth = 4;                                 // measured: 2 is 5 % slower with groups of 1024 elements, 8 is 13 % slower everywhere
+
+template <int DEPTH>
+__device__ __forceinline__ int lookback(const uint64_t *flags, uint32_t gw, uint32_t first, int lane, bool block,
+                                        unsigned limit, uint64_t *excl_out)
+{
+    uint64_t excl = 0;
+    int64_t idx = (int64_t)gw - 1 - lane;                         // lane's nearest predecessor of this round
+    unsigned polls = 0;
+    for (;;) {
+        uint64_t f[DEPTH];
+        bool done = false;                                        // a prefix (or poison) ends the walk in this round
+        for (;;) {
+#pragma unroll
+            for (int j = 0; j < DEPTH; j++) {
+                const int64_t i = idx - 32 * j;
+                f[j] = (i >= (int64_t)first) ? ld_relaxed_u64(flags + i) : (kFlagPrefix << kFlagShift);
+            }
+            bool ready = true;                                    // walk the chunks from the nearest predecessor outward
+            done = false;
+#pragma unroll
+            for (int j = 0; j < DEPTH; j++) {
+                if (!done && ready) {
+                    const uint32_t st = (uint32_t)(f[j] >> kFlagShift);
+                    const unsigned stop_mask = __ballot_sync(0xFFFFFFFFu, st == kFlagPrefix || st == kFlagPoison);
+                    const unsigned empty_mask = __ballot_sync(0xFFFFFFFFu, st == kFlagEmpty);
+                    const unsigned upto = stop_mask ? ((2u << (__ffs(stop_mask) - 1)) - 1u) : 0xFFFFFFFFu;
+                    if (empty_mask & upto) ready = false;
+                    else if (stop_mask) done = true;
+                }
+            }
+            if (ready) break;
+            if (!block) return 0;
+            if (++polls > limit) return -2;
+            __nanosleep(64);
+        }
+        // accumulate up to and including the first prefix; a poisoned predecessor fails the window
+        uint64_t v = 0;
+        bool stop = false, bad = false;
+#pragma unroll
+        for (int j = 0; j < DEPTH; j++) {
+            if (!stop) {
+                const uint32_t st = (uint32_t)(f[j] >> kFlagShift);
+                const unsigned stop_mask = __ballot_sync(0xFFFFFFFFu, st == kFlagPrefix || st == kFlagPoison);
+                const unsigned upto = stop_mask ? ((2u << (__ffs(stop_mask) - 1)) - 1u) : 0xFFFFFFFFu;
+                if (__ballot_sync(0xFFFFFFFFu, st == kFlagPoison) & upto) bad = true;
+                if ((upto >> lane) & 1u) v += f[j] & kFlagValueMask;
+                if (stop_mask) stop = true;
+            }
+        }
+        if (bad) return -1;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+        excl += v;
+        if (done) break;
+        idx -= 32 * DEPTH;
+    }
+    *excl_out = excl;
+    return 1;
+}
+
 // The streaming kernel for calls whose windows all end with one width (compress_stream.cuh; one
 // translation unit per element type).
 template <typename T, bool BATCH, bool RELU>
 cudaError_t dispatch_stream_t(uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream);
+
+// The general kernel: any mix of widths within a window (compress_general.cuh; one translation unit per element type).
+template <typename T, bool BATCH, bool RELU>
+cudaError_t dispatch_general_t(uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream);
+
+template <bool BATCH, bool RELU>
+inline cudaError_t dispatch_general(uint32_t dtype, uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
+                                    cudaStream_t stream)
+{
+    if (dtype == DAF_F32) return dispatch_general_t<float, BATCH, RELU>(chunks, args, stream);
+    if (dtype == DAF_F16) return dispatch_general_t<__half, BATCH, RELU>(chunks, args, stream);
+    return dispatch_general_t<__nv_bfloat16, BATCH, RELU>(chunks, args, stream);
+}
 
 template <bool BATCH, bool RELU>
 inline cudaError_t dispatch_stream(uint32_t dtype, uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
