@@ -28,6 +28,8 @@
 // Windows are handed out by ticket, so every window with a smaller index than the one a CTA holds
 // belongs to a CTA that is running (or done) and the look-back always makes progress.
 #pragma once
+#include <type_traits>
+
 #include "compress_shared.cuh"
 
 namespace daf {
@@ -37,7 +39,8 @@ namespace general {
 constexpr int kWorkers = kWarps;                                  // 16 worker warps: one strip of the window each
 constexpr int kDeciders = 2;
 constexpr int kCtaThreads = 32 * (kWorkers + kDeciders);
-constexpr int kRing = 4;                                          // window slots (a window is in flight for two iterations)
+constexpr int kLag = 3;                                           // pass B runs this many windows behind pass A
+constexpr int kRing = kLag + 2;                                   // window slots
 
 struct WinHead {                                                  // fixed part of a window's slot
     uint64_t stats_in;        // mbarrier: every worker's min / max of the window are in (one arrival per worker)
@@ -138,7 +141,93 @@ __device__ __forceinline__ void quantize_store(uint32_t b, const float (&x)[8], 
     }
 }
 
+// ------------------------------------------------------------------------------------------
+// The greedy of Sec. 3.4.1 on one warp, candidates in registers.  Every lane holds NK candidate raises (key, cw =
+// cost | 1 << 16, or cw = 0 for "no candidate"); slot s of lane l sorts, among equal keys, before slot s' > s of
+// any lane and before slot s of lane l' > l.  Accepted is the longest prefix, in the order (key descending, then
+// that order), whose summed cost is at most rem; take[s] says whether this lane's slot s is in it.  F(t), the cost
+// of all raises with key >= t, falls as t grows, so the prefix is every raise with a key above Kp, the largest t
+// with F(t) > rem, and then the raises with key Kp in order while they fit.  One warp reduction gives F(t) and N(t),
+// the number of raises with key >= t; the interval that holds Kp starts from the keys' common leading bits and is
+// halved bit by bit; as soon as a single raise is left in it, its key is Kp.
+// ------------------------------------------------------------------------------------------
+template <int NK, bool BOUNDS>
+__device__ __forceinline__ void accept_prefix(const uint32_t (&key)[NK], const uint32_t (&cw)[NK],
+                                              const uint32_t (&slot_cost)[NK], uint32_t rem, uint32_t hi, uint32_t lo,
+                                              int lane, bool (&take)[NK])
+{
+    if (!BOUNDS) {
+        hi = 0u;
+        lo = 0xFFFFFFFFu;
+#pragma unroll
+        for (int s = 0; s < NK; s++)
+            if (cw[s] != 0u) {
+                hi = max(hi, key[s]);
+                lo = min(lo, key[s]);
+            }
+        hi = __reduce_max_sync(0xFFFFFFFFu, hi);
+        lo = __reduce_min_sync(0xFFFFFFFFu, lo);
+    }
+    auto from = [&](uint32_t t) {                                 // F(t) | N(t) << 16
+        uint32_t f = 0;
+#pragma unroll
+        for (int s = 0; s < NK; s++) f += key[s] >= t ? cw[s] : 0u;
+        return __reduce_add_sync(0xFFFFFFFFu, f);
+    };
+    uint32_t Kp = 0u, at_lo = from(0u), at_hi;                    // F | N at the two ends of the interval
+    if ((at_lo & 0xFFFFu) > rem) {
+        const uint32_t diff = hi ^ lo;
+        int bit = diff != 0u ? 31 - __clz(diff) : -1;             // the interval is [Kp, Kp + 2^(bit+1))
+        Kp = diff != 0u ? hi & ~((2u << bit) - 1u) : hi;
+        at_hi = 0u;
+        while (bit >= 0 && (at_lo >> 16) - (at_hi >> 16) > 1u) {
+            const uint32_t t = Kp | (1u << bit);
+            const uint32_t e = from(t);
+            if ((e & 0xFFFFu) > rem) {
+                Kp = t;
+                at_lo = e;
+            } else {
+                at_hi = e;
+            }
+            bit--;
+        }
+        if (bit >= 0) {                                           // one raise left in the interval: Kp is its key
+            const uint32_t sh = (uint32_t)bit + 1u;
+            uint32_t only = 0u;
+#pragma unroll
+            for (int s = 0; s < NK; s++)
+                if (cw[s] != 0u && (sh >= 32u || (key[s] >> sh) == (Kp >> sh))) only = key[s];
+            Kp = __reduce_max_sync(0xFFFFFFFFu, only);
+        }
+    } else {
+        at_hi = from(1u);                                         // every raise fits (Kp = 0)
+    }
+    uint32_t left = rem - (at_hi & 0xFFFFu);                      // after every raise with a key above Kp
+    bool open = true;                                             // no raise has been turned down yet
+    const uint32_t below = (1u << lane) - 1u;
+#pragma unroll
+    for (int s = 0; s < NK; s++) {
+        const bool on = cw[s] != 0u, tie = on && key[s] == Kp;
+        const uint32_t ties = __ballot_sync(0xFFFFFFFFu, tie);
+        uint32_t fit = 0u;
+        if (ties != 0u && open) {
+            const uint32_t cnt = (uint32_t)__popc(ties);
+            fit = min(cnt, left / slot_cost[s]);
+            left -= fit * slot_cost[s];
+            open = fit == cnt;                                    // the walk stops at the first raise that does not fit
+        }
+        take[s] = on && (key[s] > Kp || (tie && (uint32_t)__popc(ties & below) < fit));
+    }
+}
+
 }  // namespace general
+
+// Development aid: time stamps of the first CTA's deciders into the (here unused) first descriptor array.
+#ifdef DAF_STAMPS
+#define DAF_GSTAMP(k) do { if (blockIdx.x == 0 && lane == 0 && it < 24u) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); a.flags[it * 8u + (k)] = t_; } } while (0)
+#else
+#define DAF_GSTAMP(k) do { } while (0)
+#endif
 
 template <typename T, int CHUNKS, bool BATCH, bool RELU>
 __global__ void __launch_bounds__(general::kCtaThreads, 2)
@@ -151,6 +240,8 @@ general_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_M
 
     extern __shared__ __align__(16) unsigned char smem[];        // kRing window slots
     __shared__ uint32_t s_gw[kRing];                              // window of iteration i (slot i % kRing)
+    __shared__ uint32_t s_tag[kRing];                             // i + 1 once that window is known
+    __shared__ uint32_t s_claim;                                  // the last iteration whose window somebody has set out to draw
     __shared__ uint32_t s_abort;                                  // a wait ran out, or a window before ours failed: the CTA leaves
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -170,7 +261,9 @@ general_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_M
     if (tid == 0) {
         s_abort = 0u;
         s_gw[0] = atomicAdd(&a.hdr->ticket2, 1u);
-        s_gw[1] = atomicAdd(&a.hdr->ticket2, 1u);
+        s_tag[0] = 1u;
+        for (int r = 1; r < kRing; r++) s_tag[r] = 0u;
+        s_claim = 0u;
     }
     __syncthreads();
 
@@ -206,11 +299,67 @@ general_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_M
     if (warp >= kWorkers) {
         // ============================================================ decider warps: warp d settles windows d, d + 2, ...
         const uint32_t nl = a.m - 1u;                             // raises per group
+        uint32_t pend_it = 0xFFFFFFFFu, pend_gw = 0u, pend_total = 0u;   // the window whose place is still to be looked up
+        // Looks up the pending window's place in the packed buffer (bounded decoupled look-back over the windows
+        // before it), publishes its inclusive prefix, writes its offset and lets the workers have the slot.
+        // block: wait (bounded) for the windows before it; else give up for now when one of them has not published yet.
+        auto finish = [&](bool block) {
+            if (pend_it == 0xFFFFFFFFu) return;
+            WinHead &ph = head(pend_it);
+            const TensorDesc &td = a.t[BATCH ? ph.ti : 0u];
+            const uint32_t w = pend_gw - td.first_window;
+            uint64_t excl = 0;
+            int state = 1;
+            if (w != 0u) {
+                state = lookback<kLookDepth>(a.flags2, pend_gw, td.first_window, lane, block, a.poll_limit, &excl);
+                if (state == 0) return;                           // not yet
+                if (lane == 0)
+                    st_relaxed_u64(a.flags2 + pend_gw, state == 1 ? ((kFlagPrefix << kFlagShift) | (excl + pend_total))
+                                                                   : (kFlagPoison << kFlagShift));
+            }
+            bool store = state == 1;
+            if (store) {
+                if (lane == 0) {
+                    td.woff[w] = excl;
+                    if (w + 1u == td.n_windows) td.woff[w + 1u] = excl + pend_total;
+                }
+                if (excl + pend_total > td.capacity) {            // no room: nothing of the window is stored
+                    store = false;
+                    if (lane == 0) record_error(DAF_ERR_CAPACITY, pend_gw, 12u);
+                }
+            } else {
+                if (state == -2 && lane == 0) record_error(DAF_ERR_TIMEOUT, pend_gw, 13u);   // (a poisoned predecessor has reported itself)
+                st_volatile_shared(&s_abort, 1u);                 // the windows behind a failed one are lost: the CTA leaves
+            }
+            if (lane == 0) {
+                ph.out = td.packed + excl;
+                ph.store = store ? 1u : 0u;
+            }
+            __syncwarp();
+            if (lane == 0) bar_arrive(&ph.ready);                 // (release: the slot is visible to who sees the phase)
+            pend_it = 0xFFFFFFFFu;
+        };
         for (uint32_t it = (uint32_t)warp - kWorkers;; it += kDeciders) {
             WinHead &h = head(it);
-            if (!wait(&h.stats_in, (it / kRing) & 1u, 0xFFFFFFFFu, 11u)) break;
+            // wait for the window's statistics; meanwhile keep trying to place the window this warp settled last
+            bool go = true;
+            for (unsigned polls = 0;; polls++) {
+                if (bar_try_wait(&h.stats_in, (it / kRing) & 1u)) break;
+                if (ld_volatile_shared(&s_abort) != 0u) { go = false; break; }
+                if (polls > a.poll_limit) {
+                    if (lane == 0) record_error(DAF_ERR_TIMEOUT, 0xFFFFFFFFu, 11u);
+                    st_volatile_shared(&s_abort, 1u);
+                    go = false;
+                    break;
+                }
+                if (pend_it != 0xFFFFFFFFu) finish(false);
+                else __nanosleep(200);
+            }
+            finish(true);                                         // (the workers ask for that window next)
+            if (!go) break;
             const uint32_t gw = ld_volatile_shared(&s_gw[it % kRing]);
             if (gw >= a.total_windows) break;
+            DAF_GSTAMP(0);
             const uint32_t ti = tensor_index(gw);
             const TensorDesc &td = a.t[ti];
             const uint32_t w = gw - td.first_window;
@@ -267,13 +416,39 @@ general_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_M
                 uniform = kmin >= kmax;
             }
 
+            DAF_GSTAMP(1);
             // ---- general choice (Sec. 3.4.1): the greedy accepts the longest prefix of the raises, sorted by (key
             // descending, level ascending, group ascending), whose summed cost fits.  F(t), the cost of all raises with
             // key >= t, falls as t grows, so the prefix is every raise with a key above Kp = max{t : F(t) > rem}, and then
             // the raises with key Kp in order while they fit.  Kp is built bit by bit from the top.
             uint32_t Kp = 0u, left = 0u;                          // left: budget after every raise with a key above Kp
             uint32_t fit[3] = {0u, 0u, 0u};                       // raises of level k with key Kp that are accepted
-            if (!uniform) {
+            uint32_t level_reg[4] = {0u, 0u, 0u, 0u};             // up to 128 groups: the levels come out of the register version
+            const bool in_regs = !uniform && n <= 128u;
+            if (in_regs) {
+                // candidates in registers: slot k * Q + q is raise k of group q * 32 + lane
+                auto run = [&](auto qtag) {
+                    constexpr int Q = decltype(qtag)::value;
+                    uint32_t key[3 * Q], cw[3 * Q], slot_cost[3 * Q];
+                    bool take[3 * Q];
+#pragma unroll
+                    for (int k = 0; k < 3; k++)
+#pragma unroll
+                        for (int q = 0; q < Q; q++) {
+                            const uint32_t g = (uint32_t)lane + 32u * q;
+                            const bool on = (uint32_t)k < nl && g < n;
+                            key[k * Q + q] = on ? s_key[k * n_max + g] : 0u;
+                            cw[k * Q + q] = on ? a.cost[k] | 0x10000u : 0u;
+                            slot_cost[k * Q + q] = a.cost[k];
+                        }
+                    accept_prefix<3 * Q, false>(key, cw, slot_cost, rem, 0u, 0u, lane, take);
+#pragma unroll
+                    for (int q = 0; q < Q; q++) level_reg[q] = (uint32_t)take[q] + take[Q + q] + take[2 * Q + q];
+                };
+                if (n <= 64u) run(std::integral_constant<int, 2>{});
+                else run(std::integral_constant<int, 4>{});
+            }
+            if (!uniform && !in_regs) {
                 auto from = [&](uint32_t t) -> uint32_t {         // F(t) | (number of raises with key >= t) << 16
                     uint32_t f = 0u;
                     for (uint32_t k = 0; k < nl; k++) {
@@ -334,6 +509,7 @@ general_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_M
                 }
             }
 
+            DAF_GSTAMP(2);
             // ---- widths, byte offsets of the groups within the window (exclusive scan in group order), records
             uint32_t run = 0u;                                    // bytes of the groups before this round of 32
             uint32_t seen[3] = {0u, 0u, 0u};                      // raises with key Kp met so far, per level
@@ -342,7 +518,9 @@ general_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_M
                 const uint32_t g = g32 + (uint32_t)lane;
                 const bool on = g < n;
                 uint32_t level = ell;
-                if (!uniform) {
+                if (in_regs) {
+                    level = level_reg[(g32 >> 5) & 3u];
+                } else if (!uniform) {
                     level = 0u;
                     for (uint32_t k = 0; k < nl; k++) {
                         const uint32_t key = on ? s_key[k * n_max + g] : 0u;
@@ -381,41 +559,19 @@ general_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_M
             }
             const uint32_t total = run;                           // packed bytes of the window
 
-            // ---- the window's place in the packed buffer: publish its size, look back over the windows before it
-            uint64_t excl = 0;
-            int state = 1;
-            if (w == 0u) {
-                if (lane == 0) st_relaxed_u64(a.flags2 + gw, (kFlagPrefix << kFlagShift) | total);
-            } else {
-                if (lane == 0) st_relaxed_u64(a.flags2 + gw, (kFlagAggregate << kFlagShift) | total);
-                state = lookback<kLookDepth>(a.flags2, gw, td.first_window, lane, true, a.poll_limit, &excl);
-                if (lane == 0)
-                    st_relaxed_u64(a.flags2 + gw, state == 1 ? ((kFlagPrefix << kFlagShift) | (excl + total))
-                                                              : (kFlagPoison << kFlagShift));
-            }
-            bool store = state == 1;
-            if (store) {
-                if (lane == 0) {
-                    td.woff[w] = excl;
-                    if (w + 1u == td.n_windows) td.woff[w + 1u] = excl + total;
-                }
-                if (excl + total > td.capacity) {                 // no room: nothing of the window is stored
-                    store = false;
-                    if (lane == 0) record_error(DAF_ERR_CAPACITY, gw, 12u);
-                }
-            } else {
-                if (state == -2 && lane == 0) record_error(DAF_ERR_TIMEOUT, gw, 13u);   // (a poisoned predecessor has reported itself)
-                st_volatile_shared(&s_abort, 1u);                 // the windows behind a failed one are lost: the CTA leaves
-            }
+            DAF_GSTAMP(3);
+            // ---- publish the window's size at once; its place in the packed buffer is looked up when this warp comes
+            // back for its next window, two iterations from now, when the windows before it have long published theirs
+            if (lane == 0) st_relaxed_u64(a.flags2 + gw, ((w == 0u ? kFlagPrefix : kFlagAggregate) << kFlagShift) | total);
             if (BATCH && lane < 10) philox_store_round_keys(h.rkeys, td.seed, lane);
             if (lane == 0) {
-                h.out = td.packed + excl;
                 h.n_elems = n_elems;
-                h.store = store ? 1u : 0u;
                 h.ti = ti;
             }
-            __syncwarp();
-            if (lane == 0) bar_arrive(&h.ready);                  // (release: the slot is visible to who sees the phase)
+            pend_it = it;
+            pend_gw = gw;
+            pend_total = total;
+            finish(false);                                        // (a tensor's first window, or windows before it that are all placed)
             (void)clamp_any;
         }
         return;
@@ -424,10 +580,27 @@ general_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_M
     // ================================================================ worker warps
     const uint32_t strip0 = (uint32_t)warp * STRIP;               // the strip's first element within its window
     const uint32_t e0 = strip0 + (uint32_t)lane * 8u;             // the lane's first element of chunk 0
-    uint32_t gw_prev = 0xFFFFFFFFu;
+    uint32_t hist[kLag];                                          // windows of the last kLag iterations (hist[0]: the oldest)
+#pragma unroll
+    for (int j = 0; j < kLag; j++) hist[j] = 0xFFFFFFFFu;
+    uint32_t drain = 0;                                           // iterations since the windows ran out
     for (uint32_t it = 0;; it++) {
-        if (tid == 0) st_volatile_shared(&s_gw[(it + 2u) % kRing], atomicAdd(&a.hdr->ticket2, 1u));   // the window of iteration it + 2
-        const uint32_t gw = ld_volatile_shared(&s_gw[it % kRing]);
+        // ---- this iteration's window (drawn by the first worker that finished pass A of the iteration before)
+        uint32_t gw = 0xFFFFFFFFu;
+        if (drain == 0u) {
+            unsigned polls = 0;
+            while (ld_volatile_shared(&s_tag[it % kRing]) != it + 1u) {
+                if (ld_volatile_shared(&s_abort) != 0u) break;
+                if (++polls > a.poll_limit) {
+                    if (lane == 0) record_error(DAF_ERR_TIMEOUT, 0xFFFFFFFFu, 15u);
+                    st_volatile_shared(&s_abort, 1u);
+                    break;
+                }
+                __nanosleep(32);
+            }
+            __threadfence_block();
+            gw = ld_volatile_shared(&s_gw[it % kRing]);
+        }
         const bool valid = gw < a.total_windows;
         if (ld_volatile_shared(&s_abort) != 0u) break;
 
@@ -477,17 +650,28 @@ general_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_M
             }
         }
         __syncwarp();
-        if (lane == 0) bar_arrive(&head(it).stats_in);            // (also for "no more windows": the decider then leaves)
+        // (also for "no more windows": the decider then leaves; the other decider learns it one iteration later)
+        if (lane == 0 && drain < 2u) bar_arrive(&head(it).stats_in);
+        // ---- the next iteration's window: whoever gets here first draws the ticket (just in time, so that windows are
+        // taken up in the order of their numbers, which the look-back relies on)
+        if (lane == 0 && drain == 0u && atomicCAS(&s_claim, it, it + 1u) == it) {
+            const uint32_t next = valid ? atomicAdd(&a.hdr->ticket2, 1u) : 0xFFFFFFFFu;   // (none once the windows have run out)
+            st_volatile_shared(&s_gw[(it + 1u) % kRing], next);
+            __threadfence_block();
+            st_volatile_shared(&s_tag[(it + 1u) % kRing], it + 2u);
+        }
 
-        // ---- pass B: quantize, pack and store the previous window's strip with the records its decider has left
+        // ---- pass B: quantize, pack and store the strip of the window of kLag iterations ago with the records its
+        // decider has left
+        const uint32_t gw_prev = hist[0];
         if (gw_prev != 0xFFFFFFFFu) {
-            WinHead &h = head(it - 1u);
-            if (!wait(&h.ready, ((it - 1u) / kRing) & 1u, gw_prev, 14u)) break;
+            WinHead &h = head(it - kLag);
+            if (!wait(&h.ready, ((it - kLag) / kRing) & 1u, gw_prev, 14u)) break;
             const uint32_t n_elems = h.n_elems;
             if (h.store != 0u) {
                 const TensorDesc &td = a.t[BATCH ? h.ti : 0u];
                 const uint32_t w = gw_prev - td.first_window;
-                const GroupRec *const rec = reinterpret_cast<const GroupRec *>(slot_at(it - 1u, lay.rec));
+                const GroupRec *const rec = reinterpret_cast<const GroupRec *>(slot_at(it - kLag, lay.rec));
                 unsigned char *const out = h.out;
                 const char *const src = reinterpret_cast<const char *>(td.in) + ((uint64_t)w * WE + e0) * EB;
                 char *const act = RELU ? reinterpret_cast<char *>(td.act) + ((uint64_t)w * WE + e0) * EB : nullptr;
@@ -530,14 +714,10 @@ general_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_M
                 }
             }
         }
-        if (!valid) {
-            // no more windows: the other decider waits for the next iteration's statistics; tell it too (the window
-            // of that iteration was drawn after this one, so it does not exist either)
-            __syncwarp();
-            if (lane == 0) bar_arrive(&head(it + 1u).stats_in);
-            break;
-        }
-        gw_prev = gw;
+#pragma unroll
+        for (int j = 0; j + 1 < kLag; j++) hist[j] = hist[j + 1];
+        hist[kLag - 1] = valid ? gw : 0xFFFFFFFFu;
+        if (!valid && ++drain > (uint32_t)kLag) break;            // the last windows have been through pass B
     }
     // A CTA that leaves early poisons the windows it has drawn and not settled, so that nobody waits for them.
     if (tid == 0 && ld_volatile_shared(&s_abort) != 0u) {
