@@ -74,6 +74,9 @@ daf_status make_plan(const daf_params *p, Plan *pl)
     }
     pl->beta_q8 = (uint32_t)floorf(p->bit_budget * 256.0f);
     if (pl->beta_q8 < 256u * pl->S[0]) return DAF_ERR_BUDGET;
+    // a budget above the largest width buys nothing: every group reaches that width either way, and the packed
+    // capacity and the kernels' buffers are sized from the budget
+    if (pl->beta_q8 > 256u * pl->S[pl->m - 1]) pl->beta_q8 = 256u * pl->S[pl->m - 1];
 
     pl->n_groups = p->numel / G;
     pl->n_windows = (pl->n_groups + pl->W - 1) / pl->W;

@@ -94,6 +94,24 @@ static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, uint32_t flags, Com
     return dispatch_general<BATCH, RELU>(dtype, chunks, args, stream);
 }
 
+// Shared-memory carve-up for one launch configuration.
+static SmemLayout make_layout(uint32_t we, uint32_t elem_bytes, uint32_t G, uint32_t window_cap_bytes)
+{
+    auto up = [](uint32_t v) { return (v + 127u) & ~127u; };
+    const uint32_t n_max = we / G, units = we / (G < 256u ? G : 256u);
+    SmemLayout l;
+    uint32_t at = up(we * elem_bytes);
+    l.out0 = at;
+    l.out_stride = up(window_cap_bytes < 16u ? 16u : window_cap_bytes);
+    at += 2u * l.out_stride;
+    l.umn = at; at += up(2u * 4u * units);
+    l.umx = at; at += up(2u * 4u * units);
+    l.sel = at; at += n_max > 64u ? up(4u * kGeneralSelWords) : 0u;
+    l.grp = at; at += up(16u * n_max);
+    l.total = at;
+    return l;
+}
+
 template <int NT> static void fill_common(CompressArgs<NT> &a, const Plan &pl, const daf_params *p, void *ws)
 {
     a.hdr = reinterpret_cast<WorkspaceHeader *>(ws);
@@ -105,6 +123,7 @@ template <int NT> static void fill_common(CompressArgs<NT> &a, const Plan &pl, c
     a.nearest = p->rounding == DAF_ROUND_NEAREST;
     a.poll_limit = (p->flags >> 8) ? (p->flags >> 8) : kMaxPolls;
     a.n_max = pl.We / pl.G;
+    a.bulk_store = pl.G >= 128u;                                  // every group is then a multiple of 16 bytes
     {
         const uint32_t n = a.n_max;
         a.full_rem = (uint32_t)((((uint64_t)pl.beta_q8 * n) >> 8) - (uint64_t)pl.S[0] * n);
@@ -115,6 +134,7 @@ template <int NT> static void fill_common(CompressArgs<NT> &a, const Plan &pl, c
         a.stream_v_lo = pl.v[a.full_ell > 0 ? a.full_ell - 1 : 0];
         a.stream_v_hi = pl.v[a.full_ell];
     }
+    a.lay = make_layout(pl.We, p->dtype == DAF_F32 ? 4u : 2u, pl.G, (uint32_t)((((uint64_t)pl.beta_q8 * pl.W) >> 8) * pl.G / 8));
     for (int k = 0; k < kMaxLevels; k++) {
         a.S[k] = pl.S[k];
         a.cost[k] = pl.cost[k];

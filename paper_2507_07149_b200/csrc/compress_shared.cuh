@@ -21,6 +21,12 @@ struct TensorDesc {
     void *act;               // fused producer (daf_relu_compress): where the activation itself goes
 };
 
+constexpr int kGeneralSelWords = 180;                         // shared words of the general kernel's bit choice with more than 64 groups
+
+struct SmemLayout {          // byte offsets into the general kernel's dynamic shared memory
+    uint32_t out0, out_stride, umn, umx, sel, grp, total;
+};
+
 template <int NT> struct CompressArgs {
     WorkspaceHeader *hdr;
     uint64_t *flags;          // per window: key extremes gathered by the streaming kernel
@@ -28,12 +34,13 @@ template <int NT> struct CompressArgs {
     uint32_t gated;           // the general kernel runs only if the streaming one (or its verifier) asked for it
     uint32_t poll_limit;      // polls after which a bounded wait gives up
     uint32_t total_windows, n_tensors;
-    uint32_t G, log2G, beta_q8, m, nearest, n_max;
+    uint32_t G, log2G, beta_q8, m, nearest, bulk_store, n_max;
     uint32_t full_ell, full_rem, full_rem_after;   // budget arithmetic of a full window (n_max groups)
     uint32_t full_test;       // ... whose groups share a width only if the keys of the levels around full_ell separate
     float stream_v_lo, stream_v_hi;   // importance factors of the raise into level full_ell and of the raise out of it
     uint32_t S[kMaxLevels], cost[kMaxLevels];
     float v[kMaxLevels];
+    SmemLayout lay;
     PhiloxKeys keys;          // round keys of tensor 0 (single-tensor launches)
     TensorDesc t[NT];
 };

@@ -133,7 +133,7 @@ extern "C" daf_status daf_group_offsets(const uint8_t *d_bits, uint64_t n_groups
 {
     if (!d_bits || !d_offsets || !d_ws || (reinterpret_cast<uintptr_t>(d_offsets) & 7u) || (reinterpret_cast<uintptr_t>(d_ws) & 15u))
         return DAF_ERR_INVALID_ARG;
-    if (group_size < 32u || (group_size & (group_size - 1u))) return DAF_ERR_INVALID_ARG;
+    if (group_size < 32u || group_size > 16384u || (group_size & (group_size - 1u))) return DAF_ERR_INVALID_ARG;   // (also keeps a tile's 32-bit byte count in range)
     if (n_groups == 0) return DAF_ERR_SHAPE;
     const uint64_t tiles = (n_groups + kScanTile - 1) / kScanTile;
     if (tiles > 0x7FFFFFFFull) return DAF_ERR_UNSUPPORTED;
