@@ -169,6 +169,13 @@ daf_status daf_decompress_relu_grad(const daf_params *params, const void *d_pack
 daf_status daf_group_offsets(const uint8_t *d_bits, uint64_t n_groups, uint32_t group_size,
                              uint64_t *d_offsets, void *d_ws, uint64_t ws_bytes, daf_stream stream);
 uint64_t   daf_group_offsets_workspace(uint64_t n_groups);
+/* The same with diagnostic flags (DAF_FLAG_KEEP_WORKSPACE, DAF_FLAG_POLL_LIMIT(n); any other bit is an error): for
+ * tests of the bounded wait.  With KEEP_WORKSPACE the caller has prepared d_ws: all zero, except for what the test
+ * plants there (the tile counter is the second 32-bit word, one 64-bit look-back descriptor per tile of 8192 groups
+ * starts at byte 256; state in the top two bits: 0 empty, 1 tile sum, 2 prefix, 3 poison). */
+daf_status daf_group_offsets_diag(const uint8_t *d_bits, uint64_t n_groups, uint32_t group_size,
+                                  uint64_t *d_offsets, void *d_ws, uint64_t ws_bytes, uint32_t flags,
+                                  daf_stream stream);
 
 /*
  * Wait for `stream` and return the device status word of a workspace that was last used by

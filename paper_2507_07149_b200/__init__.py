@@ -68,6 +68,8 @@ SIGNATURES = {
     "daf_decompress": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_uint64, _vp]),
     "daf_decompress_relu_grad": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "daf_group_offsets": (ctypes.c_int, [_vp, ctypes.c_uint64, ctypes.c_uint32, _vp, _vp, ctypes.c_uint64, _vp]),
+    "daf_group_offsets_diag": (ctypes.c_int, [_vp, ctypes.c_uint64, ctypes.c_uint32, _vp, _vp, ctypes.c_uint64, ctypes.c_uint32,
+                                              _vp]),
     "daf_group_offsets_workspace": (ctypes.c_uint64, [ctypes.c_uint64]),
     "daf_poll_status": (ctypes.c_int, [_vp, _vp]),
     "daf_batch_workspace": (ctypes.c_uint64, [ctypes.c_uint32, ctypes.POINTER(daf_params)]),
@@ -208,6 +210,12 @@ def daf_group_offsets_workspace(n_groups: int) -> int:
 def daf_group_offsets(d_bits, n_groups, group_size, d_offsets, d_ws, ws_bytes, stream=None):
     _check(lib().daf_group_offsets(_ptr(d_bits), n_groups, group_size, _ptr(d_offsets), _ptr(d_ws), ws_bytes,
                                    _stream(stream)), "daf_group_offsets")
+
+
+def daf_group_offsets_diag(d_bits, n_groups, group_size, d_offsets, d_ws, ws_bytes, flags, stream=None):
+    """daf_group_offsets with diagnostic flags (FLAG_KEEP_WORKSPACE, flag_poll_limit(n)): for tests of the bounded wait."""
+    _check(lib().daf_group_offsets_diag(_ptr(d_bits), n_groups, group_size, _ptr(d_offsets), _ptr(d_ws), ws_bytes, flags,
+                                        _stream(stream)), "daf_group_offsets_diag")
 
 
 def daf_poll_status(d_workspace, stream=None) -> int:

@@ -550,9 +550,16 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                 int state = 1;
                 if (p_gw != pd.first_window) {
                     state = lookback<kLookDepth>(flags, p_gw, pd.first_window, lane, true, a.poll_limit, &excl);
-                    if (lane == 0)
+                    if (lane == 0) {
+                        // a wait that ran out is reported before the descriptor is poisoned; the windows behind, which
+                        // only meet the poison, stop without a report of their own
+                        if (state == -2) {
+                            record_error(DAF_ERR_TIMEOUT, p_gw);
+                            __threadfence();
+                        }
                         st_relaxed_u64(flags + p_gw, state == 1 ? ((kFlagPrefix << kFlagShift) | (excl + p_total))
                                                                     : (kFlagPoison << kFlagShift));
+                    }
                 }
                 const uint32_t pw = p_gw - pd.first_window;
                 bool skip = state != 1;
@@ -564,9 +571,8 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                     skip = excl + p_total > pd.capacity;
                 }
                 if (skip) {
-                    // (a poisoned predecessor in the quick kernel is a window some CTA gave up on: the full
-                    // kernel redoes the call, nothing to report; a failed copy reports itself)
-                    if (lane == 0 && state != -1) record_error(state == -2 ? DAF_ERR_TIMEOUT : DAF_ERR_CAPACITY, p_gw);
+                    // no room: nothing of the window is stored (a failed wait has reported itself above)
+                    if (lane == 0 && state == 1) record_error(DAF_ERR_CAPACITY, p_gw);
                 } else if (a.bulk_store) {
                     if (lane == 0 && p_total) {
                         bulk_store(pd.packed + excl, src, p_total);

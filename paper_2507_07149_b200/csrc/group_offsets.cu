@@ -14,6 +14,7 @@ struct ScanArgs {
     uint64_t *offsets;
     uint64_t n_groups;
     uint32_t n_tiles, bytes_per_bit;                              // bytes_per_bit = G / 8
+    uint32_t poll_limit;                                          // polls after which the bounded look-back wait gives up
     WorkspaceHeader *hdr;
     uint64_t *flags;
 };
@@ -67,7 +68,7 @@ __global__ void __launch_bounds__(kThreads) group_offsets_kernel(const __grid_co
         if (warp == 0) {
             // decoupled look-back over the tile descriptors (state in the top two bits)
             uint64_t excl = 0;
-            int bad = 0, tmo = 0;
+            int bad = 0;                                          // 1: a tile before this one failed; 2: this tile's wait ran out
             if (tile == 0) {
                 if (lane == 0) st_relaxed_u64(a.flags, (kFlagPrefix << kFlagShift) | total);
             } else {
@@ -83,10 +84,10 @@ __global__ void __launch_bounds__(kThreads) group_offsets_kernel(const __grid_co
                         const unsigned empty_mask = __ballot_sync(0xFFFFFFFFu, st == kFlagEmpty);
                         upto = stop_mask ? ((2u << (__ffs(stop_mask) - 1)) - 1u) : 0xFFFFFFFFu;
                         if ((empty_mask & upto) == 0u) break;
-                        if (++polls > kMaxPolls) { tmo = 1; break; }
+                        if (++polls > a.poll_limit) { bad = 2; break; }
                         __nanosleep(64);
                     }
-                    if (tmo) { bad = 1; break; }
+                    if (bad) break;
                     if (__ballot_sync(0xFFFFFFFFu, (uint32_t)(f >> kFlagShift) == kFlagPoison) & upto) { bad = 1; break; }
                     uint64_t v = ((upto >> lane) & 1u) ? (f & kFlagValueMask) : 0ull;
 #pragma unroll
@@ -95,12 +96,16 @@ __global__ void __launch_bounds__(kThreads) group_offsets_kernel(const __grid_co
                     if (stop_mask) break;
                     idx -= 32;
                 }
-                if (lane == 0)
+                if (lane == 0) {
+                    // the tile whose wait ran out reports it BEFORE it poisons its descriptor; tiles that only meet the
+                    // poison stop without a report of their own
+                    if (bad == 2 && atomicCAS(&a.hdr->status, 0u, (unsigned)DAF_ERR_TIMEOUT) == 0u) a.hdr->fail_window = tile;
+                    __threadfence();
                     st_relaxed_u64(a.flags + tile,
                                    bad ? (kFlagPoison << kFlagShift) : ((kFlagPrefix << kFlagShift) | (excl + total)));
+                }
             }
             if (lane == 0) {
-                if (bad) atomicCAS(&a.hdr->status, 0u, (unsigned)(tmo ? DAF_ERR_TIMEOUT : DAF_ERR_CAPACITY));
                 s_excl = excl;
                 s_failed = bad;
             }
@@ -128,19 +133,21 @@ extern "C" uint64_t daf_group_offsets_workspace(uint64_t n_groups)
     return sizeof(WorkspaceHeader) + 8ull * (tiles ? tiles : 1);
 }
 
-extern "C" daf_status daf_group_offsets(const uint8_t *d_bits, uint64_t n_groups, uint32_t group_size,
-                                        uint64_t *d_offsets, void *d_ws, uint64_t ws_bytes, daf_stream stream)
+static daf_status group_offsets_impl(const uint8_t *d_bits, uint64_t n_groups, uint32_t group_size, uint64_t *d_offsets,
+                                     void *d_ws, uint64_t ws_bytes, uint32_t flags, daf_stream stream)
 {
     if (!d_bits || !d_offsets || !d_ws || (reinterpret_cast<uintptr_t>(d_offsets) & 7u) || (reinterpret_cast<uintptr_t>(d_ws) & 15u))
         return DAF_ERR_INVALID_ARG;
-    if (group_size < 32u || group_size > 16384u || (group_size & (group_size - 1u))) return DAF_ERR_INVALID_ARG;   // (also keeps a tile's 32-bit byte count in range)
+    // (the upper bound also keeps a tile's 32-bit byte count in range)
+    if (group_size < 32u || group_size > 16384u || (group_size & (group_size - 1u))) return DAF_ERR_INVALID_ARG;
+    if (flags & 0xFBu) return DAF_ERR_INVALID_ARG;                // only DAF_FLAG_KEEP_WORKSPACE and DAF_FLAG_POLL_LIMIT mean something here
     if (n_groups == 0) return DAF_ERR_SHAPE;
     const uint64_t tiles = (n_groups + kScanTile - 1) / kScanTile;
     if (tiles > 0x7FFFFFFFull) return DAF_ERR_UNSUPPORTED;
     const uint64_t need = daf_group_offsets_workspace(n_groups);
     if (ws_bytes < need) return DAF_ERR_CAPACITY;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    if (cudaMemsetAsync(d_ws, 0, need, s) != cudaSuccess) return DAF_ERR_CUDA;
+    if (!(flags & DAF_FLAG_KEEP_WORKSPACE) && cudaMemsetAsync(d_ws, 0, need, s) != cudaSuccess) return DAF_ERR_CUDA;
     int max_ctas = 0;
     if (persistent_ctas(reinterpret_cast<const void *>(&group_offsets_kernel), kThreads, 0, &max_ctas) != cudaSuccess) return DAF_ERR_CUDA;
     ScanArgs a;
@@ -149,9 +156,23 @@ extern "C" daf_status daf_group_offsets(const uint8_t *d_bits, uint64_t n_groups
     a.n_groups = n_groups;
     a.n_tiles = (uint32_t)tiles;
     a.bytes_per_bit = group_size / 8u;
+    a.poll_limit = (flags >> 8) ? (flags >> 8) : kMaxPolls;
     a.hdr = reinterpret_cast<WorkspaceHeader *>(d_ws);
     a.flags = reinterpret_cast<uint64_t *>(reinterpret_cast<char *>(d_ws) + sizeof(WorkspaceHeader));
     const uint32_t grid = a.n_tiles < (uint32_t)max_ctas ? a.n_tiles : (uint32_t)max_ctas;
     group_offsets_kernel<<<grid, kThreads, 0, s>>>(a);
     return cudaGetLastError() == cudaSuccess ? DAF_OK : DAF_ERR_CUDA;
+}
+
+extern "C" daf_status daf_group_offsets(const uint8_t *d_bits, uint64_t n_groups, uint32_t group_size,
+                                        uint64_t *d_offsets, void *d_ws, uint64_t ws_bytes, daf_stream stream)
+{
+    return group_offsets_impl(d_bits, n_groups, group_size, d_offsets, d_ws, ws_bytes, 0u, stream);
+}
+
+extern "C" daf_status daf_group_offsets_diag(const uint8_t *d_bits, uint64_t n_groups, uint32_t group_size,
+                                             uint64_t *d_offsets, void *d_ws, uint64_t ws_bytes, uint32_t flags,
+                                             daf_stream stream)
+{
+    return group_offsets_impl(d_bits, n_groups, group_size, d_offsets, d_ws, ws_bytes, flags, stream);
 }

@@ -586,3 +586,75 @@ def test_seeded_tie_heavy_configurations(case):
     label = f"ties/{case}/{dtype}/G{G}/We{We}/{widths}/{beta}"
     xd, c, ref = assert_compress_parity(a, dtype, G, widths, beta, window_elems=We, seed=case, label=label)
     assert_decompress_parity(c, ref, dtype, label)
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# Bounded waits.  Nothing here faults, traps or spins without limit: a window (tile) that is never produced leaves
+# its look-back descriptor empty, the kernels behind it poll a few thousand times, give up, record DAF_ERR_TIMEOUT,
+# poison their own descriptors and return; the context stays usable.
+# ---------------------------------------------------------------------------------------------------------------
+HEADER_BYTES = 256                                                   # status, ticket, fail_window, fail_site, retry, ticket2, ...
+_POISON = np.uint64(3) << np.uint64(62)
+
+
+def _prepared_workspace(nbytes, ticket_word, first_ticket, poison_at=None, descriptors_at=HEADER_BYTES):
+    """An all-zero workspace whose ticket counter starts at `first_ticket` (window / tile 0 is then never handed out),
+    optionally with one pre-poisoned descriptor."""
+    ws = np.zeros(nbytes, np.uint8)
+    ws[4 * ticket_word:4 * ticket_word + 4] = np.array([first_ticket], np.uint32).view(np.uint8)
+    if poison_at is not None:
+        o = descriptors_at + 8 * poison_at
+        ws[o:o + 8] = np.array([_POISON], np.uint64).view(np.uint8)
+    return torch.from_numpy(ws).cuda()
+
+
+@pytest.mark.parametrize("poisoned", [False, True])
+def test_compress_look_back_gives_up_when_a_window_is_never_produced(poisoned):
+    """The general kernel with its ticket counter started at 1: window 0 is never taken, so window 1's look-back
+    finds an empty descriptor (and runs out), or a poisoned one (and stops at once, without a report of its own).
+    Either way nothing is stored, the guard bands stay intact, and the next ordinary call succeeds."""
+    n_windows, G, widths, beta = 8, 256, (1, 2, 4, 8), 3.0
+    a = wl.generate(77, 0, wl.TensorSpec("t", (n_windows * 16384,), "f32", "logscale", 3))
+    x = torch.from_numpy(a).cuda()
+    flags = daf.FLAG_STREAM_NEVER | daf.FLAG_KEEP_WORKSPACE | daf.flag_poll_limit(3000)
+    p = daf.make_params(daf.F32, x.numel(), G, widths, beta, seed=3, flags=flags)
+    sz = daf.daf_sizes(p)
+    guard = 4096
+    packed = torch.full((sz.packed_capacity + guard,), 0xA5, dtype=torch.uint8, device="cuda")
+    woff = torch.full((sz.n_windows + 1 + 8,), -1, dtype=torch.int64, device="cuda")
+    c = daf.alloc_outputs(p, "cuda")
+    # descriptors of the general kernel: the second array behind the header; ticket2 is 32-bit word 5 of the header
+    ws = _prepared_workspace(sz.workspace, 5, 1, poison_at=0 if poisoned else None,
+                             descriptors_at=HEADER_BYTES + 8 * sz.n_windows)
+    daf.daf_compress(p, x, packed, sz.packed_capacity, c.bits, c.min, c.scale, woff, ws, sz.workspace)
+    status = daf.daf_poll_status(ws)
+    assert status == (daf.OK if poisoned else daf.ERR_TIMEOUT)
+    torch.cuda.synchronize()
+    assert bool((packed == 0xA5).all()), "a window behind the missing one was stored"
+    assert bool((woff == -1).all()), "a window behind the missing one got an offset"
+    d = ws[HEADER_BYTES + 8 * sz.n_windows:HEADER_BYTES + 16 * sz.n_windows].cpu().numpy().view(np.uint64)
+    assert all(int(v) >> 62 == 3 for v in d[1:]), "every window behind the missing one must end up poisoned"
+    # the context is fine: the same tensor through an ordinary call
+    assert_compress_parity(a, "f32", G, widths, beta, seed=3, label="after a timed-out call")
+
+
+@pytest.mark.parametrize("poisoned", [False, True])
+def test_group_offsets_look_back_gives_up_when_a_tile_is_never_produced(poisoned):
+    n_groups = 8192 * 6 + 100                                        # 7 tiles
+    rng = np.random.default_rng(11)
+    bits = rng.choice(np.array([1, 2, 4, 8], np.uint8), n_groups)
+    d_bits = torch.from_numpy(bits).cuda()
+    off = torch.full((n_groups + 1 + 8,), -1, dtype=torch.int64, device="cuda")
+    nbytes = daf.daf_group_offsets_workspace(n_groups)
+    ws = _prepared_workspace(nbytes, 1, 1, poison_at=0 if poisoned else None)   # the tile counter is word 1 of the header
+    daf.daf_group_offsets_diag(d_bits, n_groups, 64, off, ws, nbytes, daf.FLAG_KEEP_WORKSPACE | daf.flag_poll_limit(3000))
+    assert daf.daf_poll_status(ws) == (daf.OK if poisoned else daf.ERR_TIMEOUT)
+    torch.cuda.synchronize()
+    assert bool((off == -1).all()), "a tile behind the missing one wrote offsets"
+    d = ws[HEADER_BYTES:HEADER_BYTES + 8 * 7].cpu().numpy().view(np.uint64)
+    assert all(int(v) >> 62 == 3 for v in d[1:])
+    # and the ordinary call on the same workspace is right
+    daf.daf_group_offsets(d_bits, n_groups, 64, off, ws, nbytes)
+    assert daf.daf_poll_status(ws) == daf.OK
+    want = np.concatenate([[0], np.cumsum(bits.astype(np.uint64) * 8)])
+    assert np.array_equal(off[:n_groups + 1].cpu().numpy().view(np.uint64), want)

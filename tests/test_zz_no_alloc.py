@@ -5,6 +5,7 @@ call reuses the same fixed scratch array inside the library.  Collected last on 
 import numpy as np
 import pytest
 
+import oracle
 import paper_2507_07149_b200 as daf
 from paper_2507_07149_b200 import workloads as wl
 
@@ -37,16 +38,29 @@ def test_static_scratch_entry_point_matches_daf_compress_on_two_calls_in_a_row()
         assert daf.daf_poll_status(ws) == daf.OK
         got, _ = _outputs(params)
         status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
-        daf.daf_compress_static(params, x, got["packed"], sz.packed_capacity, got["bits"], got["mn"], got["scale"],
-                                got["woff"], status)
         torch.cuda.synchronize()
-        assert int(status.item()) == daf.OK
+        # the call must not allocate: neither through torch's allocator nor behind its back
+        held, (free, _) = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()
+        daf.daf_compress_static(params, x, got["packed"], sz.packed_capacity, got["bits"], got["mn"], got["scale"],
+                                got["woff"], status if k == 0 else None)     # the status word is optional
+        torch.cuda.synchronize()
+        if k > 0:                                                     # (the first call on a device may load the kernels)
+            assert torch.cuda.memory_allocated() == held and torch.cuda.mem_get_info()[0] == free
+        else:
+            assert int(status.item()) == daf.OK
         total = int(ref["woff"][-1].item())
         assert total > 0 and torch.equal(got["woff"], ref["woff"])
         assert torch.equal(got["bits"], ref["bits"])
         assert torch.equal(got["mn"].view(torch.int32), ref["mn"].view(torch.int32))          # bit-exact, as everywhere
         assert torch.equal(got["scale"].view(torch.int32), ref["scale"].view(torch.int32))
         assert torch.equal(got["packed"][:total], ref["packed"][:total])
+        # and against the CPU oracle, like every other entry point
+        want = oracle.compress(a, G, widths, beta, dtype="bf16" if spec.dtype == "bf16" else None, seed=spec.philox_seed)
+        assert np.array_equal(got["bits"].cpu().numpy(), want.bits)
+        assert np.array_equal(got["mn"].cpu().numpy().view(np.uint32), want.mn.view(np.uint32))
+        assert np.array_equal(got["scale"].cpu().numpy().view(np.uint32), want.scale.view(np.uint32))
+        assert np.array_equal(got["woff"].cpu().numpy().view(np.uint64), want.window_offsets)
+        assert total == want.packed.size and np.array_equal(got["packed"][:total].cpu().numpy(), want.packed)
 
 
 def test_static_scratch_entry_point_rejects_tensors_beyond_its_fixed_size():
