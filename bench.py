@@ -29,9 +29,24 @@ UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per element seen by ncu (dram__bytes_read.sum + dram__bytes_write.sum) for one launch
-# on a 2^27-element fp32 slice of this workload (G = 256, budget 4): profiles/*_cfg5_G256_b4.md.
+# on a 2^27-element fp32 slice of this workload (G = 256, budget 4): profiles/stream_compress_kernel_cfg5_G256_b4.md
+# (546.50 MB read + 66.13 MB written) and profiles/decompress_kernel_cfg5_G256_b4.md (71.91 + 477.73 MB).
 # Traffic grows in proportion to the element count, so it is scaled to the launch being timed.
-NCU_TRAFFIC_BYTES_PER_ELEM = {"compress": 599.04e6 / (1 << 27), "decompress": 549.83e6 / (1 << 27)}
+NCU_TRAFFIC_BYTES_PER_ELEM = {"compress": 612.62e6 / (1 << 27), "decompress": 549.83e6 / (1 << 27)}
+# (The decompress capture is a 512 MiB output: part of its stores still sits in L2 when the kernel ends, so the scaled
+# figure understates the traffic of a full-size launch by the same amount.)
+KERNEL_NAME = {"compress": "stream_compress_kernel", "decompress": "decompress_kernel"}
+# Kernels of this library launched per step on this workload: the streaming compress kernel, its verify kernel, the
+# general compress kernel (which finds nothing to redo and returns), the decompress kernel.
+LAUNCHES_PER_STEP = 4
+
+
+def config_of(w, numel, dtype, G, beta, widths):
+    """The `config` object of the JSON line: the same keys for the CUDA arm and the reference arm."""
+    return {"workload": f"{w.name} ({numel} {dtype} Laplace(0,1) elements per GPU)",
+            "numel_per_gpu": numel, "group_size": G, "bit_budget": beta, "widths": list(widths),
+            "window_elems": 16384,
+            "l2": "inputs (4 GiB) far exceed the 126 MB L2; no flush needed"}
 
 
 def parse():
@@ -164,10 +179,10 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": float(np.mean([d for _, d in vals]) * 1e3), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": args.dtype, "data": "synthetic",
-            "config": {"workload": w.name, "numel": args.numel, "group_size": args.group, "bit_budget": args.budget,
-                       "widths": list(w.widths)},
+            "config": config_of(w, args.numel, args.dtype, args.group, args.budget, w.widths),
             "cpu_baseline": {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
-                             "sample": f"first {a.size} elements of the tensor per step, compress+decompress"},
+                             "sample": f"first {a.size} elements of the tensor per step (a bounded sample of the workload "
+                                       "named in config), compress+decompress"},
             "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
@@ -261,7 +276,7 @@ def run_cuda(args):
     def roof(kernel, ms):
         a = alg / (ms * 1e-3) / 1e9
         tr = NCU_TRAFFIC_BYTES_PER_ELEM[kernel] if profiled else None
-        return {"bound": "hbm", "kernel": f"{kernel}_kernel", "achieved": a, "peak": peak, "unit": "GB/s",
+        return {"bound": "hbm", "kernel": KERNEL_NAME[kernel], "achieved": a, "peak": peak, "unit": "GB/s",
                 "frac": a / peak, "peak_source": peak_src, "frac_of_nominal_8TBs": a / NOMINAL_HBM_GBS,
                 "algorithmic_bytes_per_launch": alg, "avg_launch_ms": ms,
                 "traffic": None if tr is None else tr * spec.numel}
@@ -338,13 +353,10 @@ def run_cuda(args):
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
                 "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": args.dtype, "data": "synthetic",
-                "config": {"workload": f"{w.name} ({spec.numel} {args.dtype} Laplace(0,1) elements per GPU)",
-                           "numel_per_gpu": spec.numel, "group_size": G, "bit_budget": beta, "widths": list(widths),
-                           "window_elems": 16384, "packed_bytes": packed_bytes,
-                           "l2": "inputs (4 GiB) far exceed the 126 MB L2; no flush needed"},
+                "config": config_of(w, spec.numel, args.dtype, G, beta, widths), "packed_bytes": packed_bytes,
                 "compress_gbs": nbytes / (t_c.mean() * 1e-3) / 1e9, "decompress_gbs": nbytes / (t_d.mean() * 1e-3) / 1e9,
                 "compress_ms": float(t_c.mean()), "decompress_ms": float(t_d.mean()),
-                "clocks": clocks, "e2e": e2e, "gpu_launches": 3 * K, "roofline": roofline, "roofline_other": roofline_other,
+                "clocks": clocks, "e2e": e2e, "gpu_launches": LAUNCHES_PER_STEP * K, "roofline": roofline, "roofline_other": roofline_other,
                 "cpu_baseline": cpu,
                 "parity": parity}
         print(json.dumps(line))

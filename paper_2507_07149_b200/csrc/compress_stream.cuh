@@ -161,7 +161,7 @@ stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MA
         float *const mn_p = td.mn + g0, *const scale_p = td.scale + g0;
         // Each group's (minimum, range) is parked in one lane while the chunks are quantized; afterwards one pass over the
         // lanes works out the scales and the importance keys and stores the metadata of the whole strip.
-        float p_mn = 0.0f, p_R = 0.0f, inv_min = __int_as_float(0x7f800000);
+        float p_mn = 0.0f, p_R = 0.0f;
         uint32_t p_idx = 0xFFFFFFFFu;                             // the parked group's index within the strip (none yet)
         // Philox + Eq. 1 + pack + store of chunk c with the group's minimum and 1/scale
         auto quantize = [&](auto chunk_tag, float mn, float inv) {
@@ -214,7 +214,6 @@ stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MA
                     p_R = R;
                     p_idx = (((uint32_t)c << 8) >> log2G) + ((uint32_t)lane >> (log2G - 3u));
                 }
-                if (R > 0.0f) inv_min = fminf(inv_min, inv);
                 quantize(ct, lo, inv);
             });
         } else if (GC == 1) {
@@ -241,8 +240,7 @@ stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MA
                         p_R = R;
                         p_idx = j;
                     }
-                    if (R > 0.0f) inv_min = fminf(inv_min, inv);
-                    mn_pair = lo;
+                        mn_pair = lo;
                     inv_pair = inv;
                 }
                 quantize(ct, mn_pair, inv_pair);
@@ -285,7 +283,6 @@ stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MA
                 p_R = R;
                 p_idx = 0u;
             }
-            if (R > 0.0f) inv_min = fminf(inv_min, inv);
             for_chunks([&](auto ct) { quantize(ct, lo, inv); });
         }
 
@@ -304,8 +301,9 @@ stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MA
             }
             kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
             kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
-            // 1/scale not a normal number: the codes may need the clamp, which this kernel does not have
-            bool give_up = __any_sync(0xFFFFFFFFu, inv_min < 0x1p-126f);
+            // 1/scale = L / R is not a normal number when R passes about 2^126: the codes may then need the clamp, which
+            // this kernel does not have.  (Any range above 2^125 is sent to the general kernel: sooner than needed is fine.)
+            bool give_up = __any_sync(0xFFFFFFFFu, p_R > 0x1p125f);
             if (lane == 0) {
                 if (a.full_test != 0u) {
                     // every raise below level ell must sort ahead of every raise from level ell upward: the window's
