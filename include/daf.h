@@ -18,7 +18,13 @@
  *     status word inside the workspace and read back with daf_poll_status; the
  *     kernels never store out of bounds, trap or spin without limit.
  *   - Device pointers must be 16-byte aligned unless stated otherwise.
- *   - No entry point throws; none keeps global state between calls.
+ *   - No entry point throws.  State the library keeps between calls: a table, one entry per
+ *     (kernel, device), of how many CTAs of that kernel the device holds at once, filled at
+ *     the first launch on each device and guarded by a mutex; and the scratch array of
+ *     daf_compress_static.  Entry points may be called from several threads and on several
+ *     devices at once (work goes to the device that is current in the calling thread) as
+ *     long as calls that overlap on the GPU use different workspaces.  daf_pool and
+ *     daf_store objects are not thread safe: one thread at a time per object.
  *
  * Data layout (all tensors are flat, contiguous, row-major)
  *   group   : G consecutive elements (G a power of two, 32 <= G <= window_elems)
@@ -110,12 +116,15 @@ daf_status daf_sizes(const daf_params *params, uint64_t *n_groups, uint64_t *n_w
  *   d_window_offsets out: n_windows + 1 uint64
  *   d_workspace          : workspace_bytes of scratch, contents irrelevant on entry; also
  *                          holds the device status word afterwards (see daf_poll_status)
- * A fused kernel reads the input once.  (The call enqueues a quick kernel, which handles
- * windows whose groups all end at the same width, and behind it the full kernel, which does
- * nothing unless the quick one met a window it does not handle; then it redoes the call.
- * A call of at most 4096 windows goes to the full kernel alone (one launch is then cheaper than the pair); the
- * environment variable DAF_QUICK_MIN_WINDOWS, read at every call, overrides that number.
- * Every output is final when the call's work on the stream is done.)  If the packed output
+ * The input is read once.  The call enqueues, in this order: a streaming kernel, which
+ * assumes that in every window all groups end at one and the same width (the one the budget
+ * gives a window of equal groups) and writes every output on that assumption while it records
+ * what is needed to check it; a small kernel that checks it for every window and writes the
+ * window offsets; and the general kernel, which returns at once unless the check failed
+ * somewhere and then redoes the whole call with the window-by-window greedy choice.  A call of
+ * at most 4096 windows, or one whose parameters rule out one-width windows, goes to the
+ * general kernel alone; params->flags can force either route.  Both routes give the same
+ * bytes.  Every output is final when the call's work on the stream is done.  If the packed output
  * of a window would pass packed_capacity, nothing of that window is stored and the status
  * word becomes DAF_ERR_CAPACITY.  Inputs must be finite; behaviour on NaN / Inf is unspecified but
  * memory safe.  Calls sharing a workspace must not overlap on the GPU.
@@ -256,6 +265,72 @@ daf_status daf_pool_free(daf_pool *pool, uint64_t handle);
 /* Frees the live allocation with the lowest importance per byte; returns its handle (0 if none). */
 uint64_t   daf_pool_evict_lowest(daf_pool *pool);
 daf_status daf_pool_get_stats(const daf_pool *pool, daf_pool_stats *stats);
+
+/*
+ * Importance-aware store: which saved activations are kept, at which width, and where in a paged
+ * arena (Sec. 3.4).  Host bookkeeping only, like daf_pool: the caller owns the arena, compresses
+ * into the offsets the store hands out, and performs the moves a shrinking budget asks for.
+ *
+ *   Sec. 3.4.1  Greedy choice across activations under a memory AND a time budget: while a budget
+ *               is exceeded, the constraint with the smaller remaining proportion is the tighter
+ *               one, and the activation worth least per unit of that resource gives way (ties:
+ *               least per unit of the other resource).  Width 0 = the activation is not stored.
+ *   Alg. 3      Two ordered indices (red-black trees) over the same activations, keyed
+ *               importance / size and importance / time, always updated together.  Under memory
+ *               pressure an activation not yet placed this iteration gives way by going one width
+ *               down (below the smallest allowed width it is dropped); one that already occupies
+ *               pages is evicted; under time pressure the victim is always evicted.  The paper
+ *               does not say at which end of an index the victim sits; here it is the entry with
+ *               the LEAST importance per unit.
+ *   Sec. 3.4.2  First fit over the free pages.
+ *   Sec. 3.4.4  The arena starts at one step (step_bytes, 100 MB when 0), grows by a step (never
+ *               past the memory budget) when an allocation finds no run, and shrinks in steps when
+ *               daf_store_set_budget lowers the budget: allocations beyond the new end move to the
+ *               first fit below it (reported as moves) or are evicted.
+ *
+ * Sizes: an activation of numel elements at width b counts numel*b/8 + 9*numel/G +
+ * 8*(ceil(numel/16384)+1) bytes (codes, per-group metadata, window offsets), rounded up to pages.
+ * Time: the caller's estimate of what storing the activation costs per iteration (compress +
+ * decompress), in any unit; it counts while the activation is kept, at any width.
+ *
+ * Per iteration: daf_store_estimate for every activation (Alg. 3, pre-iteration estimation, with
+ * the moving-average importance), then, in forward order, daf_store_admit when the activation and
+ * its measured importance arrive (returns the width to compress at and the arena offset), and
+ * daf_store_release once the backward pass has consumed it.
+ * Errors: DAF_ERR_INVALID_ARG for null handles, unknown ids, negative or NaN importance / time,
+ * numel not a multiple of group_size, an activation admitted twice.  Output arrays: *n on entry is
+ * the array's capacity, on return the number of items there were (items beyond the capacity are
+ * not written).
+ */
+typedef struct daf_store daf_store;
+typedef struct daf_store_config {
+    uint64_t mem_budget_bytes;   /* B_mem: upper bound on the arena                          */
+    double   time_budget;        /* B_time, in the unit of the time costs                     */
+    uint64_t page_bytes;         /* 0 => 65536                                                */
+    uint64_t step_bytes;         /* arena growth / shrink step; 0 => 100 MB (100 * 2^20)      */
+    uint32_t width_mask;         /* allowed widths, as in daf_params                          */
+    uint32_t reserved;           /* 0                                                         */
+} daf_store_config;
+typedef struct daf_store_move { uint64_t id, from_offset, to_offset, bytes; } daf_store_move;
+typedef struct daf_store_stats {
+    uint64_t arena_bytes, mem_budget_bytes, used_bytes, planned_bytes;
+    double   time_budget, used_time;
+    uint64_t entries, kept, evictions, resizes, grows, shrinks, moves;
+} daf_store_stats;
+daf_store *daf_store_create(const daf_store_config *config);       /* NULL on bad config */
+void       daf_store_destroy(daf_store *store);
+daf_status daf_store_estimate(daf_store *store, uint64_t id, uint64_t numel, uint32_t group_size,
+                              double importance, double time_cost, uint32_t *width);
+daf_status daf_store_admit(daf_store *store, uint64_t id, double importance, uint32_t *width,
+                           uint64_t *offset /* UINT64_MAX when not stored */,
+                           uint64_t *evicted_ids, uint32_t *n_evicted);
+/* Current width (0 = dropped) and offset (UINT64_MAX = not in pages) of an activation. */
+daf_status daf_store_width(const daf_store *store, uint64_t id, uint32_t *width, uint64_t *offset);
+daf_status daf_store_release(daf_store *store, uint64_t id);
+daf_status daf_store_set_budget(daf_store *store, uint64_t mem_budget_bytes, double time_budget,
+                                daf_store_move *moves, uint32_t *n_moves,
+                                uint64_t *evicted_ids, uint32_t *n_evicted);
+daf_status daf_store_get_stats(const daf_store *store, daf_store_stats *stats);
 
 const char *daf_status_string(daf_status status);
 uint32_t    daf_version(void);

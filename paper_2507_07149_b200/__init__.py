@@ -46,6 +46,21 @@ class daf_pool_stats(ctypes.Structure):
                                                "evictions")]
 
 
+class daf_store_config(ctypes.Structure):
+    _fields_ = [("mem_budget_bytes", ctypes.c_uint64), ("time_budget", ctypes.c_double), ("page_bytes", ctypes.c_uint64),
+                ("step_bytes", ctypes.c_uint64), ("width_mask", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+
+
+class daf_store_move(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_uint64) for n in ("id", "from_offset", "to_offset", "bytes")]
+
+
+class daf_store_stats(ctypes.Structure):
+    _fields_ = ([(n, ctypes.c_uint64) for n in ("arena_bytes", "mem_budget_bytes", "used_bytes", "planned_bytes")]
+                + [("time_budget", ctypes.c_double), ("used_time", ctypes.c_double)]
+                + [(n, ctypes.c_uint64) for n in ("entries", "kept", "evictions", "resizes", "grows", "shrinks", "moves")])
+
+
 class DafError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -82,6 +97,17 @@ SIGNATURES = {
     "daf_pool_free": (ctypes.c_int, [_vp, ctypes.c_uint64]),
     "daf_pool_evict_lowest": (ctypes.c_uint64, [_vp]),
     "daf_pool_get_stats": (ctypes.c_int, [_vp, ctypes.POINTER(daf_pool_stats)]),
+    "daf_store_create": (_vp, [ctypes.POINTER(daf_store_config)]),
+    "daf_store_destroy": (None, [_vp]),
+    "daf_store_estimate": (ctypes.c_int, [_vp, ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_double,
+                                          ctypes.c_double, ctypes.POINTER(ctypes.c_uint32)]),
+    "daf_store_admit": (ctypes.c_int, [_vp, ctypes.c_uint64, ctypes.c_double, ctypes.POINTER(ctypes.c_uint32), _u64p, _u64p,
+                                       ctypes.POINTER(ctypes.c_uint32)]),
+    "daf_store_width": (ctypes.c_int, [_vp, ctypes.c_uint64, ctypes.POINTER(ctypes.c_uint32), _u64p]),
+    "daf_store_release": (ctypes.c_int, [_vp, ctypes.c_uint64]),
+    "daf_store_set_budget": (ctypes.c_int, [_vp, ctypes.c_uint64, ctypes.c_double, ctypes.POINTER(daf_store_move),
+                                            ctypes.POINTER(ctypes.c_uint32), _u64p, ctypes.POINTER(ctypes.c_uint32)]),
+    "daf_store_get_stats": (ctypes.c_int, [_vp, ctypes.POINTER(daf_store_stats)]),
     "daf_status_string": (ctypes.c_char_p, [ctypes.c_int]),
     "daf_version": (ctypes.c_uint32, []),
 }
@@ -370,6 +396,68 @@ class Pool:
     def close(self):
         if self._h:
             lib().daf_pool_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Store:
+    """Importance-aware store (Sec. 3.4 of the paper): per-activation width under a memory and a time budget, two
+    ordered indices, first-fit pages in an arena that follows the budget in steps.  Bookkeeping only."""
+
+    NOT_STORED = (1 << 64) - 1
+    _MAX_OUT = 4096
+
+    def __init__(self, mem_budget_bytes: int, time_budget: float, widths=(1, 2, 4, 8), page_bytes: int = 0,
+                 step_bytes: int = 0):
+        cfg = daf_store_config(mem_budget_bytes, time_budget, page_bytes, step_bytes, width_mask(widths), 0)
+        self._h = lib().daf_store_create(ctypes.byref(cfg))
+        if not self._h:
+            raise DafError(ERR_INVALID_ARG, "daf_store_create")
+
+    def estimate(self, ident: int, numel: int, group_size: int, importance: float, time_cost: float) -> int:
+        w = ctypes.c_uint32()
+        _check(lib().daf_store_estimate(self._h, ident, numel, group_size, importance, time_cost, ctypes.byref(w)),
+               "daf_store_estimate")
+        return int(w.value)
+
+    def admit(self, ident: int, importance: float):
+        """(width, offset or None, ids evicted to make room)"""
+        w, off, n = ctypes.c_uint32(), ctypes.c_uint64(), ctypes.c_uint32(self._MAX_OUT)
+        ev = (ctypes.c_uint64 * self._MAX_OUT)()
+        _check(lib().daf_store_admit(self._h, ident, importance, ctypes.byref(w), ctypes.byref(off), ev, ctypes.byref(n)),
+               "daf_store_admit")
+        return int(w.value), (None if off.value == self.NOT_STORED else int(off.value)), [int(ev[i]) for i in range(min(n.value, self._MAX_OUT))]
+
+    def width(self, ident: int):
+        w, off = ctypes.c_uint32(), ctypes.c_uint64()
+        _check(lib().daf_store_width(self._h, ident, ctypes.byref(w), ctypes.byref(off)), "daf_store_width")
+        return int(w.value), (None if off.value == self.NOT_STORED else int(off.value))
+
+    def release(self, ident: int):
+        _check(lib().daf_store_release(self._h, ident), "daf_store_release")
+
+    def set_budget(self, mem_budget_bytes: int, time_budget: float):
+        """(moves as (id, from, to, bytes), ids evicted)"""
+        nm, ne = ctypes.c_uint32(self._MAX_OUT), ctypes.c_uint32(self._MAX_OUT)
+        mv, ev = (daf_store_move * self._MAX_OUT)(), (ctypes.c_uint64 * self._MAX_OUT)()
+        _check(lib().daf_store_set_budget(self._h, mem_budget_bytes, time_budget, mv, ctypes.byref(nm), ev, ctypes.byref(ne)),
+               "daf_store_set_budget")
+        return ([(int(m.id), int(m.from_offset), int(m.to_offset), int(m.bytes)) for m in mv[:min(nm.value, self._MAX_OUT)]],
+                [int(ev[i]) for i in range(min(ne.value, self._MAX_OUT))])
+
+    def stats(self) -> dict:
+        s = daf_store_stats()
+        _check(lib().daf_store_get_stats(self._h, ctypes.byref(s)), "daf_store_get_stats")
+        return {n: getattr(s, n) for n, _ in daf_store_stats._fields_}
+
+    def close(self):
+        if self._h:
+            lib().daf_store_destroy(self._h)
             self._h = None
 
     def __del__(self):

@@ -16,7 +16,7 @@ HEADERS = [os.path.join(CSRC, h) for h in ("common.cuh", "compress_shared.cuh", 
 
 CU_SOURCES = ["api.cu", "compress.cu", "compress_stream_f32.cu", "compress_stream_f16.cu", "compress_stream_bf16.cu", "compress_general_f32.cu", "compress_general_f16.cu",
               "compress_general_bf16.cu", "decompress.cu", "group_offsets.cu"]
-CXX_SOURCES = ["pool.cpp"]
+CXX_SOURCES = ["pool.cpp", "store.cpp"]
 
 # No fast-math, no flush-to-zero, no fused contraction beyond what the sources write out:
 # results must match IEEE binary32 arithmetic bit for bit.
