@@ -110,7 +110,8 @@ daf_status daf_sizes(const daf_params *params, uint64_t *n_groups, uint64_t *n_w
 /*
  * Compress one tensor (Eq. 1 applied per group; widths chosen greedily per window by
  * importance per bit under the budget, Sec. 3.4.1; codes packed compactly, Sec. 3.3).
- *   d_in             in : numel elements of params->dtype
+ *   d_in             in : numel elements of params->dtype; 32-byte aligned for DAF_F32 (a lane reads
+ *                          eight elements at once), 16-byte aligned otherwise
  *   d_packed         out: packed codes, at most packed_capacity bytes are written
  *   d_bits           out: n_groups bytes        d_min, d_scale  out: n_groups floats each
  *   d_window_offsets out: n_windows + 1 uint64
@@ -288,8 +289,9 @@ daf_status daf_pool_get_stats(const daf_pool *pool, daf_pool_stats *stats);
  *               daf_store_set_budget lowers the budget: allocations beyond the new end move to the
  *               first fit below it (reported as moves) or are evicted.
  *
- * Sizes: an activation of numel elements at width b counts numel*b/8 + 9*numel/G +
- * 8*(ceil(numel/16384)+1) bytes (codes, per-group metadata, window offsets), rounded up to pages.
+ * Sizes: an activation of numel elements at width b counts daf_store_bytes(numel, G, b) bytes: its
+ * window offsets (8*(ceil(numel/16384)+1)), min and scale (4*numel/G each), codes (numel*b/8) and widths
+ * (numel/G), in this order, each part rounded up to 16 bytes; the sum is rounded up to pages.
  * Time: the caller's estimate of what storing the activation costs per iteration (compress +
  * decompress), in any unit; it counts while the activation is kept, at any width.
  *
@@ -297,6 +299,9 @@ daf_status daf_pool_get_stats(const daf_pool *pool, daf_pool_stats *stats);
  * the moving-average importance), then, in forward order, daf_store_admit when the activation and
  * its measured importance arrive (returns the width to compress at and the arena offset), and
  * daf_store_release once the backward pass has consumed it.
+ * daf_store_estimate, daf_store_admit and daf_store_set_budget report the ids that lost their place in
+ * the call (the id itself included when it was dropped): what an evicted id held in the arena is no
+ * longer the caller's, the pages may be handed out again at once.
  * Errors: DAF_ERR_INVALID_ARG for null handles, unknown ids, negative or NaN importance / time,
  * numel not a multiple of group_size, an activation admitted twice.  Output arrays: *n on entry is
  * the array's capacity, on return the number of items there were (items beyond the capacity are
@@ -317,10 +322,12 @@ typedef struct daf_store_stats {
     double   time_budget, used_time;
     uint64_t entries, kept, evictions, resizes, grows, shrinks, moves;
 } daf_store_stats;
+uint64_t   daf_store_bytes(uint64_t numel, uint32_t group_size, uint32_t width);
 daf_store *daf_store_create(const daf_store_config *config);       /* NULL on bad config */
 void       daf_store_destroy(daf_store *store);
 daf_status daf_store_estimate(daf_store *store, uint64_t id, uint64_t numel, uint32_t group_size,
-                              double importance, double time_cost, uint32_t *width);
+                              double importance, double time_cost, uint32_t *width,
+                              uint64_t *evicted_ids, uint32_t *n_evicted);
 daf_status daf_store_admit(daf_store *store, uint64_t id, double importance, uint32_t *width,
                            uint64_t *offset /* UINT64_MAX when not stored */,
                            uint64_t *evicted_ids, uint32_t *n_evicted);

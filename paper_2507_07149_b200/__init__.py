@@ -97,10 +97,12 @@ SIGNATURES = {
     "daf_pool_free": (ctypes.c_int, [_vp, ctypes.c_uint64]),
     "daf_pool_evict_lowest": (ctypes.c_uint64, [_vp]),
     "daf_pool_get_stats": (ctypes.c_int, [_vp, ctypes.POINTER(daf_pool_stats)]),
+    "daf_store_bytes": (ctypes.c_uint64, [ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint32]),
     "daf_store_create": (_vp, [ctypes.POINTER(daf_store_config)]),
     "daf_store_destroy": (None, [_vp]),
     "daf_store_estimate": (ctypes.c_int, [_vp, ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_double,
-                                          ctypes.c_double, ctypes.POINTER(ctypes.c_uint32)]),
+                                          ctypes.c_double, ctypes.POINTER(ctypes.c_uint32), _u64p,
+                                          ctypes.POINTER(ctypes.c_uint32)]),
     "daf_store_admit": (ctypes.c_int, [_vp, ctypes.c_uint64, ctypes.c_double, ctypes.POINTER(ctypes.c_uint32), _u64p, _u64p,
                                        ctypes.POINTER(ctypes.c_uint32)]),
     "daf_store_width": (ctypes.c_int, [_vp, ctypes.c_uint64, ctypes.POINTER(ctypes.c_uint32), _u64p]),
@@ -174,10 +176,17 @@ def dtype_code(t) -> int:
     return {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}[t.dtype]
 
 
-def _stream(stream=None) -> int:
+def _call(fn, ref, stream, *args) -> int:
+    """Calls fn(*args, stream) with the device of tensor `ref` current in this thread (the library launches on the
+    current device) and, unless a stream is given, on torch's current stream OF THAT DEVICE.  Returns the status."""
     torch = _torch()
-    s = torch.cuda.current_stream() if stream is None else stream
-    return int(s.cuda_stream)
+    dev = ref.device
+    if stream is None:
+        stream = torch.cuda.current_stream(dev)
+    if dev.index == torch.cuda.current_device():
+        return int(fn(*args, int(stream.cuda_stream)))
+    with torch.cuda.device(dev):
+        return int(fn(*args, int(stream.cuda_stream)))
 
 
 def _ptr(t) -> int:
@@ -188,18 +197,15 @@ def _ptr(t) -> int:
 def daf_compress(params, d_in, d_packed, packed_capacity, d_bits, d_min, d_scale, d_window_offsets, d_workspace,
                  workspace_bytes, stream=None):
     """Tensors (or None) in, status checked; everything else is the C call."""
-    _check(lib().daf_compress(ctypes.byref(params), _ptr(d_in), _ptr(d_packed), packed_capacity, _ptr(d_bits), _ptr(d_min),
-                              _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_workspace), workspace_bytes, _stream(stream)),
-           "daf_compress")
+    _check(_call(lib().daf_compress, d_in, stream, ctypes.byref(params), _ptr(d_in), _ptr(d_packed), packed_capacity, _ptr(d_bits), _ptr(d_min),
+                              _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_workspace), workspace_bytes), "daf_compress")
 
 
 def daf_relu_compress(params, d_in, d_act, d_packed, packed_capacity, d_bits, d_min, d_scale, d_window_offsets, d_workspace,
                       workspace_bytes, stream=None):
     """Fused producer: d_act = max(d_in, +0) is written and compressed in one pass (d_act may be d_in)."""
-    _check(lib().daf_relu_compress(ctypes.byref(params), _ptr(d_in), _ptr(d_act), _ptr(d_packed), packed_capacity, _ptr(d_bits),
-                                   _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_workspace), workspace_bytes,
-                                   _stream(stream)),
-           "daf_relu_compress")
+    _check(_call(lib().daf_relu_compress, d_in, stream, ctypes.byref(params), _ptr(d_in), _ptr(d_act), _ptr(d_packed), packed_capacity, _ptr(d_bits),
+                                   _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_workspace), workspace_bytes), "daf_relu_compress")
 
 
 STATIC_MAX_WINDOWS = 65536
@@ -210,23 +216,20 @@ def daf_compress_static(params, d_in, d_packed, packed_capacity, d_bits, d_min, 
     """daf_compress for callers that cannot allocate a workspace: the kernel's scratch is a fixed
     array inside the library (at most STATIC_MAX_WINDOWS windows; calls must not overlap on the GPU).
     d_status: optional int32 tensor of one element that receives the device status word."""
-    _check(lib().daf_compress_static(ctypes.byref(params), _ptr(d_in), _ptr(d_packed), packed_capacity, _ptr(d_bits),
-                                     _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_status), _stream(stream)),
-           "daf_compress_static")
+    _check(_call(lib().daf_compress_static, d_in, stream, ctypes.byref(params), _ptr(d_in), _ptr(d_packed), packed_capacity, _ptr(d_bits),
+                                     _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_status)), "daf_compress_static")
 
 
 def daf_decompress_relu_grad(params, d_packed, d_bits, d_min, d_scale, d_window_offsets, d_grad_out, d_grad_in, stream=None):
     """Fused consumer: d_grad_in = d_grad_out where the restored activation is > 0, else 0 (may be in place)."""
-    _check(lib().daf_decompress_relu_grad(ctypes.byref(params), _ptr(d_packed), _ptr(d_bits), _ptr(d_min), _ptr(d_scale),
-                                          _ptr(d_window_offsets), _ptr(d_grad_out), _ptr(d_grad_in), _stream(stream)),
-           "daf_decompress_relu_grad")
+    _check(_call(lib().daf_decompress_relu_grad, d_grad_out, stream, ctypes.byref(params), _ptr(d_packed), _ptr(d_bits), _ptr(d_min), _ptr(d_scale),
+                                          _ptr(d_window_offsets), _ptr(d_grad_out), _ptr(d_grad_in)), "daf_decompress_relu_grad")
 
 
 def daf_decompress(params, d_packed, d_bits, d_min, d_scale, d_window_offsets, d_out, d_workspace=None,
                    workspace_bytes=0, stream=None):
-    _check(lib().daf_decompress(ctypes.byref(params), _ptr(d_packed), _ptr(d_bits), _ptr(d_min), _ptr(d_scale),
-                                _ptr(d_window_offsets), _ptr(d_out), _ptr(d_workspace), workspace_bytes, _stream(stream)),
-           "daf_decompress")
+    _check(_call(lib().daf_decompress, d_out, stream, ctypes.byref(params), _ptr(d_packed), _ptr(d_bits), _ptr(d_min), _ptr(d_scale),
+                                _ptr(d_window_offsets), _ptr(d_out), _ptr(d_workspace), workspace_bytes), "daf_decompress")
 
 
 def daf_group_offsets_workspace(n_groups: int) -> int:
@@ -234,18 +237,16 @@ def daf_group_offsets_workspace(n_groups: int) -> int:
 
 
 def daf_group_offsets(d_bits, n_groups, group_size, d_offsets, d_ws, ws_bytes, stream=None):
-    _check(lib().daf_group_offsets(_ptr(d_bits), n_groups, group_size, _ptr(d_offsets), _ptr(d_ws), ws_bytes,
-                                   _stream(stream)), "daf_group_offsets")
+    _check(_call(lib().daf_group_offsets, d_bits, stream, _ptr(d_bits), n_groups, group_size, _ptr(d_offsets), _ptr(d_ws), ws_bytes), "daf_group_offsets")
 
 
 def daf_group_offsets_diag(d_bits, n_groups, group_size, d_offsets, d_ws, ws_bytes, flags, stream=None):
     """daf_group_offsets with diagnostic flags (FLAG_KEEP_WORKSPACE, flag_poll_limit(n)): for tests of the bounded wait."""
-    _check(lib().daf_group_offsets_diag(_ptr(d_bits), n_groups, group_size, _ptr(d_offsets), _ptr(d_ws), ws_bytes, flags,
-                                        _stream(stream)), "daf_group_offsets_diag")
+    _check(_call(lib().daf_group_offsets_diag, d_bits, stream, _ptr(d_bits), n_groups, group_size, _ptr(d_offsets), _ptr(d_ws), ws_bytes, flags), "daf_group_offsets_diag")
 
 
 def daf_poll_status(d_workspace, stream=None) -> int:
-    return int(lib().daf_poll_status(_ptr(d_workspace), _stream(stream)))
+    return _call(lib().daf_poll_status, d_workspace, stream, _ptr(d_workspace))
 
 
 def _ptr_array(tensors):
@@ -262,17 +263,16 @@ def daf_compress_batch(params_list, d_in, d_packed, capacities, d_bits, d_min, d
     n = len(params_list)
     arr = (daf_params * n)(*params_list)
     caps = (ctypes.c_uint64 * n)(*capacities)
-    _check(lib().daf_compress_batch(n, arr, _ptr_array(d_in), _ptr_array(d_packed), caps, _ptr_array(d_bits),
+    _check(_call(lib().daf_compress_batch, d_in[0], stream, n, arr, _ptr_array(d_in), _ptr_array(d_packed), caps, _ptr_array(d_bits),
                                     _ptr_array(d_min), _ptr_array(d_scale), _ptr_array(d_window_offsets), _ptr(d_workspace),
-                                    workspace_bytes, _stream(stream)), "daf_compress_batch")
+                                    workspace_bytes), "daf_compress_batch")
 
 
 def daf_decompress_batch(params_list, d_packed, d_bits, d_min, d_scale, d_window_offsets, d_out, stream=None):
     n = len(params_list)
     arr = (daf_params * n)(*params_list)
-    _check(lib().daf_decompress_batch(n, arr, _ptr_array(d_packed), _ptr_array(d_bits), _ptr_array(d_min),
-                                      _ptr_array(d_scale), _ptr_array(d_window_offsets), _ptr_array(d_out), _stream(stream)),
-           "daf_decompress_batch")
+    _check(_call(lib().daf_decompress_batch, d_out[0], stream, n, arr, _ptr_array(d_packed), _ptr_array(d_bits), _ptr_array(d_min),
+                                      _ptr_array(d_scale), _ptr_array(d_window_offsets), _ptr_array(d_out)), "daf_decompress_batch")
 
 
 def daf_version() -> int:
@@ -405,6 +405,11 @@ class Pool:
             pass
 
 
+def store_bytes(numel: int, group_size: int, width: int) -> int:
+    """Bytes one activation occupies in a store at the given width (see daf_store_bytes)."""
+    return int(lib().daf_store_bytes(numel, group_size, width))
+
+
 class Store:
     """Importance-aware store (Sec. 3.4 of the paper): per-activation width under a memory and a time budget, two
     ordered indices, first-fit pages in an arena that follows the budget in steps.  Bookkeeping only."""
@@ -419,10 +424,14 @@ class Store:
         if not self._h:
             raise DafError(ERR_INVALID_ARG, "daf_store_create")
 
-    def estimate(self, ident: int, numel: int, group_size: int, importance: float, time_cost: float) -> int:
-        w = ctypes.c_uint32()
-        _check(lib().daf_store_estimate(self._h, ident, numel, group_size, importance, time_cost, ctypes.byref(w)),
-               "daf_store_estimate")
+    def estimate(self, ident: int, numel: int, group_size: int, importance: float, time_cost: float, evicted=None) -> int:
+        """Width planned for the activation; ids that lost their place in the call are appended to `evicted`."""
+        w, n = ctypes.c_uint32(), ctypes.c_uint32(self._MAX_OUT)
+        ev = (ctypes.c_uint64 * self._MAX_OUT)()
+        _check(lib().daf_store_estimate(self._h, ident, numel, group_size, importance, time_cost, ctypes.byref(w), ev,
+                                        ctypes.byref(n)), "daf_store_estimate")
+        if evicted is not None:
+            evicted.extend(int(ev[i]) for i in range(min(n.value, self._MAX_OUT)))
         return int(w.value)
 
     def admit(self, ident: int, importance: float):

@@ -143,6 +143,8 @@ template <int NT> static void fill_common(CompressArgs<NT> &a, const Plan &pl, c
 }
 
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+// the input is read eight elements per lane: 32 bytes at a time for binary32, 16 for the 16-bit types
+static bool aligned_in(const void *p, uint32_t dtype) { return (reinterpret_cast<uintptr_t>(p) & (dtype == DAF_F32 ? 31u : 15u)) == 0; }
 
 }  // namespace daf
 
@@ -157,7 +159,7 @@ extern "C" daf_status daf_compress(const daf_params *params, const void *d_in, v
     daf_status st = make_plan(params, &pl);
     if (st != DAF_OK) return st;
     if (!d_in || !d_packed || !d_bits || !d_min || !d_scale || !d_window_offsets || !d_workspace) return DAF_ERR_INVALID_ARG;
-    if (!aligned16(d_in) || !aligned16(d_packed) || !aligned16(d_workspace) || (reinterpret_cast<uintptr_t>(d_min) & 3u) ||
+    if (!aligned_in(d_in, params->dtype) || !aligned16(d_packed) || !aligned16(d_workspace) || (reinterpret_cast<uintptr_t>(d_min) & 3u) ||
         (reinterpret_cast<uintptr_t>(d_scale) & 3u) || (reinterpret_cast<uintptr_t>(d_window_offsets) & 7u))
         return DAF_ERR_INVALID_ARG;
     if (workspace_bytes < pl.workspace) return DAF_ERR_CAPACITY;
@@ -186,7 +188,7 @@ extern "C" daf_status daf_relu_compress(const daf_params *params, const void *d_
     if (st != DAF_OK) return st;
     if (!d_in || !d_act || !d_packed || !d_bits || !d_min || !d_scale || !d_window_offsets || !d_workspace)
         return DAF_ERR_INVALID_ARG;
-    if (!aligned16(d_in) || !aligned16(d_packed) || !aligned16(d_workspace) || (reinterpret_cast<uintptr_t>(d_act) & 31u) ||
+    if (!aligned_in(d_in, params->dtype) || !aligned16(d_packed) || !aligned16(d_workspace) || (reinterpret_cast<uintptr_t>(d_act) & 31u) ||
         (reinterpret_cast<uintptr_t>(d_min) & 3u) || (reinterpret_cast<uintptr_t>(d_scale) & 3u) ||
         (reinterpret_cast<uintptr_t>(d_window_offsets) & 7u))
         return DAF_ERR_INVALID_ARG;
@@ -222,7 +224,7 @@ extern "C" daf_status daf_compress_static(const daf_params *params, const void *
     daf_status st = make_plan(params, &pl);
     if (st != DAF_OK) return st;
     if (!d_in || !d_packed || !d_bits || !d_min || !d_scale || !d_window_offsets) return DAF_ERR_INVALID_ARG;
-    if (!aligned16(d_in) || !aligned16(d_packed) || (reinterpret_cast<uintptr_t>(d_min) & 3u) ||
+    if (!aligned_in(d_in, params->dtype) || !aligned16(d_packed) || (reinterpret_cast<uintptr_t>(d_min) & 3u) ||
         (reinterpret_cast<uintptr_t>(d_scale) & 3u) || (reinterpret_cast<uintptr_t>(d_window_offsets) & 7u) ||
         (reinterpret_cast<uintptr_t>(d_status) & 3u))
         return DAF_ERR_INVALID_ARG;
@@ -293,7 +295,7 @@ extern "C" daf_status daf_compress_batch(uint32_t n, const daf_params *params, c
         if (p->dtype != params[0].dtype || pl.G != pl0.G || pl.We != pl0.We || p->width_mask != params[0].width_mask ||
             pl.beta_q8 != pl0.beta_q8 || p->rounding != params[0].rounding || p->flags != params[0].flags)
             return DAF_ERR_INVALID_ARG;
-        if (!d_in[i] || !d_packed[i] || !d_bits[i] || !d_min[i] || !d_scale[i] || !d_window_offsets[i] || !aligned16(d_in[i]) ||
+        if (!d_in[i] || !d_packed[i] || !d_bits[i] || !d_min[i] || !d_scale[i] || !d_window_offsets[i] || !aligned_in(d_in[i], params[i].dtype) ||
             !aligned16(d_packed[i]) || (reinterpret_cast<uintptr_t>(d_min[i]) & 3u) ||
             (reinterpret_cast<uintptr_t>(d_scale[i]) & 3u) || (reinterpret_cast<uintptr_t>(d_window_offsets[i]) & 7u))
             return DAF_ERR_INVALID_ARG;

@@ -60,9 +60,7 @@ struct daf_store {
 
     uint64_t bytes_of(const Entry &e, uint32_t level) const
     {
-        if (level == kDropped) return 0;
-        const uint64_t groups = e.numel / e.group_size, windows = (e.numel + 16383) / 16384;
-        return e.numel * widths[level] / 8 + 9 * groups + 8 * (windows + 1);   // packed codes + metadata + window offsets
+        return level == kDropped ? 0 : daf_store_bytes(e.numel, e.group_size, widths[level]);
     }
     uint64_t pages_of(const Entry &e, uint32_t level) const
     {
@@ -176,6 +174,16 @@ uint32_t copy_out(const std::vector<uint64_t> &v, uint64_t *out, uint32_t *n)
 
 }  // namespace
 
+// What one activation occupies: window offsets, min, scale, packed codes, widths, each part rounded up to 16 bytes so
+// that every part can start on the boundary the kernels ask for.
+extern "C" uint64_t daf_store_bytes(uint64_t numel, uint32_t group_size, uint32_t width)
+{
+    if (group_size == 0 || width == 0) return 0;
+    auto up16 = [](uint64_t v) { return (v + 15) & ~15ull; };
+    const uint64_t groups = numel / group_size, windows = (numel + 16383) / 16384;
+    return up16(8 * (windows + 1)) + 2 * up16(4 * groups) + up16(numel * width / 8) + up16(groups);
+}
+
 extern "C" daf_store *daf_store_create(const daf_store_config *cfg)
 {
     if (!cfg || cfg->width_mask == 0 || (cfg->width_mask & ~0x116u)) return nullptr;
@@ -194,7 +202,7 @@ extern "C" daf_store *daf_store_create(const daf_store_config *cfg)
 extern "C" void daf_store_destroy(daf_store *s) { delete s; }
 
 extern "C" daf_status daf_store_estimate(daf_store *s, uint64_t id, uint64_t numel, uint32_t group_size, double importance,
-                                         double time_cost, uint32_t *width)
+                                         double time_cost, uint32_t *width, uint64_t *evicted_ids, uint32_t *n_evicted)
 {
     if (!s || numel == 0 || group_size == 0 || numel % group_size || !(importance >= 0.0) || !(time_cost >= 0.0))
         return DAF_ERR_INVALID_ARG;
@@ -216,9 +224,11 @@ extern "C" daf_status daf_store_estimate(daf_store *s, uint64_t id, uint64_t num
     s->entries[id] = e;
     s->used_time += time_cost;
     s->file(s->entries[id]);
-    enforce(s, nullptr);
+    std::vector<uint64_t> evicted;
+    enforce(s, &evicted);
     const Entry &now = s->entries[id];
     if (width) *width = now.level == kDropped ? 0u : s->widths[now.level];
+    copy_out(evicted, evicted_ids, n_evicted);
     return DAF_OK;
 }
 

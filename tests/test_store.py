@@ -13,7 +13,14 @@ MB = 1 << 20
 
 
 def nbytes(numel, G, b):
-    return numel * b // 8 + 9 * (numel // G) + 8 * ((numel + 16383) // 16384 + 1)
+    up16 = lambda v: (v + 15) & ~15
+    return up16(8 * ((numel + 16383) // 16384 + 1)) + 2 * up16(4 * (numel // G)) + up16(numel * b // 8) + up16(numel // G)
+
+
+def test_size_model():
+    assert daf.store_bytes(1 << 20, 256, 4) == 8 * 65 + 8 + 2 * 4 * 4096 + (1 << 19) + 4096 == nbytes(1 << 20, 256, 4)
+    assert daf.store_bytes(32 * 3, 32, 1) == 16 + 2 * 16 + 16 + 16
+    assert daf.store_bytes(1 << 20, 256, 0) == 0
 
 
 def pages(numel, G, b, page=PAGE):
@@ -84,13 +91,13 @@ class SortStore:
                 return i + 1 - need
         return None
 
-    def estimate(self, ident, numel, G, imp, t):
+    def estimate(self, ident, numel, G, imp, t, evicted=None):
         old = self.e.pop(ident, None)
         if old is not None and old["stored"]:
             self._free(old)
         self.e[ident] = dict(id=ident, numel=numel, G=G, imp=imp, time=t, level=len(self.widths) - 1, stored=False,
                              first=0, n=0)
-        self._enforce(None)
+        self._enforce(evicted)
         a = self.e[ident]
         return 0 if a["level"] is None else self.widths[a["level"]]
 
@@ -241,7 +248,9 @@ def test_admit_updates_keys_stored_activations_are_evicted_not_resized():
     assert st.admit(1, 0.5) == (8, p8 * PAGE, [])                     # measured importance lower than estimated: still fits
     # a third one arrives that was not in the estimate; it is worth more than activation 1, which sits in pages and so
     # cannot shrink: it is evicted, and the newcomer takes its pages
-    st.estimate(2, n, G, 3.0, 1.0)                                   # estimate: 2 is unplaced, worth 3 > 0.5 -> victim is 1
+    gone = []
+    st.estimate(2, n, G, 3.0, 1.0, gone)                             # 2 is unplaced, worth 3 > 0.5 -> the victim is 1
+    assert gone == [1]                                               # ... and the caller is told
     assert st.width(1) == (0, None)
     assert st.admit(2, 3.0) == (8, p8 * PAGE, [])
     s = st.stats()
@@ -323,7 +332,10 @@ def test_random_scenarios_match_the_sort_based_reference(seed):
         imp = (rng.integers(0, 12, n_act) / 4.0).tolist()               # few distinct values: ties on purpose
         tcost = (rng.integers(1, 5, n_act) / 2.0).tolist()
         for i in range(n_act):
-            assert st.estimate(i, numel[i], 128, imp[i], tcost[i]) == ref.estimate(i, numel[i], 128, imp[i], tcost[i])
+            gone, want_gone = [], []
+            assert st.estimate(i, numel[i], 128, imp[i], tcost[i], gone) == \
+                ref.estimate(i, numel[i], 128, imp[i], tcost[i], want_gone)
+            assert gone == want_gone
         assert [st.width(i)[0] for i in range(n_act)] == \
             [0 if ref.e[i]["level"] is None else ref.widths[ref.e[i]["level"]] for i in range(n_act)]
         live = []
