@@ -160,6 +160,22 @@ daf_status daf_decompress(const daf_params *params, const void *d_packed, const 
                           const uint64_t *d_window_offsets, void *d_out, void *d_workspace,
                           uint64_t workspace_bytes, daf_stream stream);
 
+/* The same for other activations.  act:
+ *   DAF_ACT_RELU   as daf_relu_compress.
+ *   DAF_ACT_RELU6  act = min(max(x, +0), 6), written to d_act and compressed.
+ *   DAF_ACT_GELU   d_act receives GELU(x) = x/2 * erfc(-x / sqrt 2), computed in binary32 and rounded to the input's
+ *                  type (within 8 + 2 min(x, 0)^2 units in the last place of binary32, or 2^-40 in absolute terms,
+ *                  of the exact value before that rounding); what is COMPRESSED is x itself, because the backward pass of a GELU
+ *                  needs its input: every other output is that of daf_compress(params, d_in, ...).  d_act must
+ *                  not be (or overlap) d_in.
+ * Any other value of act: DAF_ERR_INVALID_ARG.
+ */
+typedef enum daf_act { DAF_ACT_RELU = 1, DAF_ACT_RELU6 = 2, DAF_ACT_GELU = 3 } daf_act;
+daf_status daf_act_compress(const daf_params *params, uint32_t act, const void *d_in, void *d_act, void *d_packed,
+                            uint64_t packed_capacity, uint8_t *d_bits, float *d_min, float *d_scale,
+                            uint64_t *d_window_offsets, void *d_workspace, uint64_t workspace_bytes,
+                            daf_stream stream);
+
 /* Fused consumer (Sec. 3.2.3): the backward pass of a ReLU whose output was stored compressed.
  * d_grad_in[i] = d_grad_out[i] where the restored activation (exactly what daf_decompress would
  * store, in params->dtype) is > 0, else +0; the restored activation itself is never written.
@@ -169,6 +185,17 @@ daf_status daf_decompress(const daf_params *params, const void *d_packed, const 
 daf_status daf_decompress_relu_grad(const daf_params *params, const void *d_packed, const uint8_t *d_bits,
                                     const float *d_min, const float *d_scale, const uint64_t *d_window_offsets,
                                     const void *d_grad_out, void *d_grad_in, daf_stream stream);
+
+/* The consumer for the activations of daf_act_compress, r being the restored value in params->dtype:
+ *   DAF_ACT_RELU   d_grad_in = d_grad_out where r > 0, else +0
+ *   DAF_ACT_RELU6  d_grad_in = d_grad_out where 0 < r < 6, else +0
+ *   DAF_ACT_GELU   d_grad_in = d_grad_out * (Phi(r) + r phi(r)), r the restored INPUT of the GELU; the factor is
+ *                  computed in binary32 (within 2^-21 of the exact one), the product rounded to params->dtype
+ * Arguments and errors as for daf_decompress_relu_grad.
+ */
+daf_status daf_decompress_act_grad(const daf_params *params, uint32_t act, const void *d_packed, const uint8_t *d_bits,
+                                   const float *d_min, const float *d_scale, const uint64_t *d_window_offsets,
+                                   const void *d_grad_out, void *d_grad_in, daf_stream stream);
 
 /*
  * Device-wide exclusive prefix sum of the group byte lengths G*b_g/8 ("layout

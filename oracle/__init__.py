@@ -111,6 +111,38 @@ def relu(a: np.ndarray, dtype: str | None = None) -> np.ndarray:
     return np.where(a > 0, a, a.dtype.type(0)).astype(a.dtype)
 
 
+def relu6(a: np.ndarray, dtype: str | None = None) -> np.ndarray:
+    """ReLU6 as a fused producer (Sec. 3.2.3): min(max(x, +0), 6) in the array's own type."""
+    if dtype == "bf16" or a.dtype == np.uint16:
+        six = np.uint16(0x40C0)                                    # 6.0; positive bf16 patterns order like integers
+        r = np.where((a & 0x8000) != 0, np.uint16(0), a)
+        return np.where(r > six, six, r).astype(np.uint16)
+    r = np.where(a > 0, a, a.dtype.type(0))
+    return np.where(r > 6, a.dtype.type(6), r).astype(a.dtype)
+
+
+def gelu(x) -> np.ndarray:
+    """GELU(x) = x Phi(x) = x/2 erfc(-x / sqrt 2) in binary64 (the reference the fused producer is held to)."""
+    import math
+    x = np.asarray(x, np.float64)
+    erfc = np.vectorize(math.erfc, otypes=[np.float64])
+    return 0.5 * x * erfc(-x / math.sqrt(2.0))
+
+
+def gelu_grad(x) -> np.ndarray:
+    """d/dx GELU(x) = Phi(x) + x phi(x) in binary64."""
+    import math
+    x = np.asarray(x, np.float64)
+    erfc = np.vectorize(math.erfc, otypes=[np.float64])
+    return 0.5 * erfc(-x / math.sqrt(2.0)) + x * np.exp(-0.5 * x * x) / math.sqrt(2.0 * math.pi)
+
+
+def to_bf16_bits(x) -> np.ndarray:
+    """binary32 -> bf16 bit patterns, round to nearest even (the oracle's own conversion, element by element)."""
+    f = lib().daf_oracle_float_to_bf16
+    return np.array([f(float(v)) for v in np.asarray(x, np.float32).reshape(-1)], np.uint16)
+
+
 def stats(x, G: int):
     x = _c(x, np.float32).reshape(-1)
     ng = x.size // G

@@ -79,6 +79,10 @@ SIGNATURES = {
                                     ctypes.c_uint64, _vp]),
     "daf_relu_compress": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, _vp, ctypes.c_uint64, _vp, _vp, _vp, _vp, _vp,
                                          ctypes.c_uint64, _vp]),
+    "daf_act_compress": (ctypes.c_int, [ctypes.POINTER(daf_params), ctypes.c_uint32, _vp, _vp, _vp, ctypes.c_uint64, _vp, _vp,
+                                        _vp, _vp, _vp, ctypes.c_uint64, _vp]),
+    "daf_decompress_act_grad": (ctypes.c_int, [ctypes.POINTER(daf_params), ctypes.c_uint32, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
+                                               _vp]),
     "daf_compress_static": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, ctypes.c_uint64, _vp, _vp, _vp, _vp, _vp, _vp]),
     "daf_decompress": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_uint64, _vp]),
     "daf_decompress_relu_grad": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -208,6 +212,25 @@ def daf_relu_compress(params, d_in, d_act, d_packed, packed_capacity, d_bits, d_
                                    _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_workspace), workspace_bytes), "daf_relu_compress")
 
 
+ACT_RELU, ACT_RELU6, ACT_GELU = 1, 2, 3
+
+
+def daf_act_compress(params, act, d_in, d_act, d_packed, packed_capacity, d_bits, d_min, d_scale, d_window_offsets, d_workspace,
+                     workspace_bytes, stream=None):
+    """Fused producer for ReLU / ReLU6 / GELU: d_act = act(d_in) written in the same pass that compresses (the
+    activation for ReLU and ReLU6, the input for GELU)."""
+    _check(_call(lib().daf_act_compress, d_in, stream, ctypes.byref(params), act, _ptr(d_in), _ptr(d_act), _ptr(d_packed),
+                 packed_capacity, _ptr(d_bits), _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_workspace),
+                 workspace_bytes), "daf_act_compress")
+
+
+def daf_decompress_act_grad(params, act, d_packed, d_bits, d_min, d_scale, d_window_offsets, d_grad_out, d_grad_in, stream=None):
+    """Fused consumer: the gradient of the activation from its compressed form (may be in place)."""
+    _check(_call(lib().daf_decompress_act_grad, d_grad_out, stream, ctypes.byref(params), act, _ptr(d_packed), _ptr(d_bits),
+                 _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_grad_out), _ptr(d_grad_in)),
+           "daf_decompress_act_grad")
+
+
 STATIC_MAX_WINDOWS = 65536
 
 
@@ -333,20 +356,21 @@ def compress(x, group_size: int, widths, bit_budget: float, *, window_elems: int
 
 def relu_compress(x, group_size: int, widths, bit_budget: float, *, rounding: int = ROUND_STOCHASTIC, seed: int = 0,
                   elem_index_base: int = 0, flags: int | None = None, inplace: bool = False, out: CompressedTensor | None = None,
-                  check: bool = False, stream=None):
-    """(relu(x), compressed relu(x)) in one pass over x (daf_relu_compress); ``inplace`` overwrites x."""
+                  check: bool = False, stream=None, act: int = ACT_RELU):
+    """(act(x), compressed form) in one pass over x (daf_act_compress); ``inplace`` overwrites x.  The compressed
+    form holds act(x) for ReLU and ReLU6, and x itself for GELU."""
     if not x.is_cuda or not x.is_contiguous():
         raise ValueError("relu_compress expects a contiguous CUDA tensor")
     params = make_params(dtype_code(x), x.numel(), group_size, widths, bit_budget, rounding=rounding, seed=seed,
                          elem_index_base=elem_index_base, flags=flags)
     c = out if out is not None else alloc_outputs(params, x.device, x.shape)
     c.params = params
-    act = x if inplace else _torch().empty_like(x)
-    daf_relu_compress(params, x, act, c.packed, c.sizes.packed_capacity, c.bits, c.min, c.scale, c.window_offsets,
-                      c.workspace, c.sizes.workspace, stream)
+    y = x if inplace else _torch().empty_like(x)
+    daf_act_compress(params, act, x, y, c.packed, c.sizes.packed_capacity, c.bits, c.min, c.scale, c.window_offsets,
+                     c.workspace, c.sizes.workspace, stream)
     if check:
-        _check(daf_poll_status(c.workspace, stream), "daf_relu_compress (device status)")
-    return act, c
+        _check(daf_poll_status(c.workspace, stream), "daf_act_compress (device status)")
+    return y, c
 
 
 def decompress(c: CompressedTensor, out=None, stream=None):
@@ -358,14 +382,14 @@ def decompress(c: CompressedTensor, out=None, stream=None):
     return out
 
 
-def relu_grad(c: CompressedTensor, grad_out, out=None, stream=None):
-    """Gradient of a ReLU from its compressed output: grad_out where the restored output is > 0."""
+def relu_grad(c: CompressedTensor, grad_out, out=None, stream=None, act: int = ACT_RELU):
+    """Gradient of the activation from its compressed form (daf_decompress_act_grad)."""
     torch = _torch()
     if not grad_out.is_contiguous():
         grad_out = grad_out.contiguous()
     if out is None:
         out = torch.empty_like(grad_out)
-    daf_decompress_relu_grad(c.params, c.packed, c.bits, c.min, c.scale, c.window_offsets, grad_out, out, stream)
+    daf_decompress_act_grad(c.params, act, c.packed, c.bits, c.min, c.scale, c.window_offsets, grad_out, out, stream)
     return out
 
 

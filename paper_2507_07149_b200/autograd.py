@@ -44,7 +44,7 @@ import weakref
 
 import torch
 
-from . import (BATCH_MAX, ROUND_STOCHASTIC, CompressedTensor, Store, _check, daf_batch_workspace, daf_compress_batch,
+from . import (ACT_GELU, ACT_RELU, ACT_RELU6, BATCH_MAX, ROUND_STOCHASTIC, CompressedTensor, Store, _check, daf_batch_workspace, daf_compress_batch,
                daf_poll_status, daf_sizes, decompress, dtype_code, make_params, store_bytes)
 
 _DTYPES = (torch.float32, torch.float16, torch.bfloat16)
@@ -336,22 +336,23 @@ class saved_activation_compression(torch.autograd.graph.saved_tensors_hooks):
 
 
 class _ReluSavedCompressed(torch.autograd.Function):
-    """ReLU whose output is written and compressed in one pass (daf_relu_compress); the backward pass
-    masks the gradient with the output restored from the packed form (daf_decompress_relu_grad: the
-    restored output is never written)."""
+    """Activation whose output is written and whose saved tensor is compressed in one pass (daf_act_compress); the
+    backward pass forms the gradient from the packed form (daf_decompress_act_grad: the restored tensor is never
+    written).  ReLU and ReLU6 keep their output, GELU its input."""
 
     @staticmethod
     def forward(ctx, x, module):
         from . import relu_compress
         xin = _aligned_contiguous(x)
         act, c = relu_compress(xin, module.group_size, module.widths, module.bit_budget, rounding=module.rounding,
-                               seed=module.seed, elem_index_base=module._next_index, check=module.trim)
+                               seed=module.seed, elem_index_base=module._next_index, check=module.trim, act=module.act)
         module._next_index += (x.numel() + 7) & ~7
         if module.trim:
             c.packed = c.packed[:max(c.packed_bytes(), 16)].clone()
         c.workspace = None
         ctx.saved = c
         ctx.shape = x.shape
+        ctx.act = module.act
         return act.view(x.shape)
 
     @staticmethod
@@ -366,7 +367,7 @@ class _ReluSavedCompressed(torch.autograd.Function):
             g = g.contiguous() if not g.is_contiguous() else g.clone()
             if g.data_ptr() % _ALIGN:
                 g = g.clone()
-        return relu_grad(c, g).view(ctx.shape), None                # one pass: packed + gradient in, gradient out
+        return relu_grad(c, g, act=ctx.act).view(ctx.shape), None   # one pass: packed + gradient in, gradient out
 
 
 class CompressedReLU(torch.nn.Module):
@@ -376,6 +377,9 @@ class CompressedReLU(torch.nn.Module):
     not contiguous or not 32-byte aligned is copied first.  ``trim`` copies the used part of the packed buffer into
     a right-sized allocation, at the price of one device-to-host read per call; without it the buffer keeps the
     capacity the budget guarantees and the forward pass never waits for the device."""
+
+    act = ACT_RELU
+    _plain = staticmethod(torch.relu)
 
     def __init__(self, group_size: int = 256, widths=(1, 2, 4, 8), bit_budget: float = 4.0, *, seed: int = 0,
                  rounding: int = ROUND_STOCHASTIC, min_numel: int = 16384, trim: bool = False):
@@ -390,4 +394,17 @@ class CompressedReLU(torch.nn.Module):
     def forward(self, x):
         ok = (x.is_cuda and x.dtype in _DTYPES and x.numel() >= self.min_numel and x.numel() % self.group_size == 0
               and torch.is_grad_enabled() and x.requires_grad)
-        return _ReluSavedCompressed.apply(x, self) if ok else torch.relu(x)
+        return _ReluSavedCompressed.apply(x, self) if ok else self._plain(x)
+
+
+class CompressedReLU6(CompressedReLU):
+    """ReLU6 with its output kept compressed; the gradient passes where the restored output is strictly inside (0, 6)."""
+    act = ACT_RELU6
+    _plain = staticmethod(torch.nn.functional.relu6)
+
+
+class CompressedGELU(CompressedReLU):
+    """GELU (erf form) that keeps its INPUT compressed; the backward pass multiplies the gradient by GELU' at the
+    restored input."""
+    act = ACT_GELU
+    _plain = staticmethod(torch.nn.functional.gelu)

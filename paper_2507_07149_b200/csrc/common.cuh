@@ -287,4 +287,27 @@ daf_status make_plan(const daf_params *p, Plan *plan);
 // (kernel, device) pair and are remembered per pair; safe to call from several host threads.
 cudaError_t persistent_ctas(const void *kernel, int threads, int dyn_smem, int *ctas);
 
+// Activations of the fused producers and consumers (Sec. 3.2.3 of the paper: the statistics are taken where the
+// activation is produced, the restored value is used where the gradient is formed).
+//   ReLU   y = max(x, +0)            what is compressed: y     gradient: g where restored y > 0
+//   ReLU6  y = min(max(x, +0), 6)    what is compressed: y     gradient: g where 0 < restored y < 6
+//   GELU   y = x Phi(x) = x/2 erfc(-x / sqrt 2)    what is compressed: x (the backward pass needs the input)
+//          gradient: g * (Phi(x) + x phi(x)) at the restored x
+enum : int { kActNone = 0, kActRelu = 1, kActRelu6 = 2, kActGelu = 3 };
+__device__ __forceinline__ float gelu_f(float x) { return (0.5f * x) * erfcf(-0.70710678118654752f * x); }
+__device__ __forceinline__ float gelu_grad_f(float x)
+{
+    return 0.5f * erfcf(-0.70710678118654752f * x) + (x * 0.3989422804014327f) * expf(-0.5f * (x * x));
+}
+// x: the chunk as loaded; afterwards x = what is compressed, y = what the producer writes out.
+template <int ACT> __device__ __forceinline__ void activate8(float (&x)[8], float (&y)[8])
+{
+#pragma unroll
+    for (int i = 0; i < 8; i++) {
+        if (ACT == kActRelu) x[i] = fmaxf(x[i], 0.0f);
+        if (ACT == kActRelu6) x[i] = fminf(fmaxf(x[i], 0.0f), 6.0f);
+        y[i] = ACT == kActGelu ? gelu_f(x[i]) : x[i];
+    }
+}
+
 }  // namespace daf

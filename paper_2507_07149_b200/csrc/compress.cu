@@ -72,7 +72,7 @@ template <int NT> static uint64_t one_width_total(const CompressArgs<NT> &a, con
 // launch-bound, and one launch is cheaper than two), only the general kernel is launched.
 constexpr uint32_t kStreamMinWindows = 4096;                     // measured break-even
 
-template <bool BATCH, bool RELU = false>
+template <bool BATCH, int ACT = kActNone>
 static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, uint32_t flags, CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
                             cudaStream_t stream)
 {
@@ -85,13 +85,13 @@ static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, uint32_t flags, Com
     args.flags2 = args.flags + args.total_windows;
     args.gated = try_stream ? 1u : 0u;
     if (try_stream) {
-        cudaError_t e = dispatch_stream<BATCH, RELU>(dtype, chunks, args, stream);
+        cudaError_t e = dispatch_stream<BATCH, ACT>(dtype, chunks, args, stream);
         if (e != cudaSuccess) return e;
         verify_stream_kernel<BATCH ? DAF_BATCH_MAX : 1><<<(args.total_windows + 255u) / 256u, 256, 0, stream>>>(args, chunks * 4096u);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
-    return dispatch_general<BATCH, RELU>(dtype, chunks, args, stream);
+    return dispatch_general<BATCH, ACT>(dtype, chunks, args, stream);
 }
 
 // Shared-memory carve-up for one launch configuration.
@@ -178,11 +178,15 @@ extern "C" daf_status daf_compress(const daf_params *params, const void *d_in, v
     return dispatch<false>(params->dtype, pl.chunks, params->flags, a, s) == cudaSuccess ? DAF_OK : DAF_ERR_CUDA;
 }
 
-extern "C" daf_status daf_relu_compress(const daf_params *params, const void *d_in, void *d_act, void *d_packed,
-                                        uint64_t packed_capacity, uint8_t *d_bits, float *d_min, float *d_scale,
-                                        uint64_t *d_window_offsets, void *d_workspace, uint64_t workspace_bytes,
-                                        daf_stream stream)
+extern "C" daf_status daf_act_compress(const daf_params *params, uint32_t act, const void *d_in, void *d_act, void *d_packed,
+                                       uint64_t packed_capacity, uint8_t *d_bits, float *d_min, float *d_scale,
+                                       uint64_t *d_window_offsets, void *d_workspace, uint64_t workspace_bytes,
+                                       daf_stream stream)
 {
+    if (act != DAF_ACT_RELU && act != DAF_ACT_RELU6 && act != DAF_ACT_GELU) return DAF_ERR_INVALID_ARG;
+    // ReLU and ReLU6 may run in place (applying them twice changes nothing, so a second pass over the call still reads
+    // what it needs); GELU may not: the input is what is compressed
+    if (act == DAF_ACT_GELU && d_act == d_in) return DAF_ERR_INVALID_ARG;
     Plan pl;
     daf_status st = make_plan(params, &pl);
     if (st != DAF_OK) return st;
@@ -205,7 +209,20 @@ extern "C" daf_status daf_relu_compress(const daf_params *params, const void *d_
                         (uint32_t)pl.n_windows, d_act};
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     if (!(params->flags & DAF_FLAG_KEEP_WORKSPACE) && cudaMemsetAsync(d_workspace, 0, pl.workspace, s) != cudaSuccess) return DAF_ERR_CUDA;
-    return dispatch<false, true>(params->dtype, pl.chunks, params->flags, a, s) == cudaSuccess ? DAF_OK : DAF_ERR_CUDA;
+    cudaError_t e;
+    if (act == DAF_ACT_RELU) e = dispatch<false, kActRelu>(params->dtype, pl.chunks, params->flags, a, s);
+    else if (act == DAF_ACT_RELU6) e = dispatch<false, kActRelu6>(params->dtype, pl.chunks, params->flags, a, s);
+    else e = dispatch<false, kActGelu>(params->dtype, pl.chunks, params->flags, a, s);
+    return e == cudaSuccess ? DAF_OK : DAF_ERR_CUDA;
+}
+
+extern "C" daf_status daf_relu_compress(const daf_params *params, const void *d_in, void *d_act, void *d_packed,
+                                        uint64_t packed_capacity, uint8_t *d_bits, float *d_min, float *d_scale,
+                                        uint64_t *d_window_offsets, void *d_workspace, uint64_t workspace_bytes,
+                                        daf_stream stream)
+{
+    return daf_act_compress(params, DAF_ACT_RELU, d_in, d_act, d_packed, packed_capacity, d_bits, d_min, d_scale,
+                            d_window_offsets, d_workspace, workspace_bytes, stream);
 }
 
 // ------------------------------------------------------------------------------------------

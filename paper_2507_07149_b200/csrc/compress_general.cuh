@@ -36,18 +36,19 @@ namespace daf {
 // Staged window -> registers, then min / max per unit of LPU lanes (a full warp uses the
 // redux instruction) written to shared memory.  Chunks past a ragged window's end read
 // stale bytes; their results are never used.
-template <typename T, int CHUNKS, int LPU, bool RELU>
+template <typename T, int CHUNKS, int LPU, int ACT>
 __device__ __forceinline__ void load_and_reduce(const unsigned char *stage, int warp, int lane, float (&x)[CHUNKS][8],
                                                 float *s_umn, float *s_umx)
 {
     constexpr int kChunkBytes = 256 * Elem<T>::kBytes;
 #pragma unroll
     for (int c = 0; c < CHUNKS; c++) load8_staged<T>(stage + (warp * CHUNKS + c) * kChunkBytes, lane, x[c]);
-    if (RELU) {                                                   // fused producer: what is compressed is max(x, +0)
+    if (ACT == kActRelu || ACT == kActRelu6) {                   // fused producer: what is compressed is the activation
 #pragma unroll
-        for (int c = 0; c < CHUNKS; c++)
-#pragma unroll
-            for (int i = 0; i < 8; i++) x[c][i] = fmaxf(x[c][i], 0.0f);
+        for (int c = 0; c < CHUNKS; c++) {
+            float y[8];
+            activate8<ACT>(x[c], y);
+        }
     }
 #pragma unroll
     for (int c = 0; c < CHUNKS; c++) {
@@ -235,7 +236,7 @@ struct Budget {
 // WIDTHS: at most 64 groups per window (groups of 256 elements or more at the default window): the
 // widths warp settles every window, of one width or mixed; otherwise the compute warps that own
 // group records do (mixed windows: radix select on the keys).
-template <typename T, int CHUNKS, bool BATCH, bool WIDTHS, bool RELU>
+template <typename T, int CHUNKS, bool BATCH, bool WIDTHS, int ACT>
 __global__ void __launch_bounds__(kCompressThreads, 2)
 compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> a)
 {
@@ -625,18 +626,28 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
 
         // ---------------------------------------------------------------- staged window -> registers, unit min / max
         float x[CHUNKS][8];
-        if (G >= 256u) load_and_reduce<T, CHUNKS, 32, RELU>(s_stage, warp, lane, x, umn, umx);
-        else if (G == 128u) load_and_reduce<T, CHUNKS, 16, RELU>(s_stage, warp, lane, x, umn, umx);
-        else if (G == 64u) load_and_reduce<T, CHUNKS, 8, RELU>(s_stage, warp, lane, x, umn, umx);
-        else load_and_reduce<T, CHUNKS, 4, RELU>(s_stage, warp, lane, x, umn, umx);
-        if (RELU && !lost) {
+        if (G >= 256u) load_and_reduce<T, CHUNKS, 32, ACT>(s_stage, warp, lane, x, umn, umx);
+        else if (G == 128u) load_and_reduce<T, CHUNKS, 16, ACT>(s_stage, warp, lane, x, umn, umx);
+        else if (G == 64u) load_and_reduce<T, CHUNKS, 8, ACT>(s_stage, warp, lane, x, umn, umx);
+        else load_and_reduce<T, CHUNKS, 4, ACT>(s_stage, warp, lane, x, umn, umx);
+        if (ACT != kActNone && !lost) {
             // the activation goes out as it is compressed: one 8-element store per lane and chunk (the
             // window was staged whole before, so the output may be the input buffer)
             char *const act = reinterpret_cast<char *>(td.act) + wbase * Elem<T>::kBytes;
 #pragma unroll
             for (int c = 0; c < CHUNKS; c++) {
                 const uint32_t e = e0 + 256u * c;
-                if (e < n_elems) Elem<T>::store8(act + (size_t)e * Elem<T>::kBytes, x[c]);
+                if (e < n_elems) {
+                    if (ACT == kActGelu) {                        // x stays what is compressed; GELU(x) goes out
+                        float keep[8], y[8];
+#pragma unroll
+                        for (int i = 0; i < 8; i++) keep[i] = x[c][i];
+                        activate8<ACT>(keep, y);
+                        Elem<T>::store8(act + (size_t)e * Elem<T>::kBytes, y);
+                    } else {
+                        Elem<T>::store8(act + (size_t)e * Elem<T>::kBytes, x[c]);
+                    }
+                }
             }
         }
         // ---------------------------------------------------------------- widths, first try: one width for all
@@ -988,27 +999,27 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
 // ------------------------------------------------------------------------------------------
 // Launch
 // ------------------------------------------------------------------------------------------
-template <typename T, int CHUNKS, bool BATCH, bool WIDTHS, bool RELU = false>
+template <typename T, int CHUNKS, bool BATCH, bool WIDTHS, int ACT = kActNone>
 static cudaError_t launch(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
     const int smem = (int)args.lay.total;
     int ctas = 0;
-    const cudaError_t e = persistent_ctas(reinterpret_cast<const void *>(&compress_kernel<T, CHUNKS, BATCH, WIDTHS, RELU>),
+    const cudaError_t e = persistent_ctas(reinterpret_cast<const void *>(&compress_kernel<T, CHUNKS, BATCH, WIDTHS, ACT>),
                                           kCompressThreads, smem, &ctas);
     if (e != cudaSuccess) return e;
     const uint32_t grid = args.total_windows < (uint32_t)ctas ? args.total_windows : (uint32_t)ctas;
-    compress_kernel<T, CHUNKS, BATCH, WIDTHS, RELU><<<grid, kCompressThreads, smem, stream>>>(args);
+    compress_kernel<T, CHUNKS, BATCH, WIDTHS, ACT><<<grid, kCompressThreads, smem, stream>>>(args);
     return cudaGetLastError();
 }
 
 
-template <typename T, bool BATCH, bool RELU>
+template <typename T, bool BATCH, int ACT>
 cudaError_t dispatch_general_t(uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
     const bool widths = args.n_max <= 64u;                        // few enough groups for the widths warp
-    if constexpr (RELU) {                                         // fused producer: single tensor, default window (chunks == 4)
+    if constexpr (ACT != kActNone) {                              // fused producer: single tensor, default window (chunks == 4)
         static_assert(!BATCH, "the fused producer is compiled for single-tensor launches only");
-        return widths ? launch<T, 4, false, true, true>(args, stream) : launch<T, 4, false, false, true>(args, stream);
+        return widths ? launch<T, 4, false, true, ACT>(args, stream) : launch<T, 4, false, false, ACT>(args, stream);
     } else {
         switch (chunks) {
         case 1: return widths ? launch<T, 1, BATCH, true>(args, stream) : launch<T, 1, BATCH, false>(args, stream);
@@ -1019,8 +1030,10 @@ cudaError_t dispatch_general_t(uint32_t chunks, const CompressArgs<BATCH ? DAF_B
 }
 
 #define DAF_INSTANTIATE_GENERAL(T)                                                                                          \
-    template cudaError_t dispatch_general_t<T, false, false>(uint32_t, const CompressArgs<1> &, cudaStream_t);              \
-    template cudaError_t dispatch_general_t<T, true, false>(uint32_t, const CompressArgs<DAF_BATCH_MAX> &, cudaStream_t);   \
-    template cudaError_t dispatch_general_t<T, false, true>(uint32_t, const CompressArgs<1> &, cudaStream_t);
+    template cudaError_t dispatch_general_t<T, false, kActNone>(uint32_t, const CompressArgs<1> &, cudaStream_t);              \
+    template cudaError_t dispatch_general_t<T, true, kActNone>(uint32_t, const CompressArgs<DAF_BATCH_MAX> &, cudaStream_t);   \
+    template cudaError_t dispatch_general_t<T, false, kActRelu>(uint32_t, const CompressArgs<1> &, cudaStream_t);              \
+    template cudaError_t dispatch_general_t<T, false, kActRelu6>(uint32_t, const CompressArgs<1> &, cudaStream_t);             \
+    template cudaError_t dispatch_general_t<T, false, kActGelu>(uint32_t, const CompressArgs<1> &, cudaStream_t);
 
 }  // namespace daf

@@ -200,29 +200,29 @@ __device__ __forceinline__ int lookback(const uint64_t *flags, uint32_t gw, uint
 
 // The streaming kernel for calls whose windows all end with one width (compress_stream.cuh; one
 // translation unit per element type).
-template <typename T, bool BATCH, bool RELU>
+template <typename T, bool BATCH, int ACT>
 cudaError_t dispatch_stream_t(uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream);
 
 // The general kernel: any mix of widths within a window (compress_general.cuh; one translation unit per element type).
-template <typename T, bool BATCH, bool RELU>
+template <typename T, bool BATCH, int ACT>
 cudaError_t dispatch_general_t(uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream);
 
-template <bool BATCH, bool RELU>
+template <bool BATCH, int ACT>
 inline cudaError_t dispatch_general(uint32_t dtype, uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
                                     cudaStream_t stream)
 {
-    if (dtype == DAF_F32) return dispatch_general_t<float, BATCH, RELU>(chunks, args, stream);
-    if (dtype == DAF_F16) return dispatch_general_t<__half, BATCH, RELU>(chunks, args, stream);
-    return dispatch_general_t<__nv_bfloat16, BATCH, RELU>(chunks, args, stream);
+    if (dtype == DAF_F32) return dispatch_general_t<float, BATCH, ACT>(chunks, args, stream);
+    if (dtype == DAF_F16) return dispatch_general_t<__half, BATCH, ACT>(chunks, args, stream);
+    return dispatch_general_t<__nv_bfloat16, BATCH, ACT>(chunks, args, stream);
 }
 
-template <bool BATCH, bool RELU>
+template <bool BATCH, int ACT>
 inline cudaError_t dispatch_stream(uint32_t dtype, uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
                                    cudaStream_t stream)
 {
-    if (dtype == DAF_F32) return dispatch_stream_t<float, BATCH, RELU>(chunks, args, stream);
-    if (dtype == DAF_F16) return dispatch_stream_t<__half, BATCH, RELU>(chunks, args, stream);
-    return dispatch_stream_t<__nv_bfloat16, BATCH, RELU>(chunks, args, stream);
+    if (dtype == DAF_F32) return dispatch_stream_t<float, BATCH, ACT>(chunks, args, stream);
+    if (dtype == DAF_F16) return dispatch_stream_t<__half, BATCH, ACT>(chunks, args, stream);
+    return dispatch_stream_t<__nv_bfloat16, BATCH, ACT>(chunks, args, stream);
 }
 
 struct GroupRec {             // what the quantize pass needs per group (one 16-byte shared load)

@@ -84,7 +84,7 @@ template <int B> __device__ __forceinline__ float inverse_scale(float lo, float 
 
 }  // namespace stream
 
-template <typename T, int CHUNKS, int B, int GC, bool BATCH, bool RELU>
+template <typename T, int CHUNKS, int B, int GC, bool BATCH, int ACT>
 __global__ void __launch_bounds__(kThreads, 2)
 stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> a)
 {
@@ -142,15 +142,15 @@ stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MA
         // ---- meanwhile: has anybody asked to stop?
         stop |= retry_seen;
         retry_seen = ld_relaxed_u32(&a.hdr->retry);               // consumed one window later
-        if (RELU) {
-            // fused producer: what is compressed (and written out) is max(x, +0); a lane stores the chunk it loaded, so
-            // the output may be the input buffer
+        if (ACT != kActNone) {
+            // fused producer: the activation is written out and (ReLU, ReLU6) replaces x as what is compressed; a lane
+            // stores the chunk it loaded, so the output may be the input buffer
             char *const act = reinterpret_cast<char *>(td.act) + ((uint64_t)w * WE + e0) * EB;
 #pragma unroll
             for (int c = 0; c < CHUNKS; c++) {
-#pragma unroll
-                for (int i = 0; i < 8; i++) x[c][i] = fmaxf(x[c][i], 0.0f);
-                if (WHOLE || e0 + 256u * c < n_elems) Elem<T>::store8(act + 256u * EB * c, x[c]);
+                float y[8];
+                activate8<ACT>(x[c], y);
+                if (WHOLE || e0 + 256u * c < n_elems) Elem<T>::store8(act + 256u * EB * c, y);
             }
         }
 
@@ -342,28 +342,28 @@ stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MA
     }
 }
 
-template <typename T, int CHUNKS, int B, int GC, bool BATCH, bool RELU>
+template <typename T, int CHUNKS, int B, int GC, bool BATCH, int ACT>
 static cudaError_t launch_stream(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
     int ctas = 0;
-    const cudaError_t e = persistent_ctas(reinterpret_cast<const void *>(&stream_compress_kernel<T, CHUNKS, B, GC, BATCH, RELU>),
+    const cudaError_t e = persistent_ctas(reinterpret_cast<const void *>(&stream_compress_kernel<T, CHUNKS, B, GC, BATCH, ACT>),
                                           kThreads, 0, &ctas);
     if (e != cudaSuccess) return e;
     const uint32_t grid = args.total_windows < (uint32_t)ctas ? args.total_windows : (uint32_t)ctas;
-    stream_compress_kernel<T, CHUNKS, B, GC, BATCH, RELU><<<grid, kThreads, 0, stream>>>(args);
+    stream_compress_kernel<T, CHUNKS, B, GC, BATCH, ACT><<<grid, kThreads, 0, stream>>>(args);
     return cudaGetLastError();
 }
 
-template <typename T, int CHUNKS, bool BATCH, bool RELU>
+template <typename T, int CHUNKS, bool BATCH, int ACT>
 static cudaError_t launch_stream_c(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
     const uint32_t strip = 256u * CHUNKS;
     const int gc = args.G < 256u ? 0 : args.G < strip ? 1 : 2;
 #define DAF_CASE(BB)                                                                                                 \
     case BB:                                                                                                         \
-        if (gc == 0) return launch_stream<T, CHUNKS, BB, 0, BATCH, RELU>(args, stream);                              \
-        if constexpr (CHUNKS > 1) { if (gc == 1) return launch_stream<T, CHUNKS, BB, 1, BATCH, RELU>(args, stream); } \
-        return launch_stream<T, CHUNKS, BB, 2, BATCH, RELU>(args, stream);
+        if (gc == 0) return launch_stream<T, CHUNKS, BB, 0, BATCH, ACT>(args, stream);                              \
+        if constexpr (CHUNKS > 1) { if (gc == 1) return launch_stream<T, CHUNKS, BB, 1, BATCH, ACT>(args, stream); } \
+        return launch_stream<T, CHUNKS, BB, 2, BATCH, ACT>(args, stream);
     switch (args.S[args.full_ell]) {
         DAF_CASE(1)
         DAF_CASE(2)
@@ -376,21 +376,23 @@ static cudaError_t launch_stream_c(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1>
 
 // Launch for element type T: strip length from the window size, GC from the group size, B = the
 // width every whole window ends with.
-template <typename T, bool BATCH, bool RELU>
+template <typename T, bool BATCH, int ACT>
 cudaError_t dispatch_stream_t(uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
-    if constexpr (RELU) {                                         // fused producer: single tensor, default window
-        return launch_stream_c<T, 4, false, true>(args, stream);
+    if constexpr (ACT != kActNone) {                              // fused producer: single tensor, default window
+        return launch_stream_c<T, 4, false, ACT>(args, stream);
     } else {
-        if (chunks == 1) return launch_stream_c<T, 1, BATCH, false>(args, stream);
-        if (chunks == 2) return launch_stream_c<T, 2, BATCH, false>(args, stream);
-        return launch_stream_c<T, 4, BATCH, false>(args, stream);
+        if (chunks == 1) return launch_stream_c<T, 1, BATCH, kActNone>(args, stream);
+        if (chunks == 2) return launch_stream_c<T, 2, BATCH, kActNone>(args, stream);
+        return launch_stream_c<T, 4, BATCH, kActNone>(args, stream);
     }
 }
 
 #define DAF_INSTANTIATE_STREAM(T)                                                                                          \
-    template cudaError_t dispatch_stream_t<T, false, false>(uint32_t, const CompressArgs<1> &, cudaStream_t);              \
-    template cudaError_t dispatch_stream_t<T, true, false>(uint32_t, const CompressArgs<DAF_BATCH_MAX> &, cudaStream_t);   \
-    template cudaError_t dispatch_stream_t<T, false, true>(uint32_t, const CompressArgs<1> &, cudaStream_t);
+    template cudaError_t dispatch_stream_t<T, false, kActNone>(uint32_t, const CompressArgs<1> &, cudaStream_t);              \
+    template cudaError_t dispatch_stream_t<T, true, kActNone>(uint32_t, const CompressArgs<DAF_BATCH_MAX> &, cudaStream_t);   \
+    template cudaError_t dispatch_stream_t<T, false, kActRelu>(uint32_t, const CompressArgs<1> &, cudaStream_t);              \
+    template cudaError_t dispatch_stream_t<T, false, kActRelu6>(uint32_t, const CompressArgs<1> &, cudaStream_t);             \
+    template cudaError_t dispatch_stream_t<T, false, kActGelu>(uint32_t, const CompressArgs<1> &, cudaStream_t);
 
 }  // namespace daf

@@ -56,9 +56,10 @@ template <> __device__ __forceinline__ float as_stored<float>(float y) { return 
 template <> __device__ __forceinline__ float as_stored<__half>(float y) { return __half2float(__float2half_rn(y)); }
 template <> __device__ __forceinline__ float as_stored<__nv_bfloat16>(float y) { return __bfloat162float(__float2bfloat16_rn(y)); }
 
-// MASK: fused consumer.  Instead of the restored activation the kernel stores the gradient of a
-// ReLU that produced it: the incoming gradient where the restored value is positive, else +0.
-template <typename T, int CHUNKS, bool BATCH, bool MASK>
+// MASK != 0: fused consumer.  Instead of the restored value the kernel stores the gradient of the activation
+// whose producer stored it: ReLU, the incoming gradient where the restored output is positive, else +0; ReLU6, where
+// it lies strictly between 0 and 6; GELU, the incoming gradient times GELU'(restored input).
+template <typename T, int CHUNKS, bool BATCH, int MASK>
 __global__ void __launch_bounds__(kThreads)
 decompress_kernel(const __grid_constant__ DecompressArgs<BATCH ? DAF_BATCH_MAX : 1> a)
 {
@@ -152,20 +153,25 @@ decompress_kernel(const __grid_constant__ DecompressArgs<BATCH ? DAF_BATCH_MAX :
             float g[8];
             Elem<T>::load8(reinterpret_cast<const char *>(td.grad) + (wbase + e) * Elem<T>::kBytes, g);
 #pragma unroll
-            for (int i = 0; i < 8; i++) y[i] = as_stored<T>(y[i]) > 0.0f ? g[i] : 0.0f;
+            for (int i = 0; i < 8; i++) {
+                const float r = as_stored<T>(y[i]);
+                if (MASK == kActRelu) y[i] = r > 0.0f ? g[i] : 0.0f;
+                else if (MASK == kActRelu6) y[i] = (r > 0.0f && r < 6.0f) ? g[i] : 0.0f;
+                else y[i] = g[i] * gelu_grad_f(r);
+            }
         }
         Elem<T>::store8(out + (size_t)e * Elem<T>::kBytes, y);
     }
 }
 
-template <typename T, int CHUNKS, bool BATCH, bool MASK>
+template <typename T, int CHUNKS, bool BATCH, int MASK>
 static cudaError_t launch(const DecompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
     decompress_kernel<T, CHUNKS, BATCH, MASK><<<args.total_windows, kThreads, 0, stream>>>(args);
     return cudaGetLastError();
 }
 
-template <bool BATCH, bool MASK = false>
+template <bool BATCH, int MASK = kActNone>
 static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, const DecompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
                             cudaStream_t stream)
 {
@@ -221,10 +227,12 @@ extern "C" daf_status daf_decompress(const daf_params *params, const void *d_pac
                                                                                                                  : DAF_ERR_CUDA;
 }
 
-extern "C" daf_status daf_decompress_relu_grad(const daf_params *params, const void *d_packed, const uint8_t *d_bits,
-                                               const float *d_min, const float *d_scale, const uint64_t *d_window_offsets,
-                                               const void *d_grad_out, void *d_grad_in, daf_stream stream)
+extern "C" daf_status daf_decompress_act_grad(const daf_params *params, uint32_t act, const void *d_packed,
+                                              const uint8_t *d_bits, const float *d_min, const float *d_scale,
+                                              const uint64_t *d_window_offsets, const void *d_grad_out, void *d_grad_in,
+                                              daf_stream stream)
 {
+    if (act != DAF_ACT_RELU && act != DAF_ACT_RELU6 && act != DAF_ACT_GELU) return DAF_ERR_INVALID_ARG;
     Plan pl;
     daf_status st = make_plan(params, &pl);
     if (st != DAF_OK) return st;
@@ -239,10 +247,22 @@ extern "C" daf_status daf_decompress_relu_grad(const daf_params *params, const v
     a.log2G = pl.log2G;
     a.t[0] = DecTensor{reinterpret_cast<const uint8_t *>(d_packed), d_bits, d_min, d_scale, d_window_offsets, d_grad_in,
                        params->numel, 0u, (uint32_t)pl.n_windows, d_grad_out};
-    return dispatch<false, true>(params->dtype, pl.chunks, a, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess
-               ? DAF_OK
-               : DAF_ERR_CUDA;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    if (act == DAF_ACT_RELU) e = dispatch<false, kActRelu>(params->dtype, pl.chunks, a, s);
+    else if (act == DAF_ACT_RELU6) e = dispatch<false, kActRelu6>(params->dtype, pl.chunks, a, s);
+    else e = dispatch<false, kActGelu>(params->dtype, pl.chunks, a, s);
+    return e == cudaSuccess ? DAF_OK : DAF_ERR_CUDA;
 }
+
+extern "C" daf_status daf_decompress_relu_grad(const daf_params *params, const void *d_packed, const uint8_t *d_bits,
+                                               const float *d_min, const float *d_scale, const uint64_t *d_window_offsets,
+                                               const void *d_grad_out, void *d_grad_in, daf_stream stream)
+{
+    return daf_decompress_act_grad(params, DAF_ACT_RELU, d_packed, d_bits, d_min, d_scale, d_window_offsets, d_grad_out,
+                                   d_grad_in, stream);
+}
+
 
 extern "C" daf_status daf_decompress_batch(uint32_t n, const daf_params *params, const void *const *d_packed,
                                            const uint8_t *const *d_bits, const float *const *d_min,

@@ -400,3 +400,29 @@ def test_resnet18_under_a_memory_budget_that_binds():
     st = ctx._store.stats()
     assert st["resizes"] > 0 and st["used_bytes"] == 0
     assert all(np.isfinite(losses)) and np.mean(losses[-3:]) < losses[0]
+
+
+def test_compressed_gelu_and_relu6_layers_follow_torch_within_the_quantization_step():
+    """The layers against torch's own: forward equal (ReLU6) or within float rounding (GELU); backward equal to torch's
+    derivative taken at the restored tensor, which differs from the true one by at most a quantization step."""
+    from paper_2507_07149_b200.autograd import CompressedGELU, CompressedReLU6
+    daf.lib()
+    n, G = 16384 * 6, 256
+    xs = torch.randn(n, device="cuda") * 3
+    gw = torch.randn(n, device="cuda")
+    for layer, plain in ((CompressedReLU6(group_size=G, bit_budget=8.0, min_numel=1024), torch.nn.functional.relu6),
+                         (CompressedGELU(group_size=G, bit_budget=8.0, min_numel=1024), torch.nn.functional.gelu)):
+        x = xs.clone().requires_grad_(True)
+        y = layer(x)
+        (y * gw).sum().backward()
+        x2 = xs.clone().requires_grad_(True)
+        y2 = plain(x2)
+        (y2 * gw).sum().backward()
+        assert torch.allclose(y, y2, rtol=1e-5, atol=1e-6)
+        # at 8 bits a group of 256 normal values spans about 17 units: step 0.07; GELU' has slope <= 1.13
+        bad = (x.grad - x2.grad).abs() > 0.1 * gw.abs() + 1e-6
+        if isinstance(layer, CompressedReLU6):
+            near = (xs.abs() < 0.08) | ((xs - 6).abs() < 0.08)        # the mask may flip only next to the kinks
+            assert not (bad & ~near).any()
+        else:
+            assert not bad.any()

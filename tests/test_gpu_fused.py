@@ -26,13 +26,13 @@ def _input(rng, n, G, dtype, mixed):
     return a.astype(np.float16) if dtype == "f16" else wl.f32_to_bf16_bits(a)
 
 
-def _check(a, dtype, G, beta, inplace, seed=3):
+def _check(a, dtype, G, beta, inplace, seed=3, act_code=daf.ACT_RELU):
     x = to_device(a, dtype)
     x0 = x.clone()
-    act, c = daf.relu_compress(x, G, (1, 2, 4, 8), beta, seed=seed, inplace=inplace, check=True)
+    act, c = daf.relu_compress(x, G, (1, 2, 4, 8), beta, seed=seed, inplace=inplace, check=True, act=act_code)
     y = daf.decompress(c)
     torch.cuda.synchronize()
-    want_act = oracle.relu(a, dtype)
+    want_act = (oracle.relu if act_code == daf.ACT_RELU else oracle.relu6)(a, dtype)
     got_act = to_host(act, dtype)
     assert np.array_equal(got_act.view(np.uint32 if dtype == "f32" else np.uint16),
                           want_act.view(np.uint32 if dtype == "f32" else np.uint16))
@@ -130,3 +130,108 @@ def test_fp32_outputs_must_be_32_byte_aligned():
     assert e.value.status == daf.ERR_INVALID_ARG
     daf.daf_decompress(c.params, c.packed, c.bits, c.min, c.scale, c.window_offsets, buf[8:8 + (1 << 16)])
     torch.cuda.synchronize()
+
+
+def _scaled(a, dtype, k):
+    """The input times k (so that part of it passes 6), in its own type."""
+    if dtype == "bf16":
+        return wl.f32_to_bf16_bits(oracle.widen(a, "bf16") * np.float32(k))
+    return (a * a.dtype.type(k)).astype(a.dtype)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+@pytest.mark.parametrize("G,beta,mixed,inplace", [(256, 4.0, False, False), (256, 3.0, False, True), (64, 2.0, True, False)])
+def test_relu6_compress_matches_relu6_then_compress(dtype, G, beta, mixed, inplace):
+    rng = np.random.default_rng(G + int(beta * 10) + mixed + 100)
+    n = 16384 * 23 + G * 5
+    a = _scaled(_input(rng, n, G, dtype, mixed), dtype, 4.0)
+    want = oracle.widen(oracle.relu6(a, dtype), dtype if dtype == "bf16" else None)
+    assert (want == 6).sum() > n // 50 and (want == 0).sum() > n // 4
+    _check(a, dtype, G, beta, inplace=inplace, act_code=daf.ACT_RELU6)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+def test_relu6_grad_masks_both_ends(dtype):
+    """grad where the restored activation lies strictly between 0 and 6: saturated elements restore to exactly 6 (the
+    group maximum decodes as min + L * scale; where that rounds below 6 the gradient passes, as the oracle says)."""
+    rng = np.random.default_rng(77)
+    G, beta, n = 256, 4.0, 16384 * 5 + 256 * 3
+    a = oracle.relu6(_scaled(_input(rng, n, G, dtype, False), dtype, 4.0), dtype)
+    g32 = rng.standard_normal(n).astype(np.float32)
+    g = g32 if dtype == "f32" else (g32.astype(np.float16) if dtype == "f16" else wl.f32_to_bf16_bits(g32))
+    x = to_device(a, dtype)
+    c = daf.compress(x, G, (1, 2, 4, 8), beta, seed=4)
+    out = daf.relu_grad(c, to_device(g, dtype), act=daf.ACT_RELU6)
+    torch.cuda.synchronize()
+    ref = oracle.compress(a, G, (1, 2, 4, 8), beta, dtype="bf16" if dtype == "bf16" else None, seed=4)
+    r = oracle.widen(oracle.decompress(ref), "bf16" if dtype == "bf16" else None)
+    keep = (r > 0) & (r < 6)
+    view = np.uint32 if dtype == "f32" else np.uint16
+    want = np.where(keep, g.view(view), view(0)).astype(view)
+    assert np.array_equal(to_host(out, dtype).view(view), want)
+    assert int((r >= 6).sum()) > 0 and int((r <= 0).sum()) > 0 and int(keep.sum()) > 0
+
+
+def _ulp32(v):
+    return np.spacing(np.abs(v).astype(np.float32)).astype(np.float64)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+@pytest.mark.parametrize("G,beta,mixed", [(256, 4.0, False), (128, 3.0, True)])
+def test_gelu_compress_writes_gelu_and_compresses_the_input(dtype, G, beta, mixed):
+    """daf_act_compress(GELU): the activation written is GELU(x) to within 8 + 2 min(x, 0)^2 binary32 ulps (2^-40
+    absolute) before the rounding to the output type (the rounding of the argument of erfc is amplified by x^2 in the
+    negative tail, where the value itself vanishes); the compressed form is that of x itself, bit for bit."""
+    rng = np.random.default_rng(G + 5)
+    n = 16384 * 19 + G * 7
+    a = _scaled(_input(rng, n, G, dtype, mixed), dtype, 3.0)
+    x = to_device(a, dtype)
+    x0 = x.clone()
+    y, c = daf.relu_compress(x, G, (1, 2, 4, 8), beta, seed=6, check=True, act=daf.ACT_GELU)
+    torch.cuda.synchronize()
+    assert torch.equal(x.view(torch.int32 if dtype == "f32" else torch.int16), x0.view(torch.int32 if dtype == "f32" else torch.int16))
+    x32 = oracle.widen(a, "bf16" if dtype == "bf16" else None)
+    exact = oracle.gelu(x32)
+    got = oracle.widen(to_host(y, dtype), "bf16" if dtype == "bf16" else None).astype(np.float64)
+    tol = (8 + 2 * np.minimum(x32.astype(np.float64), 0.0) ** 2) * _ulp32(exact) + 2.0 ** -40
+    if dtype != "f32":                                            # plus the rounding to the 16-bit type (half an ulp of it)
+        mant = 11 if dtype == "f16" else 8
+        tol = tol + np.maximum(np.abs(exact) * 2.0 ** -mant, 2.0 ** -25 if dtype == "f16" else 0.0)
+    assert np.all(np.abs(got - exact) <= tol), float(np.max(np.abs(got - exact) / tol))
+    ref = oracle.compress(a, G, (1, 2, 4, 8), beta, dtype="bf16" if dtype == "bf16" else None, seed=6)
+    assert np.array_equal(c.bits.cpu().numpy(), ref.bits)
+    assert np.array_equal(c.window_offsets.cpu().numpy().view(np.uint64), ref.window_offsets)
+    assert np.array_equal(c.min.cpu().numpy().view(np.uint32), ref.mn.view(np.uint32))
+    assert np.array_equal(c.scale.cpu().numpy().view(np.uint32), ref.scale.view(np.uint32))
+    assert np.array_equal(c.packed[: ref.packed.size].cpu().numpy(), ref.packed)
+    if mixed:
+        assert len(np.unique(ref.bits)) >= 2
+    # the consumer: gradient times GELU'(restored input)
+    g32 = rng.standard_normal(n).astype(np.float32)
+    g = g32 if dtype == "f32" else (g32.astype(np.float16) if dtype == "f16" else wl.f32_to_bf16_bits(g32))
+    out = daf.relu_grad(c, to_device(g, dtype), act=daf.ACT_GELU)
+    torch.cuda.synchronize()
+    r = oracle.widen(oracle.decompress(ref), "bf16" if dtype == "bf16" else None)
+    gw = oracle.widen(g, "bf16" if dtype == "bf16" else None).astype(np.float64)
+    want = gw * oracle.gelu_grad(r)
+    got = oracle.widen(to_host(out, dtype), "bf16" if dtype == "bf16" else None).astype(np.float64)
+    # factor within 2^-21; a restored binary32 value may differ from the oracle's by one ulp (|GELU''| <= 1.13)
+    tol = np.abs(gw) * (2.0 ** -21 + 1.13 * _ulp32(r)) + _ulp32(want)
+    if dtype != "f32":
+        mant = 11 if dtype == "f16" else 8
+        tol = tol + np.maximum(np.abs(want) * 2.0 ** -mant, 2.0 ** -25 if dtype == "f16" else 0.0)
+    assert np.all(np.abs(got - want) <= tol), float(np.max(np.abs(got - want) / tol))
+
+
+def test_gelu_compress_rejects_in_place_and_unknown_activations():
+    x = torch.randn(1 << 16, device="cuda")
+    with pytest.raises(daf.DafError) as e:
+        daf.relu_compress(x, 256, (1, 2, 4, 8), 4.0, inplace=True, act=daf.ACT_GELU)
+    assert e.value.status == daf.ERR_INVALID_ARG
+    with pytest.raises(daf.DafError) as e:
+        daf.relu_compress(x, 256, (1, 2, 4, 8), 4.0, act=7)
+    assert e.value.status == daf.ERR_INVALID_ARG
+    c = daf.compress(x, 256, (1, 2, 4, 8), 4.0)
+    with pytest.raises(daf.DafError) as e:
+        daf.relu_grad(c, x, act=0)
+    assert e.value.status == daf.ERR_INVALID_ARG

@@ -421,7 +421,7 @@ def test_decode_closed_forms():
 
 @pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
 def test_constant_groups_round_trip_exactly(dtype):
-    from paper_2507_07149_b200.workloads import f32_to_bf16_bits
+    f32_to_bf16_bits = oracle.to_bf16_bits                       # the oracle's own conversion builds the oracle's input
     vals = np.float32([0.0, -0.0, 1.0, -3.5, 6.0, 1024.0, 2.0 ** -10, -65504.0])
     x = np.repeat(vals, 64)
     if dtype == "f16":
@@ -487,3 +487,34 @@ def test_relu_by_hand():
     assert np.array_equal(oracle.relu(a.astype(np.float16)).view(np.uint16), want.astype(np.float16).view(np.uint16))
     b = np.array([0xBFC0, 0x8000, 0x0000, 0x4020, 0x8001], np.uint16)          # bf16 -1.5, -0, +0, 2.5, a negative subnormal
     assert np.array_equal(oracle.relu(b, "bf16"), np.array([0, 0, 0, 0x4020, 0], np.uint16))
+
+
+def test_relu6_by_hand():
+    a = np.array([-1.5, -0.0, 0.0, 2.5, 6.0, 6.5, 1e30, -1e30], np.float32)
+    want = np.array([0.0, 0.0, 0.0, 2.5, 6.0, 6.0, 6.0, 0.0], np.float32)
+    assert np.array_equal(oracle.relu6(a).view(np.uint32), want.view(np.uint32))
+    assert np.array_equal(oracle.relu6(a.astype(np.float16)).view(np.uint16), want.astype(np.float16).view(np.uint16))
+    b = np.array([0xBFC0, 0x8000, 0x0000, 0x4020, 0x40C0, 0x40C1, 0x7F00], np.uint16)   # -1.5 -0 +0 2.5 6 6.03 huge
+    assert np.array_equal(oracle.relu6(b, "bf16"), np.array([0, 0, 0, 0x4020, 0x40C0, 0x40C0, 0x40C0], np.uint16))
+
+
+def test_gelu_and_its_derivative_against_closed_forms_and_a_library():
+    """GELU(x) = x Phi(x): values that follow from the normal distribution, the two reflection identities, the
+    derivative against a central difference, and torch's float64 GELU with its autograd derivative."""
+    x = np.concatenate([np.linspace(-9, 9, 2001), [0.0, 1.0, -1.0, 1e-8, -1e-8, 20.0, -20.0]])
+    y, d = oracle.gelu(x), oracle.gelu_grad(x)
+    assert oracle.gelu([0.0])[0] == 0.0 and oracle.gelu_grad([0.0])[0] == 0.5
+    assert abs(oracle.gelu([1.0])[0] - 0.8413447460685429) < 1e-15           # Phi(1)
+    assert abs(oracle.gelu([-1.0])[0] + 0.15865525393145707) < 1e-15         # -(1 - Phi(1))
+    assert np.allclose(y - oracle.gelu(-x), x, rtol=0, atol=1e-14)          # Phi(x) + Phi(-x) = 1
+    assert np.allclose(d + oracle.gelu_grad(-x), 1.0, rtol=0, atol=1e-14)
+    assert oracle.gelu([20.0])[0] == 20.0 and abs(oracle.gelu([-20.0])[0]) < 1e-80
+    h = 1e-5
+    num = (oracle.gelu(x + h) - oracle.gelu(x - h)) / (2 * h)
+    assert np.allclose(num, d, rtol=0, atol=1e-9)
+    torch = pytest.importorskip("torch")
+    t = torch.tensor(x, dtype=torch.float64, requires_grad=True)
+    ty = torch.nn.functional.gelu(t)
+    ty.sum().backward()
+    assert np.allclose(ty.detach().numpy(), y, rtol=1e-13, atol=1e-15)    # (the library loses the far negative tail)
+    assert np.allclose(t.grad.numpy(), d, rtol=0, atol=1e-14)
