@@ -163,9 +163,9 @@ daf_status daf_decompress(const daf_params *params, const void *d_packed, const 
 /* The same for other activations.  act:
  *   DAF_ACT_RELU   as daf_relu_compress.
  *   DAF_ACT_RELU6  act = min(max(x, +0), 6), written to d_act and compressed.
- *   DAF_ACT_GELU   d_act receives GELU(x) = x/2 * erfc(-x / sqrt 2), computed in binary32 and rounded to the input's
- *                  type (within 8 + 2 min(x, 0)^2 units in the last place of binary32, or 2^-40 in absolute terms,
- *                  of the exact value before that rounding); what is COMPRESSED is x itself, because the backward pass of a GELU
+ *   DAF_ACT_GELU   d_act receives GELU(x) = x/2 * (1 + erf(x / sqrt 2)), computed in binary32 and rounded to the
+ *                  input's type (before that rounding, within 8 units in the last place of binary32 plus
+ *                  2^-24 |x| of the exact value: the far negative tail is noise around 0); what is COMPRESSED is x itself, because the backward pass of a GELU
  *                  needs its input: every other output is that of daf_compress(params, d_in, ...).  d_act must
  *                  not be (or overlap) d_in.
  * Any other value of act: DAF_ERR_INVALID_ARG.
@@ -190,7 +190,7 @@ daf_status daf_decompress_relu_grad(const daf_params *params, const void *d_pack
  *   DAF_ACT_RELU   d_grad_in = d_grad_out where r > 0, else +0
  *   DAF_ACT_RELU6  d_grad_in = d_grad_out where 0 < r < 6, else +0
  *   DAF_ACT_GELU   d_grad_in = d_grad_out * (Phi(r) + r phi(r)), r the restored INPUT of the GELU; the factor is
- *                  computed in binary32 (within 2^-21 of the exact one), the product rounded to params->dtype
+ *                  computed in binary32 (within 2^-20 of the exact one), the product rounded to params->dtype
  * Arguments and errors as for daf_decompress_relu_grad.
  */
 daf_status daf_decompress_act_grad(const daf_params *params, uint32_t act, const void *d_packed, const uint8_t *d_bits,

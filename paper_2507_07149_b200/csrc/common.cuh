@@ -291,13 +291,15 @@ cudaError_t persistent_ctas(const void *kernel, int threads, int dyn_smem, int *
 // activation is produced, the restored value is used where the gradient is formed).
 //   ReLU   y = max(x, +0)            what is compressed: y     gradient: g where restored y > 0
 //   ReLU6  y = min(max(x, +0), 6)    what is compressed: y     gradient: g where 0 < restored y < 6
-//   GELU   y = x Phi(x) = x/2 erfc(-x / sqrt 2)    what is compressed: x (the backward pass needs the input)
+//   GELU   y = x Phi(x) = x/2 (1 + erf(x / sqrt 2))    what is compressed: x (the backward pass needs the input)
 //          gradient: g * (Phi(x) + x phi(x)) at the restored x
+// The GELU pair is bound by arithmetic, not by memory, so it takes the cheap forms: erf rather than erfc (the far
+// negative tail, where x Phi(x) is below 2^-24 |x|, is then rounding noise around 0) and the fast exponential.
 enum : int { kActNone = 0, kActRelu = 1, kActRelu6 = 2, kActGelu = 3 };
-__device__ __forceinline__ float gelu_f(float x) { return (0.5f * x) * erfcf(-0.70710678118654752f * x); }
+__device__ __forceinline__ float gelu_f(float x) { return (0.5f * x) * (1.0f + erff(0.70710678118654752f * x)); }
 __device__ __forceinline__ float gelu_grad_f(float x)
 {
-    return 0.5f * erfcf(-0.70710678118654752f * x) + (x * 0.3989422804014327f) * expf(-0.5f * (x * x));
+    return 0.5f * (1.0f + erff(0.70710678118654752f * x)) + (x * 0.3989422804014327f) * __expf(-0.5f * (x * x));
 }
 // x: the chunk as loaded; afterwards x = what is compressed, y = what the producer writes out.
 template <int ACT> __device__ __forceinline__ void activate8(float (&x)[8], float (&y)[8])

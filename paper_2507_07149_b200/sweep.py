@@ -121,7 +121,8 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--scale", type=int, default=1)
     ap.add_argument("--relu", action="store_true",
-                    help="also the fused producer on workload 5: daf_relu_compress against torch.relu followed by daf_compress")
+                    help="also the fused producers and consumers (ReLU, ReLU6, GELU) on workload 5, each against torch's own "
+                         "kernel followed / preceded by daf_compress / daf_decompress")
     args = ap.parse_args()
 
     import torch
@@ -154,38 +155,49 @@ def main():
             p = daf.make_params(daf.dtype_code(x), x.numel(), w.group_size, w.widths, w.bit_budget, seed=0)
             c = daf.alloc_outputs(p, x.device)
             act = torch.empty_like(x)
-
-            def fused():
-                daf.daf_relu_compress(p, x, act, c.packed, c.sizes.packed_capacity, c.bits, c.min, c.scale,
-                                      c.window_offsets, c.workspace, c.sizes.workspace)
-
-            def separate():
-                torch.clamp_min(x, 0, out=act)                    # relu into a preallocated tensor
-                daf.daf_compress(p, act, c.packed, c.sizes.packed_capacity, c.bits, c.min, c.scale, c.window_offsets,
-                                 c.workspace, c.sizes.workspace)
-
-            t_f = _time(torch, fused, args.steps, False)
-            assert daf.daf_poll_status(c.workspace) == daf.OK
-            packed = c.packed_bytes()
-            t_s = _time(torch, separate, args.steps, False)
-            alg = 2 * w.nbytes + packed + 9 * (x.numel() // w.group_size) + 8 * (c.sizes.n_windows + 1)
-            print(f"| {w.name} relu + compress, fused | {w.numel} | {w.nbytes / 2**30:.3f} | {packed / 2**30:.3f} | "
-                  f"{t_f:.4f} | {alg / t_f / 1e6:.0f} | — | — | torch.relu + daf_compress: {t_s:.4f} | — |", flush=True)
             g = torch.randn_like(x)
             gi = torch.empty_like(x)
+            F = torch.nn.functional
+            # name, library code, the activation and its backward as torch runs them (separate kernels)
+            variants = (
+                ("ReLU", daf.ACT_RELU, lambda: torch.clamp_min(x, 0, out=act),
+                 lambda: torch.ops.aten.threshold_backward.grad_input(g, act, 0.0, grad_input=gi)),
+                ("ReLU6", daf.ACT_RELU6, lambda: torch.clamp(x, 0, 6, out=act),
+                 lambda: torch.ops.aten.hardtanh_backward.grad_input(g, act, 0.0, 6.0, grad_input=gi)),
+                ("GELU", daf.ACT_GELU, lambda: torch.ops.aten.gelu.out(x, out=act),
+                 lambda: torch.ops.aten.gelu_backward.grad_input(g, act, grad_input=gi)))
+            for name, code, torch_fwd, torch_bwd in variants:
+                gelu = code == daf.ACT_GELU
 
-            def fused_back():
-                daf.daf_decompress_relu_grad(p, c.packed, c.bits, c.min, c.scale, c.window_offsets, g, gi)
+                def fused():
+                    daf.daf_act_compress(p, code, x, act, c.packed, c.sizes.packed_capacity, c.bits, c.min, c.scale,
+                                         c.window_offsets, c.workspace, c.sizes.workspace)
 
-            def separate_back():
-                daf.daf_decompress(p, c.packed, c.bits, c.min, c.scale, c.window_offsets, act)
-                torch.ops.aten.threshold_backward.grad_input(g, act, 0.0, grad_input=gi)   # the ReLU backward kernel of torch
+                def separate():
+                    torch_fwd()
+                    daf.daf_compress(p, x if gelu else act, c.packed, c.sizes.packed_capacity, c.bits, c.min, c.scale,
+                                     c.window_offsets, c.workspace, c.sizes.workspace)
 
-            t_fb = _time(torch, fused_back, args.steps, False)
-            t_sb = _time(torch, separate_back, args.steps, False)
-            print(f"| {w.name} ReLU gradient from the packed output, fused | {w.numel} | {w.nbytes / 2**30:.3f} | "
-                  f"{packed / 2**30:.3f} | — | — | {t_fb:.4f} | {alg / t_fb / 1e6:.0f} | — | daf_decompress + the ReLU backward kernel of torch: {t_sb:.4f} |",
-                  flush=True)
+                t_f = _time(torch, fused, args.steps, False)
+                assert daf.daf_poll_status(c.workspace) == daf.OK
+                packed = c.packed_bytes()
+                t_s = _time(torch, separate, args.steps, False)
+                alg = 2 * w.nbytes + packed + 9 * (x.numel() // w.group_size) + 8 * (c.sizes.n_windows + 1)
+                print(f"| {w.name} {name} + compress, fused | {w.numel} | {w.nbytes / 2**30:.3f} | {packed / 2**30:.3f} | "
+                      f"{t_f:.4f} | {alg / t_f / 1e6:.0f} | — | — | torch {name} + daf_compress: {t_s:.4f} | — |", flush=True)
+
+                def fused_back():
+                    daf.daf_decompress_act_grad(p, code, c.packed, c.bits, c.min, c.scale, c.window_offsets, g, gi)
+
+                def separate_back():
+                    daf.daf_decompress(p, c.packed, c.bits, c.min, c.scale, c.window_offsets, act)
+                    torch_bwd()                                       # torch's backward kernel on the restored tensor
+
+                t_fb = _time(torch, fused_back, args.steps, False)
+                t_sb = _time(torch, separate_back, args.steps, False)
+                print(f"| {w.name} {name} gradient from the packed form, fused | {w.numel} | {w.nbytes / 2**30:.3f} | "
+                      f"{packed / 2**30:.3f} | — | — | {t_fb:.4f} | {alg / t_fb / 1e6:.0f} | — | daf_decompress + torch's "
+                      f"{name} backward: {t_sb:.4f} |", flush=True)
             del act, c, g, gi
         del xs
         torch.cuda.empty_cache()

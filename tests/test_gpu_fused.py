@@ -179,9 +179,9 @@ def _ulp32(v):
 @pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
 @pytest.mark.parametrize("G,beta,mixed", [(256, 4.0, False), (128, 3.0, True)])
 def test_gelu_compress_writes_gelu_and_compresses_the_input(dtype, G, beta, mixed):
-    """daf_act_compress(GELU): the activation written is GELU(x) to within 8 + 2 min(x, 0)^2 binary32 ulps (2^-40
-    absolute) before the rounding to the output type (the rounding of the argument of erfc is amplified by x^2 in the
-    negative tail, where the value itself vanishes); the compressed form is that of x itself, bit for bit."""
+    """daf_act_compress(GELU): the activation written is GELU(x) to within 8 binary32 ulps plus 2^-24 |x| (the erf
+    form: the far negative tail is rounding noise around 0) before the rounding to the output type; the compressed
+    form is that of x itself, bit for bit."""
     rng = np.random.default_rng(G + 5)
     n = 16384 * 19 + G * 7
     a = _scaled(_input(rng, n, G, dtype, mixed), dtype, 3.0)
@@ -193,7 +193,7 @@ def test_gelu_compress_writes_gelu_and_compresses_the_input(dtype, G, beta, mixe
     x32 = oracle.widen(a, "bf16" if dtype == "bf16" else None)
     exact = oracle.gelu(x32)
     got = oracle.widen(to_host(y, dtype), "bf16" if dtype == "bf16" else None).astype(np.float64)
-    tol = (8 + 2 * np.minimum(x32.astype(np.float64), 0.0) ** 2) * _ulp32(exact) + 2.0 ** -40
+    tol = 8 * _ulp32(exact) + 2.0 ** -24 * np.abs(x32.astype(np.float64)) + 2.0 ** -40
     if dtype != "f32":                                            # plus the rounding to the 16-bit type (half an ulp of it)
         mant = 11 if dtype == "f16" else 8
         tol = tol + np.maximum(np.abs(exact) * 2.0 ** -mant, 2.0 ** -25 if dtype == "f16" else 0.0)
@@ -215,8 +215,8 @@ def test_gelu_compress_writes_gelu_and_compresses_the_input(dtype, G, beta, mixe
     gw = oracle.widen(g, "bf16" if dtype == "bf16" else None).astype(np.float64)
     want = gw * oracle.gelu_grad(r)
     got = oracle.widen(to_host(out, dtype), "bf16" if dtype == "bf16" else None).astype(np.float64)
-    # factor within 2^-21; a restored binary32 value may differ from the oracle's by one ulp (|GELU''| <= 1.13)
-    tol = np.abs(gw) * (2.0 ** -21 + 1.13 * _ulp32(r)) + _ulp32(want)
+    # factor within 2^-20; a restored binary32 value may differ from the oracle's by one ulp (|GELU''| <= 1.13)
+    tol = np.abs(gw) * (2.0 ** -20 + 1.13 * _ulp32(r)) + _ulp32(want)
     if dtype != "f32":
         mant = 11 if dtype == "f16" else 8
         tol = tol + np.maximum(np.abs(want) * 2.0 ** -mant, 2.0 ** -25 if dtype == "f16" else 0.0)
