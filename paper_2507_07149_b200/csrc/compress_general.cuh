@@ -247,7 +247,6 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     __shared__ __align__(8) uint64_t s_full;                     // mbarrier: staged window has landed (or there is none)
     __shared__ uint32_t s_next[2];                               // ticket of the window of iteration i (slot i & 1)
     __shared__ uint32_t s_lost;                                  // a staged copy did not land in time
-    __shared__ uint32_t s_abort;                                 // quick kernel: this CTA met a window it does not handle
     __shared__ __align__(16) uint32_t s_rkeys[2][20];            // batched calls: Philox round keys of the window's tensor
     __shared__ uint32_t s_tot[2];                                // packed bytes of the window of iteration i (slot i & 1)
     __shared__ uint32_t s_mode[2];                               // how that window's widths came out (see below)
@@ -307,7 +306,6 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
     if (tid == kThreads) {
         mbar_init(&s_full, 1);
         s_lost = 0u;
-        s_abort = 0u;
         s_slow[0] = s_slow[1] = 0u;
         s_kmin[0] = s_kmin[1] = 0xFFFFFFFFu;
         s_kmax[0] = s_kmax[1] = 0u;
@@ -516,7 +514,7 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
         for (uint32_t iter = 0;; iter++) {
             bar_sync(kBarStage, stage_threads);                   // every unit's min / max is visible
             const uint32_t gw = s_next[iter & 1u];
-            if (gw >= a.total_windows || s_abort != 0u) break;
+            if (gw >= a.total_windows) break;
             bool arrived = false;
             if (s_lost == 0u) uniform_widths(gw, iter, arrived);
             if (!arrived) bar_arrive(kBarWidths, kThreads + 32);  // the verdict on the window is in

@@ -46,6 +46,13 @@ def test_sizes_and_host_validation():
         q = daf.make_params(daf.BF16, n, G, (1, 2, 4, 8), beta, window_elems=We)
         assert daf.daf_sizes(q).packed_capacity == oracle.packed_capacity(n, G, We, beta)
 
+    # a budget above the largest width buys nothing: sizes are those of the largest width
+    n = 16384 * 2 + 512
+    for widths, top in (((1, 2, 4, 8), 8), ((1, 2, 4), 4), ((2,), 2)):
+        big = daf.daf_sizes(daf.make_params(daf.F32, n, 256, widths, 12.0))
+        at_top = daf.daf_sizes(daf.make_params(daf.F32, n, 256, widths, float(top)))
+        assert big.packed_capacity == at_top.packed_capacity == n * top // 8
+
     def status(**kw):
         args = dict(dtype=daf.F32, numel=16384, group_size=256, widths=(2, 4, 8), bit_budget=4.0)
         args.update(kw)

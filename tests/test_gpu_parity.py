@@ -295,6 +295,16 @@ def test_group_offsets_against_oracle(n_groups):
         assert np.array_equal(off.cpu().numpy().view(np.uint64), oracle.offsets(bits, G))
 
 
+def test_budget_above_the_largest_width():
+    """Budget 12 with widths {1,2,4}: every group ends at 4 bits, the capacity is that of 4 bits, parity as usual."""
+    rng = np.random.default_rng(12)
+    n = 16384 * 9 + 256 * 5
+    a = (rng.standard_normal(n) * np.repeat(10.0 ** rng.uniform(-2, 2, n // 256), 256)).astype(np.float32)
+    xd, c, ref = assert_compress_parity(a, "f32", 256, (1, 2, 4), 12.0, seed=3, label="budget 12")
+    assert set(np.unique(ref.bits)) == {4} and c.sizes.packed_capacity == n * 4 // 8
+    assert_decompress_parity(c, ref, "f32", "budget 12")
+
+
 # ------------------------------------------------------------------ device-detected errors, guard bands
 def test_capacity_error_is_reported_and_nothing_is_written_out_of_bounds():
     rng = np.random.default_rng(3)
