@@ -201,15 +201,19 @@ def _ptr(t) -> int:
 def daf_compress(params, d_in, d_packed, packed_capacity, d_bits, d_min, d_scale, d_window_offsets, d_workspace,
                  workspace_bytes, stream=None):
     """Tensors (or None) in, status checked; everything else is the C call."""
-    _check(_call(lib().daf_compress, d_in, stream, ctypes.byref(params), _ptr(d_in), _ptr(d_packed), packed_capacity, _ptr(d_bits), _ptr(d_min),
-                              _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_workspace), workspace_bytes), "daf_compress")
+    status = _call(lib().daf_compress, d_in, stream, ctypes.byref(params), _ptr(d_in), _ptr(d_packed),
+                   packed_capacity, _ptr(d_bits), _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets),
+                   _ptr(d_workspace), workspace_bytes)
+    _check(status, "daf_compress")
 
 
 def daf_relu_compress(params, d_in, d_act, d_packed, packed_capacity, d_bits, d_min, d_scale, d_window_offsets, d_workspace,
                       workspace_bytes, stream=None):
     """Fused producer: d_act = max(d_in, +0) is written and compressed in one pass (d_act may be d_in)."""
-    _check(_call(lib().daf_relu_compress, d_in, stream, ctypes.byref(params), _ptr(d_in), _ptr(d_act), _ptr(d_packed), packed_capacity, _ptr(d_bits),
-                                   _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_workspace), workspace_bytes), "daf_relu_compress")
+    status = _call(lib().daf_relu_compress, d_in, stream, ctypes.byref(params), _ptr(d_in), _ptr(d_act),
+                   _ptr(d_packed), packed_capacity, _ptr(d_bits), _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets),
+                   _ptr(d_workspace), workspace_bytes)
+    _check(status, "daf_relu_compress")
 
 
 ACT_RELU, ACT_RELU6, ACT_GELU = 1, 2, 3
@@ -219,16 +223,18 @@ def daf_act_compress(params, act, d_in, d_act, d_packed, packed_capacity, d_bits
                      workspace_bytes, stream=None):
     """Fused producer for ReLU / ReLU6 / GELU: d_act = act(d_in) written in the same pass that compresses (the
     activation for ReLU and ReLU6, the input for GELU)."""
-    _check(_call(lib().daf_act_compress, d_in, stream, ctypes.byref(params), act, _ptr(d_in), _ptr(d_act), _ptr(d_packed),
-                 packed_capacity, _ptr(d_bits), _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_workspace),
-                 workspace_bytes), "daf_act_compress")
+    status = _call(lib().daf_act_compress, d_in, stream, ctypes.byref(params), act, _ptr(d_in), _ptr(d_act),
+                   _ptr(d_packed), packed_capacity, _ptr(d_bits), _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets),
+                   _ptr(d_workspace), workspace_bytes)
+    _check(status, "daf_act_compress")
 
 
 def daf_decompress_act_grad(params, act, d_packed, d_bits, d_min, d_scale, d_window_offsets, d_grad_out, d_grad_in, stream=None):
     """Fused consumer: the gradient of the activation from its compressed form (may be in place)."""
-    _check(_call(lib().daf_decompress_act_grad, d_grad_out, stream, ctypes.byref(params), act, _ptr(d_packed), _ptr(d_bits),
-                 _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_grad_out), _ptr(d_grad_in)),
-           "daf_decompress_act_grad")
+    status = _call(lib().daf_decompress_act_grad, d_grad_out, stream, ctypes.byref(params), act, _ptr(d_packed),
+                   _ptr(d_bits), _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_grad_out),
+                   _ptr(d_grad_in))
+    _check(status, "daf_decompress_act_grad")
 
 
 STATIC_MAX_WINDOWS = 65536
@@ -239,20 +245,25 @@ def daf_compress_static(params, d_in, d_packed, packed_capacity, d_bits, d_min, 
     """daf_compress for callers that cannot allocate a workspace: the kernel's scratch is a fixed
     array inside the library (at most STATIC_MAX_WINDOWS windows; calls must not overlap on the GPU).
     d_status: optional int32 tensor of one element that receives the device status word."""
-    _check(_call(lib().daf_compress_static, d_in, stream, ctypes.byref(params), _ptr(d_in), _ptr(d_packed), packed_capacity, _ptr(d_bits),
-                                     _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_status)), "daf_compress_static")
+    status = _call(lib().daf_compress_static, d_in, stream, ctypes.byref(params), _ptr(d_in), _ptr(d_packed),
+                   packed_capacity, _ptr(d_bits), _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_status))
+    _check(status, "daf_compress_static")
 
 
 def daf_decompress_relu_grad(params, d_packed, d_bits, d_min, d_scale, d_window_offsets, d_grad_out, d_grad_in, stream=None):
     """Fused consumer: d_grad_in = d_grad_out where the restored activation is > 0, else 0 (may be in place)."""
-    _check(_call(lib().daf_decompress_relu_grad, d_grad_out, stream, ctypes.byref(params), _ptr(d_packed), _ptr(d_bits), _ptr(d_min), _ptr(d_scale),
-                                          _ptr(d_window_offsets), _ptr(d_grad_out), _ptr(d_grad_in)), "daf_decompress_relu_grad")
+    status = _call(lib().daf_decompress_relu_grad, d_grad_out, stream, ctypes.byref(params), _ptr(d_packed),
+                   _ptr(d_bits), _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_grad_out),
+                   _ptr(d_grad_in))
+    _check(status, "daf_decompress_relu_grad")
 
 
 def daf_decompress(params, d_packed, d_bits, d_min, d_scale, d_window_offsets, d_out, d_workspace=None,
                    workspace_bytes=0, stream=None):
-    _check(_call(lib().daf_decompress, d_out, stream, ctypes.byref(params), _ptr(d_packed), _ptr(d_bits), _ptr(d_min), _ptr(d_scale),
-                                _ptr(d_window_offsets), _ptr(d_out), _ptr(d_workspace), workspace_bytes), "daf_decompress")
+    status = _call(lib().daf_decompress, d_out, stream, ctypes.byref(params), _ptr(d_packed), _ptr(d_bits),
+                   _ptr(d_min), _ptr(d_scale), _ptr(d_window_offsets), _ptr(d_out), _ptr(d_workspace),
+                   workspace_bytes)
+    _check(status, "daf_decompress")
 
 
 def daf_group_offsets_workspace(n_groups: int) -> int:
@@ -260,12 +271,16 @@ def daf_group_offsets_workspace(n_groups: int) -> int:
 
 
 def daf_group_offsets(d_bits, n_groups, group_size, d_offsets, d_ws, ws_bytes, stream=None):
-    _check(_call(lib().daf_group_offsets, d_bits, stream, _ptr(d_bits), n_groups, group_size, _ptr(d_offsets), _ptr(d_ws), ws_bytes), "daf_group_offsets")
+    status = _call(lib().daf_group_offsets, d_bits, stream, _ptr(d_bits), n_groups, group_size, _ptr(d_offsets),
+                   _ptr(d_ws), ws_bytes)
+    _check(status, "daf_group_offsets")
 
 
 def daf_group_offsets_diag(d_bits, n_groups, group_size, d_offsets, d_ws, ws_bytes, flags, stream=None):
     """daf_group_offsets with diagnostic flags (FLAG_KEEP_WORKSPACE, flag_poll_limit(n)): for tests of the bounded wait."""
-    _check(_call(lib().daf_group_offsets_diag, d_bits, stream, _ptr(d_bits), n_groups, group_size, _ptr(d_offsets), _ptr(d_ws), ws_bytes, flags), "daf_group_offsets_diag")
+    status = _call(lib().daf_group_offsets_diag, d_bits, stream, _ptr(d_bits), n_groups, group_size, _ptr(d_offsets),
+                   _ptr(d_ws), ws_bytes, flags)
+    _check(status, "daf_group_offsets_diag")
 
 
 def daf_poll_status(d_workspace, stream=None) -> int:
@@ -286,16 +301,18 @@ def daf_compress_batch(params_list, d_in, d_packed, capacities, d_bits, d_min, d
     n = len(params_list)
     arr = (daf_params * n)(*params_list)
     caps = (ctypes.c_uint64 * n)(*capacities)
-    _check(_call(lib().daf_compress_batch, d_in[0], stream, n, arr, _ptr_array(d_in), _ptr_array(d_packed), caps, _ptr_array(d_bits),
-                                    _ptr_array(d_min), _ptr_array(d_scale), _ptr_array(d_window_offsets), _ptr(d_workspace),
-                                    workspace_bytes), "daf_compress_batch")
+    status = _call(lib().daf_compress_batch, d_in[0], stream, n, arr, _ptr_array(d_in), _ptr_array(d_packed), caps,
+                   _ptr_array(d_bits), _ptr_array(d_min), _ptr_array(d_scale), _ptr_array(d_window_offsets),
+                   _ptr(d_workspace), workspace_bytes)
+    _check(status, "daf_compress_batch")
 
 
 def daf_decompress_batch(params_list, d_packed, d_bits, d_min, d_scale, d_window_offsets, d_out, stream=None):
     n = len(params_list)
     arr = (daf_params * n)(*params_list)
-    _check(_call(lib().daf_decompress_batch, d_out[0], stream, n, arr, _ptr_array(d_packed), _ptr_array(d_bits), _ptr_array(d_min),
-                                      _ptr_array(d_scale), _ptr_array(d_window_offsets), _ptr_array(d_out)), "daf_decompress_batch")
+    status = _call(lib().daf_decompress_batch, d_out[0], stream, n, arr, _ptr_array(d_packed), _ptr_array(d_bits),
+                   _ptr_array(d_min), _ptr_array(d_scale), _ptr_array(d_window_offsets), _ptr_array(d_out))
+    _check(status, "daf_decompress_batch")
 
 
 def daf_version() -> int:
