@@ -274,6 +274,34 @@ daf_status daf_compress_static(const daf_params *params, const void *d_in, void 
                                daf_stream stream);
 
 /*
+ * Per-tensor statistics and per-tensor quantization: Eq. 1 at the granularity the paper states it (one min, max and
+ * width per activation tensor; the group-wise calls above are the refinement the library is built around), with the
+ * collective reduction of Sec. 3.2.1-3.2.2 behind it: tree reduction inside a CTA, one integer atomic per CTA and
+ * statistic across CTAs (the paper's hybrid of both; its compare-and-swap loop on floats is replaced by a native
+ * atomic max on a monotone integer key).  No workspace; nothing is allocated.
+ *
+ *   d_in / d_out : numel elements of dtype (a daf_dtype); numel a positive multiple of 8 (DAF_ERR_SHAPE otherwise);
+ *                  32-byte aligned for DAF_F32, 16 otherwise.
+ *   d_stats      : device, 32 bytes, 16-byte aligned.  daf_tensor_minmax writes float words [0] min, [1] max (under the
+ *                  order in which -0 < +0), [2] range = max - min, or 0 when that is below 2^-118 (the tensor then
+ *                  counts as constant); words 4-7 are scratch.  daf_tensor_compress reads words 0 and 2.
+ *   d_packed     : numel * width / 8 bytes, 16-byte aligned; code i occupies bits [i*width, (i+1)*width), LSB first.
+ *   d_min_scale  : device, two floats: the minimum and scale = range / (2^width - 1) (0 for a constant tensor),
+ *                  written by daf_tensor_compress, read by daf_tensor_decompress.
+ *   width in {1,2,4,8}; rounding, seed, elem_index_base (a multiple of 8) as in daf_params: element i draws the 16-bit
+ *   lane (elem_index_base + i) & 7 of Philox block (elem_index_base + i) >> 3, exactly as the group-wise path does.
+ * The code of element i is min((RNE((x_i - min) * fl(L / range) * 2^15) + r15) >> 15, L) with L = 2^width - 1, i.e. the
+ * group-wise arithmetic with the whole tensor as the one group; decompress gives fma(code, scale, min) rounded to dtype.
+ * Errors: INVALID_ARG (null or misaligned pointer, bad dtype / width / rounding / base), SHAPE, CUDA.
+ */
+daf_status daf_tensor_minmax(uint32_t dtype, const void *d_in, uint64_t numel, void *d_stats, daf_stream stream);
+daf_status daf_tensor_compress(uint32_t dtype, const void *d_in, uint64_t numel, uint32_t width, uint32_t rounding,
+                               uint64_t seed, uint64_t elem_index_base, const void *d_stats, void *d_packed,
+                               float *d_min_scale, daf_stream stream);
+daf_status daf_tensor_decompress(uint32_t dtype, const void *d_packed, uint64_t numel, uint32_t width,
+                                 const float *d_min_scale, void *d_out, daf_stream stream);
+
+/*
  * Host-side page pool for packed buffers (Sec. 3.4.2: one preallocated contiguous arena,
  * page-granular first-fit allocation; Sec. 3.4.3: every allocation carries an importance,
  * and the least important one is evicted first).  The pool does bookkeeping only: it never

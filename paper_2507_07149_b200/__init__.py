@@ -95,6 +95,10 @@ SIGNATURES = {
     "daf_compress_batch": (ctypes.c_int, [ctypes.c_uint32, ctypes.POINTER(daf_params), _vp, _vp, _u64p, _vp, _vp, _vp, _vp,
                                           _vp, ctypes.c_uint64, _vp]),
     "daf_decompress_batch": (ctypes.c_int, [ctypes.c_uint32, ctypes.POINTER(daf_params), _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "daf_tensor_minmax": (ctypes.c_int, [ctypes.c_uint32, _vp, ctypes.c_uint64, _vp, _vp]),
+    "daf_tensor_compress": (ctypes.c_int, [ctypes.c_uint32, _vp, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint32,
+                                           ctypes.c_uint64, ctypes.c_uint64, _vp, _vp, _vp, _vp]),
+    "daf_tensor_decompress": (ctypes.c_int, [ctypes.c_uint32, _vp, ctypes.c_uint64, ctypes.c_uint32, _vp, _vp, _vp]),
     "daf_pool_create": (_vp, [ctypes.c_uint64, ctypes.c_uint64]),
     "daf_pool_destroy": (None, [_vp]),
     "daf_pool_alloc": (ctypes.c_uint64, [_vp, ctypes.c_uint64, ctypes.c_double, _u64p]),
@@ -407,6 +411,46 @@ def relu_grad(c: CompressedTensor, grad_out, out=None, stream=None, act: int = A
     if out is None:
         out = torch.empty_like(grad_out)
     daf_decompress_act_grad(c.params, act, c.packed, c.bits, c.min, c.scale, c.window_offsets, grad_out, out, stream)
+    return out
+
+
+# ------------------------------------------------------------------------------------ per-tensor path
+def daf_tensor_minmax(d_in, d_stats, stream=None):
+    """min, max and range of the whole tensor into d_stats (8 x 32-bit words on the device: floats 0-2, scratch 4-7)."""
+    status = _call(lib().daf_tensor_minmax, d_in, stream, dtype_code(d_in), _ptr(d_in), d_in.numel(), _ptr(d_stats))
+    _check(status, "daf_tensor_minmax")
+
+
+def daf_tensor_compress(d_in, width, d_stats, d_packed, d_min_scale, *, rounding=ROUND_STOCHASTIC, seed=0, elem_index_base=0,
+                        stream=None):
+    status = _call(lib().daf_tensor_compress, d_in, stream, dtype_code(d_in), _ptr(d_in), d_in.numel(), width, rounding, seed,
+                   elem_index_base, _ptr(d_stats), _ptr(d_packed), _ptr(d_min_scale))
+    _check(status, "daf_tensor_compress")
+
+
+def daf_tensor_decompress(d_packed, width, d_min_scale, d_out, stream=None):
+    status = _call(lib().daf_tensor_decompress, d_out, stream, dtype_code(d_out), _ptr(d_packed), d_out.numel(), width,
+                   _ptr(d_min_scale), _ptr(d_out))
+    _check(status, "daf_tensor_decompress")
+
+
+def tensor_compress(x, width: int, *, rounding: int = ROUND_STOCHASTIC, seed: int = 0, elem_index_base: int = 0, stream=None):
+    """Eq. 1 with one min / max / width for the whole tensor: (packed uint8 tensor, min_scale float tensor, stats)."""
+    torch = _torch()
+    if not x.is_cuda or not x.is_contiguous():
+        raise ValueError("tensor_compress expects a contiguous CUDA tensor")
+    stats = torch.empty(8, dtype=torch.int32, device=x.device)
+    packed = torch.empty(max(x.numel() * width // 8, 16), dtype=torch.uint8, device=x.device)
+    min_scale = torch.empty(2, dtype=torch.float32, device=x.device)
+    daf_tensor_minmax(x, stats, stream)
+    daf_tensor_compress(x, width, stats, packed, min_scale, rounding=rounding, seed=seed, elem_index_base=elem_index_base,
+                        stream=stream)
+    return packed, min_scale, stats
+
+
+def tensor_decompress(packed, width: int, min_scale, shape, dtype, stream=None):
+    out = _torch().empty(shape, dtype=dtype, device=packed.device)
+    daf_tensor_decompress(packed, width, min_scale, out, stream)
     return out
 
 

@@ -15,7 +15,7 @@ HEADERS = [os.path.join(CSRC, h) for h in ("common.cuh", "compress_shared.cuh", 
     os.path.join(os.path.dirname(HERE), "include", "daf.h")]
 
 CU_SOURCES = ["api.cu", "compress.cu", "compress_stream_f32.cu", "compress_stream_f16.cu", "compress_stream_bf16.cu", "compress_general_f32.cu", "compress_general_f16.cu",
-              "compress_general_bf16.cu", "decompress.cu", "group_offsets.cu"]
+              "compress_general_bf16.cu", "decompress.cu", "group_offsets.cu", "tensorwise.cu"]
 CXX_SOURCES = ["pool.cpp", "store.cpp"]
 
 # No fast-math, no flush-to-zero, no fused contraction beyond what the sources write out:

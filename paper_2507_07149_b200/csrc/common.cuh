@@ -312,4 +312,23 @@ template <int ACT> __device__ __forceinline__ void activate8(float (&x)[8], floa
     }
 }
 
+// Eight codes of width B (LSB-first in w0, and w1 for B = 8) back to values: the code is widened with the power-of-two
+// offset of Eq. 5 (bits | 0x4B000000 is the float 2^23 + code), then x_hat = fma(code, scale, min).
+template <int B> __device__ __forceinline__ void decode8(uint32_t w0, uint32_t w1, float mn, float scale, float (&y)[8])
+{
+    constexpr uint32_t L = (1u << B) - 1u;
+#pragma unroll
+    for (int i = 0; i < 8; i++) {
+        uint32_t f;
+        if (B == 8) {
+            // byte i of the pair of words into the low byte of 0x4B0000xx in one permute
+            f = __byte_perm(i < 4 ? w0 : w1, 0x4B000000u, 0x7540u | (uint32_t)(i & 3));
+        } else {
+            f = ((w0 >> (B * i)) & L) | 0x4B000000u;
+        }
+        const float q = __fsub_rn(__uint_as_float(f), 8388608.0f);   // exact: f is the float 2^23 + code
+        y[i] = __fmaf_rn(q, scale, mn);
+    }
+}
+
 }  // namespace daf

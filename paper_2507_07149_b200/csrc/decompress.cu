@@ -33,23 +33,6 @@ struct DecRec {
     uint32_t b, off;
 };
 
-template <int B> __device__ __forceinline__ void decode8(uint32_t w0, uint32_t w1, float mn, float scale, float (&y)[8])
-{
-    constexpr uint32_t L = (1u << B) - 1u;
-#pragma unroll
-    for (int i = 0; i < 8; i++) {
-        uint32_t f;
-        if (B == 8) {
-            // byte i of the pair of words into the low byte of 0x4B0000xx in one permute
-            f = __byte_perm(i < 4 ? w0 : w1, 0x4B000000u, 0x7540u | (uint32_t)(i & 3));
-        } else {
-            f = ((w0 >> (B * i)) & L) | 0x4B000000u;
-        }
-        const float q = __fsub_rn(__uint_as_float(f), 8388608.0f);   // exact: f is the float 2^23 + code
-        y[i] = __fmaf_rn(q, scale, mn);
-    }
-}
-
 // The restored value as it would be stored in type T (round to nearest even), back in binary32.
 template <typename T> __device__ __forceinline__ float as_stored(float y);
 template <> __device__ __forceinline__ float as_stored<float>(float y) { return y; }

@@ -1,6 +1,6 @@
 """Times compress / decompress on the five benchmark workloads and the group-size x budget sweep.
 
-    python -m paper_2507_07149_b200.sweep [--configs 1,2,3,4,5] [--sweep] [--relu] [--steps K] [--scale S]
+    python -m paper_2507_07149_b200.sweep [--configs 1,2,3,4,5] [--sweep] [--relu] [--tensorwise] [--steps K] [--scale S]
 
 Workloads 1-4 are sets of tensors: each set goes through ONE batched call (daf_compress_batch /
 daf_decompress_batch) when it has at most DAF_BATCH_MAX tensors.  Inputs are the seeded synthetic
@@ -123,6 +123,8 @@ def main():
     ap.add_argument("--relu", action="store_true",
                     help="also the fused producers and consumers (ReLU, ReLU6, GELU) on workload 5, each against torch's own "
                          "kernel followed / preceded by daf_compress / daf_decompress")
+    ap.add_argument("--tensorwise", action="store_true",
+                    help="also the per-tensor path on workload 5: min / max reduction, Eq. 1 with one min / max / width, its inverse")
     args = ap.parse_args()
 
     import torch
@@ -199,6 +201,21 @@ def main():
                       f"{packed / 2**30:.3f} | — | — | {t_fb:.4f} | {alg / t_fb / 1e6:.0f} | — | daf_decompress + torch's "
                       f"{name} backward: {t_sb:.4f} |", flush=True)
             del act, c, g, gi
+        if cfg == 5 and args.tensorwise:
+            x = xs[0]
+            width = int(w.bit_budget)
+            stats = torch.empty(8, dtype=torch.int32, device=x.device)
+            packed = torch.empty(x.numel() * width // 8, dtype=torch.uint8, device=x.device)
+            ms = torch.empty(2, dtype=torch.float32, device=x.device)
+            y = torch.empty_like(x)
+            t_m = _time(torch, lambda: daf.daf_tensor_minmax(x, stats), args.steps, False)
+            t_q = _time(torch, lambda: daf.daf_tensor_compress(x, width, stats, packed, ms), args.steps, False)
+            t_d = _time(torch, lambda: daf.daf_tensor_decompress(packed, width, ms, y), args.steps, False)
+            nb, pb = w.nbytes, packed.numel()
+            print(f"| {w.name} per-tensor min / max | {w.numel} | {nb / 2**30:.3f} | — | {t_m:.4f} | {nb / t_m / 1e6:.0f} | — | — | — | — |")
+            print(f"| {w.name} per-tensor quantize (width {width}) / dequantize | {w.numel} | {nb / 2**30:.3f} | {pb / 2**30:.3f} | "
+                  f"{t_q:.4f} | {(nb + pb) / t_q / 1e6:.0f} | {t_d:.4f} | {(nb + pb) / t_d / 1e6:.0f} | — | — |", flush=True)
+            del stats, packed, ms, y
         del xs
         torch.cuda.empty_cache()
 
