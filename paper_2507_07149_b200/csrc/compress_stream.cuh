@@ -349,7 +349,11 @@ static cudaError_t launch_stream(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &
     const cudaError_t e = persistent_ctas(reinterpret_cast<const void *>(&stream_compress_kernel<T, CHUNKS, B, GC, BATCH, ACT>),
                                           kThreads, 0, &ctas);
     if (e != cudaSuccess) return e;
-    const uint32_t grid = args.total_windows < (uint32_t)ctas ? args.total_windows : (uint32_t)ctas;
+    // eight times the CTAs the device holds at once: no CTA waits for another here, and with several waves the block
+    // scheduler evens out the CTAs' finishing times (measured on 2^30 elements: 0.839 ms at 1x, 0.824 at 2x, 0.815 at 4x,
+    // 0.814 at 8x, 0.818 at 16x, 0.831 at 32x, 0.926 with one CTA per window)
+    const uint32_t want = (uint32_t)ctas * 8u;
+    const uint32_t grid = args.total_windows < want ? args.total_windows : want;
     stream_compress_kernel<T, CHUNKS, B, GC, BATCH, ACT><<<grid, kThreads, 0, stream>>>(args);
     return cudaGetLastError();
 }

@@ -147,10 +147,104 @@ decompress_kernel(const __grid_constant__ DecompressArgs<BATCH ? DAF_BATCH_MAX :
     }
 }
 
+// The same for windows of at most 64 groups (groups of 256 elements or more at the default window): no shared memory
+// and no meeting of the CTA's warps.  Every warp reads the widths of the window's groups itself (two per lane, 64 bytes
+// that sit in L1 after the first warp), scans their byte lengths with shuffles and serves its own chunks; a chunk lies
+// in one group, so width, offset, min and scale are the same for all its lanes.
+template <typename T, int CHUNKS, bool BATCH, int MASK>
+__global__ void __launch_bounds__(kThreads)
+decompress_few_groups_kernel(const __grid_constant__ DecompressArgs<BATCH ? DAF_BATCH_MAX : 1> a)
+{
+    constexpr uint32_t WE = kThreads * kLaneElems * CHUNKS;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t G = a.G, log2G = a.log2G;
+    const uint32_t gw = blockIdx.x;
+    uint32_t ti = 0;
+    if (BATCH) {
+        uint32_t lo = 0, hi = a.n_tensors - 1;
+        while (lo < hi) {
+            uint32_t mid = (lo + hi + 1) >> 1;
+            if (a.t[mid].first_window <= gw) lo = mid; else hi = mid - 1;
+        }
+        ti = lo;
+    }
+    const DecTensor &td = a.t[ti];
+    const uint32_t w = gw - td.first_window;
+    const uint64_t wbase = (uint64_t)w * WE;
+    const uint64_t left = td.numel - wbase;
+    const uint32_t n_elems = left < WE ? (uint32_t)left : WE;
+    const uint32_t n = n_elems >> log2G;
+    const uint64_t g0 = wbase >> log2G;
+    const uint32_t first_chunk = (uint32_t)warp * CHUNKS * 256u;
+    if (first_chunk >= n_elems) return;                           // (a ragged window: nothing for this warp)
+
+    const uint64_t window_offset = td.woff[w];
+    const uint32_t b0 = (uint32_t)lane < n ? td.bits[g0 + lane] : 0u, b1 = (uint32_t)lane + 32u < n ? td.bits[g0 + lane + 32] : 0u;
+    // min and scale of the warp's chunks' groups, asked for early
+    float mn[CHUNKS], scale[CHUNKS];
+#pragma unroll
+    for (int c = 0; c < CHUNKS; c++) {
+        const uint32_t cs = first_chunk + 256u * c;
+        const uint32_t g = cs < n_elems ? cs >> log2G : 0u;
+        mn[c] = td.mn[g0 + g];
+        scale[c] = td.scale[g0 + g];
+    }
+    const uint32_t size0 = (G >> 3) * b0, size1 = (G >> 3) * b1;
+    uint32_t incl0 = size0, incl1 = size1;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t y0 = __shfl_up_sync(0xFFFFFFFFu, incl0, off), y1 = __shfl_up_sync(0xFFFFFFFFu, incl1, off);
+        if (lane >= off) {
+            incl0 += y0;
+            incl1 += y1;
+        }
+    }
+    const uint32_t excl0 = incl0 - size0, excl1 = __shfl_sync(0xFFFFFFFFu, incl0, 31) + incl1 - size1;
+
+    const uint8_t *src = td.packed + window_offset;
+    char *out = reinterpret_cast<char *>(td.out) + wbase * Elem<T>::kBytes;
+#pragma unroll
+    for (int c = 0; c < CHUNKS; c++) {
+        const uint32_t cs = first_chunk + 256u * c;               // the chunk's first element: the same for all lanes
+        if (cs >= n_elems) break;
+        const uint32_t g = cs >> log2G, from = g & 31u;
+        const uint32_t b = __shfl_sync(0xFFFFFFFFu, g < 32u ? b0 : b1, (int)from);
+        const uint32_t goff = __shfl_sync(0xFFFFFFFFu, g < 32u ? excl0 : excl1, (int)from);
+        const uint32_t e = cs + (uint32_t)lane * 8u;
+        const uint8_t *p = src + goff + ((e & (G - 1u)) >> 3) * b;
+        float y[8];
+        switch (b) {
+        case 1: decode8<1>(*p, 0u, mn[c], scale[c], y); break;
+        case 2: decode8<2>(*reinterpret_cast<const uint16_t *>(p), 0u, mn[c], scale[c], y); break;
+        case 4: decode8<4>(*reinterpret_cast<const uint32_t *>(p), 0u, mn[c], scale[c], y); break;
+        default: {
+            const uint2 v = *reinterpret_cast<const uint2 *>(p);
+            decode8<8>(v.x, v.y, mn[c], scale[c], y);
+            break;
+        }
+        }
+        if (MASK != kActNone) {
+            float gr[8];
+            Elem<T>::load8(reinterpret_cast<const char *>(td.grad) + (wbase + e) * Elem<T>::kBytes, gr);
+#pragma unroll
+            for (int i = 0; i < 8; i++) {
+                const float r = as_stored<T>(y[i]);
+                if (MASK == kActRelu) y[i] = r > 0.0f ? gr[i] : 0.0f;
+                else if (MASK == kActRelu6) y[i] = (r > 0.0f && r < 6.0f) ? gr[i] : 0.0f;
+                else y[i] = gr[i] * gelu_grad_f(r);
+            }
+        }
+        Elem<T>::store8(out + (size_t)e * Elem<T>::kBytes, y);
+    }
+}
+
 template <typename T, int CHUNKS, bool BATCH, int MASK>
 static cudaError_t launch(const DecompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
-    decompress_kernel<T, CHUNKS, BATCH, MASK><<<args.total_windows, kThreads, 0, stream>>>(args);
+    if (args.G >= 256u)                                           // a chunk lies in one group, a window has at most 64
+        decompress_few_groups_kernel<T, CHUNKS, BATCH, MASK><<<args.total_windows, kThreads, 0, stream>>>(args);
+    else
+        decompress_kernel<T, CHUNKS, BATCH, MASK><<<args.total_windows, kThreads, 0, stream>>>(args);
     return cudaGetLastError();
 }
 
