@@ -32,10 +32,10 @@ FALLBACK_HBM_GBS = 6650.0
 # on a 2^27-element fp32 slice of this workload (G = 256, budget 4): profiles/stream_compress_kernel_cfg5_G256_b4.md
 # (546.50 MB read + 66.13 MB written) and profiles/decompress_kernel_cfg5_G256_b4.md (71.91 + 477.73 MB).
 # Traffic grows in proportion to the element count, so it is scaled to the launch being timed.
-NCU_TRAFFIC_BYTES_PER_ELEM = {"compress": 612.62e6 / (1 << 27), "decompress": 549.83e6 / (1 << 27)}
+NCU_TRAFFIC_BYTES_PER_ELEM = {"compress": 603.02e6 / (1 << 27), "decompress": 549.75e6 / (1 << 27)}
 # (The decompress capture is a 512 MiB output: part of its stores still sits in L2 when the kernel ends, so the scaled
 # figure understates the traffic of a full-size launch by the same amount.)
-KERNEL_NAME = {"compress": "stream_compress_kernel", "decompress": "decompress_kernel"}
+KERNEL_NAME = {"compress": "stream_compress_kernel", "decompress": "decompress_few_groups_kernel"}
 # Kernels of this library launched per step on this workload: the streaming compress kernel, its verify kernel, the
 # general compress kernel (which finds nothing to redo and returns), the decompress kernel.
 LAUNCHES_PER_STEP = 4
@@ -276,7 +276,10 @@ def run_cuda(args):
     def roof(kernel, ms):
         a = alg / (ms * 1e-3) / 1e9
         tr = NCU_TRAFFIC_BYTES_PER_ELEM[kernel] if profiled else None
-        return {"bound": "hbm", "kernel": KERNEL_NAME[kernel], "achieved": a, "peak": peak, "unit": "GB/s",
+        name = KERNEL_NAME[kernel]
+        if kernel == "decompress" and G < 256:
+            name = "decompress_kernel"                            # (groups below 256 elements take the variant with group records)
+        return {"bound": "hbm", "kernel": name, "achieved": a, "peak": peak, "unit": "GB/s",
                 "frac": a / peak, "peak_source": peak_src, "frac_of_nominal_8TBs": a / NOMINAL_HBM_GBS,
                 "algorithmic_bytes_per_launch": alg, "avg_launch_ms": ms,
                 "traffic": None if tr is None else tr * spec.numel}

@@ -31,6 +31,25 @@ def _device_tensor(torch, wl, cfg, ti, spec):
 
 
 _FLUSH = None
+_NVML = None
+
+
+def _sm_mhz(torch):
+    """SM clock right now (read while the GPU is still busy with the point just timed), or None without NVML."""
+    global _NVML
+    try:
+        if _NVML is None:
+            import pynvml
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(torch.cuda.current_device()).uuid)
+            _NVML = (pynvml, pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid if not uuid.startswith("GPU-") else uuid).encode()))
+        n, h = _NVML
+        return int(n.nvmlDeviceGetClockInfo(h, n.NVML_CLOCK_SM))
+    except Exception:
+        return None
+
+
+COOLDOWN_S = 0.0
 
 
 def _time(torch, fn, steps, flush):
@@ -40,16 +59,22 @@ def _time(torch, fn, steps, flush):
     global _FLUSH
     if flush and _FLUSH is None:
         _FLUSH = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    if COOLDOWN_S > 0:
+        import time
+        torch.cuda.synchronize()
+        time.sleep(COOLDOWN_S)
     for _ in range(3):
         fn()
     torch.cuda.synchronize()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    global LAST_MHZ
     for e0, e1 in ev:
         if flush:
             _FLUSH.fill_(1)
         e0.record()
         fn()
         e1.record()
+    LAST_MHZ = _sm_mhz(torch)                                      # the queue is still draining: a clock under load
     torch.cuda.synchronize()
     return float(np.median([e0.elapsed_time(e1) for e0, e1 in ev]))
 
@@ -107,11 +132,14 @@ def run_set(torch, daf, wl, w, xs, steps):
     return t_c, t_d, packed, meta, per_tensor
 
 
+LAST_MHZ = None
+
+
 def row(name, numel, nbytes, packed, meta, t_c, t_d, per_tensor=None):
     alg = nbytes + packed + meta
     each = "— | —" if per_tensor is None else f"{per_tensor[0]:.4f} | {per_tensor[1]:.4f}"
     return (f"| {name} | {numel} | {nbytes / 2**30:.3f} | {packed / 2**30:.3f} | {t_c:.4f} | {alg / t_c / 1e6:.0f} | "
-            f"{t_d:.4f} | {alg / t_d / 1e6:.0f} | {each} |")
+            f"{t_d:.4f} | {alg / t_d / 1e6:.0f} | {each} | {LAST_MHZ if LAST_MHZ is not None else '—'} |")
 
 
 def main():
@@ -123,6 +151,9 @@ def main():
     ap.add_argument("--relu", action="store_true",
                     help="also the fused producers and consumers (ReLU, ReLU6, GELU) on workload 5, each against torch's own "
                          "kernel followed / preceded by daf_compress / daf_decompress")
+    ap.add_argument("--cooldown", type=float, default=1.0,
+                    help="seconds of idle before every point, so that each is timed from the same state: back to back the points "
+                         "run into the board's power cap and the SM clock falls from 1965 to about 1600 MHz (see the last column)")
     ap.add_argument("--tensorwise", action="store_true",
                     help="also the per-tensor path on workload 5: min / max reduction, Eq. 1 with one min / max / width, its inverse")
     args = ap.parse_args()
@@ -132,9 +163,11 @@ def main():
     from paper_2507_07149_b200 import workloads as wl
 
     daf.lib()
+    global COOLDOWN_S
+    COOLDOWN_S = args.cooldown
     print("| workload | elements | tensor GiB | packed GiB | compress ms | compress GB/s | decompress ms | decompress GB/s "
-          "| compress ms, one call per tensor | decompress ms, one call per tensor |")
-    print("|---|---|---|---|---|---|---|---|---|---|")
+          "| compress ms, one call per tensor | decompress ms, one call per tensor | SM MHz under load |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|")
     S = args.scale
     for cfg in [int(c) for c in args.configs.split(",")]:
         kw = {}
