@@ -152,7 +152,7 @@ decompress_kernel(const __grid_constant__ DecompressArgs<BATCH ? DAF_BATCH_MAX :
 // that sit in L1 after the first warp), scans their byte lengths with shuffles and serves its own chunks; a chunk lies
 // in one group, so width, offset, min and scale are the same for all its lanes.
 template <typename T, int CHUNKS, bool BATCH, int MASK>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, MASK == kActGelu ? 3 : 4)   // (32 registers: four CTAs per SM; the GELU factor needs more)
 decompress_few_groups_kernel(const __grid_constant__ DecompressArgs<BATCH ? DAF_BATCH_MAX : 1> a)
 {
     constexpr uint32_t WE = kThreads * kLaneElems * CHUNKS;
