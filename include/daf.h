@@ -108,6 +108,17 @@ daf_status daf_sizes(const daf_params *params, uint64_t *n_groups, uint64_t *n_w
                      uint64_t *packed_capacity_bytes, uint64_t *workspace_bytes);
 
 /*
+ * Sharding (host only).  The path has no exchange step: a tensor is cut at window boundaries, every rank (GPU)
+ * compresses its slice with the same seed and with elem_index_base moved to the slice's first element, and the results
+ * are exactly the pieces of the unsharded result (widths, minima, scales, packed bytes; window offsets restart at 0 in
+ * every slice).  daf_shard fills *shard with the parameters of the slice of rank `rank` among `world` ranks -- whole
+ * windows, as even as possible, in order -- and *first_elem (may be NULL) with the slice's first element.  A rank
+ * beyond the number of windows gets shard->numel == 0: nothing to do.  Errors: those of daf_sizes for `whole`;
+ * INVALID_ARG for a null shard, world == 0 or rank >= world.
+ */
+daf_status daf_shard(const daf_params *whole, uint32_t rank, uint32_t world, daf_params *shard, uint64_t *first_elem);
+
+/*
  * Compress one tensor (Eq. 1 applied per group; widths chosen greedily per window by
  * importance per bit under the budget, Sec. 3.4.1; codes packed compactly, Sec. 3.3).
  *   d_in             in : numel elements of params->dtype; 32-byte aligned for DAF_F32 (a lane reads

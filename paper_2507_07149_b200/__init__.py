@@ -75,6 +75,7 @@ _vp = ctypes.c_void_p
 # name -> (restype, argtypes): every symbol include/daf.h declares
 SIGNATURES = {
     "daf_sizes": (ctypes.c_int, [ctypes.POINTER(daf_params), _u64p, _u64p, _u64p, _u64p]),
+    "daf_shard": (ctypes.c_int, [ctypes.POINTER(daf_params), ctypes.c_uint32, ctypes.c_uint32, ctypes.POINTER(daf_params), _u64p]),
     "daf_compress": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, ctypes.c_uint64, _vp, _vp, _vp, _vp, _vp,
                                     ctypes.c_uint64, _vp]),
     "daf_relu_compress": (ctypes.c_int, [ctypes.POINTER(daf_params), _vp, _vp, _vp, ctypes.c_uint64, _vp, _vp, _vp, _vp, _vp,
@@ -172,6 +173,13 @@ def daf_sizes(params: daf_params) -> Sizes:
     v = [ctypes.c_uint64() for _ in range(4)]
     _check(lib().daf_sizes(ctypes.byref(params), *[ctypes.byref(x) for x in v]), "daf_sizes")
     return Sizes(*[int(x.value) for x in v])
+
+
+def daf_shard(params: daf_params, rank: int, world: int):
+    """(parameters of rank's window-aligned slice, its first element); the slice's numel is 0 when there is none."""
+    shard, first = daf_params(), ctypes.c_uint64()
+    _check(lib().daf_shard(ctypes.byref(params), rank, world, ctypes.byref(shard), ctypes.byref(first)), "daf_shard")
+    return shard, int(first.value)
 
 
 def _torch():

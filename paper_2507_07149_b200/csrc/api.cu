@@ -103,6 +103,25 @@ extern "C" daf_status daf_sizes(const daf_params *params, uint64_t *n_groups, ui
     return DAF_OK;
 }
 
+// The window-aligned slice of a tensor that rank `rank` of `world` takes: whole windows, as even as possible, in order.
+extern "C" daf_status daf_shard(const daf_params *whole, uint32_t rank, uint32_t world, daf_params *shard, uint64_t *first_elem)
+{
+    Plan pl;
+    const daf_status st = make_plan(whole, &pl);
+    if (st != DAF_OK) return st;
+    if (!shard || world == 0 || rank >= world) return DAF_ERR_INVALID_ARG;
+    const uint64_t per = pl.n_windows / world, extra = pl.n_windows % world;
+    const uint64_t w_lo = (uint64_t)rank * per + (rank < extra ? rank : extra), w_hi = w_lo + per + (rank < extra ? 1u : 0u);
+    uint64_t lo = w_lo * pl.We, hi = w_hi * pl.We;
+    if (lo > whole->numel) lo = whole->numel;
+    if (hi > whole->numel) hi = whole->numel;
+    *shard = *whole;
+    shard->numel = hi - lo;                                       // 0: more ranks than windows, nothing for this one
+    shard->elem_index_base = whole->elem_index_base + lo;
+    if (first_elem) *first_elem = lo;
+    return DAF_OK;
+}
+
 extern "C" daf_status daf_poll_status(const void *d_workspace, daf_stream stream)
 {
     if (!d_workspace) return DAF_ERR_INVALID_ARG;

@@ -400,6 +400,34 @@ def _random_configuration(case):
     assert_decompress_parity(c, ref, dtype, label)
 
 
+def test_shards_cut_by_daf_shard_reproduce_the_unsharded_result():
+    """Three ranks' slices (daf_shard: window-aligned, bases moved) compressed one by one equal the pieces of the oracle's
+    result for the whole tensor: widths, minima, scales, packed bytes; window offsets restart in every slice."""
+    rng = np.random.default_rng(77)
+    G, widths, beta, seed = 128, (1, 2, 4, 8), 3.0, 5
+    n = 16384 * 10 + 128 * 9
+    a = (rng.standard_normal(n) * np.repeat(10.0 ** rng.uniform(-1, 1, n // G), G)).astype(np.float32)
+    ref = oracle.compress(a, G, widths, beta, seed=seed)
+    x = to_device(a, "f32")
+    whole = daf.make_params(daf.F32, n, G, widths, beta, seed=seed)
+    for rank in range(3):
+        p, first = daf.daf_shard(whole, rank, 3)
+        m = int(p.numel)
+        c = daf.alloc_outputs(p, "cuda")
+        daf.daf_compress(p, x[first:first + m], c.packed, c.sizes.packed_capacity, c.bits, c.min, c.scale, c.window_offsets,
+                         c.workspace, c.sizes.workspace)
+        assert daf.daf_poll_status(c.workspace) == daf.OK
+        g0, g1 = first // G, (first + m) // G
+        w0 = first // 16384
+        assert np.array_equal(c.bits.cpu().numpy(), ref.bits[g0:g1])
+        assert np.array_equal(c.min.cpu().numpy().view(np.uint32), ref.mn[g0:g1].view(np.uint32))
+        assert np.array_equal(c.scale.cpu().numpy().view(np.uint32), ref.scale[g0:g1].view(np.uint32))
+        woff = c.window_offsets.cpu().numpy().view(np.uint64)
+        base = int(ref.window_offsets[w0])
+        assert np.array_equal(woff + np.uint64(base), ref.window_offsets[w0:w0 + woff.size])
+        assert np.array_equal(c.packed[: int(woff[-1])].cpu().numpy(), ref.packed[base: base + int(woff[-1])])
+
+
 # ------------------------------------------------------------------ batched calls
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_batched_calls_equal_single_calls(dtype):

@@ -64,3 +64,26 @@ def test_shard_ranges_cover_the_tensor_in_whole_windows():
         assert cuts[0][0] == 0 and cuts[-1][1] == numel
         for (a, b), (c, d) in zip(cuts, cuts[1:]):
             assert b == c and a % WE == 0
+
+
+def test_daf_shard_cuts_where_the_generator_of_the_bench_does():
+    """The library's own sharding call against the window arithmetic written out here: whole windows, as even as
+    possible, in order; bases move with the slices; ranks beyond the windows get nothing."""
+    import paper_2507_07149_b200 as daf
+    for numel, we, G in ((16384 * 10 + 256 * 3, 0, 256), (4096 * 7, 4096, 64), (16384, 0, 1024), (8192 * 5 + 128, 8192, 128)):
+        WE_ = we or 16384
+        p = daf.make_params(daf.F32, numel, G, (1, 2, 4, 8), 4.0, window_elems=we, seed=9, elem_index_base=8 * 5)
+        for world in (1, 2, 3, 8, 64):
+            at = 0
+            for rank in range(world):
+                shard, first = daf.daf_shard(p, rank, world)
+                lo, hi = wl.shard_range(numel, WE_, rank, world)
+                assert (first, int(shard.numel)) == (lo, hi - lo) and first == at
+                assert int(shard.elem_index_base) == 40 + lo and int(shard.seed) == 9 and int(shard.group_size) == G
+                assert lo % WE_ == 0 or lo == numel
+                at += int(shard.numel)
+            assert at == numel
+    with pytest.raises(daf.DafError):
+        daf.daf_shard(p, 3, 3)
+    with pytest.raises(daf.DafError):
+        daf.daf_shard(p, 0, 0)
