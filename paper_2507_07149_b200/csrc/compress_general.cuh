@@ -57,6 +57,17 @@ __device__ __forceinline__ void load_and_reduce(const unsigned char *stage, int 
         if (LPU == 32) {
             asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(lo) : "f"(lo));
             asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(hi) : "f"(hi));
+        } else if (LPU == 16) {
+            // two units per chunk: a warp-wide reduction for each half, the other half's lanes holding the identity
+            const bool upper = lane >= 16;
+            const float inf = __uint_as_float(0x7F800000u), ninf = __uint_as_float(0xFF800000u);
+            float lo_a = upper ? inf : lo, lo_b = upper ? lo : inf, hi_a = upper ? ninf : hi, hi_b = upper ? hi : ninf;
+            asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(lo_a) : "f"(lo_a));
+            asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(lo_b) : "f"(lo_b));
+            asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(hi_a) : "f"(hi_a));
+            asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(hi_b) : "f"(hi_b));
+            lo = upper ? lo_b : lo_a;
+            hi = upper ? hi_b : hi_a;
         } else {
 #pragma unroll
             for (int off = 1; off < LPU; off <<= 1) {

@@ -194,17 +194,24 @@ stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MA
                 constexpr int c = decltype(ct)::value;
                 float lo, hi;
                 extremes8(x[c], lo, hi);
-                lo = fmin2(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, 1));
-                hi = fmax2(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, 1));
-                lo = fmin2(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, 2));
-                hi = fmax2(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, 2));
-                if (lpg > 4u) {
-                    lo = fmin2(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, 4));
-                    hi = fmax2(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, 4));
-                }
-                if (lpg > 8u) {
-                    lo = fmin2(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, 8));
-                    hi = fmax2(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, 8));
+                if (lpg == 16u) {
+                    // two groups per chunk: a warp-wide reduction for each half, the other half's lanes holding the
+                    // identity (four redux and four selects instead of eight shuffles and eight min / max)
+                    const bool upper = lane >= 16;
+                    const float inf = __uint_as_float(0x7F800000u), ninf = __uint_as_float(0xFF800000u);
+                    const float lo_a = warp_min(upper ? inf : lo), lo_b = warp_min(upper ? lo : inf);
+                    const float hi_a = warp_max(upper ? ninf : hi), hi_b = warp_max(upper ? hi : ninf);
+                    lo = upper ? lo_b : lo_a;
+                    hi = upper ? hi_b : hi_a;
+                } else {
+                    lo = fmin2(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, 1));
+                    hi = fmax2(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, 1));
+                    lo = fmin2(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, 2));
+                    hi = fmax2(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, 2));
+                    if (lpg > 4u) {
+                        lo = fmin2(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, 4));
+                        hi = fmax2(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, 4));
+                    }
                 }
                 float R;
                 const float inv = inverse_scale<B>(lo, hi, R);
