@@ -24,7 +24,7 @@
 // share a group exchange their extremes through shared memory at a named barrier of their own.
 //
 // The kernel is a template over the element type, the strip length, the width B, the relation
-// of group size and strip (GC: 0 = groups below 256 elements, 1 = groups of whole chunks inside
+// of group size and strip (GC: 0 = groups below 128 elements, 3 = groups of 128, 1 = groups of whole chunks inside
 // a strip, 2 = groups of one or more strips), batched calls and the fused ReLU; this header is
 // included by one translation unit per element type.
 #pragma once
@@ -186,7 +186,7 @@ stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MA
             }
         };
 
-        if (GC == 0) {
+        if (GC == 0 || GC == 3) {
             // ---- several groups per chunk: a segmented shuffle leaves every lane with its own group's extremes; the lane
             // whose position in its group equals the chunk number parks the group
             const uint32_t lpg = 1u << (log2G - 3u);              // lanes per group (4, 8 or 16)
@@ -194,7 +194,7 @@ stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MA
                 constexpr int c = decltype(ct)::value;
                 float lo, hi;
                 extremes8(x[c], lo, hi);
-                if (lpg == 16u) {
+                if (GC == 3) {
                     // two groups per chunk: a warp-wide reduction for each half, the other half's lanes holding the
                     // identity (four redux and four selects instead of eight shuffles and eight min / max)
                     const bool upper = lane >= 16;
@@ -369,10 +369,11 @@ template <typename T, int CHUNKS, bool BATCH, int ACT>
 static cudaError_t launch_stream_c(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
 {
     const uint32_t strip = 256u * CHUNKS;
-    const int gc = args.G < 256u ? 0 : args.G < strip ? 1 : 2;
+    const int gc = args.G < 128u ? 0 : args.G == 128u ? 3 : args.G < strip ? 1 : 2;
 #define DAF_CASE(BB)                                                                                                 \
     case BB:                                                                                                         \
         if (gc == 0) return launch_stream<T, CHUNKS, BB, 0, BATCH, ACT>(args, stream);                              \
+        if (gc == 3) return launch_stream<T, CHUNKS, BB, 3, BATCH, ACT>(args, stream);                              \
         if constexpr (CHUNKS > 1) { if (gc == 1) return launch_stream<T, CHUNKS, BB, 1, BATCH, ACT>(args, stream); } \
         return launch_stream<T, CHUNKS, BB, 2, BATCH, ACT>(args, stream);
     switch (args.S[args.full_ell]) {
