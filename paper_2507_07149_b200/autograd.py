@@ -44,8 +44,10 @@ import weakref
 
 import torch
 
-from . import (ACT_GELU, ACT_RELU, ACT_RELU6, BATCH_MAX, ROUND_STOCHASTIC, CompressedTensor, Store, _check, daf_batch_workspace, daf_compress_batch,
-               daf_poll_status, daf_sizes, decompress, dtype_code, make_params, store_bytes)
+import ctypes
+
+from . import (ACT_GELU, ACT_RELU, ACT_RELU6, BATCH_MAX, ROUND_STOCHASTIC, Store, _call, _check, daf_params, daf_poll_status,
+               daf_sizes, dtype_code, lib, make_params)
 
 _DTYPES = (torch.float32, torch.float16, torch.bfloat16)
 _ALIGN = 32
@@ -80,24 +82,17 @@ def _layout(params, packed_bytes=None):
     return sz, (o_min, o_scale, o_packed, o_bits, o_bits + _up16(ng))
 
 
-def _carve(block, at: int, params, shape, packed_bytes=None) -> CompressedTensor:
-    """The parts of one compressed tensor as views of `block` (uint8) from byte `at` on."""
-    sz, (o_min, o_scale, o_packed, o_bits, _) = _layout(params, packed_bytes)
-    ng, nw = sz.n_groups, sz.n_windows
-    return CompressedTensor(params, tuple(shape),
-                            block[at + o_packed:at + o_bits], block[at + o_bits:at + o_bits + ng],
-                            block[at + o_min:at + o_min + 4 * ng].view(torch.float32),
-                            block[at + o_scale:at + o_scale + 4 * ng].view(torch.float32),
-                            block[at:at + 8 * (nw + 1)].view(torch.int64), None, sz)
-
-
 class _Saved:
     """What the context keeps for one saved activation: the tensor itself while it is queued, then its parts."""
 
-    __slots__ = ("owner", "ident", "x", "c", "shape", "dtype", "device", "width", "offset", "dropped", "kept", "__weakref__")
+    # block, at, lay, params: where the compressed form lives (a uint8 tensor, the byte it starts at, the offsets of its parts
+    # as _layout gives them) and the parameters it was compressed with; set when the handle's batch has been launched
+    __slots__ = ("owner", "ident", "x", "block", "at", "lay", "params", "shape", "dtype", "device", "width", "offset",
+                 "dropped", "kept", "__weakref__")
 
     def __init__(self, owner, ident, x, shape, width, offset):
-        self.owner, self.ident, self.x, self.c = owner, ident, x, None
+        self.owner, self.ident, self.x = owner, ident, x
+        self.block, self.at, self.lay, self.params = None, 0, None, None
         self.shape, self.dtype, self.device = shape, x.dtype, x.device
         self.width, self.offset, self.dropped, self.kept = width, offset, width == 0, 0
 
@@ -141,6 +136,7 @@ class saved_activation_compression(torch.autograd.graph.saved_tensors_hooks):
         self._base, self._announced = 0, set()                      # the step's id range; ids the store has an entry for
         self._handles = weakref.WeakValueDictionary()
         self._store, self._arena = None, None
+        self._layouts = {}                                          # (dtype, numel, budget, packed bytes) -> (params, sizes, offsets)
         if mem_budget is not None:
             allowed = [w for w in self.widths if w <= self.bit_budget]
             self._store = Store(int(mem_budget), float("1e30") if time_budget is None else float(time_budget), allowed,
@@ -209,8 +205,8 @@ class saved_activation_compression(torch.autograd.graph.saved_tensors_hooks):
                 continue
             self._arena[dst:dst + nbytes].copy_(self._arena[src:src + nbytes].clone())   # the ranges may overlap
             h.offset = dst
-            if h.c is not None:
-                h.c = _carve(self._arena, dst, h.c.params, h.shape)
+            if h.block is not None:
+                h.at = dst
 
     # ---------------------------------------------------------------------------------------- hooks
     def _eligible(self, t) -> bool:
@@ -266,8 +262,7 @@ class saved_activation_compression(torch.autograd.graph.saved_tensors_hooks):
             h.x = None
             self.stats["dropped"] += 1
             return h
-        h.kept = (store_bytes(x.numel(), self.group_size, width) if self._store is not None else
-                  _layout(make_params(dtype_code(x), x.numel(), self.group_size, self.widths, float(width)))[1][4])
+        h.kept = self._layout_of(dtype_code(x), x.numel(), width)[2][4]
         self.stats["bytes_kept"] += h.kept
         self._queue.append(h)
         self._queued_bytes += nbytes
@@ -282,7 +277,7 @@ class saved_activation_compression(torch.autograd.graph.saved_tensors_hooks):
         if not h.dropped:
             self.stats["dropped"] += 1
             self.stats["bytes_kept"] -= h.kept
-        h.dropped, h.x, h.c = True, None, None
+        h.dropped, h.x, h.block = True, None, None
         if h in self._queue:
             self._queue.remove(h)
             for k in [k for k, v in self._queued_by_key.items() if v is h]:
@@ -293,9 +288,26 @@ class saved_activation_compression(torch.autograd.graph.saved_tensors_hooks):
             return s
         if s.dropped:
             return torch.zeros(s.shape, dtype=s.dtype, device=s.device)
-        if s.c is None:
+        if s.block is None:
             self.flush()
-        return decompress(s.c).view(s.shape)
+        out = torch.empty(s.shape, dtype=s.dtype, device=s.device)
+        b = s.block.data_ptr() + s.at
+        o_min, o_scale, o_packed, o_bits, _ = s.lay
+        status = _call(lib().daf_decompress, out, None, ctypes.byref(s.params), b + o_packed, b + o_bits, b + o_min, b + o_scale, b,
+                       out.data_ptr(), 0, 0)
+        _check(status, "daf_decompress")
+        return out
+
+    def _layout_of(self, code: int, numel: int, width):
+        """(parameters without seed and counter base, sizes, offsets of the parts) for a tensor of this type, size and
+        budget; remembered, since a model saves the same shapes every step."""
+        key = (code, numel, width)
+        v = self._layouts.get(key)
+        if v is None:
+            p = make_params(code, numel, self.group_size, self.widths, float(width), rounding=self.rounding)
+            sz, offs = _layout(p, numel * int(width) // 8 if self._arena is not None else None)
+            v = self._layouts[key] = (p, sz, offs)
+        return v
 
     # ---------------------------------------------------------------------------------------- the batched launch
     def flush(self) -> None:
@@ -311,28 +323,38 @@ class saved_activation_compression(torch.autograd.graph.saved_tensors_hooks):
                 self._launch(device, width, hs[i:i + BATCH_MAX])
 
     def _launch(self, device, width, hs) -> None:
-        params = []
-        for h in hs:
-            params.append(make_params(dtype_code(h.x), h.x.numel(), self.group_size, self.widths, float(width),
-                                      rounding=self.rounding, seed=self.seed, elem_index_base=self._next_index))
-            self._next_index += (h.x.numel() + 7) & ~7
+        n = len(hs)
+        lays = [self._layout_of(dtype_code(h.x), h.x.numel(), width) for h in hs]
         if self._arena is not None:
             block, starts = self._arena, [h.offset for h in hs]
-            cs = [_carve(block, at, p, h.shape, h.x.numel() * width // 8) for h, p, at in zip(hs, params, starts)]
         else:
-            sizes = [(_layout(p)[1][4] + 255) & ~255 for p in params]
-            starts = [sum(sizes[:i]) for i in range(len(sizes))]
-            block = torch.empty(sum(sizes), dtype=torch.uint8, device=device)
-            cs = [_carve(block, at, p, h.shape) for h, p, at in zip(hs, params, starts)]
-        ws_bytes = daf_batch_workspace(params)
+            starts, total = [], 0
+            for lay in lays:
+                starts.append(total)
+                total += (lay[2][4] + 255) & ~255
+            block = torch.empty(total, dtype=torch.uint8, device=device)
+        base = block.data_ptr()
+        arr = (daf_params * n)()
+        ptrs = [(ctypes.c_void_p * n)() for _ in range(6)]          # in, packed, bits, min, scale, window offsets
+        caps = (ctypes.c_uint64 * n)()
+        for i, (h, (tmpl, sz, (o_min, o_scale, o_packed, o_bits, _)), at) in enumerate(zip(hs, lays, starts)):
+            arr[i] = tmpl
+            arr[i].seed, arr[i].elem_index_base = self.seed, self._next_index
+            self._next_index += (h.x.numel() + 7) & ~7
+            b = base + at
+            ptrs[0][i], ptrs[1][i], ptrs[2][i] = h.x.data_ptr(), b + o_packed, b + o_bits
+            ptrs[3][i], ptrs[4][i], ptrs[5][i] = b + o_min, b + o_scale, b
+            caps[i] = sz.packed_capacity
+        ws_bytes = int(lib().daf_batch_workspace(n, arr))
         ws = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
-        daf_compress_batch(params, [h.x for h in hs], [c.packed for c in cs], [c.sizes.packed_capacity for c in cs],
-                           [c.bits for c in cs], [c.min for c in cs], [c.scale for c in cs], [c.window_offsets for c in cs],
-                           ws, ws_bytes)
+        status = _call(lib().daf_compress_batch, hs[0].x, None, n, arr, ptrs[0], ptrs[1], caps, ptrs[2], ptrs[3], ptrs[4], ptrs[5],
+                       ws.data_ptr(), ws_bytes)
+        _check(status, "daf_compress_batch")
         self._workspaces.append(ws)
         self.stats["launches"] += 1
-        for h, c in zip(hs, cs):
-            h.c, h.x = c, None                                      # the uncompressed tensor can go now
+        for i, (h, lay, at) in enumerate(zip(hs, lays, starts)):
+            h.block, h.at, h.lay, h.params = block, at, lay[2], daf_params.from_buffer_copy(arr[i])
+            h.x = None                                              # the uncompressed tensor can go now
 
 
 class _ReluSavedCompressed(torch.autograd.Function):
