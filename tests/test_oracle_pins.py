@@ -518,3 +518,25 @@ def test_gelu_and_its_derivative_against_closed_forms_and_a_library():
     ty.sum().backward()
     assert np.allclose(ty.detach().numpy(), y, rtol=1e-13, atol=1e-15)    # (the library loses the far negative tail)
     assert np.allclose(t.grad.numpy(), d, rtol=0, atol=1e-14)
+
+
+def test_packed_capacity_is_a_tight_bound():
+    """The capacity formula (what the budget guarantees per window) against what the oracle's own compress produces: never
+    exceeded on data with wildly different ranges, and met exactly when the budget is an allowed width."""
+    rng = np.random.default_rng(2)
+    for G, We, n_groups in ((32, 4096, 300), (256, 16384, 150), (1024, 8192, 21), (128, 16384, 129)):
+        n = G * n_groups
+        x = (rng.standard_normal(n) * np.repeat(10.0 ** rng.uniform(-4, 4, n_groups), G)).astype(np.float32)
+        for beta in (1.0, 1.5, 2.0, 2.75, 3.0, 4.0, 5.5, 8.0):
+            cap = oracle.packed_capacity(n, G, We, beta)
+            got = oracle.compress(x, G, (1, 2, 4, 8), beta, window_elems=We).packed.size
+            assert got <= cap, (G, We, beta)
+            if beta in (1.0, 2.0, 4.0, 8.0):
+                flat = oracle.compress(np.tile(np.linspace(-1, 1, G, dtype=np.float32), n_groups), G, (1, 2, 4, 8), beta,
+                                       window_elems=We).packed.size
+                assert flat == cap == n * int(beta) // 8
+            # by hand: every window of n_w groups may spend floor(beta * 256) * n_w / 256 bits per group-unit
+            W = We // G
+            full, last = divmod(n_groups, W)
+            q8 = int(np.floor(beta * 256))
+            assert cap == full * ((q8 * W) >> 8) * G // 8 + ((q8 * last) >> 8) * G // 8
