@@ -567,3 +567,56 @@ class Store:
             self.close()
         except Exception:
             pass
+
+
+class HostRoundTrip:
+    """Compress + decompress of a tensor that lives in pinned HOST memory, streamed through the device in window-aligned
+    chunks: while chunk i is compressed and restored, chunk i+1 is on its way in and chunk i-1 on its way out (three
+    streams, two sets of device buffers).  The chunks are shards in the sense of daf_shard -- same seed, counter base
+    moved -- so the restored values are exactly those of one call on the whole tensor.  The packed form of a chunk only
+    lives until the next chunk reuses its slot: this is the end-to-end path of the benchmark and of callers that want
+    the effect of the round trip (what the backward pass will see), not a way to keep the packed bytes."""
+
+    def __init__(self, dtype, group_size: int, widths, bit_budget: float, *, seed: int = 0, rounding: int = ROUND_STOCHASTIC,
+                 chunk_elems: int = 1 << 25, device="cuda"):
+        torch = _torch()
+        if chunk_elems % DEFAULT_WINDOW:
+            raise ValueError("chunk_elems must be a multiple of the window")
+        self.kw = dict(group_size=group_size, widths=tuple(widths), bit_budget=float(bit_budget), seed=seed, rounding=rounding)
+        self.chunk, self.device = int(chunk_elems), torch.device(device)
+        self.s_in, self.s_run, self.s_out = (torch.cuda.Stream(self.device) for _ in range(3))
+        self.x = [torch.empty(self.chunk, dtype=dtype, device=self.device) for _ in range(2)]
+        self.y = [torch.empty(self.chunk, dtype=dtype, device=self.device) for _ in range(2)]
+        code = dtype_code(self.x[0])
+        full = make_params(code, self.chunk, group_size, widths, bit_budget, rounding=rounding, seed=seed)
+        self.c = [alloc_outputs(full, self.device) for _ in range(2)]
+        self.free = [torch.cuda.Event() for _ in range(2)]
+
+    def __call__(self, h_in, h_out) -> None:
+        """h_in, h_out: flat pinned host tensors of the same length (a multiple of the group size).  Returns when the
+        work has been enqueued; the calling stream waits for it (so events recorded on it afterwards see it done)."""
+        torch = _torch()
+        n = h_in.numel()
+        cur = torch.cuda.current_stream(self.device)
+        for s in (self.s_in, self.s_run, self.s_out):
+            s.wait_stream(cur)
+        for i, lo in enumerate(range(0, n, self.chunk)):
+            m, k = min(self.chunk, n - lo), i & 1
+            ev_in, ev_run = torch.cuda.Event(), torch.cuda.Event()
+            with torch.cuda.stream(self.s_in):
+                if i >= 2:
+                    self.s_in.wait_event(self.free[k])            # the slot's last chunk has left the device
+                self.x[k][:m].copy_(h_in[lo:lo + m], non_blocking=True)
+                ev_in.record()
+            with torch.cuda.stream(self.s_run):
+                self.s_run.wait_event(ev_in)
+                kw = self.kw
+                c = compress(self.x[k][:m], kw["group_size"], kw["widths"], kw["bit_budget"], rounding=kw["rounding"],
+                             seed=kw["seed"], elem_index_base=lo, out=self.c[k] if m == self.chunk else None)
+                decompress(c, out=self.y[k][:m])
+                ev_run.record()
+            with torch.cuda.stream(self.s_out):
+                self.s_out.wait_event(ev_run)
+                h_out[lo:lo + m].copy_(self.y[k][:m], non_blocking=True)
+                self.free[k].record()
+        cur.wait_stream(self.s_out)

@@ -428,6 +428,24 @@ def test_shards_cut_by_daf_shard_reproduce_the_unsharded_result():
         assert np.array_equal(c.packed[: int(woff[-1])].cpu().numpy(), ref.packed[base: base + int(woff[-1])])
 
 
+def test_streamed_host_round_trip_equals_the_oracle_on_the_whole_tensor():
+    """HostRoundTrip: pinned host tensor in, restored values out, through chunks that overlap copies and kernels; the
+    result is what the oracle decodes for the whole tensor (the chunks are shards with the counter base moved)."""
+    rng = np.random.default_rng(91)
+    G, widths, beta, seed = 256, (1, 2, 4, 8), 4.0, 12
+    n = 16384 * 9 + 256 * 3                                         # two whole chunks of four windows and a ragged one
+    a = rng.laplace(size=n).astype(np.float32)
+    h_in = torch.from_numpy(a).pin_memory()
+    h_out = torch.empty_like(h_in).pin_memory()
+    rt = daf.HostRoundTrip(torch.float32, G, widths, beta, seed=seed, chunk_elems=16384 * 4)
+    for _ in range(2):                                              # twice: the slots are reused
+        h_out.zero_()
+        rt(h_in, h_out)
+        torch.cuda.synchronize()
+        want = oracle.decompress(oracle.compress(a, G, widths, beta, seed=seed))
+        assert np.array_equal(h_out.numpy().view(np.uint32), want.view(np.uint32))
+
+
 # ------------------------------------------------------------------ batched calls
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_batched_calls_equal_single_calls(dtype):
