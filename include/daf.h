@@ -85,6 +85,11 @@ typedef struct daf_params {
  *       of one width (see daf_compress) unless the call is small or the parameters rule such windows
  *       out; ALWAYS drops the size rule, NEVER goes to the general kernel directly (e.g. for data known
  *       to mix widths).  Giving both is an error.
+ *   DAF_FLAG_ONE_PASS / _TWO_PASS : windows of mixed widths are handled either by the general kernel (one pass
+ *       over the input; CTAs that wait for one another's window offsets) or by the two-pass kernels (widths first,
+ *       then offsets, then quantize + pack: the input is read twice, nothing waits).  The library chooses by
+ *       element type and group size; these flags force one or the other where both exist (two-pass: groups of 128
+ *       to 1024 elements, default window, no fused activation).  Giving both is an error.
  *   DAF_FLAG_KEEP_WORKSPACE : diagnostic.  The workspace is not cleared on entry: the caller has
  *       prepared it (all zero, except what a test of the failure paths has planted there).
  *   DAF_FLAG_POLL_LIMIT(n)  : diagnostic.  Bounded device-side waits give up after n polls
@@ -93,6 +98,8 @@ typedef struct daf_params {
 #define DAF_FLAG_STREAM_ALWAYS  0x1u
 #define DAF_FLAG_STREAM_NEVER   0x2u
 #define DAF_FLAG_KEEP_WORKSPACE 0x4u
+#define DAF_FLAG_ONE_PASS       0x8u
+#define DAF_FLAG_TWO_PASS       0x10u
 #define DAF_FLAG_POLL_LIMIT(n)  ((uint32_t)(n) << 8)
 
 /*
@@ -128,15 +135,18 @@ daf_status daf_shard(const daf_params *whole, uint32_t rank, uint32_t world, daf
  *   d_window_offsets out: n_windows + 1 uint64
  *   d_workspace          : workspace_bytes of scratch, contents irrelevant on entry; also
  *                          holds the device status word afterwards (see daf_poll_status)
- * The input is read once.  The call enqueues, in this order: a streaming kernel, which
- * assumes that in every window all groups end at one and the same width (the one the budget
- * gives a window of equal groups) and writes every output on that assumption while it records
- * what is needed to check it; a small kernel that checks it for every window and writes the
- * window offsets; and the general kernel, which returns at once unless the check failed
- * somewhere and then redoes the whole call with the window-by-window greedy choice.  A call of
- * at most 4096 windows, or one whose parameters rule out one-width windows, goes to the
- * general kernel alone; params->flags can force either route.  Both routes give the same
- * bytes.  Every output is final when the call's work on the stream is done.  If the packed output
+ * The call enqueues, in this order: a streaming kernel, which assumes that in every window
+ * all groups end at one and the same width (the one the budget gives a window of equal
+ * groups) and writes every output on that assumption while it records what is needed to
+ * check it; a small kernel that checks it for every window and writes the window offsets;
+ * and a fallback, which returns at once unless the check failed somewhere and then redoes the
+ * whole call with the window-by-window greedy choice.  The fallback is the general kernel
+ * (one launch; the input is read once), or, for calls of more than 4096 windows on 16-bit
+ * elements with groups of 128 to 1024 elements, three kernels that read the input twice:
+ * widths and metadata of every window, window offsets, quantize + pack.  A call of at most
+ * 4096 windows, or one whose parameters rule out one-width windows, goes to the fallback
+ * alone; params->flags can force each of these choices.  All routes give the same bytes.
+ * Every output is final when the call's work on the stream is done.  If the packed output
  * of a window would pass packed_capacity, nothing of that window is stored and the status
  * word becomes DAF_ERR_CAPACITY.  Inputs must be finite; behaviour on NaN / Inf is unspecified but
  * memory safe.  Calls sharing a workspace must not overlap on the GPU.

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libdaf.so")
 OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_BUDGET, ERR_CAPACITY, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED = range(8)
 F32, F16, BF16 = 0, 1, 2
 ROUND_STOCHASTIC, ROUND_NEAREST = 0, 1
-FLAG_STREAM_ALWAYS, FLAG_STREAM_NEVER, FLAG_KEEP_WORKSPACE = 1, 2, 4
+FLAG_STREAM_ALWAYS, FLAG_STREAM_NEVER, FLAG_KEEP_WORKSPACE, FLAG_ONE_PASS, FLAG_TWO_PASS = 1, 2, 4, 8, 16
 
 
 # daf_params.flags used by make_params when the caller gives none (the GPU tests set FLAG_STREAM_ALWAYS here so

@@ -47,9 +47,10 @@ static float raise_factor(uint32_t lo, uint32_t hi)
 
 daf_status make_plan(const daf_params *p, Plan *pl)
 {
-    if (!p || p->struct_size != sizeof(daf_params) || (p->flags & 0xF8u) != 0) return DAF_ERR_INVALID_ARG;
+    if (!p || p->struct_size != sizeof(daf_params) || (p->flags & 0xE0u) != 0) return DAF_ERR_INVALID_ARG;
     if (p->dtype > DAF_BF16 || p->rounding > DAF_ROUND_NEAREST) return DAF_ERR_INVALID_ARG;
     if ((p->flags & DAF_FLAG_STREAM_ALWAYS) && (p->flags & DAF_FLAG_STREAM_NEVER)) return DAF_ERR_INVALID_ARG;
+    if ((p->flags & DAF_FLAG_ONE_PASS) && (p->flags & DAF_FLAG_TWO_PASS)) return DAF_ERR_INVALID_ARG;
     const uint32_t We = p->window_elems ? p->window_elems : 16384u;
     const uint32_t G = p->group_size;
     if (!is_pow2(G) || G < 32u) return DAF_ERR_INVALID_ARG;

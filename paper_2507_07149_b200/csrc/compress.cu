@@ -2,13 +2,15 @@
 // kernels of one call.
 //
 //   daf_compress = [clear the workspace] -> streaming kernel -> verify kernel -> general kernel
+//                                                                                (or widths -> offsets -> pack)
 //
 // The streaming kernel (compress_stream.cuh) assumes that every window ends with one width; the
-// verify kernel checks that assumption window by window and writes the window offsets; the
-// general kernel (compress_general.cuh), which handles any mix of widths, runs last and returns
-// at once unless one of the two asked for it (hdr->retry), in which case it redoes the call.
-// When the parameters rule out windows of one width, or the call is small, only the general
-// kernel is launched.
+// verify kernel checks that assumption window by window and writes the window offsets; what
+// handles any mix of widths runs last and returns at once unless one of the two asked for it
+// (hdr->retry), in which case it redoes the call: the general kernel (compress_general.cuh), or,
+// for large calls on 16-bit elements, the three two-pass kernels (compress_twopass.cuh).
+// When the parameters rule out windows of one width, or the call is small, the streaming kernel
+// is not launched.
 #include "compress_shared.cuh"
 
 namespace daf {
@@ -71,6 +73,9 @@ template <int NT> static uint64_t one_width_total(const CompressArgs<NT> &a, con
 // (the general kernel then reports the overflow window by window), or when the call is small (it is
 // launch-bound, and one launch is cheaper than two), only the general kernel is launched.
 constexpr uint32_t kStreamMinWindows = 4096;                     // measured break-even
+constexpr uint32_t kTwoPassMinWindows = 4096;                    // below, one launch of the general kernel beats three (measured: sets of
+                                                                  // 16-bit tensors of 600 - 2400 windows each, one call per tensor, came out
+                                                                  // 7 % faster when mixed and 17 % slower when of one width)
 
 template <bool BATCH, int ACT = kActNone>
 static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, uint32_t flags, CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args,
@@ -95,6 +100,15 @@ static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, uint32_t flags, Com
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
+    // Windows of mixed widths.  The two-pass kernels (compress_twopass.cuh) read the input twice and never wait; the
+    // general kernel reads it once, but its warps hold a window in registers while its widths are decided.  Measured
+    // (B200, whole calls): 16-bit elements, groups of 128, mostly mixed windows: 0.86 ms two-pass against 1.10 ms
+    // general on 581 M elements; the same with windows of one width throughout: 0.93 against 0.74 ms on 671 M; binary32,
+    // groups of 256, budget between two widths: 0.73 against 0.70 ms on 466 M.  So: 16-bit elements, calls large enough
+    // that three launches do not matter, unless the caller says otherwise.
+    bool two_pass = ACT == kActNone && chunks == 4u && args.G >= 128u && args.G <= 1024u && !(flags & DAF_FLAG_ONE_PASS);
+    if (!(flags & DAF_FLAG_TWO_PASS)) two_pass = two_pass && dtype != DAF_F32 && args.total_windows > kTwoPassMinWindows;
+    if (two_pass) return dispatch_twopass<BATCH>(dtype, args, stream);
     return dispatch_general<BATCH, ACT>(dtype, chunks, args, stream);
 }
 

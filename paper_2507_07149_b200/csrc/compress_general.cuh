@@ -155,87 +155,6 @@ __device__ __forceinline__ void quantize_uniform_b(uint32_t b, const float (&x)[
     }
 }
 
-// ------------------------------------------------------------------------------------------
-// The greedy of Sec. 3.4.1 on one warp.  Every lane holds NK candidate raises (key, cw = cost
-// | 1 << 16, or cw = 0 for "no candidate"); slot s of lane l sorts, among equal keys, before
-// slot s' > s of any lane and before slot s of lane l' > l.  Accepted is the longest prefix,
-// in the order (key descending, then that order), whose summed cost is at most rem; take[s]
-// says whether this lane's slot s is in it.  F(t), the cost of all raises with key >= t, falls
-// as t grows, so the prefix is every raise with a key above Kp, the largest t with F(t) > rem,
-// and then the raises with key Kp in order while they fit.  One warp reduction gives F(t) and
-// N(t), the number of raises with key >= t; the interval that holds Kp starts from the keys'
-// common leading bits (BOUNDS: the caller passes the largest and the smallest key) and is
-// halved bit by bit; as soon as a single raise is left in it, its key is Kp.
-// ------------------------------------------------------------------------------------------
-template <int NK, bool BOUNDS>
-__device__ __forceinline__ void accept_prefix(const uint32_t (&key)[NK], const uint32_t (&cw)[NK],
-                                              const uint32_t (&slot_cost)[NK], uint32_t rem, uint32_t hi, uint32_t lo,
-                                              int lane, bool (&take)[NK])
-{
-    if (!BOUNDS) {
-        hi = 0u;
-        lo = 0xFFFFFFFFu;
-#pragma unroll
-        for (int s = 0; s < NK; s++)
-            if (cw[s] != 0u) {
-                hi = max(hi, key[s]);
-                lo = min(lo, key[s]);
-            }
-        hi = __reduce_max_sync(0xFFFFFFFFu, hi);
-        lo = __reduce_min_sync(0xFFFFFFFFu, lo);
-    }
-    auto from = [&](uint32_t t) {                                 // F(t) | N(t) << 16
-        uint32_t f = 0;
-#pragma unroll
-        for (int s = 0; s < NK; s++) f += key[s] >= t ? cw[s] : 0u;
-        return __reduce_add_sync(0xFFFFFFFFu, f);
-    };
-    uint32_t Kp = 0u, at_lo = from(0u), at_hi;                    // F | N at the two ends of the interval
-    if ((at_lo & 0xFFFFu) > rem) {
-        const uint32_t diff = hi ^ lo;
-        int bit = diff != 0u ? 31 - __clz(diff) : -1;             // the interval is [Kp, Kp + 2^(bit+1))
-        Kp = diff != 0u ? hi & ~((2u << bit) - 1u) : hi;
-        at_hi = 0u;
-        while (bit >= 0 && (at_lo >> 16) - (at_hi >> 16) > 1u) {
-            const uint32_t t = Kp | (1u << bit);
-            const uint32_t e = from(t);
-            if ((e & 0xFFFFu) > rem) {
-                Kp = t;
-                at_lo = e;
-            } else {
-                at_hi = e;
-            }
-            bit--;
-        }
-        if (bit >= 0) {                                           // one raise left in the interval: Kp is its key
-            const uint32_t sh = (uint32_t)bit + 1u;
-            uint32_t only = 0u;
-#pragma unroll
-            for (int s = 0; s < NK; s++)
-                if (cw[s] != 0u && (sh >= 32u || (key[s] >> sh) == (Kp >> sh))) only = key[s];
-            Kp = __reduce_max_sync(0xFFFFFFFFu, only);
-        }
-    } else {
-        at_hi = from(1u);                                         // every raise fits (Kp = 0)
-    }
-    uint32_t left = rem - (at_hi & 0xFFFFu);                      // after every raise with a key above Kp
-    bool open = true;                                             // no raise has been turned down yet
-    const uint32_t below = (1u << lane) - 1u;
-#pragma unroll
-    for (int s = 0; s < NK; s++) {
-        const bool on = cw[s] != 0u, tie = on && key[s] == Kp;
-        const uint32_t ties = __ballot_sync(0xFFFFFFFFu, tie);
-        uint32_t fit = 0u;
-        if (ties != 0u && open) {
-            const uint32_t cnt = (uint32_t)__popc(ties);
-            fit = min(cnt, left / slot_cost[s]);
-            left -= fit * slot_cost[s];
-            open = fit == cnt;                                    // the walk stops at the first raise that does not fit
-        }
-        take[s] = on && (key[s] > Kp || (tie && (uint32_t)__popc(ties & below) < fit));
-    }
-}
-
 // Budget arithmetic of a window of n groups.
 struct Budget {
     uint32_t ell;          // largest level every group can be raised to
@@ -952,24 +871,25 @@ compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MAX : 1> 
                     const uint32_t e = e0 + 256u * c;
                     if (e >= n_elems) break;                      // ragged last window: whole chunks are missing
                     const GroupRec rec = s_grp[e >> log2G];
-                    uint32_t o[4], w0, w1;
+                    uint32_t o[4], t[8], w0, w1;
                     draw(c, o);
+                    noisy_sums8(x[c], rec.mn, rec.inv, o, t);     // (the arithmetic all widths share stays outside the split)
                     unsigned char *p = s_out + rec.off + ((e & (G - 1u)) >> 3) * rec.b;
                     switch (rec.b) {
                     case 1:
-                        quantize8<1, false>(x[c], rec.mn, rec.inv, o, w0, w1);
+                        close_codes8<1, false>(t, w0, w1);
                         *p = (unsigned char)w0;
                         break;
                     case 2:
-                        quantize8<2, false>(x[c], rec.mn, rec.inv, o, w0, w1);
+                        close_codes8<2, false>(t, w0, w1);
                         *reinterpret_cast<uint16_t *>(p) = (uint16_t)w0;
                         break;
                     case 4:
-                        quantize8<4, false>(x[c], rec.mn, rec.inv, o, w0, w1);
+                        close_codes8<4, false>(t, w0, w1);
                         *reinterpret_cast<uint32_t *>(p) = w0;
                         break;
                     default:
-                        quantize8<8, false>(x[c], rec.mn, rec.inv, o, w0, w1);
+                        close_codes8<8, false>(t, w0, w1);
                         *reinterpret_cast<uint2 *>(p) = make_uint2(w0, w1);
                         break;
                     }

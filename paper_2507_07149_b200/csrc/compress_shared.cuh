@@ -203,6 +203,18 @@ __device__ __forceinline__ int lookback(const uint64_t *flags, uint32_t gw, uint
 template <typename T, bool BATCH, int ACT>
 cudaError_t dispatch_stream_t(uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream);
 
+// The two-pass kernels for windows of mixed widths (compress_twopass.cuh; one translation unit per element type).
+template <typename T, bool BATCH>
+cudaError_t dispatch_twopass_t(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream);
+
+template <bool BATCH>
+inline cudaError_t dispatch_twopass(uint32_t dtype, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
+{
+    if (dtype == DAF_F32) return dispatch_twopass_t<float, BATCH>(args, stream);
+    if (dtype == DAF_F16) return dispatch_twopass_t<__half, BATCH>(args, stream);
+    return dispatch_twopass_t<__nv_bfloat16, BATCH>(args, stream);
+}
+
 // The general kernel: any mix of widths within a window (compress_general.cuh; one translation unit per element type).
 template <typename T, bool BATCH, int ACT>
 cudaError_t dispatch_general_t(uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream);
@@ -238,12 +250,9 @@ struct GroupRec {             // what the quantize pass needs per group (one 16-
 // (fixed + r15) >> 15 == (2*bits(s) + h - 2*bits(256)) >> 16, which needs one add, one shift
 // and one fused subtract-and-clamp per element.
 // ------------------------------------------------------------------------------------------
-template <int B, bool CLAMP>
-__device__ __forceinline__ void quantize8(const float (&x)[8], float mn, float inv, const uint32_t (&o)[4],
-                                          uint32_t &w0, uint32_t &w1)
+// t[i] = 2 * bits(s_i) + h_i (mod 2^32): bits 16 .. 31 of t[i], less 0x8700, are code i before any clamp.
+__device__ __forceinline__ void noisy_sums8(const float (&x)[8], float mn, float inv, const uint32_t (&o)[4], uint32_t (&t)[8])
 {
-    constexpr uint32_t L = (1u << B) - 1u;
-    uint32_t t[8];
 #pragma unroll
     for (int i = 0; i < 8; i++) {
         const float d = __fsub_rn(x[i], mn);
@@ -251,6 +260,13 @@ __device__ __forceinline__ void quantize8(const float (&x)[8], float mn, float i
         const uint32_t h = (i & 1) ? (o[i >> 1] >> 16) : (o[i >> 1] & 0xFFFFu);
         t[i] = __float_as_uint(s) * 2u + h;                       // mod 2^32; 2*bits(256) = 0x87000000
     }
+}
+
+// The eight codes of width B out of t[], packed LSB first into w0 (and w1 for B = 8).
+template <int B, bool CLAMP>
+__device__ __forceinline__ void close_codes8(const uint32_t (&t)[8], uint32_t &w0, uint32_t &w1)
+{
+    constexpr uint32_t L = (1u << B) - 1u;
     if (CLAMP) {
         w0 = 0u;
         w1 = 0u;
@@ -287,6 +303,15 @@ __device__ __forceinline__ void quantize8(const float (&x)[8], float mn, float i
     }
 }
 
+template <int B, bool CLAMP>
+__device__ __forceinline__ void quantize8(const float (&x)[8], float mn, float inv, const uint32_t (&o)[4],
+                                          uint32_t &w0, uint32_t &w1)
+{
+    uint32_t t[8];
+    noisy_sums8(x, mn, inv, o, t);
+    close_codes8<B, CLAMP>(t, w0, w1);
+}
+
 // The same for a width known only at run time (and possibly different in every lane): the
 // codes are clamped to 2^b - 1, then joined pairwise with multiply-adds by 2^b, 2^2b, 2^4b.
 __device__ __forceinline__ void quantize8_any(const float (&x)[8], float mn, float inv, const uint32_t (&o)[4],
@@ -307,6 +332,87 @@ __device__ __forceinline__ void quantize8_any(const float (&x)[8], float mn, flo
     const uint32_t lo = q23 * m2 + q01, hi = q67 * m2 + q45;
     w0 = hi * m4 + lo;
     w1 = hi;
+}
+
+// ------------------------------------------------------------------------------------------
+// The greedy of Sec. 3.4.1 on one warp.  Every lane holds NK candidate raises (key, cw = cost
+// | 1 << 16, or cw = 0 for "no candidate"); slot s of lane l sorts, among equal keys, before
+// slot s' > s of any lane and before slot s of lane l' > l.  Accepted is the longest prefix,
+// in the order (key descending, then that order), whose summed cost is at most rem; take[s]
+// says whether this lane's slot s is in it.  F(t), the cost of all raises with key >= t, falls
+// as t grows, so the prefix is every raise with a key above Kp, the largest t with F(t) > rem,
+// and then the raises with key Kp in order while they fit.  One warp reduction gives F(t) and
+// N(t), the number of raises with key >= t; the interval that holds Kp starts from the keys'
+// common leading bits (BOUNDS: the caller passes the largest and the smallest key) and is
+// halved bit by bit; as soon as a single raise is left in it, its key is Kp.
+// ------------------------------------------------------------------------------------------
+template <int NK, bool BOUNDS>
+__device__ __forceinline__ void accept_prefix(const uint32_t (&key)[NK], const uint32_t (&cw)[NK],
+                                              const uint32_t (&slot_cost)[NK], uint32_t rem, uint32_t hi, uint32_t lo,
+                                              int lane, bool (&take)[NK])
+{
+    if (!BOUNDS) {
+        hi = 0u;
+        lo = 0xFFFFFFFFu;
+#pragma unroll
+        for (int s = 0; s < NK; s++)
+            if (cw[s] != 0u) {
+                hi = max(hi, key[s]);
+                lo = min(lo, key[s]);
+            }
+        hi = __reduce_max_sync(0xFFFFFFFFu, hi);
+        lo = __reduce_min_sync(0xFFFFFFFFu, lo);
+    }
+    auto from = [&](uint32_t t) {                                 // F(t) | N(t) << 16
+        uint32_t f = 0;
+#pragma unroll
+        for (int s = 0; s < NK; s++) f += key[s] >= t ? cw[s] : 0u;
+        return __reduce_add_sync(0xFFFFFFFFu, f);
+    };
+    uint32_t Kp = 0u, at_lo = from(0u), at_hi;                    // F | N at the two ends of the interval
+    if ((at_lo & 0xFFFFu) > rem) {
+        const uint32_t diff = hi ^ lo;
+        int bit = diff != 0u ? 31 - __clz(diff) : -1;             // the interval is [Kp, Kp + 2^(bit+1))
+        Kp = diff != 0u ? hi & ~((2u << bit) - 1u) : hi;
+        at_hi = 0u;
+        while (bit >= 0 && (at_lo >> 16) - (at_hi >> 16) > 1u) {
+            const uint32_t t = Kp | (1u << bit);
+            const uint32_t e = from(t);
+            if ((e & 0xFFFFu) > rem) {
+                Kp = t;
+                at_lo = e;
+            } else {
+                at_hi = e;
+            }
+            bit--;
+        }
+        if (bit >= 0) {                                           // one raise left in the interval: Kp is its key
+            const uint32_t sh = (uint32_t)bit + 1u;
+            uint32_t only = 0u;
+#pragma unroll
+            for (int s = 0; s < NK; s++)
+                if (cw[s] != 0u && (sh >= 32u || (key[s] >> sh) == (Kp >> sh))) only = key[s];
+            Kp = __reduce_max_sync(0xFFFFFFFFu, only);
+        }
+    } else {
+        at_hi = from(1u);                                         // every raise fits (Kp = 0)
+    }
+    uint32_t left = rem - (at_hi & 0xFFFFu);                      // after every raise with a key above Kp
+    bool open = true;                                             // no raise has been turned down yet
+    const uint32_t below = (1u << lane) - 1u;
+#pragma unroll
+    for (int s = 0; s < NK; s++) {
+        const bool on = cw[s] != 0u, tie = on && key[s] == Kp;
+        const uint32_t ties = __ballot_sync(0xFFFFFFFFu, tie);
+        uint32_t fit = 0u;
+        if (ties != 0u && open) {
+            const uint32_t cnt = (uint32_t)__popc(ties);
+            fit = min(cnt, left / slot_cost[s]);
+            left -= fit * slot_cost[s];
+            open = fit == cnt;                                    // the walk stops at the first raise that does not fit
+        }
+        take[s] = on && (key[s] > Kp || (tie && (uint32_t)__popc(ties & below) < fit));
+    }
 }
 
 }  // namespace daf

@@ -1,0 +1,6 @@
+// The two-pass compress kernels for f16 inputs (see compress_twopass.cuh).
+#include "compress_twopass.cuh"
+
+namespace daf {
+DAF_INSTANTIATE_TWOPASS(__half)
+}

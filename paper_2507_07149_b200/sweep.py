@@ -81,7 +81,8 @@ def _time(torch, fn, steps, flush):
 
 def run_set(torch, daf, wl, w, xs, steps):
     """(compress ms, decompress ms, packed bytes) for the tensors xs of workload w."""
-    params = [daf.make_params(daf.dtype_code(x), x.numel(), w.group_size, w.widths, w.bit_budget, seed=t.philox_seed)
+    params = [daf.make_params(daf.dtype_code(x), x.numel(), w.group_size, w.widths, w.bit_budget, seed=t.philox_seed,
+                              flags=FLAGS)
               for x, t in zip(xs, w.tensors)]
     outs = [daf.alloc_outputs(p, xs[0].device) for p in params]
     ys = [torch.empty_like(x) for x in xs]
@@ -133,6 +134,7 @@ def run_set(torch, daf, wl, w, xs, steps):
 
 
 LAST_MHZ = None
+FLAGS = 0
 
 
 def row(name, numel, nbytes, packed, meta, t_c, t_d, per_tensor=None):
@@ -156,7 +158,12 @@ def main():
                          "run into the board's power cap and the SM clock falls from 1965 to about 1600 MHz (see the last column)")
     ap.add_argument("--tensorwise", action="store_true",
                     help="also the per-tensor path on workload 5: min / max reduction, Eq. 1 with one min / max / width, its inverse")
+    ap.add_argument("--flags", type=lambda v: int(v, 0), default=0,
+                    help="daf_params.flags of every call of the five workloads (launch policy, e.g. 8 = DAF_FLAG_ONE_PASS, "
+                         "16 = DAF_FLAG_TWO_PASS, 2 = DAF_FLAG_STREAM_NEVER)")
     args = ap.parse_args()
+    global FLAGS
+    FLAGS = args.flags
 
     import torch
     import paper_2507_07149_b200 as daf

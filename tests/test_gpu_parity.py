@@ -672,7 +672,7 @@ def test_compress_look_back_gives_up_when_a_window_is_never_produced(poisoned):
     n_windows, G, widths, beta = 8, 256, (1, 2, 4, 8), 3.0
     a = wl.generate(77, 0, wl.TensorSpec("t", (n_windows * 16384,), "f32", "logscale", 3))
     x = torch.from_numpy(a).cuda()
-    flags = daf.FLAG_STREAM_NEVER | daf.FLAG_KEEP_WORKSPACE | daf.flag_poll_limit(3000)
+    flags = daf.FLAG_STREAM_NEVER | daf.FLAG_ONE_PASS | daf.FLAG_KEEP_WORKSPACE | daf.flag_poll_limit(3000)
     p = daf.make_params(daf.F32, x.numel(), G, widths, beta, seed=3, flags=flags)
     sz = daf.daf_sizes(p)
     guard = 4096
