@@ -99,11 +99,17 @@ stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MA
     __shared__ uint32_t s_first[BATCH ? DAF_BATCH_MAX : 1];       // first window of every tensor
     __shared__ __align__(16) uint32_t s_rkeys[BATCH ? kWarps : 1][20];   // Philox round keys of the warp's current tensor
 
+    __shared__ uint32_t s_late;                                   // the call was given up before this CTA started
+
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (BATCH) {
+    if (BATCH)
         for (uint32_t i = tid; i < DAF_BATCH_MAX; i += kThreads) s_first[i] = i < a.n_tensors ? a.t[i].first_window : 0xFFFFFFFFu;
-        __syncthreads();
-    }
+    // A CTA that starts after somebody has asked for the general kernel leaves at once: the grid is several times what
+    // the device holds, so after a failure in the first wave the rest of the grid costs next to nothing.  One thread
+    // reads the flag for all: warps that share a group must take the same decision.
+    if (tid == 0) s_late = ld_relaxed_u32(&a.hdr->retry);
+    __syncthreads();
+    if (s_late != 0u) return;
     const uint32_t log2G = a.log2G;
     const uint32_t strip0 = (uint32_t)warp * STRIP;               // the strip's first element within its window
     const uint32_t e0 = strip0 + (uint32_t)lane * 8u;             // the lane's first element of chunk 0
