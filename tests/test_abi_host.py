@@ -76,6 +76,12 @@ def test_sizes_and_host_validation():
     assert status(window_elems=2048) == daf.ERR_UNSUPPORTED
     assert status(window_elems=5000) == daf.ERR_INVALID_ARG
     assert status(elem_index_base=4) == daf.ERR_INVALID_ARG
+    # launch-policy flags: each alone and sensible pairs are fine, contradictory pairs and unknown bits are not
+    for ok in (daf.FLAG_STREAM_ALWAYS, daf.FLAG_STREAM_NEVER, daf.FLAG_ONE_PASS, daf.FLAG_TWO_PASS, daf.FLAG_KEEP_WORKSPACE,
+               daf.FLAG_STREAM_NEVER | daf.FLAG_TWO_PASS, daf.FLAG_STREAM_ALWAYS | daf.FLAG_ONE_PASS | daf.flag_poll_limit(100)):
+        assert status(flags=ok) == daf.OK
+    for bad_flags in (daf.FLAG_STREAM_ALWAYS | daf.FLAG_STREAM_NEVER, daf.FLAG_ONE_PASS | daf.FLAG_TWO_PASS, 0x20, 0x40, 0x80):
+        assert status(flags=bad_flags) == daf.ERR_INVALID_ARG
     bad = daf.make_params(daf.F32, 16384, 256, (4,), 4.0)
     bad.struct_size = 8
     with pytest.raises(daf.DafError):
