@@ -104,17 +104,28 @@ stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MA
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (BATCH)
         for (uint32_t i = tid; i < DAF_BATCH_MAX; i += kThreads) s_first[i] = i < a.n_tensors ? a.t[i].first_window : 0xFFFFFFFFu;
-    // A CTA that starts after somebody has asked for the general kernel leaves at once: the grid is several times what
-    // the device holds, so after a failure in the first wave the rest of the grid costs next to nothing.  One thread
-    // reads the flag for all: warps that share a group must take the same decision.
-    if (tid == 0) s_late = ld_relaxed_u32(&a.hdr->retry);
-    __syncthreads();
-    if (s_late != 0u) return;
+    // Whoever starts after somebody has asked for the fallback leaves at once: the grid is several times what the
+    // device holds, so after a failure in the first wave the rest of the grid costs next to nothing.  Warps that
+    // share a group (GC = 2) must take the same decision: there one thread reads the flag for the CTA.
+    // Independent warps read the flag themselves: at once (groups of 128 elements and more; 8-bit codes), or with the
+    // wait for it moved behind the first strip's loads (smaller groups) -- whichever the instantiation runs faster
+    // with when nothing fails (differences of half a percent, measured on the 16 sweep points).
+    constexpr bool kWaitAtStart = GC != 0 || B == 8;
+    uint32_t retry_seen = 0u;
+    if (GC == 2) {
+        if (tid == 0) s_late = ld_relaxed_u32(&a.hdr->retry);
+        __syncthreads();
+        if (s_late != 0u) return;
+    } else {
+        if (BATCH) __syncthreads();
+        retry_seen = ld_relaxed_u32(&a.hdr->retry);
+        if (kWaitAtStart && retry_seen != 0u) return;
+    }
     const uint32_t log2G = a.log2G;
     const uint32_t strip0 = (uint32_t)warp * STRIP;               // the strip's first element within its window
     const uint32_t e0 = strip0 + (uint32_t)lane * 8u;             // the lane's first element of chunk 0
     uint32_t cur_keys = 0xFFFFFFFFu;
-    uint32_t stop = 0u, retry_seen = 0u;
+    uint32_t stop = 0u;
     uint32_t it = 0;
 
     // One strip.  WHOLE: the window has all its elements (no predicates anywhere).
@@ -148,6 +159,7 @@ stream_compress_kernel(const __grid_constant__ CompressArgs<BATCH ? DAF_BATCH_MA
         // ---- meanwhile: has anybody asked to stop?
         stop |= retry_seen;
         retry_seen = ld_relaxed_u32(&a.hdr->retry);               // consumed one window later
+        if (GC != 2 && !kWaitAtStart && stop != 0u) return;       // (nobody waits for this warp: the strip is dropped here)
         if (ACT != kActNone) {
             // fused producer: the activation is written out and (ReLU, ReLU6) replaces x as what is compressed; a lane
             // stores the chunk it loaded, so the output may be the input buffer
