@@ -11,10 +11,10 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libdaf.so")
-HEADERS = [os.path.join(CSRC, h) for h in ("common.cuh", "compress_shared.cuh", "compress_stream.cuh", "compress_general.cuh", "compress_twopass.cuh", "launch_cache.hpp")] + [
+HEADERS = [os.path.join(CSRC, h) for h in ("common.cuh", "compress_shared.cuh", "compress_stream.cuh", "compress_general.cuh", "compress_twopass.cuh", "compress_twowidth.cuh", "launch_cache.hpp")] + [
     os.path.join(os.path.dirname(HERE), "include", "daf.h")]
 
-CU_SOURCES = ["api.cu", "compress.cu", "compress_stream_f32.cu", "compress_stream_f16.cu", "compress_stream_bf16.cu", "compress_twopass_f32.cu", "compress_twopass_f16.cu", "compress_twopass_bf16.cu", "compress_general_f32.cu", "compress_general_f16.cu",
+CU_SOURCES = ["api.cu", "compress.cu", "compress_stream_f32.cu", "compress_stream_f16.cu", "compress_stream_bf16.cu", "compress_twowidth_f32.cu", "compress_twowidth_f16.cu", "compress_twowidth_bf16.cu", "compress_twopass_f32.cu", "compress_twopass_f16.cu", "compress_twopass_bf16.cu", "compress_general_f32.cu", "compress_general_f16.cu",
               "compress_general_bf16.cu", "decompress.cu", "group_offsets.cu", "tensorwise.cu"]
 CXX_SOURCES = ["pool.cpp", "store.cpp"]
 

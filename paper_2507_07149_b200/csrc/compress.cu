@@ -91,8 +91,48 @@ static cudaError_t dispatch(uint32_t dtype, uint32_t chunks, uint32_t flags, Com
     if ((ACT == kActRelu || ACT == kActRelu6) && !(flags & DAF_FLAG_STREAM_ALWAYS)) try_stream = false;
     for (uint32_t i = 0; try_stream && i < args.n_tensors; i++)
         try_stream = one_width_total(args, args.t[i], chunks * 4096u) <= args.t[i].capacity;
+    // A budget between two widths: the two-width streaming kernel, if the group size is one it handles and the packed
+    // buffer holds what it would write (its sizes do not depend on the data).
+    bool try_two = !args.nearest && ACT == kActNone && !all_max && !need_sep && chunks == 4u && args.G >= 256u && args.G <= 1024u &&
+                   !(flags & DAF_FLAG_STREAM_NEVER) && (args.total_windows > kStreamMinWindows || (flags & DAF_FLAG_STREAM_ALWAYS));
+    args.tw_k = 0u;
+    if (try_two) {
+        const uint32_t kk = args.full_rem_after / args.cost[args.full_ell];
+        args.tw_k = kk < args.n_max ? kk : args.n_max;
+        const uint64_t lo = (uint64_t)(args.G >> 3) * args.S[args.full_ell];
+        const uint64_t up = (uint64_t)(args.G >> 3) * (args.S[args.full_ell + 1u] - args.S[args.full_ell]);
+        const uint64_t we = chunks * 4096u, wb = args.n_max * lo + args.tw_k * up;   // elements and packed bytes of a whole window
+        args.tw_blo = args.S[args.full_ell];
+        args.tw_bhi = args.S[args.full_ell + 1u];
+        args.tw_size_lo = (uint32_t)lo;
+        args.tw_size_up = (uint32_t)up;
+        args.tw_lf_lo = (float)((1u << args.tw_blo) - 1u);
+        args.tw_lf_hi = (float)((1u << args.tw_bhi) - 1u);
+        args.tw_wbytes = wb;
+        args.tw_v_my = args.v[args.full_ell];
+        args.tw_test_lo = args.full_ell > 0u;
+        args.tw_test_hi = args.full_ell + 2u < args.m;
+        args.tw_v_lo = args.tw_test_lo ? args.v[args.full_ell - 1u] : 0.0f;
+        args.tw_v_hi = args.tw_test_hi ? args.v[args.full_ell + 1u] : 0.0f;
+        for (uint32_t i = 0; try_two && i < args.n_tensors; i++) {
+            const uint64_t tail = args.t[i].numel % we;           // elements of a ragged last window (0: none)
+            uint64_t total = (uint64_t)(args.t[i].n_windows - (tail ? 1u : 0u)) * wb;
+            if (tail) {                                           // its own budget arithmetic, as the kernel does it
+                const uint64_t n = tail >> args.log2G, base = (uint64_t)(args.S[args.full_ell] - args.S[0]) * n;
+                const uint64_t rem = (((uint64_t)args.beta_q8 * n) >> 8) - (uint64_t)args.S[0] * n;
+                uint64_t kl = base <= rem ? (rem - base) / args.cost[args.full_ell] : 0u;   // (base > rem: the kernel gives the window up)
+                if (kl > n) kl = n;
+                total += n * lo + kl * up;
+            }
+            try_two = total <= args.t[i].capacity;
+        }
+    }
     args.flags2 = args.flags + args.total_windows;
-    args.gated = try_stream ? 1u : 0u;
+    args.gated = (try_stream || try_two) ? 1u : 0u;
+    if (try_two) {
+        const cudaError_t e = dispatch_two_width<BATCH>(dtype, args, stream);
+        if (e != cudaSuccess) return e;
+    }
     if (try_stream) {
         cudaError_t e = dispatch_stream<BATCH, ACT>(dtype, chunks, args, stream);
         if (e != cudaSuccess) return e;

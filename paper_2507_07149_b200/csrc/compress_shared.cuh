@@ -37,6 +37,13 @@ template <int NT> struct CompressArgs {
     uint32_t G, log2G, beta_q8, m, nearest, bulk_store, n_max;
     uint32_t full_ell, full_rem, full_rem_after;   // budget arithmetic of a full window (n_max groups)
     uint32_t full_test;       // ... whose groups share a width only if the keys of the levels around full_ell separate
+    // two-width streaming kernel: groups of a full window that are raised above level full_ell; the two widths, their
+    // largest codes as floats, bytes of a group at the lower width and what the raise adds, bytes of a whole window
+    uint32_t tw_k, tw_blo, tw_bhi, tw_size_lo, tw_size_up;
+    float tw_lf_lo, tw_lf_hi;
+    float tw_v_my, tw_v_lo, tw_v_hi;   // importance factors of the raise out of level full_ell, into it, and of the next one
+    uint32_t tw_test_lo, tw_test_hi;   // ... the latter two exist
+    uint64_t tw_wbytes;
     float stream_v_lo, stream_v_hi;   // importance factors of the raise into level full_ell and of the raise out of it
     uint32_t S[kMaxLevels], cost[kMaxLevels];
     float v[kMaxLevels];
@@ -202,6 +209,19 @@ __device__ __forceinline__ int lookback(const uint64_t *flags, uint32_t gw, uint
 // translation unit per element type).
 template <typename T, bool BATCH, int ACT>
 cudaError_t dispatch_stream_t(uint32_t chunks, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream);
+
+// The streaming kernel for calls whose windows end with two neighbouring widths (compress_twowidth.cuh; one translation
+// unit per element type).
+template <typename T, bool BATCH>
+cudaError_t dispatch_two_width_t(const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream);
+
+template <bool BATCH>
+inline cudaError_t dispatch_two_width(uint32_t dtype, const CompressArgs<BATCH ? DAF_BATCH_MAX : 1> &args, cudaStream_t stream)
+{
+    if (dtype == DAF_F32) return dispatch_two_width_t<float, BATCH>(args, stream);
+    if (dtype == DAF_F16) return dispatch_two_width_t<__half, BATCH>(args, stream);
+    return dispatch_two_width_t<__nv_bfloat16, BATCH>(args, stream);
+}
 
 // The two-pass kernels for windows of mixed widths (compress_twopass.cuh; one translation unit per element type).
 template <typename T, bool BATCH>
