@@ -37,6 +37,12 @@ template <int NT> struct CompressArgs {
     uint32_t G, log2G, beta_q8, m, nearest, bulk_store, n_max;
     uint32_t full_ell, full_rem, full_rem_after;   // budget arithmetic of a full window (n_max groups)
     uint32_t full_test;       // ... whose groups share a width only if the keys of the levels around full_ell separate
+    float stream_v_lo, stream_v_hi;   // importance factors of the raise into level full_ell and of the raise out of it
+    uint32_t S[kMaxLevels], cost[kMaxLevels];
+    float v[kMaxLevels];
+    SmemLayout lay;
+    PhiloxKeys keys;          // round keys of tensor 0 (single-tensor launches)
+    TensorDesc t[NT];
     // two-width streaming kernel: groups of a full window that are raised above level full_ell; the two widths, their
     // largest codes as floats, bytes of a group at the lower width and what the raise adds, bytes of a whole window
     uint32_t tw_k, tw_blo, tw_bhi, tw_size_lo, tw_size_up;
@@ -44,12 +50,6 @@ template <int NT> struct CompressArgs {
     float tw_v_my, tw_v_lo, tw_v_hi;   // importance factors of the raise out of level full_ell, into it, and of the next one
     uint32_t tw_test_lo, tw_test_hi;   // ... the latter two exist
     uint64_t tw_wbytes;
-    float stream_v_lo, stream_v_hi;   // importance factors of the raise into level full_ell and of the raise out of it
-    uint32_t S[kMaxLevels], cost[kMaxLevels];
-    float v[kMaxLevels];
-    SmemLayout lay;
-    PhiloxKeys keys;          // round keys of tensor 0 (single-tensor launches)
-    TensorDesc t[NT];
 };
 
 // ------------------------------------------------------------------------------------------
