@@ -82,8 +82,8 @@ typedef struct daf_params {
 
 /* daf_params.flags.  None of them changes a result.
  *   DAF_FLAG_STREAM_ALWAYS / _NEVER : daf_compress first runs a streaming kernel that assumes windows
- *       of one width (see daf_compress) unless the call is small or the parameters rule such windows
- *       out; ALWAYS drops the size rule, NEVER goes to the general kernel directly (e.g. for data known
+ *       of one width, or of two neighbouring widths (see daf_compress), unless the call is small or the
+ *       parameters rule such windows out; ALWAYS drops the size rule, NEVER goes to the general kernel directly (e.g. for data known
  *       to mix widths).  Giving both is an error.
  *   DAF_FLAG_ONE_PASS / _TWO_PASS : windows of mixed widths are handled either by the general kernel (one pass
  *       over the input; CTAs that wait for one another's window offsets) or by the two-pass kernels (widths first,
@@ -140,7 +140,11 @@ daf_status daf_shard(const daf_params *whole, uint32_t rank, uint32_t world, daf
  * groups) and writes every output on that assumption while it records what is needed to
  * check it; a small kernel that checks it for every window and writes the window offsets;
  * and a fallback, which returns at once unless the check failed somewhere and then redoes the
- * whole call with the window-by-window greedy choice.  The fallback is the general kernel
+ * whole call with the window-by-window greedy choice.  Where the budget lies between two
+ * allowed widths (groups of 256 to 1024 elements, default window) the streaming kernel is
+ * another one: it assumes that in every window the groups end at those two widths, the k
+ * groups with the largest ranges at the larger one (k follows from the budget alone), checks
+ * that itself window by window, and asks for the fallback where the assumption fails.  The fallback is the general kernel
  * (one launch; the input is read once), or, for calls of more than 4096 windows on 16-bit
  * elements with groups of 128 to 1024 elements, three kernels that read the input twice:
  * widths and metadata of every window, window offsets, quantize + pack.  A call of at most
